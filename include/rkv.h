@@ -1,0 +1,248 @@
+/*
+ * rkv.h -- C ABI of librkv: bulk verification of candidate-kernel outputs on
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the numerical-correctness step of the robust-kbench
+ * evaluation loop (arxiv 2509.14279): the outputs of K candidate kernels are
+ * compared with one reference output, for seeded test inputs drawn from several
+ * value distributions, and outputs that exploit a loophole are flagged.
+ *
+ *   - App. "Kernel Evaluation Environment": a kernel is correct iff it passes
+ *     all tests (input sizes x initialisation settings x seeds); absolute and
+ *     relative tolerance 1e-5.  -> rkv_verify_batch / rkv_verify_multi, the
+ *     per-element rule |c - r| <= atol + rtol*|r| and the joint verdict.
+ *   - Sec. 5 "Kernel Translation & Optimization": the candidate's result is
+ *     compared with the torch reference.  -> one reference, K candidates.
+ *   - Sec. 3 (harness): "diverse initialization states to prevent hardcoding";
+ *     forward and backward passes (a backward candidate returns several
+ *     gradient tensors).  -> rkv_gen_inputs, rkv_verify_multi.
+ *   - Sec. 3, App. A.1 and the listing "Level 2 - Task 13": constant outputs,
+ *     pass-through of the input, low-magnitude outputs.  -> the flags.
+ *
+ * Conventions.  Every function returns an rkv_status (0 = RKV_OK, < 0 = error)
+ * unless stated otherwise; none throws, aborts or prints.  Unless a parameter is
+ * marked HOST, a data pointer is caller-owned DEVICE memory of the current CUDA
+ * device, 16-byte aligned; the library reads inputs and writes outputs
+ * stream-ordered on the given stream and never synchronises it, except where a
+ * function says so.  bf16 tensors are raw 16-bit patterns.  Tensors are flat,
+ * contiguous, row-major; a shape is only a product.
+ */
+#ifndef RKV_H
+#define RKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum rkv_status {
+    RKV_OK = 0,
+    RKV_ERR_INVALID_ARG = -1,  /* null pointer, K < 1, n < 1, bad enum, negative / non-finite tolerance */
+    RKV_ERR_UNSUPPORTED = -2,  /* legal request outside this build's limits (see each function) */
+    RKV_ERR_ALIGNMENT = -3,    /* a device pointer is not 16-byte aligned */
+    RKV_ERR_WORKSPACE = -4,    /* workspace missing or smaller than rkv_workspace_bytes() */
+    RKV_ERR_CUDA = -5,         /* a CUDA runtime call failed (no device, launch error, ...) */
+    RKV_ERR_TIMEOUT = -6       /* device side: a bounded wait on a bulk copy ran out */
+} rkv_status;
+
+enum { RKV_F32 = 0, RKV_BF16 = 1 };
+
+/* Value distributions of the input generator. */
+enum {
+    RKV_DIST_NORMAL = 0,      /* N(0,1), Box-Muller                                   */
+    RKV_DIST_UNIFORM_PM1 = 1, /* uniform on [-1, 1), multiples of 2^-23               */
+    RKV_DIST_STUDENT_T2 = 2,  /* Student-t with 2 degrees of freedom (heavy-tailed)   */
+    RKV_DIST_SPARSE90 = 3,    /* exact +0 with probability 0.9, else N(0,1)           */
+    RKV_DIST_NORMAL_1E4 = 4   /* N(0,1) * 1e4 (large magnitude)                       */
+};
+
+/* Where a reference / input tensor comes from. */
+enum {
+    RKV_SRC_NONE = 0,      /* input only: no input tensor, copy-of-input flags stay clear */
+    RKV_SRC_POINTER = 1,   /* read from device memory                                     */
+    RKV_SRC_GENERATED = 2  /* regenerated on the fly from an rkv_gen_spec (fused path)    */
+};
+
+/* rkv_stats.verdict bits; a candidate passes iff verdict == 0. */
+enum {
+    RKV_FAIL_TOL = 1u << 0,            /* n_over_tol > 0                                        */
+    RKV_FAIL_NAN = 1u << 1,            /* the candidate holds a NaN                             */
+    RKV_FAIL_INF_MISMATCH = 1u << 2,   /* an infinity on one side not matched on the other      */
+    RKV_FAIL_LOOPHOLE_CONST = 1u << 3, /* candidate constant, reference not, n > 1              */
+    RKV_FAIL_LOOPHOLE_COPY = 1u << 4   /* candidate is a bit copy of the input, reference is not */
+};
+
+/* rkv_stats.flags bits. */
+enum {
+    RKV_FLAG_CAND_CONST = 1u << 0,         /* every candidate element bit-equal to element 0 */
+    RKV_FLAG_CAND_COPY_OF_INPUT = 1u << 1, /* every candidate element bit-equal to input[i]  */
+    RKV_FLAG_REF_CONST = 1u << 2,
+    RKV_FLAG_REF_COPY_OF_INPUT = 1u << 3,
+    RKV_FLAG_HAS_NAN = 1u << 4,
+    RKV_FLAG_HAS_INF = 1u << 5
+};
+
+#define RKV_NO_INDEX UINT64_MAX
+
+/*
+ * Result for one candidate and one tensor (88 bytes, little-endian, 8-aligned).
+ * With c the candidate and r the reference, both as fp32 (bf16 is upcast
+ * exactly), an element is COMPARABLE when c and r are finite.  For comparable
+ * elements e = |c - r| (one fp32 subtraction) and the element is over tolerance
+ * when !(e <= atol + rtol*|r|), the product and the sum each rounded to fp32.
+ * Equal infinities match and are not comparable; any other non-finite
+ * involvement counts as over tolerance.  Indices are flat element offsets, the
+ * first (smallest) index attaining the maximum; RKV_NO_INDEX when no element
+ * qualifies.  max_rel_err ranges over comparable elements with r != 0.
+ */
+typedef struct rkv_stats {
+    uint32_t verdict;
+    uint32_t flags;
+    uint64_t n_over_tol;
+    uint64_t n_nan;           /* NaN elements of the candidate            */
+    uint64_t n_inf;           /* infinite elements of the candidate       */
+    uint64_t n_inf_mismatch;  /* non-comparable, not matching, an infinity on either side */
+    uint64_t n_comparable;
+    uint64_t argmax_abs_err;
+    uint64_t argmax_rel_err;
+    double sum_abs_err;       /* sum of e over comparable elements        */
+    float max_abs_err;        /* 0 when nothing is comparable             */
+    float max_rel_err;
+    float mean_abs_err;       /* (float)(sum_abs_err / n_comparable), 0 if none */
+    uint32_t reserved;
+} rkv_stats;
+
+/* A Philox stream: which (seed, stream_id, distribution) tensor to generate.
+ * Element i is produced by word (i & 3) of Philox4x32-10 block (i >> 2) with
+ * key = seed and counter = (block index, stream_id).  RKV_DIST_SPARSE90 also
+ * consumes the stream stream_id + 1 (its zero mask). */
+typedef struct rkv_gen_spec {
+    uint64_t seed;
+    uint64_t stream_id;
+    int32_t dist;
+    int32_t reserved;
+} rkv_gen_spec;
+
+/* One tensor of a verification case. */
+typedef struct rkv_tensor_desc {
+    uint64_t n;                /* elements; 1 <= n < 2^40                                      */
+    const void *ref;           /* DEVICE, n elements of ref_dtype; used when ref_src == POINTER */
+    const void *input;         /* DEVICE, n elements of cand_dtype; used when input_src == POINTER */
+    const void *const *cands;  /* HOST array of K DEVICE pointers, n elements of cand_dtype each */
+    rkv_gen_spec ref_gen;      /* used when ref_src == GENERATED   */
+    rkv_gen_spec input_gen;    /* used when input_src == GENERATED */
+    int32_t cand_dtype;        /* RKV_F32 | RKV_BF16 */
+    int32_t ref_dtype;         /* RKV_F32 | RKV_BF16; a generated reference is rounded to it */
+    int32_t ref_src;           /* RKV_SRC_POINTER | RKV_SRC_GENERATED */
+    int32_t input_src;         /* RKV_SRC_NONE | RKV_SRC_POINTER | RKV_SRC_GENERATED; the input
+                                  has the candidates' dtype (a copy is a bit copy) */
+    float atol;                /* finite, >= 0 */
+    float rtol;                /* finite, >= 0 */
+} rkv_tensor_desc;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int rkv_version(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char *rkv_status_string(int status);
+
+/* Stream used by the two calls that take none (rkv_gen_inputs,
+ * rkv_verify_batch).  cuda_stream is a cudaStream_t; NULL = default stream.
+ * Process-wide; not synchronised against concurrent callers. */
+int rkv_set_stream(void *cuda_stream);
+
+/*
+ * Input generator (Sec. 3: diverse initialisation states; App. "Kernel
+ * Evaluation Environment": multiple random seeds).  Fills out with the tensor
+ * (seed, stream 0, dist).
+ *   shape  HOST array of ndim extents (>= 1 each); only the product is used
+ *   dtype  RKV_F32 | RKV_BF16 (fp32 value rounded to nearest-even)
+ *   out    DEVICE, product(shape) elements, 16-byte aligned
+ * Runs on the stream set by rkv_set_stream.  Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+int rkv_gen_inputs(uint64_t seed, int dist, const int64_t *shape, int ndim, int dtype, void *out);
+
+/*
+ * Same generator with every knob: elements first_elem .. first_elem + n - 1 of
+ * the tensor (seed, stream_id, dist) are written to out[0 .. n).  first_elem
+ * must be a multiple of 4 (one Philox block serves four elements).
+ */
+int rkv_gen_inputs_ex(uint64_t seed, uint64_t stream_id, int dist, uint64_t n,
+                      uint64_t first_elem, int dtype, void *out, void *cuda_stream);
+
+/*
+ * Verify K candidates against one reference (App. "Kernel Evaluation
+ * Environment"; Sec. 5).  Both sides have dtype `dtype`; no input tensor, so the
+ * copy-of-input flags stay clear.
+ *   ref        DEVICE, n elements
+ *   cands      HOST array of K DEVICE pointers, n elements each
+ *   stats_out  DEVICE, K rkv_stats, written stream-ordered
+ * Runs on the stream set by rkv_set_stream.  Uses a library-owned scratch
+ * buffer that grows on demand (cudaMalloc on first use / growth: not safe
+ * during stream capture; concurrent calls on different streams would share it,
+ * so serialise them).  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+int rkv_verify_batch(const void *ref, const void *const *cands, int K, uint64_t n, int dtype,
+                     float atol, float rtol, rkv_stats *stats_out);
+
+/*
+ * General form: T tensors per candidate, verified in one launch; candidate k
+ * passes jointly iff it passes on every tensor (the paper's "passes all tests";
+ * a backward candidate returns three gradients).
+ *   tensors     HOST array of T descriptors (1 <= T <= 64); tensors[t].cands HOST array of K
+ *   stats_out   DEVICE, K*T rkv_stats, entry [k*T + t]
+ *   joint_pass  DEVICE, K uint32 (1 = pass on all T tensors), may be NULL
+ *   workspace   DEVICE scratch, >= rkv_workspace_bytes(tensors, T, K) bytes, 256-byte
+ *               aligned; contents are undefined afterwards; must not be shared by
+ *               calls that overlap on the GPU
+ * Nothing is allocated.  The descriptors and pointer tables are copied to the
+ * workspace with one cudaMemcpyAsync from pageable host memory.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.  A device-side
+ * timeout is reported by rkv_device_status.
+ */
+int rkv_verify_multi(const rkv_tensor_desc *tensors, int T, int K, rkv_stats *stats_out,
+                     uint32_t *joint_pass, void *workspace, size_t workspace_bytes,
+                     void *cuda_stream);
+
+/* Scratch bytes rkv_verify_multi needs for this case on the current device
+ * (0 on an invalid argument).  Depends on n, the dtypes, T, K and the device's
+ * SM count only. */
+size_t rkv_workspace_bytes(const rkv_tensor_desc *tensors, int T, int K);
+
+/* Synchronises cuda_stream and returns the device-side status word the last
+ * rkv_verify_multi on this workspace left (RKV_OK or RKV_ERR_TIMEOUT), or
+ * RKV_ERR_CUDA. */
+int rkv_device_status(const void *workspace, void *cuda_stream);
+
+/*
+ * End-to-end form with HOST buffers: copies the reference and the candidates to
+ * the device in chunks (overlapped with verification on two streams), verifies,
+ * copies the K results back and synchronises.  Pinned host buffers make the
+ * copies asynchronous.  Allocates (and caches) device staging memory.
+ *   ref_host     HOST, n elements of dtype
+ *   cands_host   HOST array of K HOST pointers
+ *   stats_host   HOST, K rkv_stats
+ */
+int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, int K, uint64_t n,
+                          int dtype, float atol, float rtol, rkv_stats *stats_host);
+
+/*
+ * Host-only planning helper (no CUDA call): how a tensor is cut into slabs.
+ * A slab is the run of elements whose reference (and input) one thread block
+ * stages in shared memory and reuses for all K candidates.
+ *   smem_bytes_per_elem  reference bytes + input bytes kept per element (2..8)
+ *   num_sms              SM count of the device
+ * Writes the slab length (a multiple of 128 elements) and the slab count.
+ */
+int rkv_plan_slabs(uint64_t n, int smem_bytes_per_elem, int num_sms, uint32_t *slab_elems,
+                   uint64_t *n_slabs);
+
+/* Releases the library-owned scratch and staging buffers of all devices. */
+int rkv_release_cached(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RKV_H */

@@ -1,0 +1,304 @@
+"""ctypes binding of ``librkv.so`` (declared in ``include/rkv.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch is used for device memory (``tensor.data_ptr()``) and for the
+current stream.  There is no fallback: if the library is missing, loading
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librkv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = (
+    0, -1, -2, -3, -4, -5, -6)
+F32, BF16 = 0, 1
+DIST_NORMAL, DIST_UNIFORM_PM1, DIST_STUDENT_T2, DIST_SPARSE90, DIST_NORMAL_1E4 = range(5)
+SRC_NONE, SRC_POINTER, SRC_GENERATED = 0, 1, 2
+FAIL_TOL, FAIL_NAN, FAIL_INF_MISMATCH, FAIL_LOOPHOLE_CONST, FAIL_LOOPHOLE_COPY = 1, 2, 4, 8, 16
+(FLAG_CAND_CONST, FLAG_CAND_COPY_OF_INPUT, FLAG_REF_CONST, FLAG_REF_COPY_OF_INPUT,
+ FLAG_HAS_NAN, FLAG_HAS_INF) = 1, 2, 4, 8, 16, 32
+NO_INDEX = 2**64 - 1
+
+STATS_DTYPE = np.dtype([
+    ("verdict", "<u4"), ("flags", "<u4"), ("n_over_tol", "<u8"), ("n_nan", "<u8"),
+    ("n_inf", "<u8"), ("n_inf_mismatch", "<u8"), ("n_comparable", "<u8"),
+    ("argmax_abs_err", "<u8"), ("argmax_rel_err", "<u8"), ("sum_abs_err", "<f8"),
+    ("max_abs_err", "<f4"), ("max_rel_err", "<f4"), ("mean_abs_err", "<f4"), ("reserved", "<u4"),
+])
+STATS_BYTES = STATS_DTYPE.itemsize
+assert STATS_BYTES == 88
+
+
+class RkvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class GenSpec(ctypes.Structure):
+    _fields_ = [("seed", ctypes.c_uint64), ("stream_id", ctypes.c_uint64),
+                ("dist", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class TensorDescC(ctypes.Structure):
+    _fields_ = [
+        ("n", ctypes.c_uint64),
+        ("ref", ctypes.c_void_p),
+        ("input", ctypes.c_void_p),
+        ("cands", ctypes.POINTER(ctypes.c_void_p)),
+        ("ref_gen", GenSpec),
+        ("input_gen", GenSpec),
+        ("cand_dtype", ctypes.c_int32),
+        ("ref_dtype", ctypes.c_int32),
+        ("ref_src", ctypes.c_int32),
+        ("input_src", ctypes.c_int32),
+        ("atol", ctypes.c_float),
+        ("rtol", ctypes.c_float),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2509_14279_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, u64, i32, f32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float
+        L.rkv_version.restype = i32
+        L.rkv_version.argtypes = []
+        L.rkv_status_string.restype = ctypes.c_char_p
+        L.rkv_status_string.argtypes = [i32]
+        L.rkv_set_stream.restype = i32
+        L.rkv_set_stream.argtypes = [vp]
+        L.rkv_gen_inputs.restype = i32
+        L.rkv_gen_inputs.argtypes = [u64, i32, ctypes.POINTER(ctypes.c_int64), i32, i32, vp]
+        L.rkv_gen_inputs_ex.restype = i32
+        L.rkv_gen_inputs_ex.argtypes = [u64, u64, i32, u64, u64, i32, vp, vp]
+        L.rkv_verify_batch.restype = i32
+        L.rkv_verify_batch.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
+        L.rkv_verify_multi.restype = i32
+        L.rkv_verify_multi.argtypes = [ctypes.POINTER(TensorDescC), i32, i32, vp, vp, vp,
+                                       ctypes.c_size_t, vp]
+        L.rkv_workspace_bytes.restype = ctypes.c_size_t
+        L.rkv_workspace_bytes.argtypes = [ctypes.POINTER(TensorDescC), i32, i32]
+        L.rkv_device_status.restype = i32
+        L.rkv_device_status.argtypes = [vp, vp]
+        L.rkv_verify_batch_host.restype = i32
+        L.rkv_verify_batch_host.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
+        L.rkv_plan_slabs.restype = i32
+        L.rkv_plan_slabs.argtypes = [u64, i32, i32, ctypes.POINTER(ctypes.c_uint32),
+                                     ctypes.POINTER(ctypes.c_uint64)]
+        L.rkv_release_cached.restype = i32
+        L.rkv_release_cached.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().rkv_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise RkvError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"rkv tensors are float32 or bfloat16, got {t.dtype}")
+
+
+def _stream_ptr(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def version() -> int:
+    return int(lib().rkv_version())
+
+
+def set_stream(stream=None) -> None:
+    _check(lib().rkv_set_stream(ctypes.c_void_p(_stream_ptr(stream))), "rkv_set_stream")
+
+
+def plan_slabs(n: int, smem_bytes_per_elem: int, num_sms: int) -> tuple:
+    """Host-only: (slab_elems, n_slabs) for a tensor of n elements."""
+    s, c = ctypes.c_uint32(), ctypes.c_uint64()
+    _check(lib().rkv_plan_slabs(int(n), int(smem_bytes_per_elem), int(num_sms),
+                                ctypes.byref(s), ctypes.byref(c)), "rkv_plan_slabs")
+    return int(s.value), int(c.value)
+
+
+def gen_inputs(seed: int, dist: int, shape, dtype: torch.dtype = torch.float32,
+               out: torch.Tensor | None = None) -> torch.Tensor:
+    """rkv_gen_inputs: the tensor (seed, stream 0, dist) on the current device and stream."""
+    shape = tuple(int(s) for s in shape)
+    if out is None:
+        out = torch.empty(shape, dtype=dtype, device="cuda")
+    set_stream()
+    arr = (ctypes.c_int64 * len(shape))(*shape)
+    _check(lib().rkv_gen_inputs(int(seed), int(dist), arr, len(shape), _dtype_code(out),
+                                ctypes.c_void_p(out.data_ptr())), "rkv_gen_inputs")
+    return out
+
+
+def gen_inputs_ex(seed: int, stream_id: int, dist: int, n: int, first_elem: int = 0,
+                  dtype: torch.dtype = torch.float32, out: torch.Tensor | None = None,
+                  stream=None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty(int(n), dtype=dtype, device="cuda")
+    _check(lib().rkv_gen_inputs_ex(int(seed), int(stream_id), int(dist), int(n), int(first_elem),
+                                   _dtype_code(out), ctypes.c_void_p(out.data_ptr()),
+                                   ctypes.c_void_p(_stream_ptr(stream))), "rkv_gen_inputs_ex")
+    return out
+
+
+def stats_to_numpy(stats: torch.Tensor) -> np.ndarray:
+    """Device (or host) stats buffer -> structured numpy array (synchronises)."""
+    return stats.detach().cpu().numpy().view(STATS_DTYPE)
+
+
+def verify_batch(ref: torch.Tensor, cands, atol: float, rtol: float,
+                 stats_out: torch.Tensor | None = None) -> torch.Tensor:
+    """rkv_verify_batch: K candidates against one reference, same dtype, no input tensor.
+    Returns the device buffer of K rkv_stats (uint8, K*88 bytes)."""
+    K = len(cands)
+    n = ref.numel()
+    if stats_out is None:
+        stats_out = torch.empty(K * STATS_BYTES, dtype=torch.uint8, device=ref.device)
+    ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cands])
+    set_stream()
+    _check(lib().rkv_verify_batch(ctypes.c_void_p(ref.data_ptr()), ptrs, K, n, _dtype_code(ref),
+                                  float(atol), float(rtol), ctypes.c_void_p(stats_out.data_ptr())),
+           "rkv_verify_batch")
+    return stats_out
+
+
+@dataclass
+class TensorDesc:
+    """One tensor of a case, as torch tensors (or generator specs)."""
+    n: int
+    cands: list                       # K device tensors
+    atol: float
+    rtol: float
+    ref: torch.Tensor | None = None   # None -> regenerated from ref_gen
+    input: torch.Tensor | None = None
+    ref_gen: tuple | None = None      # (seed, stream_id, dist)
+    input_gen: tuple | None = None
+    ref_dtype: int | None = None      # for a generated reference; default fp32
+    _keep: list = field(default_factory=list, repr=False)
+
+    def to_c(self) -> TensorDescC:
+        d = TensorDescC()
+        d.n = int(self.n)
+        K = len(self.cands)
+        ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in self.cands])
+        self._keep.append(ptrs)
+        d.cands = ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p))
+        d.cand_dtype = _dtype_code(self.cands[0])
+        if self.ref is not None:
+            d.ref = self.ref.data_ptr()
+            d.ref_src = SRC_POINTER
+            d.ref_dtype = _dtype_code(self.ref)
+        else:
+            seed, stream_id, dist = self.ref_gen
+            d.ref_gen = GenSpec(int(seed), int(stream_id), int(dist), 0)
+            d.ref_src = SRC_GENERATED
+            d.ref_dtype = F32 if self.ref_dtype is None else int(self.ref_dtype)
+        if self.input is not None:
+            d.input = self.input.data_ptr()
+            d.input_src = SRC_POINTER
+        elif self.input_gen is not None:
+            seed, stream_id, dist = self.input_gen
+            d.input_gen = GenSpec(int(seed), int(stream_id), int(dist), 0)
+            d.input_src = SRC_GENERATED
+        else:
+            d.input_src = SRC_NONE
+        d.atol = float(self.atol)
+        d.rtol = float(self.rtol)
+        return d
+
+
+def _desc_array(tensors) -> ctypes.Array:
+    arr = (TensorDescC * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t.to_c()
+    return arr
+
+
+def workspace_bytes(tensors, K: int) -> int:
+    arr = _desc_array(tensors)
+    return int(lib().rkv_workspace_bytes(arr, len(tensors), int(K)))
+
+
+def verify_multi(tensors, K: int, workspace: torch.Tensor | None = None,
+                 stats_out: torch.Tensor | None = None, joint_pass: torch.Tensor | None = None,
+                 stream=None, descs=None):
+    """rkv_verify_multi.  Returns (stats [K*T*88 bytes uint8], joint_pass [K] int32, workspace).
+
+    ``descs`` may carry a prebuilt ctypes descriptor array (from ``prepare``) so
+    that a timed loop does no Python marshalling.
+    """
+    T = len(tensors)
+    arr = _desc_array(tensors) if descs is None else descs
+    dev = tensors[0].cands[0].device
+    if workspace is None:
+        need = int(lib().rkv_workspace_bytes(arr, T, int(K)))
+        if need == 0:
+            raise RkvError(ERR_INVALID_ARG, "rkv_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if stats_out is None:
+        stats_out = torch.empty(K * T * STATS_BYTES, dtype=torch.uint8, device=dev)
+    if joint_pass is None:
+        joint_pass = torch.empty(K, dtype=torch.int32, device=dev)
+    _check(lib().rkv_verify_multi(arr, T, int(K), ctypes.c_void_p(stats_out.data_ptr()),
+                                  ctypes.c_void_p(joint_pass.data_ptr()),
+                                  ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                  ctypes.c_void_p(_stream_ptr(stream))), "rkv_verify_multi")
+    return stats_out, joint_pass, workspace
+
+
+def prepare(tensors):
+    """Marshal the descriptors once; pass the result as ``descs=`` to verify_multi."""
+    return _desc_array(tensors)
+
+
+def device_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(lib().rkv_device_status(ctypes.c_void_p(workspace.data_ptr()),
+                                       ctypes.c_void_p(_stream_ptr(stream))))
+
+
+def verify_batch_host(ref: torch.Tensor, cands, atol: float, rtol: float) -> np.ndarray:
+    """rkv_verify_batch_host: HOST tensors in, structured numpy stats out (synchronous)."""
+    K = len(cands)
+    n = ref.numel()
+    assert ref.device.type == "cpu" and all(c.device.type == "cpu" for c in cands)
+    out = np.zeros(K, dtype=STATS_DTYPE)
+    ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cands])
+    set_stream()
+    _check(lib().rkv_verify_batch_host(ctypes.c_void_p(ref.data_ptr()), ptrs, K, n,
+                                       _dtype_code(ref), float(atol), float(rtol),
+                                       out.ctypes.data_as(ctypes.c_void_p)),
+           "rkv_verify_batch_host")
+    return out
+
+
+def release_cached() -> None:
+    lib().rkv_release_cached()

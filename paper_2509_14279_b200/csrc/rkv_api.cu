@@ -1,0 +1,430 @@
+// Host side of librkv: argument validation, slab planning, workspace layout,
+// launches, and the host-buffer end-to-end form.  No torch types anywhere.
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
+#include <vector>
+
+#include "rkv_internal.h"
+
+namespace rkv {
+
+// ----------------------------------------------------------------------------
+// planning
+// ----------------------------------------------------------------------------
+
+int smem_bytes_per_elem(const rkv_tensor_desc& t) {
+    // a generated reference is staged as fp32 whatever its dtype
+    const int rsz = (t.ref_src == RKV_SRC_POINTER && t.ref_dtype == RKV_BF16) ? 2 : 4;
+    const int isz = t.input_src == RKV_SRC_NONE ? 0 : (t.cand_dtype == RKV_BF16 ? 2 : 4);
+    return rsz + isz;
+}
+
+// Slab length: the smallest whole number of waves w of the resident grid
+// (num_sms * kBlocksPerSm blocks) such that n / (grid * w), rounded up to the
+// granule, fits the shared-memory budget.  Every block then gets the same number
+// of equally long slabs, so no wave is partly empty.
+static int plan_one(uint64_t n, int bytes_per_elem, int num_sms, uint32_t* slab_elems, uint64_t* n_slabs) {
+    if (n == 0 || n >= kMaxN || bytes_per_elem < 2 || bytes_per_elem > 8 || num_sms < 1)
+        return RKV_ERR_INVALID_ARG;
+    const uint64_t s_max = (uint64_t)(kSmemDataBudget / bytes_per_elem) / kSlabGranule * kSlabGranule;
+    const uint64_t grid = (uint64_t)num_sms * kBlocksPerSm;
+    uint64_t S = s_max;
+    // smallest number of waves whose slabs fit
+    uint64_t w = (n + grid * s_max - 1) / (grid * s_max);
+    if (w == 0) w = 1;
+    for (;; ++w) {
+        const uint64_t per = (n + grid * w - 1) / (grid * w);
+        const uint64_t s = (per + kSlabGranule - 1) / kSlabGranule * kSlabGranule;
+        if (s <= s_max) { S = s; break; }
+    }
+    *slab_elems = (uint32_t)S;
+    *n_slabs = (n + S - 1) / S;
+    return RKV_OK;
+}
+
+static bool finite_nonneg(float x) { return x >= 0.0f && x <= 3.402823466e38f; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool dtype_ok(int d) { return d == RKV_F32 || d == RKV_BF16; }
+static bool dist_ok(int d) { return d >= RKV_DIST_NORMAL && d <= RKV_DIST_NORMAL_1E4; }
+
+int validate_tensors(const rkv_tensor_desc* tensors, int T, int K) {
+    if (!tensors || T < 1 || K < 1) return RKV_ERR_INVALID_ARG;
+    if (T > kMaxTensors) return RKV_ERR_UNSUPPORTED;
+    for (int t = 0; t < T; ++t) {
+        const rkv_tensor_desc& d = tensors[t];
+        if (d.n < 1) return RKV_ERR_INVALID_ARG;
+        if (d.n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+        if (!dtype_ok(d.cand_dtype) || !dtype_ok(d.ref_dtype)) return RKV_ERR_INVALID_ARG;
+        if (!finite_nonneg(d.atol) || !finite_nonneg(d.rtol)) return RKV_ERR_INVALID_ARG;
+        if (d.ref_src == RKV_SRC_POINTER) {
+            if (!d.ref) return RKV_ERR_INVALID_ARG;
+            if (!aligned16(d.ref)) return RKV_ERR_ALIGNMENT;
+        } else if (d.ref_src == RKV_SRC_GENERATED) {
+            if (!dist_ok(d.ref_gen.dist)) return RKV_ERR_INVALID_ARG;
+        } else {
+            return RKV_ERR_INVALID_ARG;
+        }
+        if (d.input_src == RKV_SRC_POINTER) {
+            if (!d.input) return RKV_ERR_INVALID_ARG;
+            if (!aligned16(d.input)) return RKV_ERR_ALIGNMENT;
+        } else if (d.input_src == RKV_SRC_GENERATED) {
+            if (!dist_ok(d.input_gen.dist)) return RKV_ERR_INVALID_ARG;
+        } else if (d.input_src != RKV_SRC_NONE) {
+            return RKV_ERR_INVALID_ARG;
+        }
+        if (!d.cands) return RKV_ERR_INVALID_ARG;
+        for (int k = 0; k < K; ++k) {
+            if (!d.cands[k]) return RKV_ERR_INVALID_ARG;
+            if (!aligned16(d.cands[k])) return RKV_ERR_ALIGNMENT;
+        }
+    }
+    return RKV_OK;
+}
+
+int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* plan) {
+    uint64_t items = 0;
+    for (int t = 0; t < T; ++t) {
+        uint32_t S;
+        uint64_t ns;
+        const int rc = plan_one(tensors[t].n, smem_bytes_per_elem(tensors[t]), num_sms, &S, &ns);
+        if (rc != RKV_OK) return rc;
+        plan->slab_elems[t] = S;
+        plan->n_slabs[t] = (uint32_t)ns;
+        plan->first_item[t] = (uint32_t)items;
+        items += ns;
+        if (items > 0xFFFFFFFFull / 2) return RKV_ERR_UNSUPPORTED;
+    }
+    plan->total_items = (uint32_t)items;
+    size_t table = (size_t)T * sizeof(DevTensor) + (size_t)T * (size_t)K * sizeof(void*);
+    plan->table_bytes = (table + 255) / 256 * 256;
+    plan->partial_bytes = (size_t)items * (size_t)(K + 1) * sizeof(Partial);
+    plan->total_bytes = sizeof(WorkspaceHeader) + plan->table_bytes + plan->partial_bytes;
+    return RKV_OK;
+}
+
+int current_num_sms(int* num_sms) {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RKV_ERR_CUDA; }
+    if (dev >= 0 && dev < 64 && cached[dev]) { *num_sms = cached[dev]; return RKV_OK; }
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        return RKV_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64) cached[dev] = n;
+    *num_sms = n;
+    return RKV_OK;
+}
+
+// ----------------------------------------------------------------------------
+// library-owned buffers for the forms that take no workspace
+// ----------------------------------------------------------------------------
+namespace {
+
+struct DeviceCache {
+    void* workspace = nullptr;
+    size_t workspace_bytes = 0;
+    void* staging = nullptr;      // host-buffer form: reference + candidate chunks + stats
+    size_t staging_bytes = 0;
+    cudaStream_t copy_stream[2] = {nullptr, nullptr};
+    cudaEvent_t copied[2] = {nullptr, nullptr};
+    cudaEvent_t consumed[2] = {nullptr, nullptr};
+};
+
+std::mutex g_mutex;
+DeviceCache g_cache[64];
+cudaStream_t g_stream = nullptr;
+
+int ensure(void** buf, size_t* have, size_t want) {
+    if (*have >= want) return RKV_OK;
+    if (*buf) { cudaFree(*buf); *buf = nullptr; *have = 0; }
+    size_t bytes = (want + (size_t(1) << 20) - 1) >> 20 << 20;
+    if (cudaMalloc(buf, bytes) != cudaSuccess) { cudaGetLastError(); return RKV_ERR_CUDA; }
+    *have = bytes;
+    return RKV_OK;
+}
+
+// Build the device tables in the workspace and launch verify (+ finalize).
+int run_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k_end, bool finalize,
+             bool upload, const Plan& plan, int num_sms, rkv_stats* stats_out, uint32_t* joint_pass,
+             void* workspace, cudaStream_t stream) {
+    unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
+    DevTensor* d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
+    const void** d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) +
+                                                         (size_t)T * sizeof(DevTensor));
+    Partial* partials = reinterpret_cast<Partial*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
+    int32_t* status = reinterpret_cast<int32_t*>(ws);
+    if (upload) {
+        std::vector<unsigned char> blob(sizeof(WorkspaceHeader) + plan.table_bytes, 0);
+        DevTensor* h_t = reinterpret_cast<DevTensor*>(blob.data() + sizeof(WorkspaceHeader));
+        const void** h_p = reinterpret_cast<const void**>(blob.data() + sizeof(WorkspaceHeader) +
+                                                          (size_t)T * sizeof(DevTensor));
+        for (int t = 0; t < T; ++t) {
+            const rkv_tensor_desc& s = tensors[t];
+            DevTensor& d = h_t[t];
+            d.n = s.n;
+            d.ref = s.ref_src == RKV_SRC_POINTER ? s.ref : nullptr;
+            d.input = s.input_src == RKV_SRC_POINTER ? s.input : nullptr;
+            d.cands = d_ptrs + (size_t)t * K;
+            d.ref_seed = s.ref_gen.seed; d.ref_stream = s.ref_gen.stream_id; d.ref_dist = s.ref_gen.dist;
+            d.in_seed = s.input_gen.seed; d.in_stream = s.input_gen.stream_id; d.in_dist = s.input_gen.dist;
+            d.cand_dtype = s.cand_dtype; d.ref_dtype = s.ref_dtype;
+            d.ref_src = s.ref_src; d.input_src = s.input_src;
+            d.atol = s.atol; d.rtol = s.rtol;
+            d.slab_elems = plan.slab_elems[t]; d.n_slabs = plan.n_slabs[t];
+            d.first_item = plan.first_item[t];
+            for (int k = 0; k < K; ++k) h_p[(size_t)t * K + k] = s.cands[k];
+        }
+        if (cudaMemcpyAsync(ws, blob.data(), blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return RKV_ERR_CUDA;
+        }
+    }
+    int rc = launch_verify(d_tensors, T, K, k_begin, k_end, plan.total_items, num_sms, partials, status,
+                           stream);
+    if (rc != RKV_OK) return rc;
+    if (finalize) rc = launch_finalize(d_tensors, T, K, partials, stats_out, joint_pass, stream);
+    return rc;
+}
+
+}  // namespace
+}  // namespace rkv
+
+using namespace rkv;
+
+// ----------------------------------------------------------------------------
+// C ABI
+// ----------------------------------------------------------------------------
+extern "C" {
+
+int rkv_version(void) { return 100; }
+
+const char* rkv_status_string(int status) {
+    switch (status) {
+        case RKV_OK: return "ok";
+        case RKV_ERR_INVALID_ARG: return "invalid argument";
+        case RKV_ERR_UNSUPPORTED: return "unsupported size or combination";
+        case RKV_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case RKV_ERR_WORKSPACE: return "workspace missing or too small";
+        case RKV_ERR_CUDA: return "CUDA runtime error";
+        case RKV_ERR_TIMEOUT: return "device-side bounded wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int rkv_set_stream(void* cuda_stream) {
+    g_stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    return RKV_OK;
+}
+
+int rkv_plan_slabs(uint64_t n, int smem_bytes_per_elem, int num_sms, uint32_t* slab_elems,
+                   uint64_t* n_slabs) {
+    if (!slab_elems || !n_slabs) return RKV_ERR_INVALID_ARG;
+    if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+    return plan_one(n, smem_bytes_per_elem, num_sms, slab_elems, n_slabs);
+}
+
+int rkv_gen_inputs_ex(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t first_elem,
+                      int dtype, void* out, void* cuda_stream) {
+    if (!out || n < 1 || !dist_ok(dist) || !dtype_ok(dtype) || (first_elem & 3u))
+        return RKV_ERR_INVALID_ARG;
+    if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+    if (!aligned16(out)) return RKV_ERR_ALIGNMENT;
+    int sms = 0;
+    const int rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    return launch_gen(seed, stream_id, dist, n, first_elem, dtype, out, sms,
+                      reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int rkv_gen_inputs(uint64_t seed, int dist, const int64_t* shape, int ndim, int dtype, void* out) {
+    if (!shape || ndim < 1) return RKV_ERR_INVALID_ARG;
+    uint64_t n = 1;
+    for (int i = 0; i < ndim; ++i) {
+        if (shape[i] < 1) return RKV_ERR_INVALID_ARG;
+        if ((uint64_t)shape[i] >= kMaxN || n * (uint64_t)shape[i] >= kMaxN) return RKV_ERR_UNSUPPORTED;
+        n *= (uint64_t)shape[i];
+    }
+    return rkv_gen_inputs_ex(seed, 0, dist, n, 0, dtype, out, g_stream);
+}
+
+size_t rkv_workspace_bytes(const rkv_tensor_desc* tensors, int T, int K) {
+    if (!tensors || T < 1 || T > kMaxTensors || K < 1) return 0;
+    for (int t = 0; t < T; ++t)
+        if (tensors[t].n < 1 || tensors[t].n >= kMaxN) return 0;
+    int sms = 0;
+    if (current_num_sms(&sms) != RKV_OK) return 0;
+    Plan plan;
+    if (make_plan(tensors, T, K, sms, &plan) != RKV_OK) return 0;
+    return plan.total_bytes;
+}
+
+int rkv_verify_multi(const rkv_tensor_desc* tensors, int T, int K, rkv_stats* stats_out,
+                     uint32_t* joint_pass, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int rc = validate_tensors(tensors, T, K);
+    if (rc != RKV_OK) return rc;
+    if (!stats_out) return RKV_ERR_INVALID_ARG;
+    if (!workspace) return RKV_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return RKV_ERR_ALIGNMENT;
+    int sms = 0;
+    rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    Plan plan;
+    rc = make_plan(tensors, T, K, sms, &plan);
+    if (rc != RKV_OK) return rc;
+    if (workspace_bytes < plan.total_bytes) return RKV_ERR_WORKSPACE;
+    return run_case(tensors, T, K, 0, K, true, true, plan, sms, stats_out, joint_pass, workspace,
+                    reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int rkv_verify_batch(const void* ref, const void* const* cands, int K, uint64_t n, int dtype, float atol,
+                     float rtol, rkv_stats* stats_out) {
+    rkv_tensor_desc d;
+    memset(&d, 0, sizeof d);
+    d.n = n; d.ref = ref; d.cands = cands;
+    d.cand_dtype = dtype; d.ref_dtype = dtype;
+    d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
+    d.atol = atol; d.rtol = rtol;
+    int rc = validate_tensors(&d, 1, K);
+    if (rc != RKV_OK) return rc;
+    if (!stats_out) return RKV_ERR_INVALID_ARG;
+    int sms = 0;
+    rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    Plan plan;
+    rc = make_plan(&d, 1, K, sms, &plan);
+    if (rc != RKV_OK) return rc;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCache& c = g_cache[dev & 63];
+    rc = ensure(&c.workspace, &c.workspace_bytes, plan.total_bytes);
+    if (rc != RKV_OK) return rc;
+    return run_case(&d, 1, K, 0, K, true, true, plan, sms, stats_out, nullptr, c.workspace, g_stream);
+}
+
+int rkv_device_status(const void* workspace, void* cuda_stream) {
+    if (!workspace) return RKV_ERR_INVALID_ARG;
+    int32_t st = 0;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(&st, workspace, sizeof st, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return RKV_ERR_CUDA;
+    }
+    return st;
+}
+
+int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, int K, uint64_t n,
+                          int dtype, float atol, float rtol, rkv_stats* stats_host) {
+    if (!ref_host || !cands_host || !stats_host || K < 1 || n < 1 || !dtype_ok(dtype) ||
+        !finite_nonneg(atol) || !finite_nonneg(rtol))
+        return RKV_ERR_INVALID_ARG;
+    if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+    for (int k = 0; k < K; ++k)
+        if (!cands_host[k]) return RKV_ERR_INVALID_ARG;
+    int sms = 0;
+    int rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCache& c = g_cache[dev & 63];
+
+    const size_t esz = dtype == RKV_BF16 ? 2 : 4;
+    const size_t tensor_bytes = ((size_t)n * esz + 255) / 256 * 256;
+    // candidates travel in chunks of kc tensors, two chunks in flight
+    size_t kc = (size_t(512) << 20) / tensor_bytes;
+    if (kc < 1) kc = 1;
+    if (kc > (size_t)K) kc = (size_t)K;
+    if (kc > 16) kc = 16;
+    const size_t stats_bytes = ((size_t)K * sizeof(rkv_stats) + 255) / 256 * 256;
+    const size_t need = tensor_bytes * (1 + 2 * kc) + stats_bytes;
+    rc = ensure(&c.staging, &c.staging_bytes, need);
+    if (rc != RKV_OK) return rc;
+    for (int i = 0; i < 2; ++i) {
+        if (!c.copy_stream[i] &&
+            (cudaStreamCreateWithFlags(&c.copy_stream[i], cudaStreamNonBlocking) != cudaSuccess ||
+             cudaEventCreateWithFlags(&c.copied[i], cudaEventDisableTiming) != cudaSuccess ||
+             cudaEventCreateWithFlags(&c.consumed[i], cudaEventDisableTiming) != cudaSuccess)) {
+            cudaGetLastError();
+            return RKV_ERR_CUDA;
+        }
+    }
+    unsigned char* base = reinterpret_cast<unsigned char*>(c.staging);
+    unsigned char* d_ref = base;
+    unsigned char* d_chunk[2] = {base + tensor_bytes, base + tensor_bytes * (1 + kc)};
+    rkv_stats* d_stats = reinterpret_cast<rkv_stats*>(base + tensor_bytes * (1 + 2 * kc));
+
+    // device pointers of every candidate: candidate k lives in slot k % kc of buffer (k / kc) % 2
+    std::vector<const void*> ptrs((size_t)K);
+    for (int k = 0; k < K; ++k)
+        ptrs[(size_t)k] = d_chunk[((size_t)k / kc) & 1] + ((size_t)k % kc) * tensor_bytes;
+    rkv_tensor_desc d;
+    memset(&d, 0, sizeof d);
+    d.n = n; d.ref = d_ref; d.cands = ptrs.data();
+    d.cand_dtype = dtype; d.ref_dtype = dtype;
+    d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
+    d.atol = atol; d.rtol = rtol;
+    Plan plan;
+    rc = make_plan(&d, 1, K, sms, &plan);
+    if (rc != RKV_OK) return rc;
+    rc = ensure(&c.workspace, &c.workspace_bytes, plan.total_bytes);
+    if (rc != RKV_OK) return rc;
+
+    cudaStream_t main = g_stream;
+    bool fail = false;
+    fail |= cudaMemcpyAsync(d_ref, ref_host, (size_t)n * esz, cudaMemcpyHostToDevice, main) != cudaSuccess;
+    const int n_chunks = (int)(((size_t)K + kc - 1) / kc);
+    for (int ch = 0; ch < n_chunks && !fail; ++ch) {
+        const int b = ch & 1;
+        const int k0 = ch * (int)kc;
+        const int k1 = (k0 + (int)kc) < K ? (k0 + (int)kc) : K;
+        // the buffer may be overwritten once the verification of chunk ch-2 is done
+        if (ch >= 2) fail |= cudaStreamWaitEvent(c.copy_stream[b], c.consumed[b], 0) != cudaSuccess;
+        for (int k = k0; k < k1; ++k)
+            fail |= cudaMemcpyAsync(const_cast<void*>(ptrs[(size_t)k]), cands_host[k], (size_t)n * esz,
+                                    cudaMemcpyHostToDevice, c.copy_stream[b]) != cudaSuccess;
+        fail |= cudaEventRecord(c.copied[b], c.copy_stream[b]) != cudaSuccess;
+        fail |= cudaStreamWaitEvent(main, c.copied[b], 0) != cudaSuccess;
+        if (fail) break;
+        rc = run_case(&d, 1, K, k0, k1, k1 == K, ch == 0, plan, sms, d_stats, nullptr, c.workspace, main);
+        if (rc != RKV_OK) { fail = true; break; }
+        fail |= cudaEventRecord(c.consumed[b], main) != cudaSuccess;
+    }
+    if (!fail)
+        fail |= cudaMemcpyAsync(stats_host, d_stats, (size_t)K * sizeof(rkv_stats), cudaMemcpyDeviceToHost,
+                                main) != cudaSuccess;
+    const bool sync_fail = cudaStreamSynchronize(main) != cudaSuccess;
+    cudaStreamSynchronize(c.copy_stream[0]);
+    cudaStreamSynchronize(c.copy_stream[1]);
+    if (fail || sync_fail) { cudaGetLastError(); return rc != RKV_OK ? rc : RKV_ERR_CUDA; }
+    return RKV_OK;
+}
+
+int rkv_release_cached(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int cur = 0;
+    const bool have_dev = cudaGetDevice(&cur) == cudaSuccess;
+    for (int dev = 0; dev < 64; ++dev) {
+        DeviceCache& c = g_cache[dev];
+        if (!c.workspace && !c.staging && !c.copy_stream[0]) continue;
+        cudaSetDevice(dev);
+        if (c.workspace) cudaFree(c.workspace);
+        if (c.staging) cudaFree(c.staging);
+        for (int i = 0; i < 2; ++i) {
+            if (c.copy_stream[i]) cudaStreamDestroy(c.copy_stream[i]);
+            if (c.copied[i]) cudaEventDestroy(c.copied[i]);
+            if (c.consumed[i]) cudaEventDestroy(c.consumed[i]);
+        }
+        c = DeviceCache();
+    }
+    if (have_dev) cudaSetDevice(cur);
+    cudaGetLastError();
+    return RKV_OK;
+}
+
+}  // extern "C"

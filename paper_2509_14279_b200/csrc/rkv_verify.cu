@@ -1,0 +1,693 @@
+// Fused single-pass verification kernel and its finalize kernel (sm_100a).
+//
+// Work decomposition.  Every tensor is cut into slabs (runs of at most ~12-24 K
+// elements, a multiple of 128).  A persistent thread block takes slabs round
+// robin.  For a slab it stages the reference (and the input tensor, when the
+// copy-of-input flag is wanted) in shared memory ONCE -- by a bulk asynchronous
+// copy (cp.async.bulk, completion on an mbarrier) or by regenerating it from its
+// Philox stream -- and then streams the same slab of all K candidates from HBM
+// with 128-bit read-once loads.  Candidate bytes are the only traffic that
+// scales with K; the reference costs 1/K of it.
+//
+// Per element the fast path is: one subtraction, the tolerance product and sum
+// (two separately rounded operations), a compare, a running maximum, a filter
+// for the relative-error maximum, two xor/or accumulations for the loophole
+// flags.  Anything non-finite makes the 4- or 8-element vector sum non-finite,
+// which sends that vector down the general path; a slab whose reference holds a
+// non-finite value uses the general path throughout.
+//
+// Reductions are deterministic: integer sums, lexicographic (value descending,
+// index ascending) maxima, and a fixed-order fp64 sum.  No float atomics.
+#include "rkv_internal.h"
+#include "rkv_philox.cuh"
+
+namespace rkv {
+
+namespace {
+
+constexpr int kWarps = kThreads / 32;
+constexpr uint32_t kFullMask = 0xFFFFFFFFu;
+
+// ----------------------------------------------------------------------------
+// shared-memory layout
+// ----------------------------------------------------------------------------
+constexpr int kOffMbar = 0;                               // 8 bytes
+constexpr int kOffFirst = 16;                             // scratch words
+constexpr int kOffHintE = 64;
+constexpr int kOffHintQ = kOffHintE + kHintK * 4;
+constexpr int kOffWarpPart = kOffHintQ + kHintK * 4;      // 16-aligned
+constexpr int kOffDataRaw = kOffWarpPart + kChunkK * kWarps * (int)sizeof(Partial);
+constexpr int kOffData = (kOffDataRaw + 127) / 128 * 128;
+static_assert(kOffWarpPart % 16 == 0, "warp partials must be 16-byte aligned");
+
+// ----------------------------------------------------------------------------
+// small PTX helpers
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(mbar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bulk asynchronous copy global -> this block's shared memory; bytes is a
+// multiple of 16, both addresses 16-byte aligned.  No multicast.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(mbar)
+        : "memory");
+}
+
+// 128-bit read-once load of candidate data: no L1 allocation.
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
+__device__ __forceinline__ bool bits_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
+__device__ __forceinline__ bool bits_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
+
+// Largest float strictly below q for q > 0; a negative value otherwise.  A
+// threshold taken from another thread's maximum is lowered by one step so that
+// an element whose quotient ties that maximum still gets divided.
+__device__ __forceinline__ float just_below(float q) {
+    return q > 0.0f ? __uint_as_float(__float_as_uint(q) - 1u) : -1.0f;
+}
+
+// ----------------------------------------------------------------------------
+// per-thread accumulators for one (slab, candidate)
+// ----------------------------------------------------------------------------
+struct Acc {
+    uint32_t n_over;
+    float emax; uint32_t eidx; float ethr;
+    float qmax; uint32_t qidx; float qthr;
+    double sum;
+    uint32_t cacc, pacc;
+    uint32_t n_noncomp, n_nan, n_inf, n_infmis;
+};
+
+__device__ __forceinline__ void acc_reset(Acc& a, float hint_e, float hint_q) {
+    a.n_over = 0;
+    a.emax = -1.0f; a.eidx = 0xFFFFFFFFu; a.ethr = hint_e;
+    a.qmax = -1.0f; a.qidx = 0xFFFFFFFFu; a.qthr = just_below(hint_q);
+    a.sum = 0.0;
+    a.cacc = 0; a.pacc = 0;
+    a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
+}
+
+// The comparison rule for one element, every case included.
+__device__ __forceinline__ void elem_general(Acc& a, uint32_t cb, uint32_t rb, uint32_t idx, float atol,
+                                             float rtol) {
+    if (bits_nan(cb)) a.n_nan++;
+    if (bits_inf(cb)) a.n_inf++;
+    if (bits_finite(cb) && bits_finite(rb)) {
+        const float c = __uint_as_float(cb), r = __uint_as_float(rb);
+        const float e = fabsf(__fsub_rn(c, r));
+        const float thr = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r)));
+        if (!(e <= thr)) a.n_over++;
+        if (e > a.emax) { a.emax = e; a.eidx = idx; }
+        if (r != 0.0f) {
+            const float q = __fdiv_rn(e, fabsf(r));
+            if (q > a.qmax) { a.qmax = q; a.qidx = idx; }
+        }
+        a.sum += (double)e;
+    } else if (bits_inf(cb) && cb == rb) {
+        a.n_noncomp++;
+    } else {
+        a.n_noncomp++;
+        a.n_over++;
+        if (bits_inf(cb) || bits_inf(rb)) a.n_infmis++;
+    }
+}
+
+// VEC consecutive elements, candidate bits c[] and reference bits r[] as fp32
+// patterns, idx0 the slab-local index of the first.
+template <int VEC>
+__device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const uint32_t (&r)[VEC],
+                                         uint32_t idx0, float atol, float rtol, bool general) {
+    float e[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j)
+        e[j] = fabsf(__fsub_rn(__uint_as_float(c[j]), __uint_as_float(r[j])));
+    float s;
+    if (VEC == 4) {
+        s = __fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3]));
+    } else {
+        s = __fadd_rn(__fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3])),
+                      __fadd_rn(__fadd_rn(e[4 % VEC], e[5 % VEC]), __fadd_rn(e[6 % VEC], e[7 % VEC])));
+    }
+    if (general || !(s < __int_as_float(0x7F800000))) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) elem_general(a, c[j], r[j], idx0 + j, atol, rtol);
+        a.ethr = fmaxf(a.ethr, a.emax);
+        a.qthr = fmaxf(a.qthr, a.qmax);
+        return;
+    }
+    // fast path: all 2*VEC values are finite
+    float m = e[0];
+    bool relhit = false;
+    bool rp[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        const float ar = fabsf(__uint_as_float(r[j]));
+        const float thr = __fadd_rn(atol, __fmul_rn(rtol, ar));
+        if (!(e[j] <= thr)) a.n_over++;
+        m = fmaxf(m, e[j]);
+        rp[j] = (e[j] >= __fmul_rn(a.qthr, ar)) && (ar != 0.0f);
+        relhit |= rp[j];
+    }
+    a.sum += (double)s;
+    if (m >= a.ethr) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j)
+            if (e[j] > a.emax) { a.emax = e[j]; a.eidx = idx0 + j; }
+        a.ethr = fmaxf(a.ethr, a.emax);
+    }
+    if (relhit) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            if (rp[j]) {
+                const float q = __fdiv_rn(e[j], fabsf(__uint_as_float(r[j])));
+                if (q > a.qmax) { a.qmax = q; a.qidx = idx0 + j; }
+            }
+        }
+        a.qthr = fmaxf(a.qthr, a.qmax);
+    }
+}
+
+// ----------------------------------------------------------------------------
+// warp reduction of the accumulators -> one Partial in shared memory
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ void warp_reduce_store(const Acc& a, Partial* dst, int lane) {
+    const uint32_t n_over = __reduce_add_sync(kFullMask, a.n_over);
+    const uint32_t rare = a.n_noncomp | a.n_nan | a.n_inf | a.n_infmis;
+    uint32_t n_noncomp = 0, n_nan = 0, n_inf = 0, n_infmis = 0;
+    if (__any_sync(kFullMask, rare != 0)) {
+        n_noncomp = __reduce_add_sync(kFullMask, a.n_noncomp);
+        n_nan = __reduce_add_sync(kFullMask, a.n_nan);
+        n_inf = __reduce_add_sync(kFullMask, a.n_inf);
+        n_infmis = __reduce_add_sync(kFullMask, a.n_infmis);
+    }
+    // non-negative floats (and the -1 sentinel) order like their bit patterns as signed ints
+    const int eb = __float_as_int(a.emax);
+    const int ebm = __reduce_max_sync(kFullMask, eb);
+    const uint32_t eidx = __reduce_min_sync(kFullMask, eb == ebm ? a.eidx : 0xFFFFFFFFu);
+    const int qb = __float_as_int(a.qmax);
+    const int qbm = __reduce_max_sync(kFullMask, qb);
+    const uint32_t qidx = __reduce_min_sync(kFullMask, qb == qbm ? a.qidx : 0xFFFFFFFFu);
+    const uint32_t cacc = __reduce_or_sync(kFullMask, a.cacc);
+    const uint32_t pacc = __reduce_or_sync(kFullMask, a.pacc);
+    double sum = a.sum;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFullMask, sum, off);
+    if (lane == 0) {
+        Partial p;
+        p.n_over = n_over; p.n_noncomp = n_noncomp; p.n_nan = n_nan; p.n_inf = n_inf;
+        p.n_infmis = n_infmis;
+        p.mismatch = (cacc ? 1u : 0u) | (pacc ? 2u : 0u);
+        p.emax = __int_as_float(ebm); p.eidx = eidx;
+        p.qmax = __int_as_float(qbm); p.qidx = qidx;
+        p.sum = sum;
+        *dst = p;
+    }
+}
+
+__device__ __forceinline__ void partial_merge(Partial& a, const Partial& b) {
+    a.n_over += b.n_over; a.n_noncomp += b.n_noncomp; a.n_nan += b.n_nan; a.n_inf += b.n_inf;
+    a.n_infmis += b.n_infmis; a.mismatch |= b.mismatch;
+    if (b.emax > a.emax || (b.emax == a.emax && b.eidx < a.eidx)) { a.emax = b.emax; a.eidx = b.eidx; }
+    if (b.qmax > a.qmax || (b.qmax == a.qmax && b.qidx < a.qidx)) { a.qmax = b.qmax; a.qidx = b.qidx; }
+    a.sum += b.sum;
+}
+
+// ----------------------------------------------------------------------------
+// staging of the reference / input slab
+// ----------------------------------------------------------------------------
+
+// Generate `len` elements starting at tensor element `start` (a multiple of 4)
+// into shared memory, as fp32 bit patterns or as bf16 bit patterns.
+template <bool OUT_BF16, bool ROUND_BF16>
+__device__ __forceinline__ void stage_generated(unsigned char* dst, uint64_t seed, uint64_t stream_id,
+                                                int dist, uint64_t start, uint32_t len, int tid) {
+    const PhiloxKey key = philox_key(seed);
+    const uint32_t n_blocks = (len + 3u) >> 2;
+    for (uint32_t b = tid; b < n_blocks; b += kThreads) {
+        float v[4];
+        gen_block_dyn(dist, (start >> 2) + b, stream_id, key, v);
+        if (OUT_BF16) {
+            uint2 w;
+            w.x = bf16_rne_bits(v[0]) | (bf16_rne_bits(v[1]) << 16);
+            w.y = bf16_rne_bits(v[2]) | (bf16_rne_bits(v[3]) << 16);
+            *reinterpret_cast<uint2*>(dst + (size_t)b * 8) = w;
+        } else {
+            uint4 w;
+            w.x = __float_as_uint(v[0]); w.y = __float_as_uint(v[1]);
+            w.z = __float_as_uint(v[2]); w.w = __float_as_uint(v[3]);
+            if (ROUND_BF16) {
+                w.x = bf16_rne_bits(v[0]) << 16; w.y = bf16_rne_bits(v[1]) << 16;
+                w.z = bf16_rne_bits(v[2]) << 16; w.w = bf16_rne_bits(v[3]) << 16;
+            }
+            *reinterpret_cast<uint4*>(dst + (size_t)b * 16) = w;
+        }
+    }
+}
+
+// Element 0 of a tensor as an fp32 bit pattern (upcast), from memory or generated.
+__device__ __forceinline__ uint32_t first_elem_bits(const void* ptr, int src, int dtype, uint64_t seed,
+                                                    uint64_t stream_id, int dist) {
+    if (src == RKV_SRC_POINTER) {
+        if (dtype == RKV_BF16) return (uint32_t)(*reinterpret_cast<const uint16_t*>(ptr)) << 16;
+        return *reinterpret_cast<const uint32_t*>(ptr);
+    }
+    const PhiloxKey key = philox_key(seed);
+    float v[4];
+    gen_block_dyn(dist, 0, stream_id, key, v);
+    if (dtype == RKV_BF16) return bf16_rne_bits(v[0]) << 16;
+    return __float_as_uint(v[0]);
+}
+
+template <bool B16>
+__device__ __forceinline__ uint32_t smem_elem_bits(const unsigned char* base, uint32_t i) {
+    if (B16) return (uint32_t)reinterpret_cast<const uint16_t*>(base)[i] << 16;
+    return reinterpret_cast<const uint32_t*>(base)[i];
+}
+
+// ----------------------------------------------------------------------------
+// one slab, all candidates
+//   CB16   candidates (and the staged input) are bf16
+//   RB16   the staged reference is bf16 (only a bf16 reference read from memory)
+//   HAS_IN an input tensor is staged and the copy flag computed
+// ----------------------------------------------------------------------------
+template <bool CB16, bool RB16, bool HAS_IN>
+__device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, int K, int k_begin, int k_end,
+                                             Partial* __restrict__ partials, unsigned char* smem,
+                                             uint32_t& phase, int32_t* status) {
+    constexpr int VEC = CB16 ? 8 : 4;
+    constexpr int CSZ = CB16 ? 2 : 4;
+    constexpr int RSZ = RB16 ? 2 : 4;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t S = D.slab_elems;
+    const uint32_t slab = item - D.first_item;
+    const uint64_t start = (uint64_t)slab * S;
+    const uint32_t len = (uint32_t)((D.n - start) < (uint64_t)S ? (D.n - start) : (uint64_t)S);
+    const float atol = D.atol, rtol = D.rtol;
+
+    unsigned char* ref_s = smem + kOffData;
+    unsigned char* in_s = ref_s + (((size_t)S * RSZ + 127) & ~(size_t)127);
+    const uint32_t mbar = smem_u32(smem + kOffMbar);
+    float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
+    float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
+    Partial* warp_part = reinterpret_cast<Partial*>(smem + kOffWarpPart);
+
+    // ---- stage reference and input -------------------------------------------------
+    uint32_t bulk_total = 0;
+    const uint32_t ref_bulk = (D.ref_src == RKV_SRC_POINTER) ? (len * RSZ) & ~15u : 0u;
+    const uint32_t in_bulk = (HAS_IN && D.input_src == RKV_SRC_POINTER) ? (len * CSZ) & ~15u : 0u;
+    bulk_total = ref_bulk + in_bulk;
+    if (tid == 0 && bulk_total) {
+        mbar_expect_tx(mbar, bulk_total);
+        const unsigned char* g = reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ;
+        for (uint32_t off = 0; off < ref_bulk; off += 32768u) {
+            const uint32_t bytes = (ref_bulk - off) < 32768u ? (ref_bulk - off) : 32768u;
+            bulk_g2s(smem_u32(ref_s + off), g + off, bytes, mbar);
+        }
+        if (in_bulk) {
+            const unsigned char* gi = reinterpret_cast<const unsigned char*>(D.input) + start * CSZ;
+            for (uint32_t off = 0; off < in_bulk; off += 32768u) {
+                const uint32_t bytes = (in_bulk - off) < 32768u ? (in_bulk - off) : 32768u;
+                bulk_g2s(smem_u32(in_s + off), gi + off, bytes, mbar);
+            }
+        }
+    }
+    if (D.ref_src == RKV_SRC_POINTER) {
+        // the last (< 16) bytes of a ragged slab come by plain loads
+        for (uint32_t i = ref_bulk / RSZ + tid; i < len; i += kThreads) {
+            if (RB16)
+                reinterpret_cast<uint16_t*>(ref_s)[i] =
+                    reinterpret_cast<const uint16_t*>(D.ref)[start + i];
+            else
+                reinterpret_cast<uint32_t*>(ref_s)[i] =
+                    reinterpret_cast<const uint32_t*>(D.ref)[start + i];
+        }
+    } else {
+        if (D.ref_dtype == RKV_BF16)
+            stage_generated<false, true>(ref_s, D.ref_seed, D.ref_stream, D.ref_dist, start, len, tid);
+        else
+            stage_generated<false, false>(ref_s, D.ref_seed, D.ref_stream, D.ref_dist, start, len, tid);
+    }
+    if (HAS_IN) {
+        if (D.input_src == RKV_SRC_POINTER) {
+            for (uint32_t i = in_bulk / CSZ + tid; i < len; i += kThreads) {
+                if (CB16)
+                    reinterpret_cast<uint16_t*>(in_s)[i] =
+                        reinterpret_cast<const uint16_t*>(D.input)[start + i];
+                else
+                    reinterpret_cast<uint32_t*>(in_s)[i] =
+                        reinterpret_cast<const uint32_t*>(D.input)[start + i];
+            }
+        } else {
+            stage_generated<CB16, false>(in_s, D.in_seed, D.in_stream, D.in_dist, start, len, tid);
+        }
+    }
+    bool waited_ok = true;
+    if (bulk_total) {
+        waited_ok = false;
+        const long long t0 = clock64();
+        for (uint32_t spin = 0; spin < (1u << 24); ++spin) {
+            if (mbar_try_wait(mbar, phase)) { waited_ok = true; break; }
+            if (clock64() - t0 > 2000000000LL) break;      // about a second
+        }
+        phase ^= 1u;
+    }
+    if (__syncthreads_or(!waited_ok)) {
+        if (tid == 0) atomicExch(status, (int32_t)RKV_ERR_TIMEOUT);
+        return false;
+    }
+
+    // ---- scan the staged slab: non-finite reference values, reference flags ---------
+    const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed, D.ref_stream,
+                                             D.ref_dist);
+    uint32_t r_nonfinite = 0, r_cacc = 0, r_pacc = 0;
+    for (uint32_t i = tid; i < len; i += kThreads) {
+        const uint32_t rb = smem_elem_bits<RB16>(ref_s, i);
+        r_nonfinite |= bits_finite(rb) ? 0u : 1u;
+        r_cacc |= rb ^ r_first;
+        if (HAS_IN) r_pacc |= rb ^ smem_elem_bits<CB16>(in_s, i);
+    }
+    // __syncthreads_or is a boolean any(), one call per flag
+    const bool general = __syncthreads_or((int)r_nonfinite) != 0;
+    const bool ref_differs_first = __syncthreads_or(r_cacc != 0u) != 0;
+    const bool ref_differs_input = HAS_IN ? (__syncthreads_or(r_pacc != 0u) != 0) : false;
+    if (tid == 0 && k_begin == 0) {
+        Partial p = {};
+        p.mismatch = (ref_differs_first ? 1u : 0u) | (ref_differs_input ? 2u : 0u);
+        p.emax = -1.0f; p.qmax = -1.0f; p.eidx = 0xFFFFFFFFu; p.qidx = 0xFFFFFFFFu;
+        partials[(size_t)item * (K + 1) + K] = p;
+    }
+
+    // ---- stream the candidates -------------------------------------------------------
+    const uint32_t nvec = len / VEC;
+    const uint32_t tail0 = nvec * VEC;
+    constexpr int U = CB16 ? 2 : 4;                         // 16-byte loads in flight per thread
+    for (int kc0 = k_begin; kc0 < k_end; kc0 += kChunkK) {
+        const int kc1 = (kc0 + kChunkK) < k_end ? (kc0 + kChunkK) : k_end;
+        for (int k = kc0; k < kc1; ++k) {
+            const unsigned char* cp = reinterpret_cast<const unsigned char*>(D.cands[k]);
+            uint32_t c_first;
+            if (CB16) {
+                c_first = *reinterpret_cast<const uint16_t*>(cp);
+                c_first |= c_first << 16;
+            } else {
+                c_first = *reinterpret_cast<const uint32_t*>(cp);
+            }
+            cp += start * CSZ;
+            Acc a;
+            acc_reset(a, k < kHintK ? hint_e[k] : -1.0f, k < kHintK ? hint_q[k] : -1.0f);
+
+            for (uint32_t v0 = tid; v0 < nvec; v0 += U * kThreads) {
+                uint4 cv[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t v = v0 + u * kThreads;
+                    if (v < nvec) cv[u] = ldg_stream(cp + (size_t)v * 16);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t v = v0 + u * kThreads;
+                    if (v < nvec) {
+                        uint32_t c[VEC], r[VEC];
+                        if (!CB16) {
+                            c[0] = cv[u].x; c[1] = cv[u].y; c[2] = cv[u].z; c[3] = cv[u].w;
+                            a.cacc |= (c[0] ^ c_first) | (c[1] ^ c_first) | (c[2] ^ c_first) |
+                                      (c[3] ^ c_first);
+                            if (HAS_IN) {
+                                const uint4 iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
+                                a.pacc |= (c[0] ^ iv.x) | (c[1] ^ iv.y) | (c[2] ^ iv.z) | (c[3] ^ iv.w);
+                            }
+                            if (RB16) {
+                                const uint2 rv = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
+                                r[0] = rv.x << 16; r[1] = rv.x & 0xFFFF0000u;
+                                r[2] = rv.y << 16; r[3] = rv.y & 0xFFFF0000u;
+                            } else {
+                                const uint4 rv = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                                r[0] = rv.x; r[1] = rv.y; r[2] = rv.z; r[3] = rv.w;
+                            }
+                        } else {
+                            const uint32_t w[4] = {cv[u].x, cv[u].y, cv[u].z, cv[u].w};
+                            a.cacc |= (w[0] ^ c_first) | (w[1] ^ c_first) | (w[2] ^ c_first) |
+                                      (w[3] ^ c_first);
+                            if (HAS_IN) {
+                                const uint4 iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
+                                a.pacc |= (w[0] ^ iv.x) | (w[1] ^ iv.y) | (w[2] ^ iv.z) | (w[3] ^ iv.w);
+                            }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                c[2 * q] = w[q] << 16;
+                                c[2 * q + 1] = w[q] & 0xFFFF0000u;
+                            }
+                            if (RB16) {
+                                const uint4 rv = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                                const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    r[2 * q] = rw[q] << 16;
+                                    r[2 * q + 1] = rw[q] & 0xFFFF0000u;
+                                }
+                            } else {
+                                const uint4 r0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
+                                const uint4 r1 =
+                                    *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
+                                r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
+                                r[4 % VEC] = r1.x; r[5 % VEC] = r1.y; r[6 % VEC] = r1.z; r[7 % VEC] = r1.w;
+                            }
+                        }
+                        step_vec<VEC>(a, c, r, v * VEC, atol, rtol, general);
+                    }
+                }
+            }
+            // ragged end of the tensor: fewer than VEC elements, one thread, element by element
+            if (tid == 0) {
+                for (uint32_t i = tail0; i < len; ++i) {
+                    uint32_t cb;
+                    if (CB16) cb = (uint32_t)reinterpret_cast<const uint16_t*>(cp)[i] << 16;
+                    else cb = reinterpret_cast<const uint32_t*>(cp)[i];
+                    const uint32_t cf = CB16 ? (c_first << 16) : c_first;
+                    a.cacc |= cb ^ cf;
+                    if (HAS_IN) a.pacc |= cb ^ smem_elem_bits<CB16>(in_s, i);
+                    elem_general(a, cb, smem_elem_bits<RB16>(ref_s, i), i, atol, rtol);
+                }
+            }
+            warp_reduce_store(a, &warp_part[(k - kc0) * kWarps + warp], lane);
+        }
+        __syncthreads();
+        if (tid < kc1 - kc0) {
+            const int k = kc0 + tid;
+            Partial p = warp_part[tid * kWarps];
+#pragma unroll
+            for (int w = 1; w < kWarps; ++w) partial_merge(p, warp_part[tid * kWarps + w]);
+            partials[(size_t)item * (K + 1) + k] = p;
+            if (k < kHintK) {
+                hint_e[k] = fmaxf(hint_e[k], p.emax);
+                hint_q[k] = fmaxf(hint_q[k], p.qmax);
+            }
+        }
+        __syncthreads();
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
+verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end,
+              uint32_t total_items, Partial* __restrict__ partials, int32_t* status) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        mbar_init(smem_u32(smem + kOffMbar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t phase = 0;
+    int cur_t = -1;
+    for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x) {
+        int t = 0;
+        while (t + 1 < T && item >= tensors[t + 1].first_item) ++t;
+        const DevTensor D = tensors[t];
+        if (t != cur_t) {
+            // thresholds carried from earlier slabs are per tensor
+            float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
+            float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
+            for (int i = tid; i < kHintK; i += kThreads) { hint_e[i] = -1.0f; hint_q[i] = -1.0f; }
+            cur_t = t;
+        }
+        const bool cb16 = D.cand_dtype == RKV_BF16;
+        const bool rb16 = D.ref_dtype == RKV_BF16 && D.ref_src == RKV_SRC_POINTER;
+        const bool has_in = D.input_src != RKV_SRC_NONE;
+        bool ok;
+        if (!cb16) {
+            if (!rb16) ok = has_in ? process_item<false, false, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
+                                   : process_item<false, false, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
+            else       ok = has_in ? process_item<false, true, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
+                                   : process_item<false, true, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
+        } else {
+            if (!rb16) ok = has_in ? process_item<true, false, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
+                                   : process_item<true, false, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
+            else       ok = has_in ? process_item<true, true, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
+                                   : process_item<true, true, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
+        }
+        if (!ok) return;
+    }
+}
+
+// ----------------------------------------------------------------------------
+// finalize: merge the per-slab partials of each (candidate, tensor) in a fixed
+// order, derive flags and verdict, and the joint verdict over tensors
+// ----------------------------------------------------------------------------
+constexpr int kFinThreads = 128;
+
+struct Wide {
+    uint64_t n_over, n_noncomp, n_nan, n_inf, n_infmis;
+    uint64_t eidx, qidx;
+    double sum;
+    float emax, qmax;
+    uint32_t mismatch;
+};
+
+__device__ __forceinline__ void wide_merge(Wide& a, const Wide& b) {
+    a.n_over += b.n_over; a.n_noncomp += b.n_noncomp; a.n_nan += b.n_nan; a.n_inf += b.n_inf;
+    a.n_infmis += b.n_infmis; a.mismatch |= b.mismatch;
+    if (b.emax > a.emax || (b.emax == a.emax && b.eidx < a.eidx)) { a.emax = b.emax; a.eidx = b.eidx; }
+    if (b.qmax > a.qmax || (b.qmax == a.qmax && b.qidx < a.qidx)) { a.qmax = b.qmax; a.qidx = b.qidx; }
+    a.sum += b.sum;
+}
+
+__global__ void __launch_bounds__(kFinThreads)
+finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Partial* __restrict__ partials,
+                rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ joint_pass) {
+    __shared__ Wide red[kFinThreads];
+    __shared__ uint32_t ref_mismatch_s;
+    const int k = blockIdx.x, tid = threadIdx.x;
+    uint32_t all_pass = 1;
+    for (int t = 0; t < T; ++t) {
+        const DevTensor D = tensors[t];
+        Wide w = {};
+        w.emax = -1.0f; w.qmax = -1.0f; w.eidx = RKV_NO_INDEX; w.qidx = RKV_NO_INDEX;
+        uint32_t ref_mm = 0;
+        for (uint32_t s = tid; s < D.n_slabs; s += kFinThreads) {
+            const size_t row = (size_t)(D.first_item + s) * (K + 1);
+            const Partial p = partials[row + k];
+            Wide b;
+            b.n_over = p.n_over; b.n_noncomp = p.n_noncomp; b.n_nan = p.n_nan; b.n_inf = p.n_inf;
+            b.n_infmis = p.n_infmis; b.mismatch = p.mismatch;
+            const uint64_t base = (uint64_t)s * D.slab_elems;
+            b.emax = p.emax; b.eidx = p.emax < 0.0f ? RKV_NO_INDEX : base + p.eidx;
+            b.qmax = p.qmax; b.qidx = p.qmax < 0.0f ? RKV_NO_INDEX : base + p.qidx;
+            b.sum = p.sum;
+            wide_merge(w, b);
+            ref_mm |= partials[row + K].mismatch;
+        }
+        red[tid] = w;
+        if (tid == 0) ref_mismatch_s = 0;
+        __syncthreads();
+        if (ref_mm) atomicOr(&ref_mismatch_s, ref_mm);
+        for (int off = kFinThreads / 2; off > 0; off >>= 1) {
+            if (tid < off) {
+                Wide a = red[tid];
+                wide_merge(a, red[tid + off]);
+                red[tid] = a;
+            }
+            __syncthreads();
+        }
+        if (tid == 0) {
+            const Wide r = red[0];
+            const uint32_t ref_mismatch = ref_mismatch_s;
+            rkv_stats st;
+            st.n_over_tol = r.n_over;
+            st.n_nan = r.n_nan;
+            st.n_inf = r.n_inf;
+            st.n_inf_mismatch = r.n_infmis;
+            st.n_comparable = D.n - r.n_noncomp;
+            st.argmax_abs_err = r.emax < 0.0f ? RKV_NO_INDEX : r.eidx;
+            st.argmax_rel_err = r.qmax < 0.0f ? RKV_NO_INDEX : r.qidx;
+            st.sum_abs_err = r.sum;
+            st.max_abs_err = r.emax < 0.0f ? 0.0f : r.emax;
+            st.max_rel_err = r.qmax < 0.0f ? 0.0f : r.qmax;
+            st.mean_abs_err = st.n_comparable ? (float)(r.sum / (double)st.n_comparable) : 0.0f;
+            st.reserved = 0;
+            const bool has_in = D.input_src != RKV_SRC_NONE;
+            uint32_t flags = 0;
+            if (!(r.mismatch & 1u)) flags |= RKV_FLAG_CAND_CONST;
+            if (has_in && !(r.mismatch & 2u)) flags |= RKV_FLAG_CAND_COPY_OF_INPUT;
+            if (!(ref_mismatch & 1u)) flags |= RKV_FLAG_REF_CONST;
+            if (has_in && !(ref_mismatch & 2u)) flags |= RKV_FLAG_REF_COPY_OF_INPUT;
+            if (r.n_nan) flags |= RKV_FLAG_HAS_NAN;
+            if (r.n_inf) flags |= RKV_FLAG_HAS_INF;
+            uint32_t verdict = 0;
+            if (r.n_over) verdict |= RKV_FAIL_TOL;
+            if (r.n_nan) verdict |= RKV_FAIL_NAN;
+            if (r.n_infmis) verdict |= RKV_FAIL_INF_MISMATCH;
+            if ((flags & RKV_FLAG_CAND_CONST) && !(flags & RKV_FLAG_REF_CONST) && D.n > 1)
+                verdict |= RKV_FAIL_LOOPHOLE_CONST;
+            if ((flags & RKV_FLAG_CAND_COPY_OF_INPUT) && !(flags & RKV_FLAG_REF_COPY_OF_INPUT))
+                verdict |= RKV_FAIL_LOOPHOLE_COPY;
+            st.flags = flags;
+            st.verdict = verdict;
+            stats_out[(size_t)k * T + t] = st;
+            if (verdict) all_pass = 0;
+        }
+        __syncthreads();
+    }
+    if (tid == 0 && joint_pass) joint_pass[k] = all_pass;
+}
+
+}  // namespace
+
+int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
+                  uint32_t total_items, int num_sms, Partial* partials, int32_t* status,
+                  cudaStream_t stream) {
+    const int smem = kOffData + kSmemDataBudget + 256;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RKV_ERR_CUDA;
+    if (dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+            cudaSuccess)
+            return RKV_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    uint32_t grid = (uint32_t)num_sms * kBlocksPerSm;
+    if (grid > total_items) grid = total_items;
+    verify_kernel<<<grid, kThreads, smem, stream>>>(d_tensors, T, K, k_begin, k_end, total_items,
+                                                    partials, status);
+    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+int launch_finalize(const DevTensor* d_tensors, int T, int K, const Partial* partials,
+                    rkv_stats* stats_out, uint32_t* joint_pass, cudaStream_t stream) {
+    finalize_kernel<<<K, kFinThreads, 0, stream>>>(d_tensors, T, K, partials, stats_out, joint_pass);
+    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+}  // namespace rkv

@@ -1,0 +1,175 @@
+"""CPU-only checks of the C ABI: the library loads, exports every declared
+symbol, validates arguments before touching CUDA, and plans slabs sensibly.
+No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2509_14279_b200 import binding as rkv
+from paper_2509_14279_b200 import build as rkv_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HAS_GPU = torch.cuda.is_available()
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    rkv_build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rkv_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert {"rkv_gen_inputs", "rkv_verify_batch", "rkv_verify_multi", "rkv_workspace_bytes",
+            "rkv_gen_inputs_ex", "rkv_verify_batch_host", "rkv_plan_slabs"} <= set(names)
+    L = ctypes.CDLL(rkv.LIB_PATH)
+    for name in names:
+        assert hasattr(L, name), name
+
+
+def test_version_and_status_strings():
+    assert rkv.version() >= 100
+    seen = set()
+    for code in range(0, -7, -1):
+        s = rkv.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 7
+    assert rkv.status_string(-99) == "unknown status"
+
+
+def test_stats_struct_is_88_bytes():
+    text = open(os.path.join(ROOT, "include", "rkv.h")).read()
+    assert "88 bytes" in text
+    assert rkv.STATS_BYTES == 88
+    assert ctypes.sizeof(rkv.TensorDescC) == 8 * 4 + 24 * 2 + 4 * 4 + 8
+
+
+@pytest.mark.parametrize("bpe", [2, 4, 6, 8])
+@pytest.mark.parametrize("n", [1, 127, 128, 129, 4096, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
+def test_slab_plan_properties(n, bpe):
+    S, cnt = rkv.plan_slabs(n, bpe, 148)
+    assert S % 128 == 0 and S >= 128
+    assert S * bpe <= 96 * 1024
+    assert (cnt - 1) * S < n <= cnt * S
+    grid = 148 * 2
+    if n >= grid * 128 * 4:
+        waves = -(-cnt // grid)
+        assert cnt / (waves * grid) > 0.97          # no wave is mostly empty
+    if n <= 128:
+        assert cnt == 1
+
+
+def test_slab_plan_rejects_bad_arguments():
+    for args in [(0, 4, 148), (1000, 1, 148), (1000, 9, 148), (1000, 4, 0)]:
+        with pytest.raises(rkv.RkvError) as e:
+            rkv.plan_slabs(*args)
+        assert e.value.status == rkv.ERR_INVALID_ARG
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.plan_slabs(1 << 40, 4, 148)
+    assert e.value.status == rkv.ERR_UNSUPPORTED
+
+
+def _desc(n=1024, ref=0x1000, cand=0x2000, K=1, atol=1e-5, rtol=1e-5, cand_dtype=0, ref_dtype=0,
+          ref_src=1, input_src=0, inp=0, ref_dist=0):
+    d = rkv.TensorDescC()
+    d.n = n
+    d.ref = ref
+    d.input = inp
+    ptrs = (ctypes.c_void_p * K)(*[cand + 0x100000 * k for k in range(K)])
+    d.cands = ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p))
+    d.cand_dtype, d.ref_dtype, d.ref_src, d.input_src = cand_dtype, ref_dtype, ref_src, input_src
+    d.ref_gen = rkv.GenSpec(0, 0, ref_dist, 0)
+    d.atol, d.rtol = atol, rtol
+    return d, ptrs
+
+
+def _call_multi(d, K=1, stats=0x3000, ws=0x4000, ws_bytes=1 << 30):
+    arr = (rkv.TensorDescC * 1)(d)
+    return rkv.lib().rkv_verify_multi(arr, 1, K, ctypes.c_void_p(stats), None, ctypes.c_void_p(ws),
+                                      ws_bytes, None)
+
+
+def test_verify_multi_validates_before_any_cuda_call():
+    bad = [
+        (dict(n=0), rkv.ERR_INVALID_ARG),
+        (dict(n=1 << 40), rkv.ERR_UNSUPPORTED),
+        (dict(ref=0), rkv.ERR_INVALID_ARG),
+        (dict(ref=0x1004), rkv.ERR_ALIGNMENT),
+        (dict(cand=0x2008), rkv.ERR_ALIGNMENT),
+        (dict(cand=0), rkv.ERR_INVALID_ARG),
+        (dict(atol=float("nan")), rkv.ERR_INVALID_ARG),
+        (dict(rtol=float("inf")), rkv.ERR_INVALID_ARG),
+        (dict(atol=-1e-5), rkv.ERR_INVALID_ARG),
+        (dict(cand_dtype=2), rkv.ERR_INVALID_ARG),
+        (dict(ref_dtype=-1), rkv.ERR_INVALID_ARG),
+        (dict(ref_src=0), rkv.ERR_INVALID_ARG),
+        (dict(ref_src=2, ref_dist=9), rkv.ERR_INVALID_ARG),
+        (dict(input_src=1, inp=0), rkv.ERR_INVALID_ARG),
+        (dict(input_src=1, inp=0x5002), rkv.ERR_ALIGNMENT),
+        (dict(input_src=3), rkv.ERR_INVALID_ARG),
+    ]
+    for kw, want in bad:
+        d, keep = _desc(**kw)
+        assert _call_multi(d) == want, kw
+    d, keep = _desc()
+    assert _call_multi(d, K=0) == rkv.ERR_INVALID_ARG
+    assert _call_multi(d, stats=0) == rkv.ERR_INVALID_ARG
+    assert _call_multi(d, ws=0) == rkv.ERR_WORKSPACE
+    assert _call_multi(d, ws=0x4010) == rkv.ERR_ALIGNMENT
+    arr = (rkv.TensorDescC * 1)(d)
+    assert rkv.lib().rkv_verify_multi(arr, 65, 1, ctypes.c_void_p(0x3000), None,
+                                      ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_UNSUPPORTED
+    assert rkv.lib().rkv_verify_multi(None, 1, 1, ctypes.c_void_p(0x3000), None,
+                                      ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_INVALID_ARG
+
+
+def test_gen_and_batch_validate_before_any_cuda_call():
+    L = rkv.lib()
+    assert L.rkv_gen_inputs_ex(0, 0, 0, 16, 0, 0, None, None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs_ex(0, 0, 5, 16, 0, 0, ctypes.c_void_p(0x1000), None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs_ex(0, 0, 0, 0, 0, 0, ctypes.c_void_p(0x1000), None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs_ex(0, 0, 0, 16, 3, 0, ctypes.c_void_p(0x1000), None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs_ex(0, 0, 0, 16, 0, 3, ctypes.c_void_p(0x1000), None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs_ex(0, 0, 0, 16, 0, 0, ctypes.c_void_p(0x1008), None) == rkv.ERR_ALIGNMENT
+    shape = (ctypes.c_int64 * 2)(4, 0)
+    assert L.rkv_gen_inputs(0, 0, shape, 2, 0, ctypes.c_void_p(0x1000)) == rkv.ERR_INVALID_ARG
+    assert L.rkv_gen_inputs(0, 0, None, 2, 0, ctypes.c_void_p(0x1000)) == rkv.ERR_INVALID_ARG
+    ptrs = (ctypes.c_void_p * 2)(0x2000, 0x3000)
+    assert L.rkv_verify_batch(None, ptrs, 2, 16, 0, 1e-5, 1e-5, ctypes.c_void_p(0x9000)) == rkv.ERR_INVALID_ARG
+    assert L.rkv_verify_batch(ctypes.c_void_p(0x1000), ptrs, 2, 16, 0, 1e-5, 1e-5, None) == rkv.ERR_INVALID_ARG
+    assert L.rkv_verify_batch(ctypes.c_void_p(0x1000), ptrs, 0, 16, 0, 1e-5, 1e-5,
+                              ctypes.c_void_p(0x9000)) == rkv.ERR_INVALID_ARG
+    assert L.rkv_verify_batch_host(None, ptrs, 2, 16, 0, 1e-5, 1e-5, ctypes.c_void_p(0x9000)) == rkv.ERR_INVALID_ARG
+    assert L.rkv_device_status(None, None) == rkv.ERR_INVALID_ARG
+
+
+@pytest.mark.skipif(HAS_GPU, reason="only meaningful without a device")
+def test_no_device_is_an_error_not_a_fallback():
+    d, keep = _desc()
+    assert _call_multi(d) == rkv.ERR_CUDA
+    assert rkv.lib().rkv_gen_inputs_ex(0, 0, 0, 16, 0, 0, ctypes.c_void_p(0x1000), None) == rkv.ERR_CUDA
+    arr = (rkv.TensorDescC * 1)(d)
+    assert rkv.lib().rkv_workspace_bytes(arr, 1, 1) == 0
+
+
+def test_population_plans_are_seeded_and_cover_the_kinds():
+    from paper_2509_14279_b200 import population as pop
+    a = pop.plan_mixed(64, 1 << 20, seed=1, fault_rate=0.4)
+    b = pop.plan_mixed(64, 1 << 20, seed=1, fault_rate=0.4)
+    assert a == b and a != pop.plan_mixed(64, 1 << 20, seed=2, fault_rate=0.4)
+    kinds = {c.kind for c in a}
+    assert pop.NOISE in kinds and len(kinds & set(pop.FAULT_KINDS)) >= 3
+    c3 = pop.plan_mixed(64, 1 << 20, seed=2, fault_rate=0.01, bf16=True)
+    assert any(c.kind in pop.FAULT_KINDS for c in c3)              # at least one fault is forced
+    m = pop.plan_multi(128, (1 << 20, 4096, 4096), seed=3, fault_rate=0.1)
+    assert len(m) == 128 and all(len(r) == 3 for r in m)
+    assert all(sum(c.kind in pop.FAULT_KINDS for c in r) <= 1 for r in m)

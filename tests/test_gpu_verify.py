@@ -1,0 +1,253 @@
+"""GPU parity: the verification path through the C ABI against the oracle.
+
+Bit-exact on verdicts, flags, counts, maxima and their indices; 1e-6 relative
+on the error sum and mean (see rkv_testlib.MEAN_RTOL).  The reference / input
+tensors handed to the oracle come from the oracle's own generator; the GPU
+either reads the same bytes or regenerates them with its own generator.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_14279_b200 import binding as rkv
+from paper_2509_14279_b200 import population as pop
+from rkv_testlib import (assert_stats_equal, build_case_cpu, mixed_plan, oracle_case,
+                         oracle_gen_tensor)
+
+pytestmark = pytest.mark.gpu
+
+ATOL = RTOL = 1e-5
+
+
+def run_gpu(ref_cpu, cands_cpu, atol, rtol, inp_cpu=None, gen_ref=None, gen_inp=None, ref_dtype=None):
+    dev = "cuda"
+    cands = [c.to(dev) for c in cands_cpu]
+    desc = rkv.TensorDesc(
+        n=cands[0].numel(), cands=cands, atol=atol, rtol=rtol,
+        ref=None if gen_ref else ref_cpu.to(dev),
+        input=None if (gen_inp or inp_cpu is None) else inp_cpu.to(dev),
+        ref_gen=gen_ref, input_gen=gen_inp, ref_dtype=ref_dtype)
+    stats, joint, ws = rkv.verify_multi([desc], len(cands))
+    assert rkv.device_status(ws) == rkv.OK
+    return rkv.stats_to_numpy(stats), joint.cpu().numpy()
+
+
+def check_case(ref_cpu, cands_cpu, atol, rtol, inp_cpu=None, where="", **kw):
+    got, joint = run_gpu(ref_cpu, cands_cpu, atol, rtol, inp_cpu, **kw)
+    want = oracle_case(pop.bits_numpy(ref_cpu), [pop.bits_numpy(c) for c in cands_cpu], atol, rtol,
+                       None if inp_cpu is None else pop.bits_numpy(inp_cpu))
+    for k, w in enumerate(want):
+        assert_stats_equal(got[k], w, f"{where} k={k}")
+        assert int(joint[k]) == int(w["verdict"] == 0)
+    return got, want
+
+
+def test_config1_population():
+    n = 256 * 1024
+    ref = oracle_gen_tensor(0, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(0, 2, oracle.NORMAL, n, "f32")
+    plan = pop.plan_c1(n, seed=0)
+    cands = build_case_cpu(plan, ref, inp, "f32")
+    got, want = check_case(ref, cands, ATOL, RTOL, inp, where="c1")
+    assert [int(g["verdict"]) == 0 for g in got] == [True, False, False, False, False, False, True, False]
+    assert int(got[1]["argmax_abs_err"]) == plan[1].indices[0]
+    # same case with the reference and the input regenerated on the device
+    got2, _ = run_gpu(ref, cands, ATOL, RTOL, gen_ref=(0, 0, rkv.DIST_NORMAL), gen_inp=(0, 2, rkv.DIST_NORMAL))
+    assert got2.tobytes() == got.tobytes()
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 31, 32, 33, 127, 128, 129, 4095, 4096, 4097, 50001])
+def test_small_and_ragged_sizes_fp32(n):
+    ref = oracle_gen_tensor(20 + n, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(20 + n, 2, oracle.NORMAL, n, "f32")
+    for K in (1, 2, 7, 9, 12):
+        cands = build_case_cpu(mixed_plan(K, n, seed=n + K), ref, inp, "f32")
+        check_case(ref, cands, ATOL, RTOL, inp, where=f"n={n} K={K}")
+    cands = build_case_cpu(mixed_plan(5, n, seed=n), ref, inp, "f32")
+    check_case(ref, cands, ATOL, RTOL, None, where=f"n={n} no input")
+
+
+@pytest.mark.parametrize("K", [33, 65, 300])
+def test_many_candidates_cross_the_merge_chunk_and_hint_limits(K):
+    n = 30011
+    ref = oracle_gen_tensor(3, 0, oracle.STUDENT_T2, n, "f32")
+    inp = oracle_gen_tensor(3, 2, oracle.STUDENT_T2, n, "f32")
+    cands = build_case_cpu(mixed_plan(K, n, seed=K), ref, inp, "f32")
+    check_case(ref, cands, ATOL, RTOL, inp, where=f"K={K}")
+
+
+@pytest.mark.parametrize("dist", oracle.DISTS)
+def test_every_distribution_several_slabs_per_block(dist):
+    n = 296 * 128 * 3 + 77            # three slabs per block on a 148-SM part, ragged tail
+    ref = oracle_gen_tensor(7, 0, dist, n, "f32")
+    inp = oracle_gen_tensor(7, 2, dist, n, "f32")
+    cands = build_case_cpu(mixed_plan(12, n, seed=dist), ref, inp, "f32")
+    check_case(ref, cands, ATOL, RTOL, inp, where=f"dist={dist}")
+    # fused: reference and input regenerated on the device
+    got_a, _ = run_gpu(ref, cands, ATOL, RTOL, inp)
+    got_b, _ = run_gpu(ref, cands, ATOL, RTOL, gen_ref=(7, 0, dist), gen_inp=(7, 2, dist))
+    assert got_a.tobytes() == got_b.tobytes()
+
+
+@pytest.mark.parametrize("cand_dtype,ref_dtype", [("bf16", "f32"), ("bf16", "bf16"), ("f32", "bf16")])
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 1000, 4099, 120001])
+def test_bf16_combinations(cand_dtype, ref_dtype, n):
+    ref = oracle_gen_tensor(31, 0, oracle.NORMAL, n, ref_dtype)
+    inp = oracle_gen_tensor(31, 2, oracle.NORMAL, n, cand_dtype)
+    cands = build_case_cpu(mixed_plan(12, n, seed=n, bf16=True), ref, inp, cand_dtype)
+    check_case(ref, cands, 1e-2, 1.6e-2, inp, where=f"{cand_dtype}/{ref_dtype} n={n}")
+    check_case(ref, cands[:5], 1e-2, 1.6e-2, None, where=f"{cand_dtype}/{ref_dtype} n={n} no input")
+    # generated reference rounded to ref_dtype, generated input in the candidates' dtype
+    got_a, _ = run_gpu(ref, cands, 1e-2, 1.6e-2, inp)
+    got_b, _ = run_gpu(ref, cands, 1e-2, 1.6e-2, gen_ref=(31, 0, rkv.DIST_NORMAL),
+                       gen_inp=(31, 2, rkv.DIST_NORMAL),
+                       ref_dtype=rkv.F32 if ref_dtype == "f32" else rkv.BF16)
+    assert got_a.tobytes() == got_b.tobytes()
+
+
+def test_nonfinite_everywhere():
+    n = 40000
+    ref = oracle_gen_tensor(41, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(41, 2, oracle.NORMAL, n, "f32")
+    r2 = ref.clone()
+    r2[5] = float("inf"); r2[6] = float("-inf"); r2[7] = float("nan"); r2[30000] = float("inf")
+    big = ref.clone(); big[100] = 3e38
+    cands = []
+    c = r2.clone(); cands.append(c)                                   # matches, NaN vs NaN fails
+    c = r2.clone(); c[5] = float("-inf"); cands.append(c)             # sign mismatch
+    c = ref.clone(); c[5] = 1.0; cands.append(c)                      # finite vs infinite ref
+    c = ref.clone(); c[100] = -3e38; cands.append(c)                  # finite difference overflows
+    c = ref.clone(); c[n - 1] = float("nan"); c[0] = float("inf"); cands.append(c)
+    c = torch.full((n,), float("nan")); cands.append(c)
+    c = torch.full((n,), float("inf")); cands.append(c)
+    check_case(r2, cands, ATOL, RTOL, inp, where="nonfinite ref")
+    check_case(big, cands, ATOL, RTOL, inp, where="huge ref")
+    check_case(ref, cands, ATOL, RTOL, None, where="finite ref")
+
+
+def test_ties_resolve_to_the_first_index():
+    n = 296 * 128 * 2 + 5
+    ref = torch.full((n,), 2.0)
+    ref[::3] = 4.0
+    ref[1::7] = 0.0
+    inp = oracle_gen_tensor(1, 2, oracle.UNIFORM_PM1, n, "f32")
+    cands = []
+    c = ref.clone(); c += 0.5; cands.append(c)                        # same error everywhere
+    c = ref.clone(); c[n // 2:] += 0.5; cands.append(c)               # first hit mid-tensor
+    c = ref.clone(); c[n - 1] += 0.5; c[n - 3] += 0.5; cands.append(c)
+    c = ref.clone(); c[40000] -= 1.0; c[123] += 1.0; c[124] += 1.0; cands.append(c)
+    c = ref * 1.5; cands.append(c)                                    # equal relative error
+    got, want = check_case(ref, cands, ATOL, RTOL, inp, where="ties")
+    assert int(got[0]["argmax_abs_err"]) == 0
+    assert int(got[1]["argmax_abs_err"]) == n // 2
+
+
+def test_multi_tensor_joint_verdict():
+    shapes = [70001, 4096, 4096]
+    tols = [(1e-5, 1e-5), (1e-5, 1e-5), (1e-4, 1e-5)]
+    K = 10
+    plans = pop.plan_multi(K, tuple(shapes), seed=3, fault_rate=0.4)
+    refs, inps, cands = [], [], []
+    for t, n in enumerate(shapes):
+        refs.append(oracle_gen_tensor(3, (t << 32) | 0, oracle.NORMAL, n, "f32"))
+        inps.append(oracle_gen_tensor(3, (t << 32) | 2, oracle.NORMAL, n, "f32"))
+        cands.append([pop.materialize(plans[k][t], refs[t], inps[t], "f32") for k in range(K)])
+    descs = [rkv.TensorDesc(n=n, cands=[c.cuda() for c in cands[t]], atol=tols[t][0], rtol=tols[t][1],
+                            ref=refs[t].cuda(), input=inps[t].cuda()) for t, n in enumerate(shapes)]
+    stats, joint, ws = rkv.verify_multi(descs, K)
+    got = rkv.stats_to_numpy(stats).reshape(K, len(shapes))
+    verdicts = []
+    for k in range(K):
+        row = []
+        for t in range(len(shapes)):
+            w = oracle.verify(pop.bits_numpy(refs[t]), pop.bits_numpy(cands[t][k]), tols[t][0], tols[t][1],
+                              input=pop.bits_numpy(inps[t]))
+            assert_stats_equal(got[k, t], w, f"k={k} t={t}")
+            row.append(w["verdict"])
+        verdicts.append(row)
+    assert joint.cpu().tolist() == oracle.joint_pass(verdicts)
+    assert 0 < sum(joint.cpu().tolist()) < K
+    # fused variant: references and inputs regenerated per tensor stream
+    descs_f = [rkv.TensorDesc(n=n, cands=descs[t].cands, atol=tols[t][0], rtol=tols[t][1],
+                              ref_gen=(3, (t << 32) | 0, rkv.DIST_NORMAL),
+                              input_gen=(3, (t << 32) | 2, rkv.DIST_NORMAL)) for t, n in enumerate(shapes)]
+    stats_f, joint_f, _ = rkv.verify_multi(descs_f, K)
+    assert rkv.stats_to_numpy(stats_f).tobytes() == rkv.stats_to_numpy(stats).tobytes()
+    assert torch.equal(joint, joint_f)
+
+
+def test_mixed_dtype_pair_like_the_large_sweep():
+    """Two tensors per candidate pair: an fp32 and a bf16 output of one reference."""
+    n, K = 90000, 6
+    ref = oracle_gen_tensor(10, 0, oracle.SPARSE90, n, "f32")
+    inp32 = oracle_gen_tensor(10, 2, oracle.SPARSE90, n, "f32")
+    inp16 = oracle_gen_tensor(10, 2, oracle.SPARSE90, n, "bf16")
+    c32 = build_case_cpu(mixed_plan(K, n, seed=1), ref, inp32, "f32")
+    c16 = build_case_cpu(mixed_plan(K, n, seed=2, bf16=True), ref, inp16, "bf16")
+    descs = [
+        rkv.TensorDesc(n=n, cands=[c.cuda() for c in c32], atol=1e-5, rtol=1e-5,
+                       ref_gen=(10, 0, rkv.DIST_SPARSE90), input_gen=(10, 2, rkv.DIST_SPARSE90)),
+        rkv.TensorDesc(n=n, cands=[c.cuda() for c in c16], atol=1e-2, rtol=1.6e-2,
+                       ref_gen=(10, 0, rkv.DIST_SPARSE90), input_gen=(10, 2, rkv.DIST_SPARSE90)),
+    ]
+    stats, joint, _ = rkv.verify_multi(descs, K)
+    got = rkv.stats_to_numpy(stats).reshape(K, 2)
+    for k in range(K):
+        assert_stats_equal(got[k, 0], oracle.verify(pop.bits_numpy(ref), pop.bits_numpy(c32[k]), 1e-5, 1e-5,
+                                                     input=pop.bits_numpy(inp32)), f"f32 k={k}")
+        assert_stats_equal(got[k, 1], oracle.verify(pop.bits_numpy(ref), pop.bits_numpy(c16[k]), 1e-2, 1.6e-2,
+                                                     input=pop.bits_numpy(inp16)), f"bf16 k={k}")
+
+
+def test_runs_are_deterministic():
+    n, K = 200003, 9
+    ref = oracle_gen_tensor(5, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(5, 2, oracle.NORMAL, n, "f32")
+    cands = build_case_cpu(mixed_plan(K, n, seed=5), ref, inp, "f32")
+    a, _ = run_gpu(ref, cands, ATOL, RTOL, inp)
+    for _ in range(3):
+        b, _ = run_gpu(ref, cands, ATOL, RTOL, inp)
+        assert a.tobytes() == b.tobytes()
+
+
+def test_north_star_two_call_form():
+    shape = (256, 1024)
+    ref = rkv.gen_inputs(0, rkv.DIST_NORMAL, shape)
+    n = ref.numel()
+    ref_cpu = oracle_gen_tensor(0, 0, oracle.NORMAL, n, "f32")
+    cands_cpu = build_case_cpu(mixed_plan(8, n, seed=0), ref_cpu, ref_cpu, "f32")
+    stats = rkv.verify_batch(ref, [c.cuda() for c in cands_cpu], ATOL, RTOL)
+    got = rkv.stats_to_numpy(stats)
+    want = oracle_case(pop.bits_numpy(ref_cpu), [pop.bits_numpy(c) for c in cands_cpu], ATOL, RTOL)
+    for k in range(8):
+        assert_stats_equal(got[k], want[k], f"k={k}")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_host_buffer_form(dtype):
+    n, K = 150001, 37
+    ref = oracle_gen_tensor(6, 0, oracle.NORMAL, n, dtype)
+    cands = build_case_cpu(mixed_plan(K, n, seed=6, bf16=dtype == "bf16"), ref, ref, dtype)
+    got = rkv.verify_batch_host(ref, cands, 1e-2, 1.6e-2)
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], 1e-2, 1.6e-2)
+    for k in range(K):
+        assert_stats_equal(got[k], want[k], f"host k={k}")
+
+
+def test_error_codes_on_device():
+    n = 1024
+    ref = torch.zeros(n + 4, device="cuda")
+    cand = torch.zeros(n, device="cuda")
+    d = rkv.TensorDesc(n=n, cands=[cand], atol=1e-5, rtol=1e-5, ref=ref[1:n + 1])
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.verify_multi([d], 1)
+    assert e.value.status == rkv.ERR_ALIGNMENT
+    d = rkv.TensorDesc(n=n, cands=[cand], atol=1e-5, rtol=1e-5, ref=ref[:n])
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.verify_multi([d], 1, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == rkv.ERR_WORKSPACE
+    d = rkv.TensorDesc(n=n, cands=[cand], atol=-1.0, rtol=1e-5, ref=ref[:n])
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.verify_multi([d], 1)
+    assert e.value.status == rkv.ERR_INVALID_ARG
