@@ -85,6 +85,7 @@ int validate_tensors(const rkv_tensor_desc* tensors, int T, int K) {
 
 int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* plan) {
     uint64_t items = 0;
+    for (int v = 0; v < 8; ++v) plan->variant_items[v] = 0;
     for (int t = 0; t < T; ++t) {
         uint32_t S;
         uint64_t ns;
@@ -93,6 +94,11 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* p
         plan->slab_elems[t] = S;
         plan->n_slabs[t] = (uint32_t)ns;
         plan->first_item[t] = (uint32_t)items;
+        const rkv_tensor_desc& d = tensors[t];
+        const int variant = (d.cand_dtype == RKV_BF16 ? 4 : 0) +
+                            ((d.ref_dtype == RKV_BF16 && d.ref_src == RKV_SRC_POINTER) ? 2 : 0) +
+                            (d.input_src != RKV_SRC_NONE ? 1 : 0);
+        plan->variant_items[variant] += (uint32_t)ns;
         items += ns;
         if (items > 0xFFFFFFFFull / 2) return RKV_ERR_UNSUPPORTED;
     }
@@ -183,7 +189,7 @@ int run_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k_en
             return RKV_ERR_CUDA;
         }
     }
-    int rc = launch_verify(d_tensors, T, K, k_begin, k_end, plan.total_items, num_sms, partials, status,
+    int rc = launch_verify(d_tensors, T, K, k_begin, k_end, plan.variant_items, num_sms, partials, status,
                            stream);
     if (rc != RKV_OK) return rc;
     if (finalize) rc = launch_finalize(d_tensors, T, K, partials, stats_out, joint_pass, stream);

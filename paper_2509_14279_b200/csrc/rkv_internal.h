@@ -13,7 +13,8 @@ constexpr int kThreads = 256;          // threads per verification block
 constexpr int kBlocksPerSm = 2;        // resident verification blocks per SM
 constexpr int kSlabGranule = 128;      // slab lengths are multiples of this many elements
 constexpr int kSmemDataBudget = 96 * 1024;  // bytes of reference + input one block stages
-constexpr int kChunkK = 32;            // candidates between two block-level merges
+constexpr int kChunkK = 16;            // candidates between two block-level merges
+constexpr int kPreK = 512;             // candidates whose pointer and first element are preloaded
 constexpr int kHintK = 256;            // candidates with a cross-slab threshold hint
 constexpr int kMaxTensors = 64;
 constexpr uint64_t kMaxN = 1ull << 40;
@@ -63,6 +64,7 @@ struct Plan {
     uint32_t n_slabs[kMaxTensors];
     uint32_t first_item[kMaxTensors];
     uint32_t total_items;
+    uint32_t variant_items[8];
     size_t table_bytes;     // descriptors + pointer tables, rounded to 256
     size_t partial_bytes;
     size_t total_bytes;
@@ -74,8 +76,10 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* p
 int current_num_sms(int* num_sms);   // RKV_ERR_CUDA without a device
 
 // kernels (rkv_verify.cu / rkv_gen.cu)
+// variant_items[v]: slabs of the tensors whose storage variant is v =
+// 4*(candidates bf16) + 2*(reference staged as bf16) + (input present)
 int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
-                  uint32_t total_items, int num_sms, Partial* partials, int32_t* status,
+                  const uint32_t variant_items[8], int num_sms, Partial* partials, int32_t* status,
                   cudaStream_t stream);
 int launch_finalize(const DevTensor* d_tensors, int T, int K, const Partial* partials,
                     rkv_stats* stats_out, uint32_t* joint_pass, cudaStream_t stream);

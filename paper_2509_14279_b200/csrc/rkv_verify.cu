@@ -26,17 +26,21 @@ namespace rkv {
 namespace {
 
 constexpr int kWarps = kThreads / 32;
+constexpr int kGroupK = 2;        // candidates processed per pass over a reference vector
+constexpr int kLoadsF32 = 2;      // 16-byte candidate loads per thread, candidate and batch (fp32)
+constexpr int kLoadsBf16 = 2;     // same for bf16 candidates
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 
 // ----------------------------------------------------------------------------
 // shared-memory layout
 // ----------------------------------------------------------------------------
 constexpr int kOffMbar = 0;                               // 8 bytes
-constexpr int kOffFirst = 16;                             // scratch words
 constexpr int kOffHintE = 64;
 constexpr int kOffHintQ = kOffHintE + kHintK * 4;
 constexpr int kOffWarpPart = kOffHintQ + kHintK * 4;      // 16-aligned
-constexpr int kOffDataRaw = kOffWarpPart + kChunkK * kWarps * (int)sizeof(Partial);
+constexpr int kOffCandPtr = kOffWarpPart + kChunkK * kWarps * (int)sizeof(Partial);
+constexpr int kOffCandFirst = kOffCandPtr + kPreK * 8;
+constexpr int kOffDataRaw = kOffCandFirst + kPreK * 4;
 constexpr int kOffData = (kOffDataRaw + 127) / 128 * 128;
 static_assert(kOffWarpPart % 16 == 0, "warp partials must be 16-byte aligned");
 
@@ -90,13 +94,6 @@ __device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000
 __device__ __forceinline__ bool bits_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
 __device__ __forceinline__ bool bits_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
 
-// Largest float strictly below q for q > 0; a negative value otherwise.  A
-// threshold taken from another thread's maximum is lowered by one step so that
-// an element whose quotient ties that maximum still gets divided.
-__device__ __forceinline__ float just_below(float q) {
-    return q > 0.0f ? __uint_as_float(__float_as_uint(q) - 1u) : -1.0f;
-}
-
 // ----------------------------------------------------------------------------
 // per-thread accumulators for one (slab, candidate)
 // ----------------------------------------------------------------------------
@@ -112,7 +109,7 @@ struct Acc {
 __device__ __forceinline__ void acc_reset(Acc& a, float hint_e, float hint_q) {
     a.n_over = 0;
     a.emax = -1.0f; a.eidx = 0xFFFFFFFFu; a.ethr = hint_e;
-    a.qmax = -1.0f; a.qidx = 0xFFFFFFFFu; a.qthr = just_below(hint_q);
+    a.qmax = -1.0f; a.qidx = 0xFFFFFFFFu; a.qthr = hint_q;
     a.sum = 0.0;
     a.cacc = 0; a.pacc = 0;
     a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
@@ -143,15 +140,46 @@ __device__ __forceinline__ void elem_general(Acc& a, uint32_t cb, uint32_t rb, u
     }
 }
 
-// VEC consecutive elements, candidate bits c[] and reference bits r[] as fp32
-// patterns, idx0 the slab-local index of the first.
+// Per-vector values that depend on the reference only; computed once and used
+// for every candidate of a group.
 template <int VEC>
-__device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const uint32_t (&r)[VEC],
+struct RefVec {
+    uint32_t r[VEC];      // reference bits (fp32 patterns)
+    float thr[VEC];       // atol + rtol*|r|, product and sum each rounded
+    float arp[VEC];       // |r|, or +inf where r == 0 (such elements never enter the relative maximum)
+};
+
+template <int VEC>
+__device__ __forceinline__ void refvec_prepare(RefVec<VEC>& rv, float atol, float rtol) {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        const float ar = fabsf(__uint_as_float(rv.r[j]));
+        rv.thr[j] = __fadd_rn(atol, __fmul_rn(rtol, ar));
+        rv.arp[j] = ar != 0.0f ? ar : __int_as_float(0x7F800000);
+    }
+}
+
+// VEC consecutive elements of one candidate: bits c[] against the prepared
+// reference vector; idx0 is the slab-local index of the first element.
+//
+// Fast path (all values finite).  The three per-element tests only set a
+// predicate; the work behind them runs when a predicate fired:
+//   over : !(e <= thr)                      -> recount the vector
+//   abs  : e > ethr, ethr >= running max    -> update (max, first index)
+//   rel  : e > RD(qthr * |r|)               -> divide, update (max, first index)
+// RD is the product rounded toward -inf.  If fl(e/|r|) > qthr then, rounding
+// being monotone, e/|r| > qthr exactly, so e > qthr*|r| >= RD(qthr*|r|): the
+// test never skips an element that beats qthr.  Thresholds always come from
+// elements with SMALLER indices (the thread's own earlier elements, earlier
+// batches of the block, earlier slabs), so a tie may be skipped: the first
+// index keeps the maximum.
+template <int VEC>
+__device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const RefVec<VEC>& rv,
                                          uint32_t idx0, float atol, float rtol, bool general) {
     float e[VEC];
 #pragma unroll
     for (int j = 0; j < VEC; ++j)
-        e[j] = fabsf(__fsub_rn(__uint_as_float(c[j]), __uint_as_float(r[j])));
+        e[j] = fabsf(__fsub_rn(__uint_as_float(c[j]), __uint_as_float(rv.r[j])));
     float s;
     if (VEC == 4) {
         s = __fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3]));
@@ -161,36 +189,36 @@ __device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const
     }
     if (general || !(s < __int_as_float(0x7F800000))) {
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) elem_general(a, c[j], r[j], idx0 + j, atol, rtol);
+        for (int j = 0; j < VEC; ++j) elem_general(a, c[j], rv.r[j], idx0 + j, atol, rtol);
         a.ethr = fmaxf(a.ethr, a.emax);
         a.qthr = fmaxf(a.qthr, a.qmax);
         return;
     }
-    // fast path: all 2*VEC values are finite
-    float m = e[0];
-    bool relhit = false;
-    bool rp[VEC];
+    bool over = false, absh = false, relh = false;
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-        const float ar = fabsf(__uint_as_float(r[j]));
-        const float thr = __fadd_rn(atol, __fmul_rn(rtol, ar));
-        if (!(e[j] <= thr)) a.n_over++;
-        m = fmaxf(m, e[j]);
-        rp[j] = (e[j] >= __fmul_rn(a.qthr, ar)) && (ar != 0.0f);
-        relhit |= rp[j];
+        over |= !(e[j] <= rv.thr[j]);
+        absh |= e[j] > a.ethr;
+        relh |= e[j] > __fmul_rd(a.qthr, rv.arp[j]);
     }
     a.sum += (double)s;
-    if (m >= a.ethr) {
+    if (over) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j)
+            if (!(e[j] <= rv.thr[j])) a.n_over++;
+    }
+    if (absh) {
 #pragma unroll
         for (int j = 0; j < VEC; ++j)
             if (e[j] > a.emax) { a.emax = e[j]; a.eidx = idx0 + j; }
         a.ethr = fmaxf(a.ethr, a.emax);
     }
-    if (relhit) {
+    if (relh) {
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
-            if (rp[j]) {
-                const float q = __fdiv_rn(e[j], fabsf(__uint_as_float(r[j])));
+            const float ar = fabsf(__uint_as_float(rv.r[j]));
+            if (ar != 0.0f && e[j] > __fmul_rd(a.qthr, ar)) {
+                const float q = __fdiv_rn(e[j], ar);
                 if (q > a.qmax) { a.qmax = q; a.qidx = idx0 + j; }
             }
         }
@@ -301,7 +329,7 @@ __device__ __forceinline__ uint32_t smem_elem_bits(const unsigned char* base, ui
 //   RB16   the staged reference is bf16 (only a bf16 reference read from memory)
 //   HAS_IN an input tensor is staged and the copy flag computed
 // ----------------------------------------------------------------------------
-template <bool CB16, bool RB16, bool HAS_IN>
+template <bool CB16, bool RB16, bool HAS_IN, int KB, int U>
 __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, int K, int k_begin, int k_end,
                                              Partial* __restrict__ partials, unsigned char* smem,
                                              uint32_t& phase, int32_t* status) {
@@ -409,98 +437,140 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
     }
 
     // ---- stream the candidates -------------------------------------------------------
+    // Candidates are taken KB at a time: the reference vector is read from shared
+    // memory and prepared once per KB candidate vectors.  Loads of the next batch
+    // are issued before the current batch is processed.
     const uint32_t nvec = len / VEC;
     const uint32_t tail0 = nvec * VEC;
-    constexpr int U = CB16 ? 2 : 4;                         // 16-byte loads in flight per thread
+    const uint32_t nbatch = (nvec + U * kThreads - 1) / (U * kThreads);
+    const unsigned char* const* cptr_s = reinterpret_cast<const unsigned char* const*>(smem + kOffCandPtr);
+    const uint32_t* cfirst_s = reinterpret_cast<const uint32_t*>(smem + kOffCandFirst);
     for (int kc0 = k_begin; kc0 < k_end; kc0 += kChunkK) {
         const int kc1 = (kc0 + kChunkK) < k_end ? (kc0 + kChunkK) : k_end;
-        for (int k = kc0; k < kc1; ++k) {
-            const unsigned char* cp = reinterpret_cast<const unsigned char*>(D.cands[k]);
-            uint32_t c_first;
-            if (CB16) {
-                c_first = *reinterpret_cast<const uint16_t*>(cp);
-                c_first |= c_first << 16;
-            } else {
-                c_first = *reinterpret_cast<const uint32_t*>(cp);
+        for (int kg = kc0; kg < kc1; kg += KB) {
+            const unsigned char* cp[KB];
+            uint32_t c_first[KB];
+            Acc a[KB];
+#pragma unroll
+            for (int i = 0; i < KB; ++i) {
+                // a group that runs past the chunk repeats its last candidate (result dropped)
+                const int k = (kg + i) < kc1 ? (kg + i) : (kc1 - 1);
+                if (k < kPreK) {
+                    cp[i] = cptr_s[k];
+                    c_first[i] = cfirst_s[k];
+                } else {
+                    cp[i] = reinterpret_cast<const unsigned char*>(D.cands[k]);
+                    c_first[i] = CB16 ? (uint32_t)(*reinterpret_cast<const uint16_t*>(cp[i]))
+                                      : *reinterpret_cast<const uint32_t*>(cp[i]);
+                }
+                if (CB16) c_first[i] = (c_first[i] & 0xFFFFu) * 0x10001u;
+                cp[i] += start * CSZ;
+                acc_reset(a[i], k < kHintK ? hint_e[k] : -1.0f, k < kHintK ? hint_q[k] : -1.0f);
             }
-            cp += start * CSZ;
-            Acc a;
-            acc_reset(a, k < kHintK ? hint_e[k] : -1.0f, k < kHintK ? hint_q[k] : -1.0f);
 
-            for (uint32_t v0 = tid; v0 < nvec; v0 += U * kThreads) {
-                uint4 cv[U];
+            uint4 cur[KB][U], nxt[KB][U];
+#pragma unroll
+            for (int i = 0; i < KB; ++i)
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const uint32_t v = v0 + u * kThreads;
-                    if (v < nvec) cv[u] = ldg_stream(cp + (size_t)v * 16);
+                    const uint32_t v = u * kThreads + tid;
+                    if (v < nvec) cur[i][u] = ldg_stream(cp[i] + (size_t)v * 16);
+                }
+            for (uint32_t b = 0; b < nbatch; ++b) {
+                const uint32_t vb = b * U * kThreads + tid;
+                if (b + 1 < nbatch) {
+#pragma unroll
+                    for (int i = 0; i < KB; ++i)
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            const uint32_t v = vb + (U + u) * kThreads;
+                            if (v < nvec) nxt[i][u] = ldg_stream(cp[i] + (size_t)v * 16);
+                        }
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const uint32_t v = v0 + u * kThreads;
+                    const uint32_t v = vb + u * kThreads;
                     if (v < nvec) {
-                        uint32_t c[VEC], r[VEC];
+                        RefVec<VEC> rv;
+                        uint4 iv = make_uint4(0, 0, 0, 0);
+                        if (HAS_IN) iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
                         if (!CB16) {
-                            c[0] = cv[u].x; c[1] = cv[u].y; c[2] = cv[u].z; c[3] = cv[u].w;
-                            a.cacc |= (c[0] ^ c_first) | (c[1] ^ c_first) | (c[2] ^ c_first) |
-                                      (c[3] ^ c_first);
-                            if (HAS_IN) {
-                                const uint4 iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
-                                a.pacc |= (c[0] ^ iv.x) | (c[1] ^ iv.y) | (c[2] ^ iv.z) | (c[3] ^ iv.w);
-                            }
                             if (RB16) {
-                                const uint2 rv = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
-                                r[0] = rv.x << 16; r[1] = rv.x & 0xFFFF0000u;
-                                r[2] = rv.y << 16; r[3] = rv.y & 0xFFFF0000u;
+                                const uint2 t = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
+                                rv.r[0] = t.x << 16; rv.r[1] = t.x & 0xFFFF0000u;
+                                rv.r[2] = t.y << 16; rv.r[3] = t.y & 0xFFFF0000u;
                             } else {
-                                const uint4 rv = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                                r[0] = rv.x; r[1] = rv.y; r[2] = rv.z; r[3] = rv.w;
+                                const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                                rv.r[0] = t.x; rv.r[1] = t.y; rv.r[2] = t.z; rv.r[3] = t.w;
                             }
                         } else {
-                            const uint32_t w[4] = {cv[u].x, cv[u].y, cv[u].z, cv[u].w};
-                            a.cacc |= (w[0] ^ c_first) | (w[1] ^ c_first) | (w[2] ^ c_first) |
-                                      (w[3] ^ c_first);
-                            if (HAS_IN) {
-                                const uint4 iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
-                                a.pacc |= (w[0] ^ iv.x) | (w[1] ^ iv.y) | (w[2] ^ iv.z) | (w[3] ^ iv.w);
-                            }
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                c[2 * q] = w[q] << 16;
-                                c[2 * q + 1] = w[q] & 0xFFFF0000u;
-                            }
                             if (RB16) {
-                                const uint4 rv = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                                const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
+                                const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                                const uint32_t rw[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
                                 for (int q = 0; q < 4; ++q) {
-                                    r[2 * q] = rw[q] << 16;
-                                    r[2 * q + 1] = rw[q] & 0xFFFF0000u;
+                                    rv.r[(2 * q) % VEC] = rw[q] << 16;
+                                    rv.r[(2 * q + 1) % VEC] = rw[q] & 0xFFFF0000u;
                                 }
                             } else {
-                                const uint4 r0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
-                                const uint4 r1 =
-                                    *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
-                                r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
-                                r[4 % VEC] = r1.x; r[5 % VEC] = r1.y; r[6 % VEC] = r1.z; r[7 % VEC] = r1.w;
+                                const uint4 t0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
+                                const uint4 t1 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
+                                rv.r[0] = t0.x; rv.r[1] = t0.y; rv.r[2] = t0.z; rv.r[3] = t0.w;
+                                rv.r[4 % VEC] = t1.x; rv.r[5 % VEC] = t1.y;
+                                rv.r[6 % VEC] = t1.z; rv.r[7 % VEC] = t1.w;
                             }
                         }
-                        step_vec<VEC>(a, c, r, v * VEC, atol, rtol, general);
+                        refvec_prepare<VEC>(rv, atol, rtol);
+#pragma unroll
+                        for (int i = 0; i < KB; ++i) {
+                            const uint32_t w[4] = {cur[i][u].x, cur[i][u].y, cur[i][u].z, cur[i][u].w};
+                            a[i].cacc |= (w[0] ^ c_first[i]) | (w[1] ^ c_first[i]) | (w[2] ^ c_first[i]) |
+                                         (w[3] ^ c_first[i]);
+                            if (HAS_IN) a[i].pacc |= (w[0] ^ iv.x) | (w[1] ^ iv.y) | (w[2] ^ iv.z) | (w[3] ^ iv.w);
+                            uint32_t c[VEC];
+                            if (!CB16) {
+                                c[0] = w[0]; c[1] = w[1]; c[2] = w[2]; c[3] = w[3];
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    c[(2 * q) % VEC] = w[q] << 16;
+                                    c[(2 * q + 1) % VEC] = w[q] & 0xFFFF0000u;
+                                }
+                            }
+                            step_vec<VEC>(a[i], c, rv, v * VEC, atol, rtol, general);
+                        }
                     }
                 }
+                // share the running maxima across the warp: every element of this batch has
+                // a smaller index than every element of the next one
+#pragma unroll
+                for (int i = 0; i < KB; ++i) {
+                    a[i].ethr = fmaxf(a[i].ethr, __int_as_float(__reduce_max_sync(kFullMask, __float_as_int(a[i].emax))));
+                    a[i].qthr = fmaxf(a[i].qthr, __int_as_float(__reduce_max_sync(kFullMask, __float_as_int(a[i].qmax))));
+                }
+#pragma unroll
+                for (int i = 0; i < KB; ++i)
+#pragma unroll
+                    for (int u = 0; u < U; ++u) cur[i][u] = nxt[i][u];
             }
             // ragged end of the tensor: fewer than VEC elements, one thread, element by element
             if (tid == 0) {
-                for (uint32_t i = tail0; i < len; ++i) {
-                    uint32_t cb;
-                    if (CB16) cb = (uint32_t)reinterpret_cast<const uint16_t*>(cp)[i] << 16;
-                    else cb = reinterpret_cast<const uint32_t*>(cp)[i];
-                    const uint32_t cf = CB16 ? (c_first << 16) : c_first;
-                    a.cacc |= cb ^ cf;
-                    if (HAS_IN) a.pacc |= cb ^ smem_elem_bits<CB16>(in_s, i);
-                    elem_general(a, cb, smem_elem_bits<RB16>(ref_s, i), i, atol, rtol);
+#pragma unroll
+                for (int i = 0; i < KB; ++i) {
+                    for (uint32_t e = tail0; e < len; ++e) {
+                        uint32_t cb;
+                        if (CB16) cb = (uint32_t)reinterpret_cast<const uint16_t*>(cp[i])[e] << 16;
+                        else cb = reinterpret_cast<const uint32_t*>(cp[i])[e];
+                        const uint32_t cf = CB16 ? (c_first[i] << 16) : c_first[i];
+                        a[i].cacc |= cb ^ cf;
+                        if (HAS_IN) a[i].pacc |= cb ^ smem_elem_bits<CB16>(in_s, e);
+                        elem_general(a[i], cb, smem_elem_bits<RB16>(ref_s, e), e, atol, rtol);
+                    }
                 }
             }
-            warp_reduce_store(a, &warp_part[(k - kc0) * kWarps + warp], lane);
+#pragma unroll
+            for (int i = 0; i < KB; ++i)
+                if (kg + i < kc1) warp_reduce_store(a[i], &warp_part[(kg + i - kc0) * kWarps + warp], lane);
         }
         __syncthreads();
         if (tid < kc1 - kc0) {
@@ -519,10 +589,22 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
     return true;
 }
 
+__device__ __forceinline__ int variant_of(const DevTensor& D) {
+    const int cb16 = D.cand_dtype == RKV_BF16;
+    const int rb16 = D.ref_dtype == RKV_BF16 && D.ref_src == RKV_SRC_POINTER;
+    const int has_in = D.input_src != RKV_SRC_NONE;
+    return cb16 * 4 + rb16 * 2 + has_in;
+}
+
+// One kernel per storage variant (candidate dtype, staged reference dtype,
+// input present), so that each gets its own register allocation.  A launch
+// handles the slabs of every tensor of its variant; `n_items` counts them.
+template <bool CB16, bool RB16, bool HAS_IN>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSm)
 verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end,
-              uint32_t total_items, Partial* __restrict__ partials, int32_t* status) {
+              uint32_t n_items, Partial* __restrict__ partials, int32_t* status) {
     extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int kVariant = (CB16 ? 4 : 0) + (RB16 ? 2 : 0) + (HAS_IN ? 1 : 0);
     const int tid = threadIdx.x;
     if (tid == 0) {
         mbar_init(smem_u32(smem + kOffMbar), 1);
@@ -531,33 +613,39 @@ verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, 
     __syncthreads();
     uint32_t phase = 0;
     int cur_t = -1;
-    for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x) {
+    for (uint32_t it = blockIdx.x; it < n_items; it += gridDim.x) {
+        // it-th slab among the tensors of this variant
         int t = 0;
-        while (t + 1 < T && item >= tensors[t + 1].first_item) ++t;
+        uint32_t slab = it;
+        for (; t < T; ++t) {
+            if (variant_of(tensors[t]) != kVariant) continue;
+            const uint32_t ns = tensors[t].n_slabs;
+            if (slab < ns) break;
+            slab -= ns;
+        }
+        if (t >= T) return;
         const DevTensor D = tensors[t];
+        const uint32_t item = D.first_item + slab;
         if (t != cur_t) {
-            // thresholds carried from earlier slabs are per tensor
+            // per-tensor block state: thresholds carried from earlier slabs, and the
+            // candidates' base pointers and first elements (the constant-output test)
             float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
             float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
+            const unsigned char** cptr_s = reinterpret_cast<const unsigned char**>(smem + kOffCandPtr);
+            uint32_t* cfirst_s = reinterpret_cast<uint32_t*>(smem + kOffCandFirst);
+            __syncthreads();
             for (int i = tid; i < kHintK; i += kThreads) { hint_e[i] = -1.0f; hint_q[i] = -1.0f; }
+            for (int k = tid; k < K && k < kPreK; k += kThreads) {
+                const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k]);
+                cptr_s[k] = p;
+                cfirst_s[k] = CB16 ? (uint32_t)(*reinterpret_cast<const uint16_t*>(p))
+                                   : *reinterpret_cast<const uint32_t*>(p);
+            }
             cur_t = t;
         }
-        const bool cb16 = D.cand_dtype == RKV_BF16;
-        const bool rb16 = D.ref_dtype == RKV_BF16 && D.ref_src == RKV_SRC_POINTER;
-        const bool has_in = D.input_src != RKV_SRC_NONE;
-        bool ok;
-        if (!cb16) {
-            if (!rb16) ok = has_in ? process_item<false, false, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
-                                   : process_item<false, false, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
-            else       ok = has_in ? process_item<false, true, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
-                                   : process_item<false, true, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
-        } else {
-            if (!rb16) ok = has_in ? process_item<true, false, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
-                                   : process_item<true, false, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
-            else       ok = has_in ? process_item<true, true, true>(D, item, K, k_begin, k_end, partials, smem, phase, status)
-                                   : process_item<true, true, false>(D, item, K, k_begin, k_end, partials, smem, phase, status);
-        }
-        if (!ok) return;
+        if (!process_item<CB16, RB16, HAS_IN, kGroupK, CB16 ? kLoadsBf16 : kLoadsF32>(
+                D, item, K, k_begin, k_end, partials, smem, phase, status))
+            return;
     }
 }
 
@@ -664,24 +752,48 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Parti
 
 }  // namespace
 
-int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
-                  uint32_t total_items, int num_sms, Partial* partials, int32_t* status,
-                  cudaStream_t stream) {
+template <bool CB16, bool RB16, bool HAS_IN>
+static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
+                          int num_sms, Partial* partials, int32_t* status, cudaStream_t stream) {
     const int smem = kOffData + kSmemDataBudget + 256;
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return RKV_ERR_CUDA;
-    if (dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-            cudaSuccess)
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        if (cudaFuncSetAttribute(verify_kernel<CB16, RB16, HAS_IN>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return RKV_ERR_CUDA;
-        attr_set[dev] = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     uint32_t grid = (uint32_t)num_sms * kBlocksPerSm;
-    if (grid > total_items) grid = total_items;
-    verify_kernel<<<grid, kThreads, smem, stream>>>(d_tensors, T, K, k_begin, k_end, total_items,
-                                                    partials, status);
+    if (grid > n_items) grid = n_items;
+    verify_kernel<CB16, RB16, HAS_IN><<<grid, kThreads, smem, stream>>>(d_tensors, T, K, k_begin, k_end,
+                                                                      n_items, partials, status);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
+                  const uint32_t variant_items[8], int num_sms, Partial* partials, int32_t* status,
+                  cudaStream_t stream) {
+    int rc = RKV_OK;
+    for (int v = 0; v < 8 && rc == RKV_OK; ++v) {
+        const uint32_t n = variant_items[v];
+        if (!n) continue;
+#define RKV_LAUNCH(CB, RB, IN) \
+    launch_variant<CB, RB, IN>(d_tensors, T, K, k_begin, k_end, n, num_sms, partials, status, stream)
+        switch (v) {
+            case 0: rc = RKV_LAUNCH(false, false, false); break;
+            case 1: rc = RKV_LAUNCH(false, false, true); break;
+            case 2: rc = RKV_LAUNCH(false, true, false); break;
+            case 3: rc = RKV_LAUNCH(false, true, true); break;
+            case 4: rc = RKV_LAUNCH(true, false, false); break;
+            case 5: rc = RKV_LAUNCH(true, false, true); break;
+            case 6: rc = RKV_LAUNCH(true, true, false); break;
+            default: rc = RKV_LAUNCH(true, true, true); break;
+        }
+#undef RKV_LAUNCH
+    }
+    return rc;
 }
 
 int launch_finalize(const DevTensor* d_tensors, int T, int K, const Partial* partials,
