@@ -18,6 +18,8 @@
 //
 // Reductions are deterministic: integer sums, lexicographic (value descending,
 // index ascending) maxima, and a fixed-order fp64 sum.  No float atomics.
+#include <type_traits>
+
 #include "rkv_internal.h"
 #include "rkv_philox.cuh"
 
@@ -37,7 +39,8 @@ constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr int kOffMbar = 0;                               // 8 bytes
 constexpr int kOffHintE = 64;
 constexpr int kOffHintQ = kOffHintE + kHintK * 4;
-constexpr int kOffWarpPart = kOffHintQ + kHintK * 4;      // 16-aligned
+constexpr int kOffHintF = kOffHintQ + kHintK * 4;
+constexpr int kOffWarpPart = kOffHintF + kHintK * 4;      // 16-aligned
 constexpr int kOffCandPtr = kOffWarpPart + kChunkK * kWarps * (int)sizeof(Partial);
 constexpr int kOffCandFirst = kOffCandPtr + kPreK * 8;
 constexpr int kOffDataRaw = kOffCandFirst + kPreK * 4;
@@ -103,7 +106,9 @@ struct Acc {
     float qmax; uint32_t qidx; float qthr;
     double sum;
     uint32_t cacc, pacc;
-    uint32_t n_noncomp, n_nan, n_inf, n_infmis;
+    // four 8-bit counters (a thread sees < 256 elements of one slab):
+    // byte 0 non-comparable, 1 NaN, 2 Inf, 3 infinity mismatch
+    uint32_t rare;
 };
 
 __device__ __forceinline__ void acc_reset(Acc& a, float hint_e, float hint_q) {
@@ -112,14 +117,14 @@ __device__ __forceinline__ void acc_reset(Acc& a, float hint_e, float hint_q) {
     a.qmax = -1.0f; a.qidx = 0xFFFFFFFFu; a.qthr = hint_q;
     a.sum = 0.0;
     a.cacc = 0; a.pacc = 0;
-    a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
+    a.rare = 0;
 }
 
 // The comparison rule for one element, every case included.
 __device__ __forceinline__ void elem_general(Acc& a, uint32_t cb, uint32_t rb, uint32_t idx, float atol,
                                              float rtol) {
-    if (bits_nan(cb)) a.n_nan++;
-    if (bits_inf(cb)) a.n_inf++;
+    if (bits_nan(cb)) a.rare += 1u << 8;
+    if (bits_inf(cb)) a.rare += 1u << 16;
     if (bits_finite(cb) && bits_finite(rb)) {
         const float c = __uint_as_float(cb), r = __uint_as_float(rb);
         const float e = fabsf(__fsub_rn(c, r));
@@ -132,11 +137,11 @@ __device__ __forceinline__ void elem_general(Acc& a, uint32_t cb, uint32_t rb, u
         }
         a.sum += (double)e;
     } else if (bits_inf(cb) && cb == rb) {
-        a.n_noncomp++;
+        a.rare += 1u;
     } else {
-        a.n_noncomp++;
+        a.rare += 1u;
         a.n_over++;
-        if (bits_inf(cb) || bits_inf(rb)) a.n_infmis++;
+        if (bits_inf(cb) || bits_inf(rb)) a.rare += 1u << 24;
     }
 }
 
@@ -146,36 +151,98 @@ template <int VEC>
 struct RefVec {
     uint32_t r[VEC];      // reference bits (fp32 patterns)
     float thr[VEC];       // atol + rtol*|r|, product and sum each rounded
-    float arp[VEC];       // |r|, or +inf where r == 0 (such elements never enter the relative maximum)
+    float minarp;         // smallest non-zero |r| of the vector, +inf if all are zero
 };
 
 template <int VEC>
 __device__ __forceinline__ void refvec_prepare(RefVec<VEC>& rv, float atol, float rtol) {
+    // |r| as an integer orders like the float; subtracting one wraps zero to the top
+    uint32_t mn = 0xFFFFFFFFu;
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-        const float ar = fabsf(__uint_as_float(rv.r[j]));
-        rv.thr[j] = __fadd_rn(atol, __fmul_rn(rtol, ar));
-        rv.arp[j] = ar != 0.0f ? ar : __int_as_float(0x7F800000);
+        const uint32_t ab = rv.r[j] & 0x7FFFFFFFu;
+        rv.thr[j] = __fadd_rn(atol, __fmul_rn(rtol, __uint_as_float(ab)));
+        mn = min(mn, ab - 1u);
     }
+    rv.minarp = mn == 0xFFFFFFFFu ? __int_as_float(0x7F800000) : __uint_as_float(mn + 1u);
+}
+
+// The rarely taken parts of a vector step live out of line, so that the hot loop
+// stays small enough for the instruction cache.  Arguments travel by value.
+struct Best {
+    float emax; uint32_t eidx;
+    float qmax; uint32_t qidx;
+};
+
+template <int VEC>
+struct VecErr {
+    float e[VEC];
+    uint32_t r[VEC];
+};
+
+// All values finite: new running maxima of |c - r| and of |c - r| / |r|.
+template <int VEC>
+__device__ __noinline__ Best rare_finite(Best b, float qthr, VecErr<VEC> x, uint32_t idx0) {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        if (x.e[j] > b.emax) { b.emax = x.e[j]; b.eidx = idx0 + j; }
+        const float ar = fabsf(__uint_as_float(x.r[j]));
+        if (ar != 0.0f && x.e[j] > __fmul_rd(qthr, ar)) {
+            const float q = __fdiv_rn(x.e[j], ar);
+            if (q > b.qmax) { b.qmax = q; b.qidx = idx0 + j; }
+        }
+    }
+    return b;
+}
+
+template <int VEC>
+struct VecBits {
+    uint32_t c[VEC];
+    uint32_t r[VEC];
+};
+
+struct GenState {
+    Best b;
+    uint32_t n_over;
+    uint32_t rare;
+    double sum;
+};
+
+// A vector with a non-finite value somewhere: the general rule, element by element.
+template <int VEC>
+__device__ __noinline__ GenState rare_general(GenState g, VecBits<VEC> x, uint32_t idx0, float atol,
+                                              float rtol) {
+    Acc a;
+    a.n_over = g.n_over; a.rare = g.rare; a.sum = g.sum;
+    a.emax = g.b.emax; a.eidx = g.b.eidx; a.qmax = g.b.qmax; a.qidx = g.b.qidx;
+    a.ethr = 0.0f; a.qthr = 0.0f; a.cacc = 0; a.pacc = 0;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) elem_general(a, x.c[j], x.r[j], idx0 + j, atol, rtol);
+    g.n_over = a.n_over; g.rare = a.rare; g.sum = a.sum;
+    g.b.emax = a.emax; g.b.eidx = a.eidx; g.b.qmax = a.qmax; g.b.qidx = a.qidx;
+    return g;
 }
 
 // VEC consecutive elements of one candidate: bits c[] against the prepared
 // reference vector; idx0 is the slab-local index of the first element.
 //
-// Fast path (all values finite).  The three per-element tests only set a
-// predicate; the work behind them runs when a predicate fired:
+// The common path only evaluates predicates; everything behind them sits in one
+// rarely taken region:
+//   !(s < s_limit)                          a non-finite value somewhere in the
+//                                           vector (or a slab whose reference
+//                                           has one: s_limit = -1) -> general rule
 //   over : !(e <= thr)                      -> recount the vector
 //   abs  : e > ethr, ethr >= running max    -> update (max, first index)
-//   rel  : e > RD(qthr * |r|)               -> divide, update (max, first index)
+//   rel  : max e > RD(qthr * min|r|)        -> per element e > RD(qthr*|r|): divide, update
 // RD is the product rounded toward -inf.  If fl(e/|r|) > qthr then, rounding
 // being monotone, e/|r| > qthr exactly, so e > qthr*|r| >= RD(qthr*|r|): the
 // test never skips an element that beats qthr.  Thresholds always come from
 // elements with SMALLER indices (the thread's own earlier elements, earlier
-// batches of the block, earlier slabs), so a tie may be skipped: the first
-// index keeps the maximum.
+// rounds of the warp, earlier slabs of the block), so a tie may be skipped: the
+// first index keeps the maximum.
 template <int VEC>
 __device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const RefVec<VEC>& rv,
-                                         uint32_t idx0, float atol, float rtol, bool general) {
+                                         uint32_t idx0, float atol, float rtol, float s_limit) {
     float e[VEC];
 #pragma unroll
     for (int j = 0; j < VEC; ++j)
@@ -187,41 +254,40 @@ __device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const
         s = __fadd_rn(__fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3])),
                       __fadd_rn(__fadd_rn(e[4 % VEC], e[5 % VEC]), __fadd_rn(e[6 % VEC], e[7 % VEC])));
     }
-    if (general || !(s < __int_as_float(0x7F800000))) {
+    const bool finite = s < s_limit;
+    bool rare = !finite;
+    float m = e[0];
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) elem_general(a, c[j], rv.r[j], idx0 + j, atol, rtol);
-        a.ethr = fmaxf(a.ethr, a.emax);
-        a.qthr = fmaxf(a.qthr, a.qmax);
-        return;
-    }
-    bool over = false, absh = false, relh = false;
+    for (int j = 1; j < VEC; ++j) m = fmaxf(m, e[j]);
+    rare |= m > a.ethr;
+    // vector-level relative-error filter: e_j > qthr*|r_j| for some j implies m > qthr*min|r|
+    rare |= m > __fmul_rd(a.qthr, rv.minarp);
+    // over-tolerance elements are common in failing candidates: counted unconditionally
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-        over |= !(e[j] <= rv.thr[j]);
-        absh |= e[j] > a.ethr;
-        relh |= e[j] > __fmul_rd(a.qthr, rv.arp[j]);
-    }
-    a.sum += (double)s;
-    if (over) {
+    for (int j = 0; j < VEC; ++j)
+        if (!(e[j] <= rv.thr[j]) && finite) a.n_over++;
+    a.sum += (double)(finite ? s : 0.0f);
+    if (rare) {
+        if (!finite) {
+            GenState g;
+            g.b.emax = a.emax; g.b.eidx = a.eidx; g.b.qmax = a.qmax; g.b.qidx = a.qidx;
+            g.n_over = a.n_over; g.rare = a.rare; g.sum = a.sum;
+            VecBits<VEC> x;
 #pragma unroll
-        for (int j = 0; j < VEC; ++j)
-            if (!(e[j] <= rv.thr[j])) a.n_over++;
-    }
-    if (absh) {
+            for (int j = 0; j < VEC; ++j) { x.c[j] = c[j]; x.r[j] = rv.r[j]; }
+            g = rare_general<VEC>(g, x, idx0, atol, rtol);
+            a.emax = g.b.emax; a.eidx = g.b.eidx; a.qmax = g.b.qmax; a.qidx = g.b.qidx;
+            a.n_over = g.n_over; a.rare = g.rare; a.sum = g.sum;
+        } else {
+            Best b;
+            b.emax = a.emax; b.eidx = a.eidx; b.qmax = a.qmax; b.qidx = a.qidx;
+            VecErr<VEC> x;
 #pragma unroll
-        for (int j = 0; j < VEC; ++j)
-            if (e[j] > a.emax) { a.emax = e[j]; a.eidx = idx0 + j; }
-        a.ethr = fmaxf(a.ethr, a.emax);
-    }
-    if (relh) {
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-            const float ar = fabsf(__uint_as_float(rv.r[j]));
-            if (ar != 0.0f && e[j] > __fmul_rd(a.qthr, ar)) {
-                const float q = __fdiv_rn(e[j], ar);
-                if (q > a.qmax) { a.qmax = q; a.qidx = idx0 + j; }
-            }
+            for (int j = 0; j < VEC; ++j) { x.e[j] = e[j]; x.r[j] = rv.r[j]; }
+            b = rare_finite<VEC>(b, a.qthr, x, idx0);
+            a.emax = b.emax; a.eidx = b.eidx; a.qmax = b.qmax; a.qidx = b.qidx;
         }
+        a.ethr = fmaxf(a.ethr, a.emax);
         a.qthr = fmaxf(a.qthr, a.qmax);
     }
 }
@@ -231,13 +297,12 @@ __device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const
 // ----------------------------------------------------------------------------
 __device__ __forceinline__ void warp_reduce_store(const Acc& a, Partial* dst, int lane) {
     const uint32_t n_over = __reduce_add_sync(kFullMask, a.n_over);
-    const uint32_t rare = a.n_noncomp | a.n_nan | a.n_inf | a.n_infmis;
     uint32_t n_noncomp = 0, n_nan = 0, n_inf = 0, n_infmis = 0;
-    if (__any_sync(kFullMask, rare != 0)) {
-        n_noncomp = __reduce_add_sync(kFullMask, a.n_noncomp);
-        n_nan = __reduce_add_sync(kFullMask, a.n_nan);
-        n_inf = __reduce_add_sync(kFullMask, a.n_inf);
-        n_infmis = __reduce_add_sync(kFullMask, a.n_infmis);
+    if (__any_sync(kFullMask, a.rare != 0)) {
+        n_noncomp = __reduce_add_sync(kFullMask, a.rare & 0xFFu);
+        n_nan = __reduce_add_sync(kFullMask, (a.rare >> 8) & 0xFFu);
+        n_inf = __reduce_add_sync(kFullMask, (a.rare >> 16) & 0xFFu);
+        n_infmis = __reduce_add_sync(kFullMask, a.rare >> 24);
     }
     // non-negative floats (and the -1 sentinel) order like their bit patterns as signed ints
     const int eb = __float_as_int(a.emax);
@@ -348,6 +413,7 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
     const uint32_t mbar = smem_u32(smem + kOffMbar);
     float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
     float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
+    uint32_t* hint_f = reinterpret_cast<uint32_t*>(smem + kOffHintF);
     Partial* warp_part = reinterpret_cast<Partial*>(smem + kOffWarpPart);
 
     // ---- stage reference and input -------------------------------------------------
@@ -438,11 +504,17 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
 
     // ---- stream the candidates -------------------------------------------------------
     // Candidates are taken KB at a time: the reference vector is read from shared
-    // memory and prepared once per KB candidate vectors.  Loads of the next batch
-    // are issued before the current batch is processed.
+    // memory and prepared once per KB candidate vectors.  Each thread keeps U
+    // 16-byte loads per candidate in flight: a register slot is reloaded with the
+    // vector U rounds ahead right after it has been consumed.
     const uint32_t nvec = len / VEC;
     const uint32_t tail0 = nvec * VEC;
-    const uint32_t nbatch = (nvec + U * kThreads - 1) / (U * kThreads);
+    // this thread's vectors are v = tid + i*kThreads, i < n_mine; the first lane of a
+    // warp has the most (n_first), which gives the warp-uniform trip count
+    const uint32_t n_mine = nvec > (uint32_t)tid ? (nvec - tid + kThreads - 1) / kThreads : 0u;
+    const uint32_t tid_first = (uint32_t)tid & ~31u;
+    const uint32_t n_first = nvec > tid_first ? (nvec - tid_first + kThreads - 1) / kThreads : 0u;
+    const float s_limit = general ? -1.0f : __int_as_float(0x7F800000);
     const unsigned char* const* cptr_s = reinterpret_cast<const unsigned char* const*>(smem + kOffCandPtr);
     const uint32_t* cfirst_s = reinterpret_cast<const uint32_t*>(smem + kOffCandFirst);
     for (int kc0 = k_begin; kc0 < k_end; kc0 += kChunkK) {
@@ -464,94 +536,122 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
                                       : *reinterpret_cast<const uint32_t*>(cp[i]);
                 }
                 if (CB16) c_first[i] = (c_first[i] & 0xFFFFu) * 0x10001u;
-                cp[i] += start * CSZ;
+                cp[i] += start * CSZ + (size_t)tid * 16;
                 acc_reset(a[i], k < kHintK ? hint_e[k] : -1.0f, k < kHintK ? hint_q[k] : -1.0f);
             }
 
-            uint4 cur[KB][U], nxt[KB][U];
+            // The loophole flags are OR-reductions over the whole tensor: once an earlier
+            // slab of this block has reported "differs" for every candidate of the group,
+            // the xor/or work is skipped and the settled value reported again.
+            uint32_t settled = 3u;
 #pragma unroll
-            for (int i = 0; i < KB; ++i)
+            for (int i = 0; i < KB; ++i) {
+                const int k = (kg + i) < kc1 ? (kg + i) : (kc1 - 1);
+                settled &= k < kHintK ? hint_f[k] : 0u;
+            }
+            constexpr uint32_t kWanted = HAS_IN ? 3u : 1u;
+            const bool need_flags = (settled & kWanted) != kWanted;
+            if (!need_flags) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t v = u * kThreads + tid;
-                    if (v < nvec) cur[i][u] = ldg_stream(cp[i] + (size_t)v * 16);
-                }
-            for (uint32_t b = 0; b < nbatch; ++b) {
-                const uint32_t vb = b * U * kThreads + tid;
-                if (b + 1 < nbatch) {
-#pragma unroll
-                    for (int i = 0; i < KB; ++i)
-#pragma unroll
-                        for (int u = 0; u < U; ++u) {
-                            const uint32_t v = vb + (U + u) * kThreads;
-                            if (v < nvec) nxt[i][u] = ldg_stream(cp[i] + (size_t)v * 16);
-                        }
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t v = vb + u * kThreads;
-                    if (v < nvec) {
-                        RefVec<VEC> rv;
-                        uint4 iv = make_uint4(0, 0, 0, 0);
-                        if (HAS_IN) iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
-                        if (!CB16) {
-                            if (RB16) {
-                                const uint2 t = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
-                                rv.r[0] = t.x << 16; rv.r[1] = t.x & 0xFFFF0000u;
-                                rv.r[2] = t.y << 16; rv.r[3] = t.y & 0xFFFF0000u;
-                            } else {
-                                const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                                rv.r[0] = t.x; rv.r[1] = t.y; rv.r[2] = t.z; rv.r[3] = t.w;
-                            }
-                        } else {
-                            if (RB16) {
-                                const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                                const uint32_t rw[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    rv.r[(2 * q) % VEC] = rw[q] << 16;
-                                    rv.r[(2 * q + 1) % VEC] = rw[q] & 0xFFFF0000u;
-                                }
-                            } else {
-                                const uint4 t0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
-                                const uint4 t1 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
-                                rv.r[0] = t0.x; rv.r[1] = t0.y; rv.r[2] = t0.z; rv.r[3] = t0.w;
-                                rv.r[4 % VEC] = t1.x; rv.r[5 % VEC] = t1.y;
-                                rv.r[6 % VEC] = t1.z; rv.r[7 % VEC] = t1.w;
-                            }
-                        }
-                        refvec_prepare<VEC>(rv, atol, rtol);
-#pragma unroll
-                        for (int i = 0; i < KB; ++i) {
-                            const uint32_t w[4] = {cur[i][u].x, cur[i][u].y, cur[i][u].z, cur[i][u].w};
-                            a[i].cacc |= (w[0] ^ c_first[i]) | (w[1] ^ c_first[i]) | (w[2] ^ c_first[i]) |
-                                         (w[3] ^ c_first[i]);
-                            if (HAS_IN) a[i].pacc |= (w[0] ^ iv.x) | (w[1] ^ iv.y) | (w[2] ^ iv.z) | (w[3] ^ iv.w);
-                            uint32_t c[VEC];
-                            if (!CB16) {
-                                c[0] = w[0]; c[1] = w[1]; c[2] = w[2]; c[3] = w[3];
-                            } else {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    c[(2 * q) % VEC] = w[q] << 16;
-                                    c[(2 * q + 1) % VEC] = w[q] & 0xFFFF0000u;
-                                }
-                            }
-                            step_vec<VEC>(a[i], c, rv, v * VEC, atol, rtol, general);
-                        }
-                    }
-                }
-                // share the running maxima across the warp: every element of this batch has
-                // a smaller index than every element of the next one
-#pragma unroll
-                for (int i = 0; i < KB; ++i) {
-                    a[i].ethr = fmaxf(a[i].ethr, __int_as_float(__reduce_max_sync(kFullMask, __float_as_int(a[i].emax))));
-                    a[i].qthr = fmaxf(a[i].qthr, __int_as_float(__reduce_max_sync(kFullMask, __float_as_int(a[i].qmax))));
-                }
+                for (int i = 0; i < KB; ++i) { a[i].cacc = 1u; a[i].pacc = 1u; }
+            }
+
+            // Two register buffers of U vectors per candidate.  All loads of a batch are
+            // issued together, one batch ahead of their use, and consumed together.
+            uint4 bufA[KB][U], bufB[KB][U];
+            auto load_batch = [&](uint4 (&buf)[KB][U], const uint32_t r0) {
 #pragma unroll
                 for (int i = 0; i < KB; ++i)
 #pragma unroll
-                    for (int u = 0; u < U; ++u) cur[i][u] = nxt[i][u];
+                    for (int u = 0; u < U; ++u)
+                        if (r0 + u < n_mine)
+                            buf[i][u] = ldg_stream(cp[i] + (size_t)(r0 + u) * (kThreads * 16));
+            };
+
+            // one vector position of this thread: round r (v = tid + r*kThreads)
+            auto do_vector = [&](const uint4 (&buf)[KB][U], const int u, const uint32_t r) {
+                const uint32_t v = (uint32_t)tid + r * kThreads;
+                RefVec<VEC> rv;
+                if (!CB16) {
+                    if (RB16) {
+                        const uint2 t = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
+                        rv.r[0] = t.x << 16; rv.r[1] = t.x & 0xFFFF0000u;
+                        rv.r[2] = t.y << 16; rv.r[3] = t.y & 0xFFFF0000u;
+                    } else {
+                        const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                        rv.r[0] = t.x; rv.r[1] = t.y; rv.r[2] = t.z; rv.r[3] = t.w;
+                    }
+                } else {
+                    if (RB16) {
+                        const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
+                        const uint32_t rw[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            rv.r[(2 * q) % VEC] = rw[q] << 16;
+                            rv.r[(2 * q + 1) % VEC] = rw[q] & 0xFFFF0000u;
+                        }
+                    } else {
+                        const uint4 t0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
+                        const uint4 t1 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
+                        rv.r[0] = t0.x; rv.r[1] = t0.y; rv.r[2] = t0.z; rv.r[3] = t0.w;
+                        rv.r[4 % VEC] = t1.x; rv.r[5 % VEC] = t1.y;
+                        rv.r[6 % VEC] = t1.z; rv.r[7 % VEC] = t1.w;
+                    }
+                }
+                refvec_prepare<VEC>(rv, atol, rtol);
+                if (need_flags) {
+                    uint4 iv = make_uint4(0, 0, 0, 0);
+                    if (HAS_IN) iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
+#pragma unroll
+                    for (int i = 0; i < KB; ++i) {
+                        const uint4 w = buf[i][u];
+                        a[i].cacc |= (w.x ^ c_first[i]) | (w.y ^ c_first[i]) | (w.z ^ c_first[i]) |
+                                     (w.w ^ c_first[i]);
+                        if (HAS_IN) a[i].pacc |= (w.x ^ iv.x) | (w.y ^ iv.y) | (w.z ^ iv.z) | (w.w ^ iv.w);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < KB; ++i) {
+                    const uint32_t w[4] = {buf[i][u].x, buf[i][u].y, buf[i][u].z, buf[i][u].w};
+                    uint32_t c[VEC];
+                    if (!CB16) {
+                        c[0] = w[0]; c[1] = w[1]; c[2] = w[2]; c[3] = w[3];
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            c[(2 * q) % VEC] = w[q] << 16;
+                            c[(2 * q + 1) % VEC] = w[q] & 0xFFFF0000u;
+                        }
+                    }
+                    step_vec<VEC>(a[i], c, rv, v * VEC, atol, rtol, s_limit);
+                }
+            };
+
+            auto compute_batch = [&](const uint4 (&buf)[KB][U], const uint32_t r0) {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (r0 + u < n_mine) do_vector(buf, u, r0 + u);
+                if (r0 < 2 * U) {
+                    // share the running maxima across the warp: every element seen so far has
+                    // a smaller index than every element of the batches to come
+#pragma unroll
+                    for (int i = 0; i < KB; ++i) {
+                        a[i].ethr = fmaxf(a[i].ethr, __int_as_float(__reduce_max_sync(
+                                                         kFullMask, __float_as_int(a[i].emax))));
+                        a[i].qthr = fmaxf(a[i].qthr, __int_as_float(__reduce_max_sync(
+                                                         kFullMask, __float_as_int(a[i].qmax))));
+                    }
+                }
+            };
+
+            // n_first rounds: what the first lane of the warp needs (the most), so that the
+            // trip count is uniform across the warp
+            load_batch(bufA, 0);
+            for (uint32_t r0 = 0; r0 < n_first; r0 += 2 * U) {
+                load_batch(bufB, r0 + U);
+                compute_batch(bufA, r0);
+                load_batch(bufA, r0 + 2 * U);
+                if (r0 + U < n_first) compute_batch(bufB, r0 + U);
             }
             // ragged end of the tensor: fewer than VEC elements, one thread, element by element
             if (tid == 0) {
@@ -582,6 +682,7 @@ __device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, 
             if (k < kHintK) {
                 hint_e[k] = fmaxf(hint_e[k], p.emax);
                 hint_q[k] = fmaxf(hint_q[k], p.qmax);
+                hint_f[k] |= p.mismatch;
             }
         }
         __syncthreads();
@@ -634,7 +735,8 @@ verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, 
             const unsigned char** cptr_s = reinterpret_cast<const unsigned char**>(smem + kOffCandPtr);
             uint32_t* cfirst_s = reinterpret_cast<uint32_t*>(smem + kOffCandFirst);
             __syncthreads();
-            for (int i = tid; i < kHintK; i += kThreads) { hint_e[i] = -1.0f; hint_q[i] = -1.0f; }
+            uint32_t* hint_f = reinterpret_cast<uint32_t*>(smem + kOffHintF);
+            for (int i = tid; i < kHintK; i += kThreads) { hint_e[i] = -1.0f; hint_q[i] = -1.0f; hint_f[i] = 0u; }
             for (int k = tid; k < K && k < kPreK; k += kThreads) {
                 const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k]);
                 cptr_s[k] = p;
