@@ -229,6 +229,48 @@ int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, i
                           int dtype, float atol, float rtol, rkv_stats *stats_host);
 
 /*
+ * rkv_verify_batch with no allocation of any kind.  (The paper has no
+ * counterpart: this form exists for the way the library gets embedded.)
+ *
+ * Who needs it: a caller that may not allocate device memory at the point of the
+ * call -- a harness that has handed all of the GPU's memory to its own pool and
+ * left the driver nothing to give out, a host thread that must not block on the
+ * allocator's device-wide synchronisation, a process running under a memory
+ * budget that counts every allocation it makes.  rkv_verify_batch grows a
+ * library-owned buffer with cudaMalloc; rkv_verify_multi wants a workspace the
+ * caller had to allocate at some point.  This form needs neither: its scratch
+ * (per-slab partial results and the descriptor tables) is an 8 MiB array that is
+ * part of the library's device image.  Every GPU that loads the library holds
+ * those 8 MiB until the process exits, whether or not this function is called.
+ *
+ * Same arguments, same results and same comparison rule as rkv_verify_batch,
+ * plus the stream to run on (a cudaStream_t; NULL = default stream).  ref, cands
+ * and stats_out are the caller's; inputs are only read.
+ *
+ * Limits: K <= 256, and the scratch the case needs (rkv_workspace_bytes of the
+ * single-tensor case, which grows with n * K) must fit in 8 MiB; e.g. fp32,
+ * n = 2^24 with K = 128, or n = 2^25 with K = 64, fit.  A larger case is rejected
+ * with RKV_ERR_UNSUPPORTED before anything is launched.  Other errors:
+ * INVALID_ARG, ALIGNMENT, CUDA.
+ *
+ * First call on a device: looks up the array's device address once (with that
+ * device current) and sets a kernel attribute.  Make that first call outside any
+ * stream capture.
+ *
+ * All calls on a device share the one array, and it keeps whatever the previous
+ * call left there.  The library rewrites the status word and the tables at the
+ * start of every call and the kernels overwrite every partial result they later
+ * read, so a call never depends on old contents.  Two calls whose work overlaps
+ * on the GPU (different streams, or several host threads) race on the array and
+ * give undefined results: run them one after the other.
+ *
+ * Calls no cudaMalloc / cudaFree and no allocating library routine; the small
+ * descriptor table is built on the host stack and sent with one cudaMemcpyAsync.
+ */
+int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, uint64_t n, int dtype,
+                            float atol, float rtol, rkv_stats *stats_out, void *cuda_stream);
+
+/*
  * Host-only planning helper (no CUDA call): how a tensor is cut into slabs.
  * A slab is the run of elements whose reference (and input) one thread block
  * stages in shared memory and reuses for all K candidates.

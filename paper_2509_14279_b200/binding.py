@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.rkv_device_status.argtypes = [vp, vp]
         L.rkv_verify_batch_host.restype = i32
         L.rkv_verify_batch_host.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
+        L.rkv_verify_batch_static.restype = i32
+        L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
         L.rkv_plan_slabs.restype = i32
         L.rkv_plan_slabs.argtypes = [u64, i32, i32, ctypes.POINTER(ctypes.c_uint32),
                                      ctypes.POINTER(ctypes.c_uint64)]
@@ -188,6 +190,23 @@ def verify_batch(ref: torch.Tensor, cands, atol: float, rtol: float,
     _check(lib().rkv_verify_batch(ctypes.c_void_p(ref.data_ptr()), ptrs, K, n, _dtype_code(ref),
                                   float(atol), float(rtol), ctypes.c_void_p(stats_out.data_ptr())),
            "rkv_verify_batch")
+    return stats_out
+
+
+def verify_batch_static(ref: torch.Tensor, cands, atol: float, rtol: float,
+                        stats_out: torch.Tensor, stream=None) -> torch.Tensor:
+    """rkv_verify_batch_static: like ``verify_batch`` but nothing is allocated, here or in
+    the library -- the scratch is a fixed 8 MiB array inside the library, so the caller must
+    pass ``stats_out`` (K*88 bytes, uint8, on the device).  For callers that cannot allocate
+    device memory when they verify (all memory already in their own pool, or no allocator
+    calls allowed on this thread).  Calls share that array: do not overlap them on the GPU."""
+    K = len(cands)
+    ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cands])
+    _check(lib().rkv_verify_batch_static(ctypes.c_void_p(ref.data_ptr()), ptrs, K, ref.numel(),
+                                         _dtype_code(ref), float(atol), float(rtol),
+                                         ctypes.c_void_p(stats_out.data_ptr()),
+                                         ctypes.c_void_p(_stream_ptr(stream))),
+           "rkv_verify_batch_static")
     return stats_out
 
 

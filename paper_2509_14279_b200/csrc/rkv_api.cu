@@ -411,6 +411,107 @@ int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, i
     return RKV_OK;
 }
 
+// ----------------------------------------------------------------------------
+// rkv_verify_batch_static: the same verification with its scratch in a fixed
+// device array that is part of the library image -- nothing is allocated.
+// ----------------------------------------------------------------------------
+}  // extern "C"
+
+namespace rkv {
+namespace {
+
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;
+constexpr int kStaticMaxK = 256;
+
+// Lives in the global memory of every device that loads the library, until the
+// process exits.  On the host this name is only a handle for
+// cudaGetSymbolAddress: it is not a device address and is never passed to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on each device, looked up once per device
+// with that device current.
+void* g_static_scratch_addr[64] = {};
+
+int static_scratch_address(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RKV_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return RKV_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return RKV_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return RKV_OK;
+}
+
+}  // namespace
+}  // namespace rkv
+
+extern "C" {
+
+int rkv_verify_batch_static(const void* ref, const void* const* cands, int K, uint64_t n, int dtype,
+                            float atol, float rtol, rkv_stats* stats_out, void* cuda_stream) {
+    rkv_tensor_desc d;
+    memset(&d, 0, sizeof d);
+    d.n = n; d.ref = ref; d.cands = cands;
+    d.cand_dtype = dtype; d.ref_dtype = dtype;
+    d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
+    d.atol = atol; d.rtol = rtol;
+    int rc = validate_tensors(&d, 1, K);
+    if (rc != RKV_OK) return rc;
+    if (!stats_out) return RKV_ERR_INVALID_ARG;
+    if (K > kStaticMaxK) return RKV_ERR_UNSUPPORTED;
+    int sms = 0;
+    rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    Plan plan;
+    rc = make_plan(&d, 1, K, sms, &plan);
+    if (rc != RKV_OK) return rc;
+    if (plan.total_bytes > kStaticScratchBytes) return RKV_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != RKV_OK) return rc;
+
+    // header (status word = 0) + descriptor + pointer table, built on the stack
+    constexpr size_t kBlobMax = sizeof(WorkspaceHeader) +
+                                (sizeof(DevTensor) + kStaticMaxK * sizeof(void*) + 255) / 256 * 256;
+    alignas(16) unsigned char blob[kBlobMax];
+    const size_t blob_bytes = sizeof(WorkspaceHeader) + plan.table_bytes;
+    if (blob_bytes > kBlobMax) return RKV_ERR_UNSUPPORTED;
+    memset(blob, 0, blob_bytes);
+    unsigned char* ws = reinterpret_cast<unsigned char*>(scratch);
+    DevTensor* d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
+    const void** d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) + sizeof(DevTensor));
+    Partial* partials = reinterpret_cast<Partial*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
+    DevTensor* h_t = reinterpret_cast<DevTensor*>(blob + sizeof(WorkspaceHeader));
+    const void** h_p = reinterpret_cast<const void**>(blob + sizeof(WorkspaceHeader) + sizeof(DevTensor));
+    h_t->n = n;
+    h_t->ref = ref;
+    h_t->input = nullptr;
+    h_t->cands = d_ptrs;
+    h_t->cand_dtype = dtype; h_t->ref_dtype = dtype;
+    h_t->ref_src = RKV_SRC_POINTER; h_t->input_src = RKV_SRC_NONE;
+    h_t->atol = atol; h_t->rtol = rtol;
+    h_t->slab_elems = plan.slab_elems[0]; h_t->n_slabs = plan.n_slabs[0];
+    h_t->first_item = plan.first_item[0];
+    for (int k = 0; k < K; ++k) h_p[k] = cands[k];
+
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(ws, blob, blob_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return RKV_ERR_CUDA;
+    }
+    rc = launch_verify(d_tensors, 1, K, 0, K, plan.variant_items, sms, partials,
+                       reinterpret_cast<int32_t*>(ws), stream);
+    if (rc != RKV_OK) return rc;
+    return launch_finalize(d_tensors, 1, K, partials, stats_out, nullptr, stream);
+}
+
 int rkv_release_cached(void) {
     std::lock_guard<std::mutex> lock(g_mutex);
     int cur = 0;
