@@ -197,8 +197,9 @@ int rkv_verify_batch(const void *ref, const void *const *cands, int K, uint64_t 
  *   workspace   DEVICE scratch, >= rkv_workspace_bytes(tensors, T, K) bytes, 256-byte
  *               aligned; contents are undefined afterwards; must not be shared by
  *               calls that overlap on the GPU
- * Nothing is allocated.  The descriptors and pointer tables are copied to the
- * workspace with one cudaMemcpyAsync from pageable host memory.
+ * Nothing is allocated on the device.  The descriptors and pointer tables are
+ * copied to the workspace with one cudaMemcpyAsync from pageable host memory and
+ * the rest of the workspace is cleared with one cudaMemsetAsync.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.  A device-side
  * timeout is reported by rkv_device_status.
  */
@@ -239,7 +240,7 @@ int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, i
  * budget that counts every allocation it makes.  rkv_verify_batch grows a
  * library-owned buffer with cudaMalloc; rkv_verify_multi wants a workspace the
  * caller had to allocate at some point.  This form needs neither: its scratch
- * (per-slab partial results and the descriptor tables) is an 8 MiB array that is
+ * (per-block partial results, per-candidate state and the descriptor tables) is an 8 MiB array that is
  * part of the library's device image.  Every GPU that loads the library holds
  * those 8 MiB until the process exits, whether or not this function is called.
  *
@@ -248,8 +249,8 @@ int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, i
  * and stats_out are the caller's; inputs are only read.
  *
  * Limits: K <= 256, and the scratch the case needs (rkv_workspace_bytes of the
- * single-tensor case, which grows with n * K) must fit in 8 MiB; e.g. fp32,
- * n = 2^24 with K = 128, or n = 2^25 with K = 64, fit.  A larger case is rejected
+ * single-tensor case: about 48 bytes * K * 2 * SM count, whatever n is) must fit
+ * in 8 MiB; on a 148-SM part every K <= 256 fits.  A larger case is rejected
  * with RKV_ERR_UNSUPPORTED before anything is launched.  Other errors:
  * INVALID_ARG, ALIGNMENT, CUDA.
  *
@@ -258,9 +259,9 @@ int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, i
  * stream capture.
  *
  * All calls on a device share the one array, and it keeps whatever the previous
- * call left there.  The library rewrites the status word and the tables at the
- * start of every call and the kernels overwrite every partial result they later
- * read, so a call never depends on old contents.  Two calls whose work overlaps
+ * call left there.  The library rewrites the status word and the tables and
+ * clears the per-candidate state and the partial results at the start of every
+ * call (stream-ordered), so a call never depends on old contents.  Two calls whose work overlaps
  * on the GPU (different streams, or several host threads) race on the array and
  * give undefined results: run them one after the other.
  *
@@ -271,15 +272,21 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
                             float atol, float rtol, rkv_stats *stats_out, void *cuda_stream);
 
 /*
- * Host-only planning helper (no CUDA call): how a tensor is cut into slabs.
- * A slab is the run of elements whose reference (and input) one thread block
- * stages in shared memory and reuses for all K candidates.
- *   smem_bytes_per_elem  reference bytes + input bytes kept per element (2..8)
- *   num_sms              SM count of the device
- * Writes the slab length (a multiple of 128 elements) and the slab count.
+ * Host-only planning helper (no CUDA call): how the work of one tensor is cut.
+ * The tensor is cut into *n_tiles tiles of *tile_elems elements.  One work item is
+ * one tile against a part of the K candidates: a thread block keeps the tile's
+ * reference values in registers and streams that tile of each candidate of the
+ * part past them.  A large tensor has two groups of items: the first *warm_tiles
+ * tiles, with parts of *part_k_warm candidates (small, so that every resident
+ * block -- 2 per SM -- gets an item), are verified first; the running maxima and
+ * loophole flags they publish let the remaining tiles, with parts of
+ * *part_k_main (<= 64) candidates, skip nearly all rare-path work.  A smaller
+ * tensor has one group: *warm_tiles == *n_tiles and *part_k_main == 0.
+ *   num_sms   SM count of the device
+ * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, null), UNSUPPORTED (n >= 2^40).
  */
-int rkv_plan_slabs(uint64_t n, int smem_bytes_per_elem, int num_sms, uint32_t *slab_elems,
-                   uint64_t *n_slabs);
+int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t *tile_elems, uint32_t *n_tiles,
+                   uint32_t *warm_tiles, uint32_t *part_k_warm, uint32_t *part_k_main);
 
 /* Releases the library-owned scratch and staging buffers of all devices. */
 int rkv_release_cached(void);

@@ -101,9 +101,9 @@ def lib() -> ctypes.CDLL:
         L.rkv_verify_batch_host.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
         L.rkv_verify_batch_static.restype = i32
         L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
-        L.rkv_plan_slabs.restype = i32
-        L.rkv_plan_slabs.argtypes = [u64, i32, i32, ctypes.POINTER(ctypes.c_uint32),
-                                     ctypes.POINTER(ctypes.c_uint64)]
+        u32p = ctypes.POINTER(ctypes.c_uint32)
+        L.rkv_plan_items.restype = i32
+        L.rkv_plan_items.argtypes = [u64, i32, i32, u32p, u32p, u32p, u32p, u32p]
         L.rkv_release_cached.restype = i32
         L.rkv_release_cached.argtypes = []
         _lib = L
@@ -140,12 +140,13 @@ def set_stream(stream=None) -> None:
     _check(lib().rkv_set_stream(ctypes.c_void_p(_stream_ptr(stream))), "rkv_set_stream")
 
 
-def plan_slabs(n: int, smem_bytes_per_elem: int, num_sms: int) -> tuple:
-    """Host-only: (slab_elems, n_slabs) for a tensor of n elements."""
-    s, c = ctypes.c_uint32(), ctypes.c_uint64()
-    _check(lib().rkv_plan_slabs(int(n), int(smem_bytes_per_elem), int(num_sms),
-                                ctypes.byref(s), ctypes.byref(c)), "rkv_plan_slabs")
-    return int(s.value), int(c.value)
+def plan_items(n: int, K: int, num_sms: int) -> tuple:
+    """Host-only: (tile_elems, n_tiles, warm_tiles, part_k_warm, part_k_main) for a tensor of
+    n elements and K candidates."""
+    v = [ctypes.c_uint32() for _ in range(5)]
+    _check(lib().rkv_plan_items(int(n), int(K), int(num_sms), *[ctypes.byref(x) for x in v]),
+           "rkv_plan_items")
+    return tuple(int(x.value) for x in v)
 
 
 def gen_inputs(seed: int, dist: int, shape, dtype: torch.dtype = torch.float32,

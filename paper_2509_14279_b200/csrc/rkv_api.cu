@@ -14,34 +14,27 @@ namespace rkv {
 // planning
 // ----------------------------------------------------------------------------
 
-int smem_bytes_per_elem(const rkv_tensor_desc& t) {
-    // a generated reference is staged as fp32 whatever its dtype
-    const int rsz = (t.ref_src == RKV_SRC_POINTER && t.ref_dtype == RKV_BF16) ? 2 : 4;
-    const int isz = t.input_src == RKV_SRC_NONE ? 0 : (t.cand_dtype == RKV_BF16 ? 2 : 4);
-    return rsz + isz;
+// How one tensor is cut: tiles of kTileElems elements; a large tensor's first
+// kWarmTiles tiles form the warm-up group (see DevTensor).
+static int plan_one(uint64_t n, uint32_t* n_tiles, uint32_t* warm_tiles) {
+    if (n == 0 || n >= kMaxN) return RKV_ERR_INVALID_ARG;
+    const uint64_t tiles = (n + kTileElems - 1) / kTileElems;
+    if (tiles > 0x3FFFFFFFull) return RKV_ERR_UNSUPPORTED;
+    *n_tiles = (uint32_t)tiles;
+    *warm_tiles = tiles >= (uint64_t)kWarmMinTiles ? (uint32_t)kWarmTiles : (uint32_t)tiles;
+    return RKV_OK;
 }
 
-// Slab length: the smallest whole number of waves w of the resident grid
-// (num_sms * kBlocksPerSm blocks) such that n / (grid * w), rounded up to the
-// granule, fits the shared-memory budget.  Every block then gets the same number
-// of equally long slabs, so no wave is partly empty.
-static int plan_one(uint64_t n, int bytes_per_elem, int num_sms, uint32_t* slab_elems, uint64_t* n_slabs) {
-    if (n == 0 || n >= kMaxN || bytes_per_elem < 2 || bytes_per_elem > 8 || num_sms < 1)
-        return RKV_ERR_INVALID_ARG;
-    const uint64_t s_max = (uint64_t)(kSmemDataBudget / bytes_per_elem) / kSlabGranule * kSlabGranule;
-    const uint64_t grid = (uint64_t)num_sms * kBlocksPerSm;
-    uint64_t S = s_max;
-    // smallest number of waves whose slabs fit
-    uint64_t w = (n + grid * s_max - 1) / (grid * s_max);
-    if (w == 0) w = 1;
-    for (;; ++w) {
-        const uint64_t per = (n + grid * w - 1) / (grid * w);
-        const uint64_t s = (per + kSlabGranule - 1) / kSlabGranule * kSlabGranule;
-        if (s <= s_max) { S = s; break; }
+// Work items of one tensor for a launch over k_count candidates.
+static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t k_count, uint32_t grid) {
+    uint64_t items = 0;
+    const uint32_t groups[2] = {warm_tiles, n_tiles - warm_tiles};
+    for (int g = 0; g < 2; ++g) {
+        if (!groups[g]) continue;
+        const uint32_t pk = part_size(groups[g], k_count, grid);
+        items += (uint64_t)groups[g] * ((k_count + pk - 1) / pk);
     }
-    *slab_elems = (uint32_t)S;
-    *n_slabs = (n + S - 1) / S;
-    return RKV_OK;
+    return items;
 }
 
 static bool finite_nonneg(float x) { return x >= 0.0f && x <= 3.402823466e38f; }
@@ -83,30 +76,36 @@ int validate_tensors(const rkv_tensor_desc* tensors, int T, int K) {
     return RKV_OK;
 }
 
-int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* plan) {
-    uint64_t items = 0;
-    for (int v = 0; v < 8; ++v) plan->variant_items[v] = 0;
+static uint32_t variant_of(const rkv_tensor_desc& d) {
+    return (d.cand_dtype == RKV_BF16 ? 2u : 0u) +
+           ((d.ref_dtype == RKV_BF16 && d.ref_src == RKV_SRC_POINTER) ? 1u : 0u);
+}
+
+int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num_sms, Plan* plan) {
+    if (k_count < 1 || k_count > K) return RKV_ERR_INVALID_ARG;
+    const uint32_t grid = (uint32_t)(num_sms * kBlocksPerSm);
+    plan->grid = grid;
+    uint64_t rows = 0, total_items[4] = {0, 0, 0, 0};
     for (int t = 0; t < T; ++t) {
-        uint32_t S;
-        uint64_t ns;
-        const int rc = plan_one(tensors[t].n, smem_bytes_per_elem(tensors[t]), num_sms, &S, &ns);
+        uint32_t tiles, warm;
+        const int rc = plan_one(tensors[t].n, &tiles, &warm);
         if (rc != RKV_OK) return rc;
-        plan->slab_elems[t] = S;
-        plan->n_slabs[t] = (uint32_t)ns;
-        plan->first_item[t] = (uint32_t)items;
-        const rkv_tensor_desc& d = tensors[t];
-        const int variant = (d.cand_dtype == RKV_BF16 ? 4 : 0) +
-                            ((d.ref_dtype == RKV_BF16 && d.ref_src == RKV_SRC_POINTER) ? 2 : 0) +
-                            (d.input_src != RKV_SRC_NONE ? 1 : 0);
-        plan->variant_items[variant] += (uint32_t)ns;
-        items += ns;
-        if (items > 0xFFFFFFFFull / 2) return RKV_ERR_UNSUPPORTED;
+        plan->n_tiles[t] = tiles;
+        plan->warm_tiles[t] = warm;
+        plan->variant[t] = variant_of(tensors[t]);
+        const uint64_t items = items_of(tiles, warm, (uint32_t)k_count, grid);
+        total_items[plan->variant[t]] += items;
+        if (total_items[plan->variant[t]] > 0x7FFFFFFFull) return RKV_ERR_UNSUPPORTED;
+        // a tensor with a group B gets one row per block, a small one a row per item at most
+        plan->n_slots[t] = (warm < tiles || items >= grid) ? grid : (uint32_t)items;
+        plan->slot_base[t] = (uint32_t)rows;
+        rows += plan->n_slots[t];
     }
-    plan->total_items = (uint32_t)items;
     size_t table = (size_t)T * sizeof(DevTensor) + (size_t)T * (size_t)K * sizeof(void*);
     plan->table_bytes = (table + 255) / 256 * 256;
-    plan->partial_bytes = (size_t)items * (size_t)(K + 1) * sizeof(Partial);
-    plan->total_bytes = sizeof(WorkspaceHeader) + plan->table_bytes + plan->partial_bytes;
+    plan->state_bytes = ((size_t)T * (size_t)(K + 1) * sizeof(CandState) + 255) / 256 * 256;
+    plan->partial_bytes = (size_t)rows * (size_t)K * sizeof(Partial);
+    plan->total_bytes = sizeof(WorkspaceHeader) + plan->table_bytes + plan->state_bytes + plan->partial_bytes;
     return RKV_OK;
 }
 
@@ -153,47 +152,81 @@ int ensure(void** buf, size_t* have, size_t want) {
     return RKV_OK;
 }
 
-// Build the device tables in the workspace and launch verify (+ finalize).
-int run_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k_end, bool finalize,
-             bool upload, const Plan& plan, int num_sms, rkv_stats* stats_out, uint32_t* joint_pass,
-             void* workspace, cudaStream_t stream) {
+// Fill the device-side descriptor of tensor t.
+void fill_dev_tensor(DevTensor& d, const rkv_tensor_desc& s, const Plan& plan, int t, const void** d_ptrs, int K) {
+    memset(&d, 0, sizeof d);
+    d.n = s.n;
+    d.ref = s.ref_src == RKV_SRC_POINTER ? s.ref : nullptr;
+    d.input = s.input_src == RKV_SRC_POINTER ? s.input : nullptr;
+    d.cands = d_ptrs + (size_t)t * K;
+    d.ref_seed = s.ref_gen.seed; d.ref_stream = s.ref_gen.stream_id; d.ref_dist = s.ref_gen.dist;
+    d.in_seed = s.input_gen.seed; d.in_stream = s.input_gen.stream_id; d.in_dist = s.input_gen.dist;
+    d.cand_dtype = s.cand_dtype; d.ref_dtype = s.ref_dtype;
+    d.ref_src = s.ref_src; d.input_src = s.input_src;
+    d.atol = s.atol; d.rtol = s.rtol;
+    d.n_tiles = plan.n_tiles[t]; d.warm_tiles = plan.warm_tiles[t];
+    d.n_slots = plan.n_slots[t]; d.slot_base = plan.slot_base[t];
+    d.variant = plan.variant[t];
+}
+
+// Workspace pieces.
+struct Layout {
+    int32_t* status;
+    DevTensor* d_tensors;
+    const void** d_ptrs;
+    CandState* state;
+    Partial* partials;
+};
+
+Layout layout_of(void* workspace, const Plan& plan, int T) {
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
-    DevTensor* d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
-    const void** d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) +
-                                                         (size_t)T * sizeof(DevTensor));
-    Partial* partials = reinterpret_cast<Partial*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
-    int32_t* status = reinterpret_cast<int32_t*>(ws);
+    Layout L;
+    L.status = reinterpret_cast<int32_t*>(ws);
+    L.d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
+    L.d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) + (size_t)T * sizeof(DevTensor));
+    L.state = reinterpret_cast<CandState*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
+    L.partials = reinterpret_cast<Partial*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes + plan.state_bytes);
+    return L;
+}
+
+// Launch verify over candidates [k_begin, k_end) (+ finalize); the tables must be in place.
+int launch_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k_end, bool finalize,
+                const Plan& plan, const Layout& L, rkv_stats* stats_out, uint32_t* joint_pass,
+                cudaStream_t stream) {
+    uint32_t items[4] = {0, 0, 0, 0};
+    const uint32_t kcount = (uint32_t)(k_end - k_begin);
+    for (int t = 0; t < T; ++t)
+        items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], kcount, plan.grid);
+    (void)tensors;
+    int rc = launch_verify(L.d_tensors, T, K, k_begin, k_end, items, (int)plan.grid, L.state, L.partials,
+                           L.status, stream);
+    if (rc != RKV_OK) return rc;
+    if (finalize) rc = launch_finalize(L.d_tensors, T, K, L.state, L.partials, stats_out, joint_pass, stream);
+    return rc;
+}
+
+// Build the device tables in the workspace, clear the per-candidate state and the
+// partials, and launch verify (+ finalize).
+int run_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k_end, bool finalize,
+             bool upload, const Plan& plan, rkv_stats* stats_out, uint32_t* joint_pass, void* workspace,
+             cudaStream_t stream) {
+    const Layout L = layout_of(workspace, plan, T);
     if (upload) {
         std::vector<unsigned char> blob(sizeof(WorkspaceHeader) + plan.table_bytes, 0);
         DevTensor* h_t = reinterpret_cast<DevTensor*>(blob.data() + sizeof(WorkspaceHeader));
         const void** h_p = reinterpret_cast<const void**>(blob.data() + sizeof(WorkspaceHeader) +
                                                           (size_t)T * sizeof(DevTensor));
         for (int t = 0; t < T; ++t) {
-            const rkv_tensor_desc& s = tensors[t];
-            DevTensor& d = h_t[t];
-            d.n = s.n;
-            d.ref = s.ref_src == RKV_SRC_POINTER ? s.ref : nullptr;
-            d.input = s.input_src == RKV_SRC_POINTER ? s.input : nullptr;
-            d.cands = d_ptrs + (size_t)t * K;
-            d.ref_seed = s.ref_gen.seed; d.ref_stream = s.ref_gen.stream_id; d.ref_dist = s.ref_gen.dist;
-            d.in_seed = s.input_gen.seed; d.in_stream = s.input_gen.stream_id; d.in_dist = s.input_gen.dist;
-            d.cand_dtype = s.cand_dtype; d.ref_dtype = s.ref_dtype;
-            d.ref_src = s.ref_src; d.input_src = s.input_src;
-            d.atol = s.atol; d.rtol = s.rtol;
-            d.slab_elems = plan.slab_elems[t]; d.n_slabs = plan.n_slabs[t];
-            d.first_item = plan.first_item[t];
-            for (int k = 0; k < K; ++k) h_p[(size_t)t * K + k] = s.cands[k];
+            fill_dev_tensor(h_t[t], tensors[t], plan, t, L.d_ptrs, K);
+            for (int k = 0; k < K; ++k) h_p[(size_t)t * K + k] = tensors[t].cands[k];
         }
-        if (cudaMemcpyAsync(ws, blob.data(), blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        if (cudaMemcpyAsync(workspace, blob.data(), blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemsetAsync(L.state, 0, plan.state_bytes + plan.partial_bytes, stream) != cudaSuccess) {
             cudaGetLastError();
             return RKV_ERR_CUDA;
         }
     }
-    int rc = launch_verify(d_tensors, T, K, k_begin, k_end, plan.variant_items, num_sms, partials, status,
-                           stream);
-    if (rc != RKV_OK) return rc;
-    if (finalize) rc = launch_finalize(d_tensors, T, K, partials, stats_out, joint_pass, stream);
-    return rc;
+    return launch_case(tensors, T, K, k_begin, k_end, finalize, plan, L, stats_out, joint_pass, stream);
 }
 
 }  // namespace
@@ -226,11 +259,18 @@ int rkv_set_stream(void* cuda_stream) {
     return RKV_OK;
 }
 
-int rkv_plan_slabs(uint64_t n, int smem_bytes_per_elem, int num_sms, uint32_t* slab_elems,
-                   uint64_t* n_slabs) {
-    if (!slab_elems || !n_slabs) return RKV_ERR_INVALID_ARG;
+int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t* tile_elems, uint32_t* n_tiles,
+                   uint32_t* warm_tiles, uint32_t* part_k_warm, uint32_t* part_k_main) {
+    if (!tile_elems || !n_tiles || !warm_tiles || !part_k_warm || !part_k_main) return RKV_ERR_INVALID_ARG;
     if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
-    return plan_one(n, smem_bytes_per_elem, num_sms, slab_elems, n_slabs);
+    if (K < 1 || num_sms < 1 || num_sms > (1 << 20)) return RKV_ERR_INVALID_ARG;
+    const int rc = plan_one(n, n_tiles, warm_tiles);
+    if (rc != RKV_OK) return rc;
+    const uint32_t grid = (uint32_t)(num_sms * kBlocksPerSm);
+    *tile_elems = kTileElems;
+    *part_k_warm = part_size(*warm_tiles, (uint32_t)K, grid);
+    *part_k_main = *warm_tiles < *n_tiles ? part_size(*n_tiles - *warm_tiles, (uint32_t)K, grid) : 0u;
+    return RKV_OK;
 }
 
 int rkv_gen_inputs_ex(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t first_elem,
@@ -264,7 +304,7 @@ size_t rkv_workspace_bytes(const rkv_tensor_desc* tensors, int T, int K) {
     int sms = 0;
     if (current_num_sms(&sms) != RKV_OK) return 0;
     Plan plan;
-    if (make_plan(tensors, T, K, sms, &plan) != RKV_OK) return 0;
+    if (make_plan(tensors, T, K, K, sms, &plan) != RKV_OK) return 0;
     return plan.total_bytes;
 }
 
@@ -279,10 +319,10 @@ int rkv_verify_multi(const rkv_tensor_desc* tensors, int T, int K, rkv_stats* st
     rc = current_num_sms(&sms);
     if (rc != RKV_OK) return rc;
     Plan plan;
-    rc = make_plan(tensors, T, K, sms, &plan);
+    rc = make_plan(tensors, T, K, K, sms, &plan);
     if (rc != RKV_OK) return rc;
     if (workspace_bytes < plan.total_bytes) return RKV_ERR_WORKSPACE;
-    return run_case(tensors, T, K, 0, K, true, true, plan, sms, stats_out, joint_pass, workspace,
+    return run_case(tensors, T, K, 0, K, true, true, plan, stats_out, joint_pass, workspace,
                     reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -301,7 +341,7 @@ int rkv_verify_batch(const void* ref, const void* const* cands, int K, uint64_t 
     rc = current_num_sms(&sms);
     if (rc != RKV_OK) return rc;
     Plan plan;
-    rc = make_plan(&d, 1, K, sms, &plan);
+    rc = make_plan(&d, 1, K, K, sms, &plan);
     if (rc != RKV_OK) return rc;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -309,7 +349,7 @@ int rkv_verify_batch(const void* ref, const void* const* cands, int K, uint64_t 
     DeviceCache& c = g_cache[dev & 63];
     rc = ensure(&c.workspace, &c.workspace_bytes, plan.total_bytes);
     if (rc != RKV_OK) return rc;
-    return run_case(&d, 1, K, 0, K, true, true, plan, sms, stats_out, nullptr, c.workspace, g_stream);
+    return run_case(&d, 1, K, 0, K, true, true, plan, stats_out, nullptr, c.workspace, g_stream);
 }
 
 int rkv_device_status(const void* workspace, void* cuda_stream) {
@@ -376,7 +416,7 @@ int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, i
     d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
     d.atol = atol; d.rtol = rtol;
     Plan plan;
-    rc = make_plan(&d, 1, K, sms, &plan);
+    rc = make_plan(&d, 1, K, (int)kc, sms, &plan);
     if (rc != RKV_OK) return rc;
     rc = ensure(&c.workspace, &c.workspace_bytes, plan.total_bytes);
     if (rc != RKV_OK) return rc;
@@ -397,7 +437,7 @@ int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, i
         fail |= cudaEventRecord(c.copied[b], c.copy_stream[b]) != cudaSuccess;
         fail |= cudaStreamWaitEvent(main, c.copied[b], 0) != cudaSuccess;
         if (fail) break;
-        rc = run_case(&d, 1, K, k0, k1, k1 == K, ch == 0, plan, sms, d_stats, nullptr, c.workspace, main);
+        rc = run_case(&d, 1, K, k0, k1, k1 == K, ch == 0, plan, d_stats, nullptr, c.workspace, main);
         if (rc != RKV_OK) { fail = true; break; }
         fail |= cudaEventRecord(c.consumed[b], main) != cudaSuccess;
     }
@@ -470,7 +510,7 @@ int rkv_verify_batch_static(const void* ref, const void* const* cands, int K, ui
     rc = current_num_sms(&sms);
     if (rc != RKV_OK) return rc;
     Plan plan;
-    rc = make_plan(&d, 1, K, sms, &plan);
+    rc = make_plan(&d, 1, K, K, sms, &plan);
     if (rc != RKV_OK) return rc;
     if (plan.total_bytes > kStaticScratchBytes) return RKV_ERR_UNSUPPORTED;
     void* scratch = nullptr;
@@ -484,32 +524,20 @@ int rkv_verify_batch_static(const void* ref, const void* const* cands, int K, ui
     const size_t blob_bytes = sizeof(WorkspaceHeader) + plan.table_bytes;
     if (blob_bytes > kBlobMax) return RKV_ERR_UNSUPPORTED;
     memset(blob, 0, blob_bytes);
-    unsigned char* ws = reinterpret_cast<unsigned char*>(scratch);
-    DevTensor* d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
-    const void** d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) + sizeof(DevTensor));
-    Partial* partials = reinterpret_cast<Partial*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
-    DevTensor* h_t = reinterpret_cast<DevTensor*>(blob + sizeof(WorkspaceHeader));
+    const Layout L = layout_of(scratch, plan, 1);
+    fill_dev_tensor(*reinterpret_cast<DevTensor*>(blob + sizeof(WorkspaceHeader)), d, plan, 0, L.d_ptrs, K);
     const void** h_p = reinterpret_cast<const void**>(blob + sizeof(WorkspaceHeader) + sizeof(DevTensor));
-    h_t->n = n;
-    h_t->ref = ref;
-    h_t->input = nullptr;
-    h_t->cands = d_ptrs;
-    h_t->cand_dtype = dtype; h_t->ref_dtype = dtype;
-    h_t->ref_src = RKV_SRC_POINTER; h_t->input_src = RKV_SRC_NONE;
-    h_t->atol = atol; h_t->rtol = rtol;
-    h_t->slab_elems = plan.slab_elems[0]; h_t->n_slabs = plan.n_slabs[0];
-    h_t->first_item = plan.first_item[0];
     for (int k = 0; k < K; ++k) h_p[k] = cands[k];
 
+    // what must start at zero in the shared array: the status word (in the blob), the
+    // per-candidate state and the partial results
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemcpyAsync(ws, blob, blob_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    if (cudaMemcpyAsync(scratch, blob, blob_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemsetAsync(L.state, 0, plan.state_bytes + plan.partial_bytes, stream) != cudaSuccess) {
         cudaGetLastError();
         return RKV_ERR_CUDA;
     }
-    rc = launch_verify(d_tensors, 1, K, 0, K, plan.variant_items, sms, partials,
-                       reinterpret_cast<int32_t*>(ws), stream);
-    if (rc != RKV_OK) return rc;
-    return launch_finalize(d_tensors, 1, K, partials, stats_out, nullptr, stream);
+    return launch_case(&d, 1, K, 0, K, true, plan, L, stats_out, nullptr, stream);
 }
 
 int rkv_release_cached(void) {

@@ -9,31 +9,49 @@
 
 namespace rkv {
 
-constexpr int kThreads = 256;          // threads per verification block
-constexpr int kBlocksPerSm = 2;        // resident verification blocks per SM
-constexpr int kSlabGranule = 128;      // slab lengths are multiples of this many elements
-constexpr int kSmemDataBudget = 96 * 1024;  // bytes of reference + input one block stages
-constexpr int kChunkK = 16;            // candidates between two block-level merges
-constexpr int kPreK = 512;             // candidates whose pointer and first element are preloaded
-constexpr int kHintK = 256;            // candidates with a cross-slab threshold hint
+// ---- verification kernel geometry ------------------------------------------------
+constexpr int kConsumerWarps = 7;                    // warps that compare
+constexpr int kConsumers = kConsumerWarps * 32;      // 224 threads
+constexpr int kThreads = kConsumers + 32;            // + one warp that issues the bulk copies = 256
+constexpr int kBlocksPerSm = 2;                      // resident verification blocks per SM
+constexpr int kElemsPerThread = 16;                  // elements of a tile one thread owns
+constexpr int kTileElems = kConsumers * kElemsPerThread;   // 3584 elements per tile
+constexpr int kStageBytes = kTileElems * 4;          // one ring stage holds a tile of fp32
+constexpr int kStages = 6;                           // ring depth (bulk copies in flight)
+constexpr int kPartK = 64;                           // candidates a block tracks at a time
+constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
+constexpr int kWarmMinTiles = 2048;                  // tensors with fewer tiles have no warm-up group
 constexpr int kMaxTensors = 64;
 constexpr uint64_t kMaxN = 1ull << 40;
 
-// Per (slab, candidate) partial result; also the per-warp record in shared memory.
+// Result of one thread block for one (tensor, candidate); merged by the finalize kernel.
 struct __align__(16) Partial {
-    uint32_t n_over;
-    uint32_t n_noncomp;
-    uint32_t n_nan;
-    uint32_t n_inf;
-    uint32_t n_infmis;
-    uint32_t mismatch;   // bit0: some element differs from element 0; bit1: differs from input
-    float emax;          // -1 when no comparable element beat the hint
-    uint32_t eidx;       // slab-local index
-    float qmax;
-    uint32_t qidx;
+    uint64_t n_over;
+    uint64_t eidx;       // tensor-wide element index of the first maximum of |c - r|
+    uint64_t qidx;       // same for |c - r| / |r|
     double sum;
+    float emax;          // -1 when the block saw no comparable element
+    float qmax;
+    uint32_t valid;      // 0 in the zero-filled workspace, 1 once a block has written the slot
+    uint32_t reserved;
 };
 static_assert(sizeof(Partial) == 48, "Partial layout");
+
+// Global per-(tensor, candidate) state, zero-filled before the launch.  Slot K of
+// a tensor belongs to the reference (only `mismatch` is used there).
+struct __align__(16) CandState {
+    // Running maxima published by all blocks, only ever used to skip work:
+    // ((bits(max) + 1) << 32) | ~tile, 0 = nothing published yet.
+    unsigned long long hint_e;
+    unsigned long long hint_q;
+    unsigned long long n_noncomp;   // elements that are not comparable
+    unsigned long long n_nan;
+    unsigned long long n_inf;
+    unsigned long long n_infmis;
+    uint32_t mismatch;              // bit0: some element differs from element 0; bit1: from the input
+    uint32_t reserved[3];
+};
+static_assert(sizeof(CandState) == 64, "CandState layout");
 
 // Device-side description of one tensor of a case.
 struct DevTensor {
@@ -47,10 +65,20 @@ struct DevTensor {
     int32_t cand_dtype, ref_dtype;
     int32_t ref_src, input_src;
     float atol, rtol;
-    uint32_t slab_elems;
-    uint32_t n_slabs;
-    uint32_t first_item;
-    uint32_t reserved;
+    // Work items.  A large tensor has two groups of items: group A covers its first
+    // warm_tiles tiles with small candidate parts (so that all blocks take part), group B
+    // the remaining tiles with parts of up to kPartK candidates.  Group A runs first: the
+    // maxima and loophole flags it publishes let group B skip almost all rare-path work.
+    // Smaller tensors only have group A.  Within a group item = part * tiles + tile, with
+    // part_size() candidates per part.
+    // Items of the tensors of one storage variant are numbered consecutively, all A
+    // groups before all B groups; block b takes items b, b + grid, ...
+    uint32_t n_tiles;       // ceil(n / kTileElems)
+    uint32_t warm_tiles;    // tiles in group A (== n_tiles when there is no group B)
+    uint32_t n_slots;       // Partial rows of this tensor
+    uint32_t slot_base;     // first Partial row (K entries per row) of this tensor
+    uint32_t variant;       // 2 * (candidates bf16) + (reference stored as bf16)
+    uint32_t reserved[3];
 };
 
 struct WorkspaceHeader {
@@ -59,30 +87,46 @@ struct WorkspaceHeader {
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header size");
 
+// How a case is cut into work items, and where everything lives in the workspace:
+//   header | tensor descriptors + pointer tables | CandState[T][K+1] | Partial[rows][K]
 struct Plan {
-    uint32_t slab_elems[kMaxTensors];
-    uint32_t n_slabs[kMaxTensors];
-    uint32_t first_item[kMaxTensors];
-    uint32_t total_items;
-    uint32_t variant_items[8];
+    uint32_t n_tiles[kMaxTensors];
+    uint32_t warm_tiles[kMaxTensors];
+    uint32_t n_slots[kMaxTensors];
+    uint32_t slot_base[kMaxTensors];
+    uint32_t variant[kMaxTensors];
+    uint32_t grid;          // blocks per launch (num_sms * kBlocksPerSm)
     size_t table_bytes;     // descriptors + pointer tables, rounded to 256
+    size_t state_bytes;     // CandState region, rounded to 256
     size_t partial_bytes;
     size_t total_bytes;
 };
 
-int smem_bytes_per_elem(const rkv_tensor_desc& t);
 int validate_tensors(const rkv_tensor_desc* tensors, int T, int K);
-int make_plan(const rkv_tensor_desc* tensors, int T, int K, int num_sms, Plan* plan);
+// k_count: candidates one launch covers (K, or the chunk length of the host-buffer form)
+int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num_sms, Plan* plan);
 int current_num_sms(int* num_sms);   // RKV_ERR_CUDA without a device
 
+// Candidates per part for `tiles` tiles and a launch over k_count candidates: balanced
+// parts of at most kPartK, more and smaller ones when there are fewer tiles than blocks.
+// The kernels and the host use this one rule.
+__host__ __device__ inline uint32_t part_size(uint32_t tiles, uint32_t k_count, uint32_t grid) {
+    uint32_t parts = (k_count + kPartK - 1) / kPartK;
+    if (tiles < grid) {
+        const uint32_t want = (grid + tiles - 1) / tiles;
+        if (want > parts) parts = want;
+    }
+    if (parts > k_count) parts = k_count;
+    return (k_count + parts - 1) / parts;
+}
+
 // kernels (rkv_verify.cu / rkv_gen.cu)
-// variant_items[v]: slabs of the tensors whose storage variant is v =
-// 4*(candidates bf16) + 2*(reference staged as bf16) + (input present)
 int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
-                  const uint32_t variant_items[8], int num_sms, Partial* partials, int32_t* status,
-                  cudaStream_t stream);
-int launch_finalize(const DevTensor* d_tensors, int T, int K, const Partial* partials,
-                    rkv_stats* stats_out, uint32_t* joint_pass, cudaStream_t stream);
+                  const uint32_t variant_items[4], int grid, CandState* state, Partial* partials,
+                  int32_t* status, cudaStream_t stream);
+int launch_finalize(const DevTensor* d_tensors, int T, int K, const CandState* state,
+                    const Partial* partials, rkv_stats* stats_out, uint32_t* joint_pass,
+                    cudaStream_t stream);
 int launch_gen(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t first_elem,
                int dtype, void* out, int num_sms, cudaStream_t stream);
 

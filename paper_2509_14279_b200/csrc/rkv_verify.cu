@@ -1,25 +1,36 @@
 // Fused single-pass verification kernel and its finalize kernel (sm_100a).
 //
-// Work decomposition.  Every tensor is cut into slabs (runs of at most ~12-24 K
-// elements, a multiple of 128).  A persistent thread block takes slabs round
-// robin.  For a slab it stages the reference (and the input tensor, when the
-// copy-of-input flag is wanted) in shared memory ONCE -- by a bulk asynchronous
-// copy (cp.async.bulk, completion on an mbarrier) or by regenerating it from its
-// Philox stream -- and then streams the same slab of all K candidates from HBM
-// with 128-bit read-once loads.  Candidate bytes are the only traffic that
-// scales with K; the reference costs 1/K of it.
+// Work decomposition.  A tensor is cut into tiles of 3584 elements; the K
+// candidates into parts of at most 64.  A work item is (tensor, part, tile).
+// A persistent thread block takes items round robin.  It has two roles:
 //
-// Per element the fast path is: one subtraction, the tolerance product and sum
-// (two separately rounded operations), a compare, a running maximum, a filter
-// for the relative-error maximum, two xor/or accumulations for the loophole
-// flags.  Anything non-finite makes the 4- or 8-element vector sum non-finite,
-// which sends that vector down the general path; a slab whose reference holds a
-// non-finite value uses the general path throughout.
+//   * one producer warp: a single thread issues bulk asynchronous copies
+//     (cp.async.bulk, completion counted on an mbarrier) that bring, for the
+//     item, the reference tile and then the same tile of every candidate of the
+//     part into a ring of shared-memory stages.  Several stages are in flight,
+//     so the copies of later candidates overlap the comparison of earlier ones;
+//   * seven consumer warps: each thread owns 16 elements of the tile.  It keeps
+//     their reference values and tolerance thresholds IN REGISTERS for the
+//     whole item and meets every candidate tile as it lands in the ring.
+//
+// Candidate bytes are read from HBM exactly once; the reference once per part.
+// When the reference is "generated" the threads regenerate their 16 values from
+// the Philox stream instead of reading them (fused generate + verify).
+//
+// Per element the common path is one subtraction, one running maximum and one
+// addition.  Counting the elements over tolerance, locating maxima, dividing for
+// the relative error and everything about non-finite values sit behind
+// predicates evaluated once per thread, candidate and tile:
+//   m > min thr              some element may be over tolerance  -> count them
+//   !(sum < inf)             a non-finite value                  -> general rule
+//   m beats/ties the hint    a new maximum is possible           -> locate it
+// The hints are running maxima that all blocks publish in global memory with
+// their tile number.  A hint only ever lets a thread skip elements that cannot
+// be the first maximum (see consider_maxima), so results do not depend on when a
+// hint becomes visible.
 //
 // Reductions are deterministic: integer sums, lexicographic (value descending,
-// index ascending) maxima, and a fixed-order fp64 sum.  No float atomics.
-#include <type_traits>
-
+// index ascending) maxima, fixed-order floating-point sums.  No float atomics.
 #include "rkv_internal.h"
 #include "rkv_philox.cuh"
 
@@ -27,25 +38,46 @@ namespace rkv {
 
 namespace {
 
-constexpr int kWarps = kThreads / 32;
-constexpr int kGroupK = 2;        // candidates processed per pass over a reference vector
-constexpr int kLoadsF32 = 2;      // 16-byte candidate loads per thread, candidate and batch (fp32)
-constexpr int kLoadsBf16 = 2;     // same for bf16 candidates
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
+constexpr int E = kElemsPerThread;
+constexpr float kInf = __builtin_huge_valf();
 
 // ----------------------------------------------------------------------------
-// shared-memory layout
+// shared-memory layout (dynamic)
 // ----------------------------------------------------------------------------
-constexpr int kOffMbar = 0;                               // 8 bytes
-constexpr int kOffHintE = 64;
-constexpr int kOffHintQ = kOffHintE + kHintK * 4;
-constexpr int kOffHintF = kOffHintQ + kHintK * 4;
-constexpr int kOffWarpPart = kOffHintF + kHintK * 4;      // 16-aligned
-constexpr int kOffCandPtr = kOffWarpPart + kChunkK * kWarps * (int)sizeof(Partial);
-constexpr int kOffCandFirst = kOffCandPtr + kPreK * 8;
-constexpr int kOffDataRaw = kOffCandFirst + kPreK * 4;
-constexpr int kOffData = (kOffDataRaw + 127) / 128 * 128;
-static_assert(kOffWarpPart % 16 == 0, "warp partials must be 16-byte aligned");
+// Per (warp, candidate of the part) running result.
+struct __align__(16) WarpRec {
+    float emax; uint32_t etile;
+    float qmax; uint32_t qtile;
+    uint32_t offs;           // eoff | qoff << 16 : element offsets inside their tiles
+    uint32_t n_over;
+    double sum;
+};
+static_assert(sizeof(WarpRec) == 32, "WarpRec layout");
+
+// Per candidate of the part, refreshed from global memory at the start of an item.
+struct __align__(16) Hint {
+    float te; uint32_t te_tile;      // published maximum of |c - r| and its tile (-1 / 0 if none)
+    float tq; uint32_t tq_tile;      // same for the relative error
+    float tq_pred;                   // largest float below tq (-1 when tq <= 0)
+    uint32_t settled;                // bit0: known to differ from element 0; bit1: from the input
+    uint32_t first;                  // storage bits of the candidate's element 0
+    uint32_t pad;
+};
+static_assert(sizeof(Hint) == 32, "Hint layout");
+
+constexpr int kOffFull = 0;                                   // kStages mbarriers
+constexpr int kOffEmpty = kOffFull + 8 * kStages;
+constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
+constexpr int kOffRefState = kOffAbort + 16;                  // 2 x uint32 settled bits of the reference (item parity)
+constexpr int kOffPtrC = 128;                                 // consumer copy of the pointers
+constexpr int kOffPtrP = kOffPtrC + kPartK * 8;               // producer copy
+constexpr int kOffHint = kOffPtrP + kPartK * 8;               // two tables (item parity)
+constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
+constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
+constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
+static_assert(kOffPtrC >= kOffRefState + 8, "layout");
+static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
 // ----------------------------------------------------------------------------
 // small PTX helpers
@@ -63,6 +95,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
                  : "memory");
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+
 __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -75,6 +111,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
     return ok != 0;
 }
 
+// Bounded wait.  Returns false when the wait ran out (about a second) or when
+// another thread of the block has already given up; the block then drains: every
+// later wait returns at once, all barriers are still reached, and the status
+// word tells the host that the results are void.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t mbar, uint32_t parity, volatile uint32_t* abort_flag) {
+    const long long t0 = clock64();
+    for (uint32_t spin = 0; spin < (1u << 26); ++spin) {
+        if (mbar_try_wait(mbar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > 2000000000LL) break;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (mbar_try_wait(mbar, parity)) return true;
+    return mbar_wait_slow(mbar, parity, abort_flag);
+}
+
 // Bulk asynchronous copy global -> this block's shared memory; bytes is a
 // multiple of 16, both addresses 16-byte aligned.  No multicast.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
@@ -84,724 +140,726 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         : "memory");
 }
 
-// 128-bit read-once load of candidate data: no L1 allocation.
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+// Barrier among the consumer threads only (the producer warp never joins).
+__device__ __forceinline__ void consumer_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
 }
 
 __device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
 __device__ __forceinline__ bool bits_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
 __device__ __forceinline__ bool bits_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
 
-// ----------------------------------------------------------------------------
-// per-thread accumulators for one (slab, candidate)
-// ----------------------------------------------------------------------------
-struct Acc {
-    uint32_t n_over;
-    float emax; uint32_t eidx; float ethr;
-    float qmax; uint32_t qidx; float qthr;
-    double sum;
-    uint32_t cacc, pacc;
-    // four 8-bit counters (a thread sees < 256 elements of one slab):
-    // byte 0 non-comparable, 1 NaN, 2 Inf, 3 infinity mismatch
-    uint32_t rare;
-};
-
-__device__ __forceinline__ void acc_reset(Acc& a, float hint_e, float hint_q) {
-    a.n_over = 0;
-    a.emax = -1.0f; a.eidx = 0xFFFFFFFFu; a.ethr = hint_e;
-    a.qmax = -1.0f; a.qidx = 0xFFFFFFFFu; a.qthr = hint_q;
-    a.sum = 0.0;
-    a.cacc = 0; a.pacc = 0;
-    a.rare = 0;
+__device__ __forceinline__ uint32_t ld_elem_bits(const void* base, int dtype, uint64_t i) {
+    if (dtype == RKV_BF16) return (uint32_t)reinterpret_cast<const uint16_t*>(base)[i] << 16;
+    return reinterpret_cast<const uint32_t*>(base)[i];
 }
 
+// ----------------------------------------------------------------------------
+// work items
+// ----------------------------------------------------------------------------
+struct Item {
+    int t;
+    uint32_t group;          // 0 = A (leading tiles, small parts), 1 = B
+    uint32_t part, tile;     // tile is the tensor-wide tile index
+    uint32_t part_k;         // candidates per part in this group
+    uint32_t first_item;     // first item of this (tensor, group) in this launch
+    uint32_t n_items;        // items of this (tensor, group)
+};
+
+// Item `id` of this launch among the tensors of `variant`; false past the end.
+__device__ __forceinline__ bool decode_item(const DevTensor* __restrict__ tensors, int T, uint32_t variant,
+                                            uint32_t k_count, uint32_t id, Item& it) {
+    uint32_t base = 0;
+    for (uint32_t g = 0; g < 2; ++g) {
+        for (int t = 0; t < T; ++t) {
+            if (tensors[t].variant != variant) continue;
+            const uint32_t warm = tensors[t].warm_tiles;
+            const uint32_t nt = g == 0 ? warm : tensors[t].n_tiles - warm;
+            if (nt == 0) continue;
+            const uint32_t pk = part_size(nt, k_count, gridDim.x);
+            const uint32_t cnt = nt * ((k_count + pk - 1) / pk);
+            if (id - base < cnt) {
+                it.t = t;
+                it.group = g;
+                it.part = (id - base) / nt;
+                it.tile = (id - base) % nt + (g == 0 ? 0u : warm);
+                it.part_k = pk;
+                it.first_item = base;
+                it.n_items = cnt;
+                return true;
+            }
+            base += cnt;
+        }
+    }
+    return false;
+}
+
+// ----------------------------------------------------------------------------
+// producer warp: feeds the ring
+// ----------------------------------------------------------------------------
+struct Ring {
+    uint32_t full0, empty0;      // shared-memory addresses of the first full / empty mbarrier
+    uint32_t stage0;             // shared-memory address of stage 0
+    volatile uint32_t* abort_flag;
+};
+
+template <bool CB16, bool RB16>
+__device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tensors, int T, int k_begin,
+                                              int k_end, uint32_t n_items, unsigned char* smem,
+                                              const Ring& ring) {
+    constexpr uint32_t CSZ = CB16 ? 2 : 4, RSZ = RB16 ? 2 : 4;
+    constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
+    const int lane = threadIdx.x & 31;
+    const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrP);
+    uint32_t n_issued = 0;
+    int cur_t = -1;
+    uint32_t cur_part = 0xFFFFFFFFu;
+
+    auto issue = [&](const unsigned char* src, uint32_t bytes) {
+        const uint32_t s = n_issued % kStages;
+        const uint32_t ph = (n_issued / kStages) & 1u;
+        // the stage is free once every consumer warp has released its previous use
+        mbar_wait(ring.empty0 + 8 * s, ph ^ 1u, ring.abort_flag);
+        if (bytes) {
+            mbar_expect_tx(ring.full0 + 8 * s, bytes);
+            bulk_g2s(ring.stage0 + s * kStageBytes, src, bytes, ring.full0 + 8 * s);
+        } else {
+            mbar_arrive(ring.full0 + 8 * s);
+        }
+        ++n_issued;
+    };
+
+    for (uint32_t id = blockIdx.x; id < n_items; id += gridDim.x) {
+        Item it;
+        if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
+        const DevTensor& D = tensors[it.t];
+        const int k0 = k_begin + (int)(it.part * it.part_k);
+        const int k1 = min(k_end, k0 + (int)it.part_k);
+        const uint32_t part_key = (it.group << 31) | it.part;
+        if (it.t != cur_t || part_key != cur_part) {
+            __syncwarp();
+            for (int k = k0 + lane; k < k1; k += 32)
+                ptrs[k - k0] = reinterpret_cast<const unsigned char*>(D.cands[k]);
+            __syncwarp();
+            cur_t = it.t;
+            cur_part = part_key;
+        }
+        if (lane == 0) {
+            const uint64_t start = (uint64_t)it.tile * kTileElems;
+            const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
+            if (D.ref_src == RKV_SRC_POINTER)
+                issue(reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ, (len * RSZ) & ~15u);
+            const uint32_t cbytes = (len * CSZ) & ~15u;
+            for (int k = k0; k < k1; ++k) issue(ptrs[k - k0] + start * CSZ, cbytes);
+        }
+    }
+    // A block that gave up must not retire with copies still landing in its shared
+    // memory: wait (bounded) for the copies issued last.
+    if (lane == 0 && *ring.abort_flag) {
+        const uint32_t pending = n_issued < (uint32_t)kStages ? n_issued : (uint32_t)kStages;
+        for (uint32_t i = 0; i < pending; ++i) {
+            const uint32_t q = n_issued - 1 - i;
+            const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
+            const long long t0 = clock64();
+            for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+                if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
+                if (clock64() - t0 > 200000000LL) break;
+            }
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------
+// consumer side: per-thread view of a tile
+// ----------------------------------------------------------------------------
+// A thread owns E = 16 elements of the tile as NV vectors of VEC elements
+// (one 16-byte piece of a candidate each): vector jv of thread tid is vector
+// jv * 224 + tid of the tile.  Element j = jv * VEC + i of the thread has the
+// tile offset below; offsets grow with j.
+template <int VEC>
+__device__ __forceinline__ uint32_t elem_off(int j, int tid) {
+    return (uint32_t)(((j / VEC) * kConsumers + tid) * VEC + (j % VEC));
+}
+
+// What a thread keeps for the whole item.
+struct RefRegs {
+    float r[E];        // reference values
+    float thr[E];      // atol + rtol*|r|, product and sum each rounded
+    float thr_min;     // smallest threshold of the thread's elements
+    float minarp;      // smallest non-zero |r|, +inf if all are zero
+    bool general;      // a non-finite reference value, or a ragged tile: element-by-element rule
+};
+
 // The comparison rule for one element, every case included.
-__device__ __forceinline__ void elem_general(Acc& a, uint32_t cb, uint32_t rb, uint32_t idx, float atol,
+struct LaneGen {
+    uint32_t n_over, n_noncomp, n_nan, n_inf, n_infmis;
+    float emax; uint32_t eoff;
+    float qmax; uint32_t qoff;
+    double sum;
+};
+
+__device__ __forceinline__ void elem_general(LaneGen& a, uint32_t cb, uint32_t rb, uint32_t off, float atol,
                                              float rtol) {
-    if (bits_nan(cb)) a.rare += 1u << 8;
-    if (bits_inf(cb)) a.rare += 1u << 16;
+    if (bits_nan(cb)) a.n_nan++;
+    if (bits_inf(cb)) a.n_inf++;
     if (bits_finite(cb) && bits_finite(rb)) {
         const float c = __uint_as_float(cb), r = __uint_as_float(rb);
         const float e = fabsf(__fsub_rn(c, r));
         const float thr = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r)));
         if (!(e <= thr)) a.n_over++;
-        if (e > a.emax) { a.emax = e; a.eidx = idx; }
+        if (e > a.emax) { a.emax = e; a.eoff = off; }
         if (r != 0.0f) {
             const float q = __fdiv_rn(e, fabsf(r));
-            if (q > a.qmax) { a.qmax = q; a.qidx = idx; }
+            if (q > a.qmax) { a.qmax = q; a.qoff = off; }
         }
         a.sum += (double)e;
     } else if (bits_inf(cb) && cb == rb) {
-        a.rare += 1u;
+        a.n_noncomp++;
     } else {
-        a.rare += 1u;
+        a.n_noncomp++;
         a.n_over++;
-        if (bits_inf(cb) || bits_inf(rb)) a.rare += 1u << 24;
+        if (bits_inf(cb) || bits_inf(rb)) a.n_infmis++;
     }
 }
 
-// Per-vector values that depend on the reference only; computed once and used
-// for every candidate of a group.
-template <int VEC>
-struct RefVec {
-    uint32_t r[VEC];      // reference bits (fp32 patterns)
-    float thr[VEC];       // atol + rtol*|r|, product and sum each rounded
-    float minarp;         // smallest non-zero |r| of the vector, +inf if all are zero
-};
-
-template <int VEC>
-__device__ __forceinline__ void refvec_prepare(RefVec<VEC>& rv, float atol, float rtol) {
-    // |r| as an integer orders like the float; subtracting one wraps zero to the top
-    uint32_t mn = 0xFFFFFFFFu;
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-        const uint32_t ab = rv.r[j] & 0x7FFFFFFFu;
-        rv.thr[j] = __fadd_rn(atol, __fmul_rn(rtol, __uint_as_float(ab)));
-        mn = min(mn, ab - 1u);
-    }
-    rv.minarp = mn == 0xFFFFFFFFu ? __int_as_float(0x7F800000) : __uint_as_float(mn + 1u);
-}
-
-// The rarely taken parts of a vector step live out of line, so that the hot loop
-// stays small enough for the instruction cache.  Arguments travel by value.
-struct Best {
-    float emax; uint32_t eidx;
-    float qmax; uint32_t qidx;
-};
-
-template <int VEC>
-struct VecErr {
-    float e[VEC];
-    uint32_t r[VEC];
-};
-
-// All values finite: new running maxima of |c - r| and of |c - r| / |r|.
-template <int VEC>
-__device__ __noinline__ Best rare_finite(Best b, float qthr, VecErr<VEC> x, uint32_t idx0) {
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-        if (x.e[j] > b.emax) { b.emax = x.e[j]; b.eidx = idx0 + j; }
-        const float ar = fabsf(__uint_as_float(x.r[j]));
-        if (ar != 0.0f && x.e[j] > __fmul_rd(qthr, ar)) {
-            const float q = __fdiv_rn(x.e[j], ar);
-            if (q > b.qmax) { b.qmax = q; b.qidx = idx0 + j; }
-        }
-    }
-    return b;
-}
-
-template <int VEC>
-struct VecBits {
-    uint32_t c[VEC];
-    uint32_t r[VEC];
-};
-
-struct GenState {
-    Best b;
-    uint32_t n_over;
-    uint32_t rare;
-    double sum;
-};
-
-// A vector with a non-finite value somewhere: the general rule, element by element.
-template <int VEC>
-__device__ __noinline__ GenState rare_general(GenState g, VecBits<VEC> x, uint32_t idx0, float atol,
-                                              float rtol) {
-    Acc a;
-    a.n_over = g.n_over; a.rare = g.rare; a.sum = g.sum;
-    a.emax = g.b.emax; a.eidx = g.b.eidx; a.qmax = g.b.qmax; a.qidx = g.b.qidx;
-    a.ethr = 0.0f; a.qthr = 0.0f; a.cacc = 0; a.pacc = 0;
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) elem_general(a, x.c[j], x.r[j], idx0 + j, atol, rtol);
-    g.n_over = a.n_over; g.rare = a.rare; g.sum = a.sum;
-    g.b.emax = a.emax; g.b.eidx = a.eidx; g.b.qmax = a.qmax; g.b.qidx = a.qidx;
-    return g;
-}
-
-// VEC consecutive elements of one candidate: bits c[] against the prepared
-// reference vector; idx0 is the slab-local index of the first element.
-//
-// The common path only evaluates predicates; everything behind them sits in one
-// rarely taken region:
-//   !(s < s_limit)                          a non-finite value somewhere in the
-//                                           vector (or a slab whose reference
-//                                           has one: s_limit = -1) -> general rule
-//   over : !(e <= thr)                      -> recount the vector
-//   abs  : e > ethr, ethr >= running max    -> update (max, first index)
-//   rel  : max e > RD(qthr * min|r|)        -> per element e > RD(qthr*|r|): divide, update
-// RD is the product rounded toward -inf.  If fl(e/|r|) > qthr then, rounding
-// being monotone, e/|r| > qthr exactly, so e > qthr*|r| >= RD(qthr*|r|): the
-// test never skips an element that beats qthr.  Thresholds always come from
-// elements with SMALLER indices (the thread's own earlier elements, earlier
-// rounds of the warp, earlier slabs of the block), so a tie may be skipped: the
-// first index keeps the maximum.
-template <int VEC>
-__device__ __forceinline__ void step_vec(Acc& a, const uint32_t (&c)[VEC], const RefVec<VEC>& rv,
-                                         uint32_t idx0, float atol, float rtol, float s_limit) {
-    float e[VEC];
-#pragma unroll
-    for (int j = 0; j < VEC; ++j)
-        e[j] = fabsf(__fsub_rn(__uint_as_float(c[j]), __uint_as_float(rv.r[j])));
-    float s;
-    if (VEC == 4) {
-        s = __fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3]));
-    } else {
-        s = __fadd_rn(__fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3])),
-                      __fadd_rn(__fadd_rn(e[4 % VEC], e[5 % VEC]), __fadd_rn(e[6 % VEC], e[7 % VEC])));
-    }
-    const bool finite = s < s_limit;
-    bool rare = !finite;
-    float m = e[0];
-#pragma unroll
-    for (int j = 1; j < VEC; ++j) m = fmaxf(m, e[j]);
-    rare |= m > a.ethr;
-    // vector-level relative-error filter: e_j > qthr*|r_j| for some j implies m > qthr*min|r|
-    rare |= m > __fmul_rd(a.qthr, rv.minarp);
-    // over-tolerance elements are common in failing candidates: counted unconditionally
-#pragma unroll
-    for (int j = 0; j < VEC; ++j)
-        if (!(e[j] <= rv.thr[j]) && finite) a.n_over++;
-    a.sum += (double)(finite ? s : 0.0f);
-    if (rare) {
-        if (!finite) {
-            GenState g;
-            g.b.emax = a.emax; g.b.eidx = a.eidx; g.b.qmax = a.qmax; g.b.qidx = a.qidx;
-            g.n_over = a.n_over; g.rare = a.rare; g.sum = a.sum;
-            VecBits<VEC> x;
-#pragma unroll
-            for (int j = 0; j < VEC; ++j) { x.c[j] = c[j]; x.r[j] = rv.r[j]; }
-            g = rare_general<VEC>(g, x, idx0, atol, rtol);
-            a.emax = g.b.emax; a.eidx = g.b.eidx; a.qmax = g.b.qmax; a.qidx = g.b.qidx;
-            a.n_over = g.n_over; a.rare = g.rare; a.sum = g.sum;
-        } else {
-            Best b;
-            b.emax = a.emax; b.eidx = a.eidx; b.qmax = a.qmax; b.qidx = a.qidx;
-            VecErr<VEC> x;
-#pragma unroll
-            for (int j = 0; j < VEC; ++j) { x.e[j] = e[j]; x.r[j] = rv.r[j]; }
-            b = rare_finite<VEC>(b, a.qthr, x, idx0);
-            a.emax = b.emax; a.eidx = b.eidx; a.qmax = b.qmax; a.qidx = b.qidx;
-        }
-        a.ethr = fmaxf(a.ethr, a.emax);
-        a.qthr = fmaxf(a.qthr, a.qmax);
-    }
-}
-
-// ----------------------------------------------------------------------------
-// warp reduction of the accumulators -> one Partial in shared memory
-// ----------------------------------------------------------------------------
-__device__ __forceinline__ void warp_reduce_store(const Acc& a, Partial* dst, int lane) {
-    const uint32_t n_over = __reduce_add_sync(kFullMask, a.n_over);
-    uint32_t n_noncomp = 0, n_nan = 0, n_inf = 0, n_infmis = 0;
-    if (__any_sync(kFullMask, a.rare != 0)) {
-        n_noncomp = __reduce_add_sync(kFullMask, a.rare & 0xFFu);
-        n_nan = __reduce_add_sync(kFullMask, (a.rare >> 8) & 0xFFu);
-        n_inf = __reduce_add_sync(kFullMask, (a.rare >> 16) & 0xFFu);
-        n_infmis = __reduce_add_sync(kFullMask, a.rare >> 24);
-    }
-    // non-negative floats (and the -1 sentinel) order like their bit patterns as signed ints
-    const int eb = __float_as_int(a.emax);
-    const int ebm = __reduce_max_sync(kFullMask, eb);
-    const uint32_t eidx = __reduce_min_sync(kFullMask, eb == ebm ? a.eidx : 0xFFFFFFFFu);
-    const int qb = __float_as_int(a.qmax);
-    const int qbm = __reduce_max_sync(kFullMask, qb);
-    const uint32_t qidx = __reduce_min_sync(kFullMask, qb == qbm ? a.qidx : 0xFFFFFFFFu);
-    const uint32_t cacc = __reduce_or_sync(kFullMask, a.cacc);
-    const uint32_t pacc = __reduce_or_sync(kFullMask, a.pacc);
-    double sum = a.sum;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFullMask, sum, off);
-    if (lane == 0) {
-        Partial p;
-        p.n_over = n_over; p.n_noncomp = n_noncomp; p.n_nan = n_nan; p.n_inf = n_inf;
-        p.n_infmis = n_infmis;
-        p.mismatch = (cacc ? 1u : 0u) | (pacc ? 2u : 0u);
-        p.emax = __int_as_float(ebm); p.eidx = eidx;
-        p.qmax = __int_as_float(qbm); p.qidx = qidx;
-        p.sum = sum;
-        *dst = p;
-    }
-}
-
-__device__ __forceinline__ void partial_merge(Partial& a, const Partial& b) {
-    a.n_over += b.n_over; a.n_noncomp += b.n_noncomp; a.n_nan += b.n_nan; a.n_inf += b.n_inf;
-    a.n_infmis += b.n_infmis; a.mismatch |= b.mismatch;
-    if (b.emax > a.emax || (b.emax == a.emax && b.eidx < a.eidx)) { a.emax = b.emax; a.eidx = b.eidx; }
-    if (b.qmax > a.qmax || (b.qmax == a.qmax && b.qidx < a.qidx)) { a.qmax = b.qmax; a.qidx = b.qidx; }
-    a.sum += b.sum;
-}
-
-// ----------------------------------------------------------------------------
-// staging of the reference / input slab
-// ----------------------------------------------------------------------------
-
-// Generate `len` elements starting at tensor element `start` (a multiple of 4)
-// into shared memory, as fp32 bit patterns or as bf16 bit patterns.
-template <bool OUT_BF16, bool ROUND_BF16>
-__device__ __forceinline__ void stage_generated(unsigned char* dst, uint64_t seed, uint64_t stream_id,
-                                                int dist, uint64_t start, uint32_t len, int tid) {
+// Four consecutive elements (tile offset off0, a multiple of 4) of a generated
+// tensor, as fp32 bit patterns; bf16 == true rounds them to bf16 first.
+__device__ __forceinline__ void gen_group(uint64_t seed, uint64_t stream_id, int dist, uint64_t start,
+                                          uint32_t off0, bool bf16, uint32_t out[4]) {
     const PhiloxKey key = philox_key(seed);
-    const uint32_t n_blocks = (len + 3u) >> 2;
-    for (uint32_t b = tid; b < n_blocks; b += kThreads) {
-        float v[4];
-        gen_block_dyn(dist, (start >> 2) + b, stream_id, key, v);
-        if (OUT_BF16) {
-            uint2 w;
-            w.x = bf16_rne_bits(v[0]) | (bf16_rne_bits(v[1]) << 16);
-            w.y = bf16_rne_bits(v[2]) | (bf16_rne_bits(v[3]) << 16);
-            *reinterpret_cast<uint2*>(dst + (size_t)b * 8) = w;
-        } else {
-            uint4 w;
-            w.x = __float_as_uint(v[0]); w.y = __float_as_uint(v[1]);
-            w.z = __float_as_uint(v[2]); w.w = __float_as_uint(v[3]);
-            if (ROUND_BF16) {
-                w.x = bf16_rne_bits(v[0]) << 16; w.y = bf16_rne_bits(v[1]) << 16;
-                w.z = bf16_rne_bits(v[2]) << 16; w.w = bf16_rne_bits(v[3]) << 16;
-            }
-            *reinterpret_cast<uint4*>(dst + (size_t)b * 16) = w;
-        }
+    float v[4];
+    gen_block_dyn(dist, (start + off0) >> 2, stream_id, key, v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        out[i] = bf16 ? (bf16_rne_bits(v[i]) << 16) : __float_as_uint(v[i]);
+}
+
+// Four consecutive elements of the input tensor as fp32 bit patterns (the input
+// has the candidates' dtype); elements at or beyond `len` come back as 0.
+template <bool CB16>
+__device__ __forceinline__ void input_group(const DevTensor& D, uint64_t start, uint32_t off0, uint32_t len,
+                                            uint32_t out[4]) {
+    if (D.input_src == RKV_SRC_GENERATED) {
+        gen_group(D.in_seed, D.in_stream, D.in_dist, start, off0, CB16, out);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            out[i] = (off0 + i < len) ? ld_elem_bits(D.input, CB16 ? RKV_BF16 : RKV_F32, start + off0 + i) : 0u;
     }
 }
 
 // Element 0 of a tensor as an fp32 bit pattern (upcast), from memory or generated.
 __device__ __forceinline__ uint32_t first_elem_bits(const void* ptr, int src, int dtype, uint64_t seed,
                                                     uint64_t stream_id, int dist) {
-    if (src == RKV_SRC_POINTER) {
-        if (dtype == RKV_BF16) return (uint32_t)(*reinterpret_cast<const uint16_t*>(ptr)) << 16;
-        return *reinterpret_cast<const uint32_t*>(ptr);
-    }
-    const PhiloxKey key = philox_key(seed);
-    float v[4];
-    gen_block_dyn(dist, 0, stream_id, key, v);
-    if (dtype == RKV_BF16) return bf16_rne_bits(v[0]) << 16;
-    return __float_as_uint(v[0]);
+    if (src == RKV_SRC_POINTER) return ld_elem_bits(ptr, dtype, 0);
+    uint32_t g[4];
+    gen_group(seed, stream_id, dist, 0, 0, dtype == RKV_BF16, g);
+    return g[0];
 }
 
-template <bool B16>
-__device__ __forceinline__ uint32_t smem_elem_bits(const unsigned char* base, uint32_t i) {
-    if (B16) return (uint32_t)reinterpret_cast<const uint16_t*>(base)[i] << 16;
-    return reinterpret_cast<const uint32_t*>(base)[i];
-}
-
-// ----------------------------------------------------------------------------
-// one slab, all candidates
-//   CB16   candidates (and the staged input) are bf16
-//   RB16   the staged reference is bf16 (only a bf16 reference read from memory)
-//   HAS_IN an input tensor is staged and the copy flag computed
-// ----------------------------------------------------------------------------
-template <bool CB16, bool RB16, bool HAS_IN, int KB, int U>
-__device__ __forceinline__ bool process_item(const DevTensor& D, uint32_t item, int K, int k_begin, int k_end,
-                                             Partial* __restrict__ partials, unsigned char* smem,
-                                             uint32_t& phase, int32_t* status) {
+// Load (or regenerate) the thread's reference values for a tile and derive what
+// depends on them alone.  `stage` holds the bulk-copied part of the tile
+// (ref_copied elements); anything beyond comes from global memory.
+template <bool CB16, bool RB16>
+__device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const DevTensor& D, uint64_t start,
+                                         uint32_t len, const unsigned char* stage, int tid) {
     constexpr int VEC = CB16 ? 8 : 4;
-    constexpr int CSZ = CB16 ? 2 : 4;
-    constexpr int RSZ = RB16 ? 2 : 4;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t S = D.slab_elems;
-    const uint32_t slab = item - D.first_item;
-    const uint64_t start = (uint64_t)slab * S;
-    const uint32_t len = (uint32_t)((D.n - start) < (uint64_t)S ? (D.n - start) : (uint64_t)S);
-    const float atol = D.atol, rtol = D.rtol;
-
-    unsigned char* ref_s = smem + kOffData;
-    unsigned char* in_s = ref_s + (((size_t)S * RSZ + 127) & ~(size_t)127);
-    const uint32_t mbar = smem_u32(smem + kOffMbar);
-    float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
-    float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
-    uint32_t* hint_f = reinterpret_cast<uint32_t*>(smem + kOffHintF);
-    Partial* warp_part = reinterpret_cast<Partial*>(smem + kOffWarpPart);
-
-    // ---- stage reference and input -------------------------------------------------
-    uint32_t bulk_total = 0;
-    const uint32_t ref_bulk = (D.ref_src == RKV_SRC_POINTER) ? (len * RSZ) & ~15u : 0u;
-    const uint32_t in_bulk = (HAS_IN && D.input_src == RKV_SRC_POINTER) ? (len * CSZ) & ~15u : 0u;
-    bulk_total = ref_bulk + in_bulk;
-    if (tid == 0 && bulk_total) {
-        mbar_expect_tx(mbar, bulk_total);
-        const unsigned char* g = reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ;
-        for (uint32_t off = 0; off < ref_bulk; off += 32768u) {
-            const uint32_t bytes = (ref_bulk - off) < 32768u ? (ref_bulk - off) : 32768u;
-            bulk_g2s(smem_u32(ref_s + off), g + off, bytes, mbar);
+    const bool full = len == (uint32_t)kTileElems;
+    if (D.ref_src == RKV_SRC_GENERATED) {
+#pragma unroll
+        for (int g = 0; g < E / 4; ++g) {
+            uint32_t v[4];
+            gen_group(D.ref_seed, D.ref_stream, D.ref_dist, start, elem_off<VEC>(4 * g, tid),
+                      D.ref_dtype == RKV_BF16, v);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rb[4 * g + i] = v[i];
         }
-        if (in_bulk) {
-            const unsigned char* gi = reinterpret_cast<const unsigned char*>(D.input) + start * CSZ;
-            for (uint32_t off = 0; off < in_bulk; off += 32768u) {
-                const uint32_t bytes = (in_bulk - off) < 32768u ? (in_bulk - off) : 32768u;
-                bulk_g2s(smem_u32(in_s + off), gi + off, bytes, mbar);
+    } else if (full) {
+#pragma unroll
+        for (int g = 0; g < E / 4; ++g) {
+            const uint32_t off0 = elem_off<VEC>(4 * g, tid);
+            if (RB16) {
+                const uint2 t = *reinterpret_cast<const uint2*>(stage + (size_t)off0 * 2);
+                rb[4 * g + 0] = t.x << 16; rb[4 * g + 1] = t.x & 0xFFFF0000u;
+                rb[4 * g + 2] = t.y << 16; rb[4 * g + 3] = t.y & 0xFFFF0000u;
+            } else {
+                const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)off0 * 4);
+                rb[4 * g + 0] = t.x; rb[4 * g + 1] = t.y; rb[4 * g + 2] = t.z; rb[4 * g + 3] = t.w;
             }
-        }
-    }
-    if (D.ref_src == RKV_SRC_POINTER) {
-        // the last (< 16) bytes of a ragged slab come by plain loads
-        for (uint32_t i = ref_bulk / RSZ + tid; i < len; i += kThreads) {
-            if (RB16)
-                reinterpret_cast<uint16_t*>(ref_s)[i] =
-                    reinterpret_cast<const uint16_t*>(D.ref)[start + i];
-            else
-                reinterpret_cast<uint32_t*>(ref_s)[i] =
-                    reinterpret_cast<const uint32_t*>(D.ref)[start + i];
         }
     } else {
-        if (D.ref_dtype == RKV_BF16)
-            stage_generated<false, true>(ref_s, D.ref_seed, D.ref_stream, D.ref_dist, start, len, tid);
-        else
-            stage_generated<false, false>(ref_s, D.ref_seed, D.ref_stream, D.ref_dist, start, len, tid);
+        constexpr uint32_t RSZ = RB16 ? 2 : 4;
+        const uint32_t copied = ((len * RSZ) & ~15u) / RSZ;
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+            const uint32_t off = elem_off<VEC>(j, tid);
+            uint32_t b = 0;
+            if (off < copied) b = ld_elem_bits(stage, RB16 ? RKV_BF16 : RKV_F32, off);
+            else if (off < len) b = ld_elem_bits(D.ref, RB16 ? RKV_BF16 : RKV_F32, start + off);
+            rb[j] = b;
+        }
     }
-    if (HAS_IN) {
-        if (D.input_src == RKV_SRC_POINTER) {
-            for (uint32_t i = in_bulk / CSZ + tid; i < len; i += kThreads) {
-                if (CB16)
-                    reinterpret_cast<uint16_t*>(in_s)[i] =
-                        reinterpret_cast<const uint16_t*>(D.input)[start + i];
-                else
-                    reinterpret_cast<uint32_t*>(in_s)[i] =
-                        reinterpret_cast<const uint32_t*>(D.input)[start + i];
+    bool nonfinite = false;
+    uint32_t mn = 0xFFFFFFFFu;
+    float tmin = kInf;
+#pragma unroll
+    for (int j = 0; j < E; ++j) {
+        const uint32_t ab = rb[j] & 0x7FFFFFFFu;
+        nonfinite |= !bits_finite(rb[j]);
+        R.r[j] = __uint_as_float(rb[j]);
+        R.thr[j] = __fadd_rn(D.atol, __fmul_rn(D.rtol, __uint_as_float(ab)));
+        tmin = fminf(tmin, R.thr[j]);
+        mn = min(mn, ab - 1u);       // |r| orders like its bits; zero wraps to the top
+    }
+    R.thr_min = tmin;
+    R.minarp = mn == 0xFFFFFFFFu ? kInf : __uint_as_float(mn + 1u);
+    R.general = nonfinite || !full;
+}
+
+__device__ __forceinline__ unsigned long long hint_key(float v, uint32_t tile) {
+    return ((unsigned long long)(__float_as_uint(v) + 1u) << 32) | (unsigned long long)(~tile);
+}
+
+// Candidate bits of element j of the thread, as an fp32 pattern.
+template <bool CB16, int NW>
+__device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[NW], int j) {
+    if (!CB16) return w[j];
+    return (j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16);
+}
+
+// One candidate tile against the thread's reference registers.
+//   w        the thread's 16-byte pieces of the candidate tile (from the ring)
+//   h        the candidate's hint entry (a snapshot; see the file header)
+//   rec      the warp's running result for this candidate (shared memory; lane 0 writes)
+//   st       the candidate's global state
+//   cand_g   the candidate tensor in global memory (only the last < 16 bytes of a
+//            ragged tensor are read from there)
+template <bool CB16>
+__device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32_t (&w)[CB16 ? E / 2 : E],
+                                                  const Hint& h, Hint* h_smem, WarpRec* rec, CandState* st,
+                                                  const DevTensor& D, const void* cand_g, uint32_t tile,
+                                                  uint64_t start, uint32_t len, uint32_t wanted_flags,
+                                                  int tid, int lane) {
+    constexpr int VEC = CB16 ? 8 : 4;
+    constexpr int NW = CB16 ? E / 2 : E;
+    constexpr uint32_t CSZ = CB16 ? 2 : 4;
+
+    // ---- common path ---------------------------------------------------------------
+    float e[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j)
+        e[j] = fabsf(__fsub_rn(__uint_as_float(cand_bits<CB16, NW>(w, j)), R.r[j]));
+    float m = fmaxf(fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])), fmaxf(fmaxf(e[4], e[5]), fmaxf(e[6], e[7])));
+    m = fmaxf(m, fmaxf(fmaxf(fmaxf(e[8], e[9]), fmaxf(e[10], e[11])),
+                       fmaxf(fmaxf(e[12], e[13]), fmaxf(e[14], e[15]))));
+    float s4[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
+        s4[g] = __fadd_rn(__fadd_rn(e[4 * g], e[4 * g + 1]), __fadd_rn(e[4 * g + 2], e[4 * g + 3]));
+    const float s = __fadd_rn(__fadd_rn(s4[0], s4[1]), __fadd_rn(s4[2], s4[3]));
+
+    // a NaN or an infinity anywhere makes the sum non-finite
+    const bool lane_gen = R.general || !(s < kInf);
+    // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
+    uint32_t cnt = 0;
+    if (__any_sync(kFullMask, m > R.thr_min)) {
+#pragma unroll
+        for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
+    }
+    // can one of these elements be the first maximum?  (te, te_tile) is a published
+    // maximum: an element equal to it in a later tile, or anything smaller, cannot.
+    bool rare = (m > h.te) || (m == h.te && tile <= h.te_tile) || lane_gen;
+    // Relative error.  fl(e/|r|) > tq implies e > tq*|r| >= RD(tq*|r|); fl(e/|r|) >= tq
+    // implies the same with the float below tq; a tie only matters at or before the hint's
+    // tile.  First a test on the thread's largest e and smallest non-zero |r|; only if that
+    // passes somewhere in the warp, the same test element by element (errors proportional to
+    // |r|, as in an all-zero output, pass the first test everywhere).
+    {
+        const float tqx = tile <= h.tq_tile ? h.tq_pred : h.tq;
+        if (__any_sync(kFullMask, m > __fmul_rd(tqx, R.minarp))) {
+            bool hit = false;
+#pragma unroll
+            for (int j = 0; j < E; ++j) {
+                const float ar = fabsf(R.r[j]);
+                hit |= (ar != 0.0f) && (e[j] > __fmul_rd(tqx, ar));
             }
+            rare |= hit;
+        }
+    }
+
+    const bool any_gen = __any_sync(kFullMask, lane_gen);
+    if (__any_sync(kFullMask, rare)) {
+        // ---- locate maxima; general rule where needed ------------------------------
+        const float rec_q = rec->qmax;
+        LaneGen a;
+        a.n_over = cnt; a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
+        a.emax = -1.0f; a.eoff = 0xFFFFu; a.qmax = -1.0f; a.qoff = 0xFFFFu; a.sum = (double)s;
+        if (lane_gen) {
+            a.n_over = 0; a.sum = 0.0;
+            const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+#pragma unroll
+            for (int j = 0; j < E; ++j) {
+                const uint32_t off = elem_off<VEC>(j, tid);
+                if (off < len) {
+                    uint32_t cb = cand_bits<CB16, NW>(w, j);
+                    if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
+                    elem_general(a, cb, __float_as_uint(R.r[j]), off, D.atol, D.rtol);
+                }
+            }
+            if (a.n_noncomp) atomicAdd(&st->n_noncomp, (unsigned long long)a.n_noncomp);
+            if (a.n_nan) atomicAdd(&st->n_nan, (unsigned long long)a.n_nan);
+            if (a.n_inf) atomicAdd(&st->n_inf, (unsigned long long)a.n_inf);
+            if (a.n_infmis) atomicAdd(&st->n_infmis, (unsigned long long)a.n_infmis);
         } else {
-            stage_generated<CB16, false>(in_s, D.in_seed, D.in_stream, D.in_dist, start, len, tid);
-        }
-    }
-    bool waited_ok = true;
-    if (bulk_total) {
-        waited_ok = false;
-        const long long t0 = clock64();
-        for (uint32_t spin = 0; spin < (1u << 24); ++spin) {
-            if (mbar_try_wait(mbar, phase)) { waited_ok = true; break; }
-            if (clock64() - t0 > 2000000000LL) break;      // about a second
-        }
-        phase ^= 1u;
-    }
-    if (__syncthreads_or(!waited_ok)) {
-        if (tid == 0) atomicExch(status, (int32_t)RKV_ERR_TIMEOUT);
-        return false;
-    }
-
-    // ---- scan the staged slab: non-finite reference values, reference flags ---------
-    const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed, D.ref_stream,
-                                             D.ref_dist);
-    uint32_t r_nonfinite = 0, r_cacc = 0, r_pacc = 0;
-    for (uint32_t i = tid; i < len; i += kThreads) {
-        const uint32_t rb = smem_elem_bits<RB16>(ref_s, i);
-        r_nonfinite |= bits_finite(rb) ? 0u : 1u;
-        r_cacc |= rb ^ r_first;
-        if (HAS_IN) r_pacc |= rb ^ smem_elem_bits<CB16>(in_s, i);
-    }
-    // __syncthreads_or is a boolean any(), one call per flag
-    const bool general = __syncthreads_or((int)r_nonfinite) != 0;
-    const bool ref_differs_first = __syncthreads_or(r_cacc != 0u) != 0;
-    const bool ref_differs_input = HAS_IN ? (__syncthreads_or(r_pacc != 0u) != 0) : false;
-    if (tid == 0 && k_begin == 0) {
-        Partial p = {};
-        p.mismatch = (ref_differs_first ? 1u : 0u) | (ref_differs_input ? 2u : 0u);
-        p.emax = -1.0f; p.qmax = -1.0f; p.eidx = 0xFFFFFFFFu; p.qidx = 0xFFFFFFFFu;
-        partials[(size_t)item * (K + 1) + K] = p;
-    }
-
-    // ---- stream the candidates -------------------------------------------------------
-    // Candidates are taken KB at a time: the reference vector is read from shared
-    // memory and prepared once per KB candidate vectors.  Each thread keeps U
-    // 16-byte loads per candidate in flight: a register slot is reloaded with the
-    // vector U rounds ahead right after it has been consumed.
-    const uint32_t nvec = len / VEC;
-    const uint32_t tail0 = nvec * VEC;
-    // this thread's vectors are v = tid + i*kThreads, i < n_mine; the first lane of a
-    // warp has the most (n_first), which gives the warp-uniform trip count
-    const uint32_t n_mine = nvec > (uint32_t)tid ? (nvec - tid + kThreads - 1) / kThreads : 0u;
-    const uint32_t tid_first = (uint32_t)tid & ~31u;
-    const uint32_t n_first = nvec > tid_first ? (nvec - tid_first + kThreads - 1) / kThreads : 0u;
-    const float s_limit = general ? -1.0f : __int_as_float(0x7F800000);
-    const unsigned char* const* cptr_s = reinterpret_cast<const unsigned char* const*>(smem + kOffCandPtr);
-    const uint32_t* cfirst_s = reinterpret_cast<const uint32_t*>(smem + kOffCandFirst);
-    for (int kc0 = k_begin; kc0 < k_end; kc0 += kChunkK) {
-        const int kc1 = (kc0 + kChunkK) < k_end ? (kc0 + kChunkK) : k_end;
-        for (int kg = kc0; kg < kc1; kg += KB) {
-            const unsigned char* cp[KB];
-            uint32_t c_first[KB];
-            Acc a[KB];
 #pragma unroll
-            for (int i = 0; i < KB; ++i) {
-                // a group that runs past the chunk repeats its last candidate (result dropped)
-                const int k = (kg + i) < kc1 ? (kg + i) : (kc1 - 1);
-                if (k < kPreK) {
-                    cp[i] = cptr_s[k];
-                    c_first[i] = cfirst_s[k];
-                } else {
-                    cp[i] = reinterpret_cast<const unsigned char*>(D.cands[k]);
-                    c_first[i] = CB16 ? (uint32_t)(*reinterpret_cast<const uint16_t*>(cp[i]))
-                                      : *reinterpret_cast<const uint32_t*>(cp[i]);
+            for (int j = 0; j < E; ++j) {
+                if (e[j] > a.emax) { a.emax = e[j]; a.eoff = elem_off<VEC>(j, tid); }
+                const float ar = fabsf(R.r[j]);
+                // the warp's own record comes from earlier tiles: only a strictly larger
+                // quotient can replace it
+                if (ar != 0.0f && e[j] > __fmul_rd(fmaxf(rec_q, a.qmax), ar)) {
+                    const float q = __fdiv_rn(e[j], ar);
+                    if (q > a.qmax) { a.qmax = q; a.qoff = elem_off<VEC>(j, tid); }
                 }
-                if (CB16) c_first[i] = (c_first[i] & 0xFFFFu) * 0x10001u;
-                cp[i] += start * CSZ + (size_t)tid * 16;
-                acc_reset(a[i], k < kHintK ? hint_e[k] : -1.0f, k < kHintK ? hint_q[k] : -1.0f);
-            }
-
-            // The loophole flags are OR-reductions over the whole tensor: once an earlier
-            // slab of this block has reported "differs" for every candidate of the group,
-            // the xor/or work is skipped and the settled value reported again.
-            uint32_t settled = 3u;
-#pragma unroll
-            for (int i = 0; i < KB; ++i) {
-                const int k = (kg + i) < kc1 ? (kg + i) : (kc1 - 1);
-                settled &= k < kHintK ? hint_f[k] : 0u;
-            }
-            constexpr uint32_t kWanted = HAS_IN ? 3u : 1u;
-            const bool need_flags = (settled & kWanted) != kWanted;
-            if (!need_flags) {
-#pragma unroll
-                for (int i = 0; i < KB; ++i) { a[i].cacc = 1u; a[i].pacc = 1u; }
-            }
-
-            // Two register buffers of U vectors per candidate.  All loads of a batch are
-            // issued together, one batch ahead of their use, and consumed together.
-            uint4 bufA[KB][U], bufB[KB][U];
-            auto load_batch = [&](uint4 (&buf)[KB][U], const uint32_t r0) {
-#pragma unroll
-                for (int i = 0; i < KB; ++i)
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-                        if (r0 + u < n_mine)
-                            buf[i][u] = ldg_stream(cp[i] + (size_t)(r0 + u) * (kThreads * 16));
-            };
-
-            // one vector position of this thread: round r (v = tid + r*kThreads)
-            auto do_vector = [&](const uint4 (&buf)[KB][U], const int u, const uint32_t r) {
-                const uint32_t v = (uint32_t)tid + r * kThreads;
-                RefVec<VEC> rv;
-                if (!CB16) {
-                    if (RB16) {
-                        const uint2 t = *reinterpret_cast<const uint2*>(ref_s + (size_t)v * 8);
-                        rv.r[0] = t.x << 16; rv.r[1] = t.x & 0xFFFF0000u;
-                        rv.r[2] = t.y << 16; rv.r[3] = t.y & 0xFFFF0000u;
-                    } else {
-                        const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                        rv.r[0] = t.x; rv.r[1] = t.y; rv.r[2] = t.z; rv.r[3] = t.w;
-                    }
-                } else {
-                    if (RB16) {
-                        const uint4 t = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 16);
-                        const uint32_t rw[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            rv.r[(2 * q) % VEC] = rw[q] << 16;
-                            rv.r[(2 * q + 1) % VEC] = rw[q] & 0xFFFF0000u;
-                        }
-                    } else {
-                        const uint4 t0 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32);
-                        const uint4 t1 = *reinterpret_cast<const uint4*>(ref_s + (size_t)v * 32 + 16);
-                        rv.r[0] = t0.x; rv.r[1] = t0.y; rv.r[2] = t0.z; rv.r[3] = t0.w;
-                        rv.r[4 % VEC] = t1.x; rv.r[5 % VEC] = t1.y;
-                        rv.r[6 % VEC] = t1.z; rv.r[7 % VEC] = t1.w;
-                    }
-                }
-                refvec_prepare<VEC>(rv, atol, rtol);
-                if (need_flags) {
-                    uint4 iv = make_uint4(0, 0, 0, 0);
-                    if (HAS_IN) iv = *reinterpret_cast<const uint4*>(in_s + (size_t)v * 16);
-#pragma unroll
-                    for (int i = 0; i < KB; ++i) {
-                        const uint4 w = buf[i][u];
-                        a[i].cacc |= (w.x ^ c_first[i]) | (w.y ^ c_first[i]) | (w.z ^ c_first[i]) |
-                                     (w.w ^ c_first[i]);
-                        if (HAS_IN) a[i].pacc |= (w.x ^ iv.x) | (w.y ^ iv.y) | (w.z ^ iv.z) | (w.w ^ iv.w);
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < KB; ++i) {
-                    const uint32_t w[4] = {buf[i][u].x, buf[i][u].y, buf[i][u].z, buf[i][u].w};
-                    uint32_t c[VEC];
-                    if (!CB16) {
-                        c[0] = w[0]; c[1] = w[1]; c[2] = w[2]; c[3] = w[3];
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            c[(2 * q) % VEC] = w[q] << 16;
-                            c[(2 * q + 1) % VEC] = w[q] & 0xFFFF0000u;
-                        }
-                    }
-                    step_vec<VEC>(a[i], c, rv, v * VEC, atol, rtol, s_limit);
-                }
-            };
-
-            auto compute_batch = [&](const uint4 (&buf)[KB][U], const uint32_t r0) {
-#pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (r0 + u < n_mine) do_vector(buf, u, r0 + u);
-                if (r0 < 2 * U) {
-                    // share the running maxima across the warp: every element seen so far has
-                    // a smaller index than every element of the batches to come
-#pragma unroll
-                    for (int i = 0; i < KB; ++i) {
-                        a[i].ethr = fmaxf(a[i].ethr, __int_as_float(__reduce_max_sync(
-                                                         kFullMask, __float_as_int(a[i].emax))));
-                        a[i].qthr = fmaxf(a[i].qthr, __int_as_float(__reduce_max_sync(
-                                                         kFullMask, __float_as_int(a[i].qmax))));
-                    }
-                }
-            };
-
-            // n_first rounds: what the first lane of the warp needs (the most), so that the
-            // trip count is uniform across the warp
-            load_batch(bufA, 0);
-            for (uint32_t r0 = 0; r0 < n_first; r0 += 2 * U) {
-                load_batch(bufB, r0 + U);
-                compute_batch(bufA, r0);
-                load_batch(bufA, r0 + 2 * U);
-                if (r0 + U < n_first) compute_batch(bufB, r0 + U);
-            }
-            // ragged end of the tensor: fewer than VEC elements, one thread, element by element
-            if (tid == 0) {
-#pragma unroll
-                for (int i = 0; i < KB; ++i) {
-                    for (uint32_t e = tail0; e < len; ++e) {
-                        uint32_t cb;
-                        if (CB16) cb = (uint32_t)reinterpret_cast<const uint16_t*>(cp[i])[e] << 16;
-                        else cb = reinterpret_cast<const uint32_t*>(cp[i])[e];
-                        const uint32_t cf = CB16 ? (c_first[i] << 16) : c_first[i];
-                        a[i].cacc |= cb ^ cf;
-                        if (HAS_IN) a[i].pacc |= cb ^ smem_elem_bits<CB16>(in_s, e);
-                        elem_general(a[i], cb, smem_elem_bits<RB16>(ref_s, e), e, atol, rtol);
-                    }
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < KB; ++i)
-                if (kg + i < kc1) warp_reduce_store(a[i], &warp_part[(kg + i - kc0) * kWarps + warp], lane);
-        }
-        __syncthreads();
-        if (tid < kc1 - kc0) {
-            const int k = kc0 + tid;
-            Partial p = warp_part[tid * kWarps];
-#pragma unroll
-            for (int w = 1; w < kWarps; ++w) partial_merge(p, warp_part[tid * kWarps + w]);
-            partials[(size_t)item * (K + 1) + k] = p;
-            if (k < kHintK) {
-                hint_e[k] = fmaxf(hint_e[k], p.emax);
-                hint_q[k] = fmaxf(hint_q[k], p.qmax);
-                hint_f[k] |= p.mismatch;
             }
         }
-        __syncthreads();
+        cnt = a.n_over;
+        // warp-wide first maximum: largest value, then smallest offset.  Non-negative
+        // floats (and the -1 sentinel) order like their bit patterns as signed ints.
+        const int eb = __float_as_int(a.emax);
+        const int ebm = __reduce_max_sync(kFullMask, eb);
+        const uint32_t eoff = __reduce_min_sync(kFullMask, eb == ebm ? a.eoff : 0xFFFFu);
+        const int qb = __float_as_int(a.qmax);
+        const int qbm = __reduce_max_sync(kFullMask, qb);
+        const uint32_t qoff = __reduce_min_sync(kFullMask, qb == qbm ? a.qoff : 0xFFFFu);
+        double sd = a.sum;
+        if (any_gen) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sd += __shfl_xor_sync(kFullMask, sd, off);
+        } else {
+            float sf = s;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+            sd = (double)sf;
+        }
+        if (lane == 0) {
+            WarpRec r = *rec;
+            const float em = __int_as_float(ebm), qm = __int_as_float(qbm);
+            if (em > r.emax) {
+                r.emax = em; r.etile = tile; r.offs = (r.offs & 0xFFFF0000u) | eoff;
+                atomicMax(&st->hint_e, hint_key(em, tile));
+            }
+            if (qm > r.qmax) {
+                r.qmax = qm; r.qtile = tile; r.offs = (r.offs & 0x0000FFFFu) | (qoff << 16);
+                atomicMax(&st->hint_q, hint_key(qm, tile));
+            }
+            r.sum += sd;
+            *rec = r;
+        }
+    } else {
+        float sf = s;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+        if (lane == 0) rec->sum += (double)sf;
     }
-    return true;
+    {
+        const uint32_t tot = __reduce_add_sync(kFullMask, cnt);
+        if (lane == 0 && tot) rec->n_over += tot;
+    }
+
+    // ---- loophole flags, until a difference has been seen ---------------------------
+    // `settled` is the one hint field other warps update while this warp reads it: take
+    // lane 0's copy so that the branch below is uniform across the warp.
+    const uint32_t need = wanted_flags & ~__shfl_sync(kFullMask, h.settled, 0);
+    if (need) {
+        uint32_t acc1 = 0, acc2 = 0;
+        const bool full = len == (uint32_t)kTileElems;
+        if (full && (need & 1u)) {
+            const uint32_t f = CB16 ? (h.first >> 16) * 0x10001u : h.first;
+#pragma unroll
+            for (int i = 0; i < NW; ++i) acc1 |= w[i] ^ f;
+        }
+        if (full && (need & 2u) && D.input_src == RKV_SRC_POINTER) {
+            // the input has the candidates' dtype: compare the 16-byte pieces as stored
+            const uint4* in = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(D.input) +
+                                                             start * CSZ) + tid;
+#pragma unroll
+            for (int jv = 0; jv < E / VEC; ++jv) {
+                const uint4 t = __ldg(in + jv * kConsumers);
+                acc2 |= (w[4 * jv] ^ t.x) | (w[4 * jv + 1] ^ t.y) | (w[4 * jv + 2] ^ t.z) | (w[4 * jv + 3] ^ t.w);
+            }
+        } else if (!full || (need & 2u)) {
+            const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+#pragma unroll
+            for (int g = 0; g < E / 4; ++g) {
+                const uint32_t off0 = elem_off<VEC>(4 * g, tid);
+                uint32_t in[4] = {0, 0, 0, 0};
+                if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t off = off0 + i;
+                    if (off < len) {
+                        uint32_t cb = cand_bits<CB16, NW>(w, 4 * g + i);
+                        if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
+                        if (!full) acc1 |= cb ^ h.first;
+                        acc2 |= cb ^ in[i];
+                    }
+                }
+            }
+        }
+        uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
+                        (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
+        seen &= need;
+        if (lane == 0 && seen) {
+            atomicOr(&st->mismatch, seen);
+            atomicOr(&h_smem->settled, seen);
+        }
+    }
 }
 
-__device__ __forceinline__ int variant_of(const DevTensor& D) {
-    const int cb16 = D.cand_dtype == RKV_BF16;
-    const int rb16 = D.ref_dtype == RKV_BF16 && D.ref_src == RKV_SRC_POINTER;
-    const int has_in = D.input_src != RKV_SRC_NONE;
-    return cb16 * 4 + rb16 * 2 + has_in;
+// Merge the warp records of every candidate of a part into the block's
+// Partial row and clear them.  Called by all consumer threads between two
+// consumer barriers.
+__device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D, int K, int k0, int kc,
+                                              uint32_t slot, Partial* __restrict__ partials, int tid) {
+    if (tid < kc) {
+        Partial p;
+        p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX; p.sum = 0.0;
+        p.emax = -1.0f; p.qmax = -1.0f; p.valid = 1u; p.reserved = 0u;
+#pragma unroll
+        for (int wp = 0; wp < kConsumerWarps; ++wp) {
+            WarpRec& r = recs[wp * kPartK + tid];
+            p.n_over += r.n_over;
+            p.sum += r.sum;
+            if (r.emax >= 0.0f) {
+                const uint64_t idx = (uint64_t)r.etile * kTileElems + (r.offs & 0xFFFFu);
+                if (r.emax > p.emax || (r.emax == p.emax && idx < p.eidx)) { p.emax = r.emax; p.eidx = idx; }
+            }
+            if (r.qmax >= 0.0f) {
+                const uint64_t idx = (uint64_t)r.qtile * kTileElems + (r.offs >> 16);
+                if (r.qmax > p.qmax || (r.qmax == p.qmax && idx < p.qidx)) { p.qmax = r.qmax; p.qidx = idx; }
+            }
+            r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
+        }
+        // the block may have written this slot before (group A, then group B): merge
+        Partial* dst = &partials[((size_t)D.slot_base + slot) * (size_t)K + (size_t)(k0 + tid)];
+        const Partial old = *dst;
+        if (old.valid) {
+            p.n_over += old.n_over;
+            p.sum = old.sum + p.sum;
+            if (old.emax > p.emax || (old.emax == p.emax && old.eidx < p.eidx)) { p.emax = old.emax; p.eidx = old.eidx; }
+            if (old.qmax > p.qmax || (old.qmax == p.qmax && old.qidx < p.qidx)) { p.qmax = old.qmax; p.qidx = old.qidx; }
+        }
+        *dst = p;
+    }
 }
 
-// One kernel per storage variant (candidate dtype, staged reference dtype,
-// input present), so that each gets its own register allocation.  A launch
-// handles the slabs of every tensor of its variant; `n_items` counts them.
-template <bool CB16, bool RB16, bool HAS_IN>
+template <bool CB16, bool RB16>
+__device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tensors, int T, int K, int k_begin,
+                                              int k_end, uint32_t n_items, CandState* __restrict__ state,
+                                              Partial* __restrict__ partials, unsigned char* smem,
+                                              const Ring& ring) {
+    constexpr int VEC = CB16 ? 8 : 4;
+    constexpr int NV = E / VEC;
+    constexpr int NW = CB16 ? E / 2 : E;
+    constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrC);
+    Hint* hints = reinterpret_cast<Hint*>(smem + kOffHint);
+    WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
+    volatile uint32_t* ref_state = reinterpret_cast<volatile uint32_t*>(smem + kOffRefState);
+    const unsigned char* stages = smem + kOffStage;
+
+    // clear the records once; flush_records leaves them cleared
+    for (int i = tid; i < kConsumerWarps * kPartK; i += kConsumers) {
+        WarpRec& r = recs[i];
+        r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
+    }
+
+    uint32_t n_used = 0;            // ring items consumed so far (same order as the producer issues)
+    uint32_t ord = 0;               // items this block has started
+    int cur_t = -1, cur_k0 = 0, cur_kc = 0;
+    uint32_t cur_part = 0xFFFFFFFFu, cur_slot = 0;
+
+    for (uint32_t id = blockIdx.x; id < n_items; id += gridDim.x, ++ord) {
+        Item it;
+        if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
+        const DevTensor& D = tensors[it.t];
+        const int k0 = k_begin + (int)(it.part * it.part_k);
+        const int kc = min(k_end, k0 + (int)it.part_k) - k0;
+        const uint32_t part_key = (it.group << 31) | it.part;
+        const uint64_t start = (uint64_t)it.tile * kTileElems;
+        const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
+        const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
+        CandState* st_t = state + (size_t)it.t * (size_t)(K + 1);
+        Hint* H = hints + (ord & 1u) * kPartK;
+
+        if (it.t != cur_t || part_key != cur_part) {
+            consumer_sync();                      // every warp is done with the previous part
+            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid);
+            if (tid < kc) ptrs[tid] = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
+            cur_t = it.t; cur_part = part_key; cur_k0 = k0; cur_kc = kc;
+            // Partial row of this block for the tensor: a tensor with a group B has one row
+            // per block; a small tensor numbers the blocks from the one that owns its first item
+            cur_slot = D.warm_tiles < D.n_tiles
+                           ? blockIdx.x
+                           : (blockIdx.x + gridDim.x - it.first_item % gridDim.x) % gridDim.x;
+        }
+        // refresh the hints of this part from the published state
+        if (tid < kc) {
+            const CandState* s = st_t + k0 + tid;
+            const unsigned long long he = __ldcg(&s->hint_e), hq = __ldcg(&s->hint_q);
+            Hint h;
+            h.te = (he >> 32) ? __uint_as_float((uint32_t)(he >> 32) - 1u) : -1.0f;
+            h.te_tile = (he >> 32) ? ~(uint32_t)he : 0u;
+            h.tq = (hq >> 32) ? __uint_as_float((uint32_t)(hq >> 32) - 1u) : -1.0f;
+            h.tq_tile = (hq >> 32) ? ~(uint32_t)hq : 0u;
+            h.tq_pred = h.tq > 0.0f ? __uint_as_float(__float_as_uint(h.tq) - 1u) : -1.0f;
+            h.settled = __ldcg(&s->mismatch);
+            h.first = ld_elem_bits(ptrs[tid], CB16 ? RKV_BF16 : RKV_F32, 0);
+            h.pad = 0;
+            H[tid] = h;
+        }
+        if (tid == kPartK) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
+
+        // ---- the thread's reference values --------------------------------------------
+        RefRegs R;
+        uint32_t rb[E];
+        if (D.ref_src == RKV_SRC_POINTER) {
+            const uint32_t s = n_used % kStages, ph = (n_used / kStages) & 1u;
+            mbar_wait(ring.full0 + 8 * s, ph, ring.abort_flag);
+            load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)s * kStageBytes, tid);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
+            ++n_used;
+        } else {
+            load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, tid);
+        }
+        consumer_sync();                          // hints, pointers and cleared records are visible
+
+        // reference flags (constant / copy of the input), until a difference has been seen
+        {
+            const uint32_t need = wanted & ~ref_state[ord & 1u];
+            if (need) {
+                const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed,
+                                                         D.ref_stream, D.ref_dist);
+                uint32_t acc1 = 0, acc2 = 0;
+#pragma unroll
+                for (int g = 0; g < E / 4; ++g) {
+                    const uint32_t off0 = elem_off<VEC>(4 * g, tid);
+                    uint32_t in[4] = {0, 0, 0, 0};
+                    if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (off0 + i < len) {
+                            acc1 |= rb[4 * g + i] ^ r_first;
+                            acc2 |= rb[4 * g + i] ^ in[i];
+                        }
+                    }
+                }
+                uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
+                                (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
+                seen &= need;
+                if (lane == 0 && seen) atomicOr(&st_t[K].mismatch, seen);
+            }
+        }
+
+        // ---- every candidate of the part ----------------------------------------------
+        for (int kk = 0; kk < kc; ++kk) {
+            const uint32_t s = n_used % kStages, ph = (n_used / kStages) & 1u;
+            const Hint h = H[kk];
+            mbar_wait(ring.full0 + 8 * s, ph, ring.abort_flag);
+            const unsigned char* stage = stages + (size_t)s * kStageBytes;
+            uint32_t w[NW];
+#pragma unroll
+            for (int jv = 0; jv < NV; ++jv) {
+                const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kConsumers + tid) * 16);
+                w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
+            ++n_used;
+            process_candidate<CB16>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+                                    it.tile, start, len, wanted, tid, lane);
+        }
+    }
+    consumer_sync();
+    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid);
+}
+
+// One kernel per storage variant (candidate dtype, stored reference dtype), so
+// that each gets its own register allocation.  A launch handles the items of
+// every tensor of its variant; `n_items` counts them.
+template <bool CB16, bool RB16>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSm)
-verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end,
-              uint32_t n_items, Partial* __restrict__ partials, int32_t* status) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int kVariant = (CB16 ? 4 : 0) + (RB16 ? 2 : 0) + (HAS_IN ? 1 : 0);
+verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
+              CandState* __restrict__ state, Partial* __restrict__ partials, int32_t* status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
+    Ring ring;
+    ring.full0 = smem_u32(smem + kOffFull);
+    ring.empty0 = smem_u32(smem + kOffEmpty);
+    ring.stage0 = smem_u32(smem + kOffStage);
+    ring.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
     if (tid == 0) {
-        mbar_init(smem_u32(smem + kOffMbar), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(ring.full0 + 8 * s, 1);                    // the producer's arrive + its bytes
+            mbar_init(ring.empty0 + 8 * s, kConsumerWarps);      // one release per consumer warp
+        }
+        *ring.abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    uint32_t phase = 0;
-    int cur_t = -1;
-    for (uint32_t it = blockIdx.x; it < n_items; it += gridDim.x) {
-        // it-th slab among the tensors of this variant
-        int t = 0;
-        uint32_t slab = it;
-        for (; t < T; ++t) {
-            if (variant_of(tensors[t]) != kVariant) continue;
-            const uint32_t ns = tensors[t].n_slabs;
-            if (slab < ns) break;
-            slab -= ns;
-        }
-        if (t >= T) return;
-        const DevTensor D = tensors[t];
-        const uint32_t item = D.first_item + slab;
-        if (t != cur_t) {
-            // per-tensor block state: thresholds carried from earlier slabs, and the
-            // candidates' base pointers and first elements (the constant-output test)
-            float* hint_e = reinterpret_cast<float*>(smem + kOffHintE);
-            float* hint_q = reinterpret_cast<float*>(smem + kOffHintQ);
-            const unsigned char** cptr_s = reinterpret_cast<const unsigned char**>(smem + kOffCandPtr);
-            uint32_t* cfirst_s = reinterpret_cast<uint32_t*>(smem + kOffCandFirst);
-            __syncthreads();
-            uint32_t* hint_f = reinterpret_cast<uint32_t*>(smem + kOffHintF);
-            for (int i = tid; i < kHintK; i += kThreads) { hint_e[i] = -1.0f; hint_q[i] = -1.0f; hint_f[i] = 0u; }
-            for (int k = tid; k < K && k < kPreK; k += kThreads) {
-                const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k]);
-                cptr_s[k] = p;
-                cfirst_s[k] = CB16 ? (uint32_t)(*reinterpret_cast<const uint16_t*>(p))
-                                   : *reinterpret_cast<const uint32_t*>(p);
-            }
-            cur_t = t;
-        }
-        if (!process_item<CB16, RB16, HAS_IN, kGroupK, CB16 ? kLoadsBf16 : kLoadsF32>(
-                D, item, K, k_begin, k_end, partials, smem, phase, status))
-            return;
+    if (tid >= kConsumers) {
+        producer_loop<CB16, RB16>(tensors, T, k_begin, k_end, n_items, smem, ring);
+    } else {
+        consumer_loop<CB16, RB16>(tensors, T, K, k_begin, k_end, n_items, state, partials, smem, ring);
+        if (tid == 0 && *ring.abort_flag) atomicExch(status, (int32_t)RKV_ERR_TIMEOUT);
     }
 }
 
 // ----------------------------------------------------------------------------
-// finalize: merge the per-slab partials of each (candidate, tensor) in a fixed
+// finalize: merge the per-block partials of each (candidate, tensor) in a fixed
 // order, derive flags and verdict, and the joint verdict over tensors
 // ----------------------------------------------------------------------------
 constexpr int kFinThreads = 128;
 
 struct Wide {
-    uint64_t n_over, n_noncomp, n_nan, n_inf, n_infmis;
+    uint64_t n_over;
     uint64_t eidx, qidx;
     double sum;
     float emax, qmax;
-    uint32_t mismatch;
 };
 
 __device__ __forceinline__ void wide_merge(Wide& a, const Wide& b) {
-    a.n_over += b.n_over; a.n_noncomp += b.n_noncomp; a.n_nan += b.n_nan; a.n_inf += b.n_inf;
-    a.n_infmis += b.n_infmis; a.mismatch |= b.mismatch;
+    a.n_over += b.n_over;
     if (b.emax > a.emax || (b.emax == a.emax && b.eidx < a.eidx)) { a.emax = b.emax; a.eidx = b.eidx; }
     if (b.qmax > a.qmax || (b.qmax == a.qmax && b.qidx < a.qidx)) { a.qmax = b.qmax; a.qidx = b.qidx; }
     a.sum += b.sum;
 }
 
 __global__ void __launch_bounds__(kFinThreads)
-finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Partial* __restrict__ partials,
-                rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ joint_pass) {
+finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandState* __restrict__ state,
+                const Partial* __restrict__ partials, rkv_stats* __restrict__ stats_out,
+                uint32_t* __restrict__ joint_pass) {
     __shared__ Wide red[kFinThreads];
-    __shared__ uint32_t ref_mismatch_s;
     const int k = blockIdx.x, tid = threadIdx.x;
     uint32_t all_pass = 1;
     for (int t = 0; t < T; ++t) {
         const DevTensor D = tensors[t];
-        Wide w = {};
+        Wide w;
+        w.n_over = 0; w.sum = 0.0;
         w.emax = -1.0f; w.qmax = -1.0f; w.eidx = RKV_NO_INDEX; w.qidx = RKV_NO_INDEX;
-        uint32_t ref_mm = 0;
-        for (uint32_t s = tid; s < D.n_slabs; s += kFinThreads) {
-            const size_t row = (size_t)(D.first_item + s) * (K + 1);
-            const Partial p = partials[row + k];
+        for (uint32_t s = tid; s < D.n_slots; s += kFinThreads) {
+            const Partial p = partials[((size_t)D.slot_base + s) * (size_t)K + (size_t)k];
+            if (!p.valid) continue;
             Wide b;
-            b.n_over = p.n_over; b.n_noncomp = p.n_noncomp; b.n_nan = p.n_nan; b.n_inf = p.n_inf;
-            b.n_infmis = p.n_infmis; b.mismatch = p.mismatch;
-            const uint64_t base = (uint64_t)s * D.slab_elems;
-            b.emax = p.emax; b.eidx = p.emax < 0.0f ? RKV_NO_INDEX : base + p.eidx;
-            b.qmax = p.qmax; b.qidx = p.qmax < 0.0f ? RKV_NO_INDEX : base + p.qidx;
-            b.sum = p.sum;
+            b.n_over = p.n_over; b.sum = p.sum;
+            b.emax = p.emax; b.eidx = p.eidx; b.qmax = p.qmax; b.qidx = p.qidx;
             wide_merge(w, b);
-            ref_mm |= partials[row + K].mismatch;
         }
         red[tid] = w;
-        if (tid == 0) ref_mismatch_s = 0;
         __syncthreads();
-        if (ref_mm) atomicOr(&ref_mismatch_s, ref_mm);
         for (int off = kFinThreads / 2; off > 0; off >>= 1) {
             if (tid < off) {
                 Wide a = red[tid];
@@ -812,13 +870,14 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Parti
         }
         if (tid == 0) {
             const Wide r = red[0];
-            const uint32_t ref_mismatch = ref_mismatch_s;
+            const CandState cs = state[(size_t)t * (size_t)(K + 1) + (size_t)k];
+            const uint32_t ref_mismatch = state[(size_t)t * (size_t)(K + 1) + (size_t)K].mismatch;
             rkv_stats st;
             st.n_over_tol = r.n_over;
-            st.n_nan = r.n_nan;
-            st.n_inf = r.n_inf;
-            st.n_inf_mismatch = r.n_infmis;
-            st.n_comparable = D.n - r.n_noncomp;
+            st.n_nan = cs.n_nan;
+            st.n_inf = cs.n_inf;
+            st.n_inf_mismatch = cs.n_infmis;
+            st.n_comparable = D.n - cs.n_noncomp;
             st.argmax_abs_err = r.emax < 0.0f ? RKV_NO_INDEX : r.eidx;
             st.argmax_rel_err = r.qmax < 0.0f ? RKV_NO_INDEX : r.qidx;
             st.sum_abs_err = r.sum;
@@ -828,16 +887,16 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Parti
             st.reserved = 0;
             const bool has_in = D.input_src != RKV_SRC_NONE;
             uint32_t flags = 0;
-            if (!(r.mismatch & 1u)) flags |= RKV_FLAG_CAND_CONST;
-            if (has_in && !(r.mismatch & 2u)) flags |= RKV_FLAG_CAND_COPY_OF_INPUT;
+            if (!(cs.mismatch & 1u)) flags |= RKV_FLAG_CAND_CONST;
+            if (has_in && !(cs.mismatch & 2u)) flags |= RKV_FLAG_CAND_COPY_OF_INPUT;
             if (!(ref_mismatch & 1u)) flags |= RKV_FLAG_REF_CONST;
             if (has_in && !(ref_mismatch & 2u)) flags |= RKV_FLAG_REF_COPY_OF_INPUT;
-            if (r.n_nan) flags |= RKV_FLAG_HAS_NAN;
-            if (r.n_inf) flags |= RKV_FLAG_HAS_INF;
+            if (cs.n_nan) flags |= RKV_FLAG_HAS_NAN;
+            if (cs.n_inf) flags |= RKV_FLAG_HAS_INF;
             uint32_t verdict = 0;
             if (r.n_over) verdict |= RKV_FAIL_TOL;
-            if (r.n_nan) verdict |= RKV_FAIL_NAN;
-            if (r.n_infmis) verdict |= RKV_FAIL_INF_MISMATCH;
+            if (cs.n_nan) verdict |= RKV_FAIL_NAN;
+            if (cs.n_infmis) verdict |= RKV_FAIL_INF_MISMATCH;
             if ((flags & RKV_FLAG_CAND_CONST) && !(flags & RKV_FLAG_REF_CONST) && D.n > 1)
                 verdict |= RKV_FAIL_LOOPHOLE_CONST;
             if ((flags & RKV_FLAG_CAND_COPY_OF_INPUT) && !(flags & RKV_FLAG_REF_COPY_OF_INPUT))
@@ -854,53 +913,49 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const Parti
 
 }  // namespace
 
-template <bool CB16, bool RB16, bool HAS_IN>
+template <bool CB16, bool RB16>
 static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
-                          int num_sms, Partial* partials, int32_t* status, cudaStream_t stream) {
-    const int smem = kOffData + kSmemDataBudget + 256;
+                          int grid_max, CandState* state, Partial* partials, int32_t* status,
+                          cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return RKV_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(verify_kernel<CB16, RB16, HAS_IN>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(verify_kernel<CB16, RB16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBytes) != cudaSuccess)
             return RKV_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    uint32_t grid = (uint32_t)num_sms * kBlocksPerSm;
-    if (grid > n_items) grid = n_items;
-    verify_kernel<CB16, RB16, HAS_IN><<<grid, kThreads, smem, stream>>>(d_tensors, T, K, k_begin, k_end,
-                                                                      n_items, partials, status);
+    // the grid is always the full resident grid: Partial rows are numbered by block
+    verify_kernel<CB16, RB16><<<grid_max, kThreads, kSmemBytes, stream>>>(d_tensors, T, K, k_begin, k_end,
+                                                                         n_items, state, partials, status);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
 int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
-                  const uint32_t variant_items[8], int num_sms, Partial* partials, int32_t* status,
-                  cudaStream_t stream) {
+                  const uint32_t variant_items[4], int grid, CandState* state, Partial* partials,
+                  int32_t* status, cudaStream_t stream) {
     int rc = RKV_OK;
-    for (int v = 0; v < 8 && rc == RKV_OK; ++v) {
+    for (int v = 0; v < 4 && rc == RKV_OK; ++v) {
         const uint32_t n = variant_items[v];
         if (!n) continue;
-#define RKV_LAUNCH(CB, RB, IN) \
-    launch_variant<CB, RB, IN>(d_tensors, T, K, k_begin, k_end, n, num_sms, partials, status, stream)
+#define RKV_LAUNCH(CB, RB) \
+    launch_variant<CB, RB>(d_tensors, T, K, k_begin, k_end, n, grid, state, partials, status, stream)
         switch (v) {
-            case 0: rc = RKV_LAUNCH(false, false, false); break;
-            case 1: rc = RKV_LAUNCH(false, false, true); break;
-            case 2: rc = RKV_LAUNCH(false, true, false); break;
-            case 3: rc = RKV_LAUNCH(false, true, true); break;
-            case 4: rc = RKV_LAUNCH(true, false, false); break;
-            case 5: rc = RKV_LAUNCH(true, false, true); break;
-            case 6: rc = RKV_LAUNCH(true, true, false); break;
-            default: rc = RKV_LAUNCH(true, true, true); break;
+            case 0: rc = RKV_LAUNCH(false, false); break;
+            case 1: rc = RKV_LAUNCH(false, true); break;
+            case 2: rc = RKV_LAUNCH(true, false); break;
+            default: rc = RKV_LAUNCH(true, true); break;
         }
 #undef RKV_LAUNCH
     }
     return rc;
 }
 
-int launch_finalize(const DevTensor* d_tensors, int T, int K, const Partial* partials,
-                    rkv_stats* stats_out, uint32_t* joint_pass, cudaStream_t stream) {
-    finalize_kernel<<<K, kFinThreads, 0, stream>>>(d_tensors, T, K, partials, stats_out, joint_pass);
+int launch_finalize(const DevTensor* d_tensors, int T, int K, const CandState* state,
+                    const Partial* partials, rkv_stats* stats_out, uint32_t* joint_pass,
+                    cudaStream_t stream) {
+    finalize_kernel<<<K, kFinThreads, 0, stream>>>(d_tensors, T, K, state, partials, stats_out, joint_pass);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 

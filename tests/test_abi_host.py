@@ -29,7 +29,7 @@ def declared_functions():
 def test_library_exports_every_declared_symbol():
     names = declared_functions()
     assert {"rkv_gen_inputs", "rkv_verify_batch", "rkv_verify_multi", "rkv_workspace_bytes",
-            "rkv_gen_inputs_ex", "rkv_verify_batch_host", "rkv_plan_slabs"} <= set(names)
+            "rkv_gen_inputs_ex", "rkv_verify_batch_host", "rkv_plan_items"} <= set(names)
     L = ctypes.CDLL(rkv.LIB_PATH)
     for name in names:
         assert hasattr(L, name), name
@@ -53,28 +53,36 @@ def test_stats_struct_is_88_bytes():
     assert ctypes.sizeof(rkv.TensorDescC) == 8 * 4 + 24 * 2 + 4 * 4 + 8
 
 
-@pytest.mark.parametrize("bpe", [2, 4, 6, 8])
-@pytest.mark.parametrize("n", [1, 127, 128, 129, 4096, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
-def test_slab_plan_properties(n, bpe):
-    S, cnt = rkv.plan_slabs(n, bpe, 148)
-    assert S % 128 == 0 and S >= 128
-    assert S * bpe <= 96 * 1024
-    assert (cnt - 1) * S < n <= cnt * S
-    grid = 148 * 2
-    if n >= grid * 128 * 4:
-        waves = -(-cnt // grid)
-        assert cnt / (waves * grid) > 0.97          # no wave is mostly empty
-    if n <= 128:
-        assert cnt == 1
+@pytest.mark.parametrize("K", [1, 2, 8, 63, 64, 65, 128, 256, 1000])
+@pytest.mark.parametrize("n", [1, 127, 3584, 3585, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
+def test_item_plan_properties(n, K):
+    sms = 148
+    grid = 2 * sms
+    tile, n_tiles, warm, pk_warm, pk_main = rkv.plan_items(n, K, sms)
+    assert tile == 3584 and tile % 8 == 0
+    assert (n_tiles - 1) * tile < n <= n_tiles * tile
+    assert 1 <= warm <= n_tiles
+    assert 1 <= pk_warm <= 64
+    parts_warm = -(-K // pk_warm)
+    if warm < grid:
+        # few tiles: the candidates are split so that most blocks get an item
+        assert warm * parts_warm >= 0.8 * min(grid, warm * K)
+    if warm < n_tiles:
+        # a large tensor: a short warm-up group, then balanced parts of at most 64
+        assert warm * tile >= 60000 and warm * 100 < n_tiles
+        parts = -(-K // 64)
+        assert pk_main == -(-K // parts)
+    else:
+        assert pk_main == 0
 
 
-def test_slab_plan_rejects_bad_arguments():
-    for args in [(0, 4, 148), (1000, 1, 148), (1000, 9, 148), (1000, 4, 0)]:
+def test_item_plan_rejects_bad_arguments():
+    for args in [(0, 4, 148), (1000, 0, 148), (1000, 4, 0)]:
         with pytest.raises(rkv.RkvError) as e:
-            rkv.plan_slabs(*args)
+            rkv.plan_items(*args)
         assert e.value.status == rkv.ERR_INVALID_ARG
     with pytest.raises(rkv.RkvError) as e:
-        rkv.plan_slabs(1 << 40, 4, 148)
+        rkv.plan_items(1 << 40, 4, 148)
     assert e.value.status == rkv.ERR_UNSUPPORTED
 
 

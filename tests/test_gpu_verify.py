@@ -77,9 +77,57 @@ def test_many_candidates_cross_the_merge_chunk_and_hint_limits(K):
     check_case(ref, cands, ATOL, RTOL, inp, where=f"K={K}")
 
 
+@pytest.mark.parametrize("cand_dtype", ["f32", "bf16"])
+def test_several_tiles_per_block_in_one_part(cand_dtype):
+    """More tiles than resident blocks: a block meets the same candidates tile after tile,
+    carries its running maxima over, and uses the maxima other blocks have published."""
+    n = 3584 * 296 * 2 + 3584 * 40 + 1234
+    ref = oracle_gen_tensor(77, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(77, 2, oracle.NORMAL, n, cand_dtype)
+    plan = mixed_plan(12, n, seed=77, bf16=cand_dtype == "bf16")
+    # equal maxima far apart: the first index must win across blocks and tiles
+    plan.append(pop.Candidate(pop.CORRUPT, delta=1.0, indices=(n - 5, n // 2, 3584 * 300 + 17)))
+    cands = build_case_cpu(plan, ref, inp, cand_dtype)
+    tol = (1e-5, 1e-5) if cand_dtype == "f32" else (1e-2, 1.6e-2)
+    check_case(ref, cands, tol[0], tol[1], inp, where=f"multi-tile {cand_dtype}")
+
+
+@pytest.mark.parametrize("cand_dtype", ["f32", "bf16"])
+def test_large_tensor_with_a_warm_up_group(cand_dtype):
+    """A tensor large enough to be cut into a leading group of tiles (verified first, by all
+    blocks) and the rest: results must not depend on which group an element falls in."""
+    tile = 3584
+    n = tile * 2100 + 77
+    ref = oracle_gen_tensor(88, 0, oracle.STUDENT_T2, n, "f32")
+    inp = oracle_gen_tensor(88, 2, oracle.STUDENT_T2, n, cand_dtype)
+    bf16 = cand_dtype == "bf16"
+    plan = [
+        pop.Candidate(pop.BF16_ULP if bf16 else pop.NOISE, sigma=1e-7, noise_seed=1),
+        # equal errors in the leading group and far behind it: the first index wins
+        pop.Candidate(pop.CORRUPT, delta=1.0, indices=(tile * 5 + 3, tile * 18 + 1, n - 2)),
+        # the only error lies behind the leading group
+        pop.Candidate(pop.CORRUPT, delta=1.0, indices=(tile * 1000 + 11,)),
+        pop.Candidate(pop.NAN_AT, indices=(tile * 17 + 3583,)),
+        pop.Candidate(pop.INF_AT, indices=(n - 1,)),
+        pop.Candidate(pop.INPUT_COPY),
+        pop.Candidate(pop.CONST, value=0.5),
+        pop.Candidate(pop.REF_EXACT),
+        pop.Candidate(pop.SCALE, factor=1.001),
+    ]
+    cands = build_case_cpu(plan, ref, inp, cand_dtype)
+    tol = (1e-5, 1e-5) if not bf16 else (1e-2, 1.6e-2)
+    got, want = check_case(ref, cands, tol[0], tol[1], inp, where=f"warm-up {cand_dtype}")
+    if not bf16:      # (bf16 rounding of the heavy tail outweighs the planted +1.0)
+        assert int(got[1]["argmax_abs_err"]) in (tile * 5 + 3, tile * 18 + 1, n - 2)
+    # and with the reference regenerated on the device
+    got2, _ = run_gpu(ref, cands, tol[0], tol[1], gen_ref=(88, 0, rkv.DIST_STUDENT_T2),
+                      gen_inp=(88, 2, rkv.DIST_STUDENT_T2))
+    assert got2.tobytes() == got.tobytes()
+
+
 @pytest.mark.parametrize("dist", oracle.DISTS)
 def test_every_distribution_several_slabs_per_block(dist):
-    n = 296 * 128 * 3 + 77            # three slabs per block on a 148-SM part, ragged tail
+    n = 296 * 128 * 3 + 77            # several tiles, ragged tail
     ref = oracle_gen_tensor(7, 0, dist, n, "f32")
     inp = oracle_gen_tensor(7, 2, dist, n, "f32")
     cands = build_case_cpu(mixed_plan(12, n, seed=dist), ref, inp, "f32")
