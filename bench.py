@@ -71,15 +71,21 @@ def kernel_source_hash() -> str:
 
 
 def recorded_traffic(workload: str, algo_bytes: float):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu
-    summary, scaled by algorithmic bytes; None if the kernel changed since."""
-    p = os.path.join(ROOT, "profiles", f"verify_kernel_{workload}.traffic.json")
+    """DRAM bytes per launch of the dominant kernel, from the committed ncu summary
+    (``profiles/verify_kernel_<workload>.md`` holds the measured DRAM bytes per
+    algorithmic byte of a smaller capture of the same kernel; traffic grows in proportion
+    to the bytes streamed).  None if there is no summary or the kernel changed since."""
+    p = os.path.join(ROOT, "profiles", f"verify_kernel_{workload}.md")
     try:
+        rec = {}
         with open(p) as fh:
-            rec = json.load(fh)
+            for line in fh:
+                if line.startswith("- ") and ":" in line:
+                    k, v = line[2:].split(":", 1)
+                    rec[k.strip()] = v.strip().strip("`")
         if rec.get("kernel_source_hash") != kernel_source_hash():
             return None
-        return rec["dram_bytes_per_algorithmic_byte"] * algo_bytes
+        return float(rec["dram_bytes_per_algorithmic_byte"]) * algo_bytes
     except Exception:
         return None
 
@@ -184,7 +190,8 @@ def build_workload(name: str, rank: int, max_dists: int = 0, cands_override: int
                 algo_bytes += W.K * n * csz + n * 4
                 launches += 2
             del cands
-        launches += 2                      # verify + finalize
+        variants = {(d.cands[0].dtype, None if d.ref is None else d.ref.dtype) for d in descs}
+        launches += len(variants) + 1      # one verify kernel per storage variant + finalize
         cases.append({"dist": dist_name, "descs": descs, "gens": gens, "K": W.K, "plan_last": plan,
                       "algo_bytes": algo_bytes, "launches": launches})
     torch.cuda.synchronize()
@@ -249,10 +256,8 @@ def run_native(args):
     barrier()
     elapsed_ms = t0.elapsed_time(t1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        tt = torch.tensor([elapsed_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
+    from paper_2509_14279_b200 import shard
+    elapsed_ms = shard.max_over_ranks(elapsed_ms, device="cuda")
 
     step_bytes = sum(c["algo_bytes"] for c in cases)
     value = world * step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
@@ -268,7 +273,8 @@ def run_native(args):
                 "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
                 "algorithmic_bytes_per_launch": launch_bytes,
                 "avg_launch_ms": round(statistics.mean(durs) * 1e3, 4),
-                "note": "events bracket rkv_verify_multi: table upload + verify_kernel + finalize_kernel",
+                "note": "events bracket rkv_verify_multi: table upload + workspace clear + verify_kernel "
+                        "(one per storage variant) + finalize_kernel",
                 "traffic": recorded_traffic(args.workload, launch_bytes)}
 
     # verdict sanity on the last case: every planted fault must fail
@@ -335,10 +341,8 @@ def run_e2e(args, W, case, world):
         rkv.verify_batch_host(ref_h, cands_h, d.atol, d.rtol)
     torch.cuda.synchronize()
     el = time.perf_counter() - t0
-    if world > 1:
-        tt = torch.tensor([el], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        el = float(tt.item())
+    from paper_2509_14279_b200 import shard
+    el = shard.max_over_ranks(el, device="cuda")
     return {"value": round(world * h2d * steps / el / 1e9, 2), "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
             "sample": f"one distribution ({case['dist']}) per step, pinned host buffers, "
@@ -377,7 +381,10 @@ def _oracle_sample_step(W, dist_id, n_s, k_s, threads, seed):
     return t_gen + t_ver, nbytes
 
 
-def cpu_baseline_sample(W):
+def cpu_baseline_sample(W, budget_s: float = 12.0):
+    """The oracle on the host cores, on a bounded sample of the workload: the first
+    distribution, a 4 Mi-element slice of the tensor, 16 candidates, repeated until
+    about `budget_s` seconds of oracle time have been spent."""
     import oracle
     from paper_2509_14279_b200 import population as pop
 
@@ -386,10 +393,15 @@ def cpu_baseline_sample(W):
     threads = min(cores, 16)
     n_s = min(W.numels[0], 1 << 22)
     k_s = 16
-    secs, nbytes = _oracle_sample_step(W, pop.DIST_IDS[W.dists[0]], n_s, k_s, threads, W.seeds[0])
+    secs, nbytes, reps = 0.0, 0, 0
+    while secs < budget_s and reps < 200:
+        s, b = _oracle_sample_step(W, pop.DIST_IDS[W.dists[0]], n_s, k_s, threads, W.seeds[0] + reps)
+        secs += s
+        nbytes += b
+        reps += 1
     return {"value": round(nbytes / secs / 1e9, 4), "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{W.dists[0]}: generate reference+input ({n_s} elements, 1 thread) and verify "
-                      f"{k_s} candidates of {n_s} elements on {threads} threads; {secs:.2f} s",
+            "sample": f"{W.dists[0]}: {reps} x (generate reference+input of {n_s} elements on 1 thread, "
+                      f"verify {k_s} candidates of {n_s} elements on {threads} threads); {secs:.1f} s of oracle time",
             "host_cores_available": cores}
 
 

@@ -277,16 +277,17 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
  * part past them.  A large tensor has two groups of items: the first *warm_tiles
- * tiles, with parts of *part_k_warm candidates (small, so that every resident
- * block -- 2 per SM -- gets an item), are verified first; the running maxima and
- * loophole flags they publish let the remaining tiles, with parts of
- * *part_k_main (<= 64) candidates, skip nearly all rare-path work.  A smaller
- * tensor has one group: *warm_tiles == *n_tiles and *part_k_main == 0.
+ * tiles, with the candidates cut into *parts_warm parts (many small ones, so that
+ * every resident block -- 2 per SM -- starts with one of these items), are
+ * verified first; the running maxima and loophole flags they publish let the
+ * remaining tiles, with *parts_main parts of at most 64 candidates, skip nearly
+ * all rare-path work.  A smaller tensor has one group: *warm_tiles == *n_tiles
+ * and *parts_main == 0.  Part p of P covers candidates [p*K/P, (p+1)*K/P).
  *   num_sms   SM count of the device
  * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, null), UNSUPPORTED (n >= 2^40).
  */
 int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t *tile_elems, uint32_t *n_tiles,
-                   uint32_t *warm_tiles, uint32_t *part_k_warm, uint32_t *part_k_main);
+                   uint32_t *warm_tiles, uint32_t *parts_warm, uint32_t *parts_main);
 
 /* Releases the library-owned scratch and staging buffers of all devices. */
 int rkv_release_cached(void);

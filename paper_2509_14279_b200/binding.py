@@ -141,7 +141,7 @@ def set_stream(stream=None) -> None:
 
 
 def plan_items(n: int, K: int, num_sms: int) -> tuple:
-    """Host-only: (tile_elems, n_tiles, warm_tiles, part_k_warm, part_k_main) for a tensor of
+    """Host-only: (tile_elems, n_tiles, warm_tiles, parts_warm, parts_main) for a tensor of
     n elements and K candidates."""
     v = [ctypes.c_uint32() for _ in range(5)]
     _check(lib().rkv_plan_items(int(n), int(K), int(num_sms), *[ctypes.byref(x) for x in v]),

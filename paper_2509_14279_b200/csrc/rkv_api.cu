@@ -31,8 +31,7 @@ static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t k_count
     const uint32_t groups[2] = {warm_tiles, n_tiles - warm_tiles};
     for (int g = 0; g < 2; ++g) {
         if (!groups[g]) continue;
-        const uint32_t pk = part_size(groups[g], k_count, grid);
-        items += (uint64_t)groups[g] * ((k_count + pk - 1) / pk);
+        items += (uint64_t)groups[g] * part_count(groups[g], k_count, grid);
     }
     return items;
 }
@@ -260,16 +259,16 @@ int rkv_set_stream(void* cuda_stream) {
 }
 
 int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t* tile_elems, uint32_t* n_tiles,
-                   uint32_t* warm_tiles, uint32_t* part_k_warm, uint32_t* part_k_main) {
-    if (!tile_elems || !n_tiles || !warm_tiles || !part_k_warm || !part_k_main) return RKV_ERR_INVALID_ARG;
+                   uint32_t* warm_tiles, uint32_t* parts_warm, uint32_t* parts_main) {
+    if (!tile_elems || !n_tiles || !warm_tiles || !parts_warm || !parts_main) return RKV_ERR_INVALID_ARG;
     if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
     if (K < 1 || num_sms < 1 || num_sms > (1 << 20)) return RKV_ERR_INVALID_ARG;
     const int rc = plan_one(n, n_tiles, warm_tiles);
     if (rc != RKV_OK) return rc;
     const uint32_t grid = (uint32_t)(num_sms * kBlocksPerSm);
     *tile_elems = kTileElems;
-    *part_k_warm = part_size(*warm_tiles, (uint32_t)K, grid);
-    *part_k_main = *warm_tiles < *n_tiles ? part_size(*n_tiles - *warm_tiles, (uint32_t)K, grid) : 0u;
+    *parts_warm = part_count(*warm_tiles, (uint32_t)K, grid);
+    *parts_main = *warm_tiles < *n_tiles ? part_count(*n_tiles - *warm_tiles, (uint32_t)K, grid) : 0u;
     return RKV_OK;
 }
 

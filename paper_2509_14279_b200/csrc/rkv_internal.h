@@ -70,7 +70,7 @@ struct DevTensor {
     // the remaining tiles with parts of up to kPartK candidates.  Group A runs first: the
     // maxima and loophole flags it publishes let group B skip almost all rare-path work.
     // Smaller tensors only have group A.  Within a group item = part * tiles + tile, with
-    // part_size() candidates per part.
+    // part_count() parts per group.
     // Items of the tensors of one storage variant are numbered consecutively, all A
     // groups before all B groups; block b takes items b, b + grid, ...
     uint32_t n_tiles;       // ceil(n / kTileElems)
@@ -107,17 +107,23 @@ int validate_tensors(const rkv_tensor_desc* tensors, int T, int K);
 int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num_sms, Plan* plan);
 int current_num_sms(int* num_sms);   // RKV_ERR_CUDA without a device
 
-// Candidates per part for `tiles` tiles and a launch over k_count candidates: balanced
-// parts of at most kPartK, more and smaller ones when there are fewer tiles than blocks.
+// Number of candidate parts for a group of `tiles` tiles in a launch over k_count
+// candidates: enough parts that none holds more than kPartK candidates, and, when the
+// group has fewer tiles than there are blocks, enough that every block gets an item
+// (tiles * parts >= grid where k_count allows).  Part p of `parts` covers the candidates
+// [p * k_count / parts, (p + 1) * k_count / parts): sizes differ by at most one.
 // The kernels and the host use this one rule.
-__host__ __device__ inline uint32_t part_size(uint32_t tiles, uint32_t k_count, uint32_t grid) {
+__host__ __device__ inline uint32_t part_count(uint32_t tiles, uint32_t k_count, uint32_t grid) {
     uint32_t parts = (k_count + kPartK - 1) / kPartK;
     if (tiles < grid) {
         const uint32_t want = (grid + tiles - 1) / tiles;
         if (want > parts) parts = want;
     }
-    if (parts > k_count) parts = k_count;
-    return (k_count + parts - 1) / parts;
+    return parts > k_count ? k_count : parts;
+}
+
+__host__ __device__ inline uint32_t part_begin(uint32_t part, uint32_t parts, uint32_t k_count) {
+    return (uint32_t)(((uint64_t)part * k_count) / parts);
 }
 
 // kernels (rkv_verify.cu / rkv_gen.cu)

@@ -161,7 +161,7 @@ struct Item {
     int t;
     uint32_t group;          // 0 = A (leading tiles, small parts), 1 = B
     uint32_t part, tile;     // tile is the tensor-wide tile index
-    uint32_t part_k;         // candidates per part in this group
+    uint32_t n_parts;        // candidate parts of this group
     uint32_t first_item;     // first item of this (tensor, group) in this launch
     uint32_t n_items;        // items of this (tensor, group)
 };
@@ -176,14 +176,14 @@ __device__ __forceinline__ bool decode_item(const DevTensor* __restrict__ tensor
             const uint32_t warm = tensors[t].warm_tiles;
             const uint32_t nt = g == 0 ? warm : tensors[t].n_tiles - warm;
             if (nt == 0) continue;
-            const uint32_t pk = part_size(nt, k_count, gridDim.x);
-            const uint32_t cnt = nt * ((k_count + pk - 1) / pk);
+            const uint32_t parts = part_count(nt, k_count, gridDim.x);
+            const uint32_t cnt = nt * parts;
             if (id - base < cnt) {
                 it.t = t;
                 it.group = g;
                 it.part = (id - base) / nt;
                 it.tile = (id - base) % nt + (g == 0 ? 0u : warm);
-                it.part_k = pk;
+                it.n_parts = parts;
                 it.first_item = base;
                 it.n_items = cnt;
                 return true;
@@ -233,8 +233,9 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
         Item it;
         if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
         const DevTensor& D = tensors[it.t];
-        const int k0 = k_begin + (int)(it.part * it.part_k);
-        const int k1 = min(k_end, k0 + (int)it.part_k);
+        const uint32_t k_count = (uint32_t)(k_end - k_begin);
+        const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
+        const int k1 = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count);
         const uint32_t part_key = (it.group << 31) | it.part;
         if (it.t != cur_t || part_key != cur_part) {
             __syncwarp();
@@ -287,7 +288,7 @@ struct RefRegs {
     float thr[E];      // atol + rtol*|r|, product and sum each rounded
     float thr_min;     // smallest threshold of the thread's elements
     float minarp;      // smallest non-zero |r|, +inf if all are zero
-    bool general;      // a non-finite reference value, or a ragged tile: element-by-element rule
+    bool general;      // a non-finite reference value: element-by-element rule
 };
 
 // The comparison rule for one element, every case included.
@@ -399,6 +400,12 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
             rb[j] = b;
         }
     }
+    if (!full) {
+        // positions past the end of the tensor hold 0 (the candidates get 0 there as well)
+#pragma unroll
+        for (int j = 0; j < E; ++j)
+            if (elem_off<VEC>(j, tid) >= len) rb[j] = 0u;
+    }
     bool nonfinite = false;
     uint32_t mn = 0xFFFFFFFFu;
     float tmin = kInf;
@@ -413,7 +420,7 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
     }
     R.thr_min = tmin;
     R.minarp = mn == 0xFFFFFFFFu ? kInf : __uint_as_float(mn + 1u);
-    R.general = nonfinite || !full;
+    R.general = nonfinite;
 }
 
 __device__ __forceinline__ unsigned long long hint_key(float v, uint32_t tile) {
@@ -513,7 +520,8 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
         } else {
 #pragma unroll
             for (int j = 0; j < E; ++j) {
-                if (e[j] > a.emax) { a.emax = e[j]; a.eoff = elem_off<VEC>(j, tid); }
+                // (positions past the end of a ragged tile hold zeros and never count)
+                if (e[j] > a.emax && elem_off<VEC>(j, tid) < len) { a.emax = e[j]; a.eoff = elem_off<VEC>(j, tid); }
                 const float ar = fabsf(R.r[j]);
                 // the warp's own record comes from earlier tiles: only a strictly larger
                 // quotient can replace it
@@ -685,8 +693,9 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         Item it;
         if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
         const DevTensor& D = tensors[it.t];
-        const int k0 = k_begin + (int)(it.part * it.part_k);
-        const int kc = min(k_end, k0 + (int)it.part_k) - k0;
+        const uint32_t k_count = (uint32_t)(k_end - k_begin);
+        const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
+        const int kc = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count) - k0;
         const uint32_t part_key = (it.group << 31) | it.part;
         const uint64_t start = (uint64_t)it.tile * kTileElems;
         const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
@@ -779,6 +788,24 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
             ++n_used;
+            if (len != (uint32_t)kTileElems) {
+                // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
+                // elements behind them come from global memory; positions past the end of the
+                // tensor get 0 against a reference of 0 (see load_ref): no error, never over
+                // tolerance, excluded from the relative error, and never the first maximum,
+                // because their offsets are larger than every real element's.
+                constexpr uint32_t CSZ = CB16 ? 2 : 4;
+                const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const uint32_t off = elem_off<VEC>(j, tid);
+                    if (off >= copied) {
+                        const uint32_t cb = off < len ? ld_elem_bits(ptrs[kk], CB16 ? RKV_BF16 : RKV_F32, start + off) : 0u;
+                        if (!CB16) w[j] = cb;
+                        else w[j >> 1] = (j & 1) ? ((w[j >> 1] & 0x0000FFFFu) | cb) : ((w[j >> 1] & 0xFFFF0000u) | (cb >> 16));
+                    }
+                }
+            }
             process_candidate<CB16>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
                                     it.tile, start, len, wanted, tid, lane);
         }

@@ -58,22 +58,20 @@ def test_stats_struct_is_88_bytes():
 def test_item_plan_properties(n, K):
     sms = 148
     grid = 2 * sms
-    tile, n_tiles, warm, pk_warm, pk_main = rkv.plan_items(n, K, sms)
+    tile, n_tiles, warm, parts_warm, parts_main = rkv.plan_items(n, K, sms)
     assert tile == 3584 and tile % 8 == 0
     assert (n_tiles - 1) * tile < n <= n_tiles * tile
     assert 1 <= warm <= n_tiles
-    assert 1 <= pk_warm <= 64
-    parts_warm = -(-K // pk_warm)
+    assert 1 <= parts_warm <= K and -(-K // parts_warm) <= 64
     if warm < grid:
-        # few tiles: the candidates are split so that most blocks get an item
-        assert warm * parts_warm >= 0.8 * min(grid, warm * K)
+        # few tiles: the candidates are split so that every block gets an item, if K allows
+        assert warm * parts_warm >= min(grid, warm * K)
     if warm < n_tiles:
-        # a large tensor: a short warm-up group, then balanced parts of at most 64
+        # a large tensor: a short warm-up group, then the fewest parts of at most 64
         assert warm * tile >= 60000 and warm * 100 < n_tiles
-        parts = -(-K // 64)
-        assert pk_main == -(-K // parts)
+        assert parts_main == -(-K // 64)
     else:
-        assert pk_main == 0
+        assert parts_main == 0
 
 
 def test_item_plan_rejects_bad_arguments():
