@@ -95,8 +95,7 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
         const uint64_t items = items_of(tiles, warm, (uint32_t)k_count, grid);
         total_items[plan->variant[t]] += items;
         if (total_items[plan->variant[t]] > 0x7FFFFFFFull) return RKV_ERR_UNSUPPORTED;
-        // a tensor with a group B gets one row per block, a small one a row per item at most
-        plan->n_slots[t] = (warm < tiles || items >= grid) ? grid : (uint32_t)items;
+        plan->n_slots[t] = grid;                 // one Partial row per block
         plan->slot_base[t] = (uint32_t)rows;
         rows += plan->n_slots[t];
     }
@@ -170,7 +169,7 @@ void fill_dev_tensor(DevTensor& d, const rkv_tensor_desc& s, const Plan& plan, i
 
 // Workspace pieces.
 struct Layout {
-    int32_t* status;
+    WorkspaceHeader* header;
     DevTensor* d_tensors;
     const void** d_ptrs;
     CandState* state;
@@ -180,7 +179,7 @@ struct Layout {
 Layout layout_of(void* workspace, const Plan& plan, int T) {
     unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
     Layout L;
-    L.status = reinterpret_cast<int32_t*>(ws);
+    L.header = reinterpret_cast<WorkspaceHeader*>(ws);
     L.d_tensors = reinterpret_cast<DevTensor*>(ws + sizeof(WorkspaceHeader));
     L.d_ptrs = reinterpret_cast<const void**>(ws + sizeof(WorkspaceHeader) + (size_t)T * sizeof(DevTensor));
     L.state = reinterpret_cast<CandState*>(ws + sizeof(WorkspaceHeader) + plan.table_bytes);
@@ -198,7 +197,7 @@ int launch_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k
         items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], kcount, plan.grid);
     (void)tensors;
     int rc = launch_verify(L.d_tensors, T, K, k_begin, k_end, items, (int)plan.grid, L.state, L.partials,
-                           L.status, stream);
+                           L.header, stream);
     if (rc != RKV_OK) return rc;
     if (finalize) rc = launch_finalize(L.d_tensors, T, K, L.state, L.partials, stats_out, joint_pass, stream);
     return rc;

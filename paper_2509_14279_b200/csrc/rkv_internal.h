@@ -72,10 +72,10 @@ struct DevTensor {
     // Smaller tensors only have group A.  Within a group item = part * tiles + tile, with
     // part_count() parts per group.
     // Items of the tensors of one storage variant are numbered consecutively, all A
-    // groups before all B groups; block b takes items b, b + grid, ...
+    // groups before all B groups; blocks take them in this order (see WorkspaceHeader).
     uint32_t n_tiles;       // ceil(n / kTileElems)
     uint32_t warm_tiles;    // tiles in group A (== n_tiles when there is no group B)
-    uint32_t n_slots;       // Partial rows of this tensor
+    uint32_t n_slots;       // Partial rows of this tensor: one per block of the grid
     uint32_t slot_base;     // first Partial row (K entries per row) of this tensor
     uint32_t variant;       // 2 * (candidates bf16) + (reference stored as bf16)
     uint32_t reserved[3];
@@ -83,7 +83,12 @@ struct DevTensor {
 
 struct WorkspaceHeader {
     int32_t status;        // rkv_status written by the device
-    uint32_t reserved[63];
+    // Work distribution of the verification kernel: every block starts with item blockIdx.x
+    // and then draws tickets; item = grid + ticket.  The last block to finish clears both
+    // words again, so that the next launch on the workspace starts from zero.
+    uint32_t next_ticket;
+    uint32_t blocks_done;
+    uint32_t reserved[61];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header size");
 
@@ -129,7 +134,7 @@ __host__ __device__ inline uint32_t part_begin(uint32_t part, uint32_t parts, ui
 // kernels (rkv_verify.cu / rkv_gen.cu)
 int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
                   const uint32_t variant_items[4], int grid, CandState* state, Partial* partials,
-                  int32_t* status, cudaStream_t stream);
+                  WorkspaceHeader* header, cudaStream_t stream);
 int launch_finalize(const DevTensor* d_tensors, int T, int K, const CandState* state,
                     const Partial* partials, rkv_stats* stats_out, uint32_t* joint_pass,
                     cudaStream_t stream);

@@ -41,6 +41,7 @@ namespace {
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr int E = kElemsPerThread;
 constexpr float kInf = __builtin_huge_valf();
+enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the producer's "no more items" mark
 
 // ----------------------------------------------------------------------------
 // shared-memory layout (dynamic)
@@ -70,13 +71,14 @@ constexpr int kOffFull = 0;                                   // kStages mbarrie
 constexpr int kOffEmpty = kOffFull + 8 * kStages;
 constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
 constexpr int kOffRefState = kOffAbort + 16;                  // 2 x uint32 settled bits of the reference (item parity)
-constexpr int kOffPtrC = 128;                                 // consumer copy of the pointers
+constexpr int kOffIds = kOffRefState + 8;                     // kStages x uint32: item id that starts in a stage
+constexpr int kOffPtrC = 256;                                 // consumer copy of the pointers
 constexpr int kOffPtrP = kOffPtrC + kPartK * 8;               // producer copy
 constexpr int kOffHint = kOffPtrP + kPartK * 8;               // two tables (item parity)
 constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
 constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
-static_assert(kOffPtrC >= kOffRefState + 8, "layout");
+static_assert(kOffPtrC >= kOffIds + 4 * kStages, "layout");
 static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
 // ----------------------------------------------------------------------------
@@ -145,6 +147,20 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
 }
 
+// The same barrier, returning whether any consumer thread passed a non-zero value.
+__device__ __forceinline__ bool consumer_sync_or(uint32_t v) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "barrier.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"(v), "n"(kConsumers)
+        : "memory");
+    return out != 0;
+}
+
 __device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
 __device__ __forceinline__ bool bits_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
 __device__ __forceinline__ bool bits_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
@@ -206,20 +222,23 @@ struct Ring {
 template <bool CB16, bool RB16>
 __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tensors, int T, int k_begin,
                                               int k_end, uint32_t n_items, unsigned char* smem,
-                                              const Ring& ring) {
+                                              const Ring& ring, WorkspaceHeader* header) {
     constexpr uint32_t CSZ = CB16 ? 2 : 4, RSZ = RB16 ? 2 : 4;
     constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
     const int lane = threadIdx.x & 31;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrP);
+    volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
     uint32_t n_issued = 0;
     int cur_t = -1;
     uint32_t cur_part = 0xFFFFFFFFu;
 
-    auto issue = [&](const unsigned char* src, uint32_t bytes) {
+    // mark: the id of the item that starts in this stage (kNoItem at the very end), else none
+    auto issue = [&](const unsigned char* src, uint32_t bytes, bool starts_item, uint32_t id) {
         const uint32_t s = n_issued % kStages;
         const uint32_t ph = (n_issued / kStages) & 1u;
         // the stage is free once every consumer warp has released its previous use
         mbar_wait(ring.empty0 + 8 * s, ph ^ 1u, ring.abort_flag);
+        if (starts_item) ids[s] = id;          // ordered before the arrive below
         if (bytes) {
             mbar_expect_tx(ring.full0 + 8 * s, bytes);
             bulk_g2s(ring.stage0 + s * kStageBytes, src, bytes, ring.full0 + 8 * s);
@@ -229,7 +248,14 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
         ++n_issued;
     };
 
-    for (uint32_t id = blockIdx.x; id < n_items; id += gridDim.x) {
+    // Every block starts with item blockIdx.x; after that lane 0 draws tickets, one ahead of
+    // the item it is issuing, so that the atomic's latency is never waited for.
+    uint32_t id = blockIdx.x;
+    for (;;) {
+        id = __shfl_sync(kFullMask, id, 0);
+        if (id >= n_items) break;
+        uint32_t next_id = 0;
+        if (lane == 0) next_id = gridDim.x + atomicAdd(&header->next_ticket, 1u);
         Item it;
         if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
         const DevTensor& D = tensors[it.t];
@@ -248,10 +274,26 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
         if (lane == 0) {
             const uint64_t start = (uint64_t)it.tile * kTileElems;
             const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
-            if (D.ref_src == RKV_SRC_POINTER)
-                issue(reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ, (len * RSZ) & ~15u);
+            bool first = true;
+            if (D.ref_src == RKV_SRC_POINTER) {
+                issue(reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ, (len * RSZ) & ~15u, true, id);
+                first = false;
+            }
             const uint32_t cbytes = (len * CSZ) & ~15u;
-            for (int k = k0; k < k1; ++k) issue(ptrs[k - k0] + start * CSZ, cbytes);
+            for (int k = k0; k < k1; ++k) {
+                issue(ptrs[k - k0] + start * CSZ, cbytes, first, id);
+                first = false;
+            }
+        }
+        id = next_id;
+    }
+    if (lane == 0) {
+        issue(nullptr, 0u, true, kNoItem);                     // tell the consumers to stop
+        // the last block to get here clears the ticket counter for the next launch
+        __threadfence();
+        if (atomicAdd(&header->blocks_done, 1u) == gridDim.x - 1u) {
+            header->next_ticket = 0u;
+            header->blocks_done = 0u;
         }
     }
     // A block that gave up must not retire with copies still landing in its shared
@@ -689,7 +731,15 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
     int cur_t = -1, cur_k0 = 0, cur_kc = 0;
     uint32_t cur_part = 0xFFFFFFFFu, cur_slot = 0;
 
-    for (uint32_t id = blockIdx.x; id < n_items; id += gridDim.x, ++ord) {
+    volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
+    for (;; ++ord) {
+        // The next item announces itself in the first ring stage it uses (which stays full
+        // until it is consumed below).  All consumers agree on stopping: at the producer's
+        // end mark, or when any thread of the block has given up on a wait.
+        const uint32_t s0 = n_used % kStages, ph0 = (n_used / kStages) & 1u;
+        const bool got = mbar_wait(ring.full0 + 8 * s0, ph0, ring.abort_flag);
+        const uint32_t id = got ? ids[s0] : kNoItem;
+        if (consumer_sync_or((id == kNoItem || id >= n_items || *ring.abort_flag) ? 1u : 0u)) break;
         Item it;
         if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
         const DevTensor& D = tensors[it.t];
@@ -708,11 +758,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid);
             if (tid < kc) ptrs[tid] = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
             cur_t = it.t; cur_part = part_key; cur_k0 = k0; cur_kc = kc;
-            // Partial row of this block for the tensor: a tensor with a group B has one row
-            // per block; a small tensor numbers the blocks from the one that owns its first item
-            cur_slot = D.warm_tiles < D.n_tiles
-                           ? blockIdx.x
-                           : (blockIdx.x + gridDim.x - it.first_item % gridDim.x) % gridDim.x;
+            cur_slot = blockIdx.x;                // one Partial row per block and tensor
         }
         // refresh the hints of this part from the published state
         if (tid < kc) {
@@ -820,7 +866,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
 template <bool CB16, bool RB16>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSm)
 verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
-              CandState* __restrict__ state, Partial* __restrict__ partials, int32_t* status) {
+              CandState* __restrict__ state, Partial* __restrict__ partials, WorkspaceHeader* header) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
     Ring ring;
@@ -838,10 +884,10 @@ verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, 
     }
     __syncthreads();
     if (tid >= kConsumers) {
-        producer_loop<CB16, RB16>(tensors, T, k_begin, k_end, n_items, smem, ring);
+        producer_loop<CB16, RB16>(tensors, T, k_begin, k_end, n_items, smem, ring, header);
     } else {
         consumer_loop<CB16, RB16>(tensors, T, K, k_begin, k_end, n_items, state, partials, smem, ring);
-        if (tid == 0 && *ring.abort_flag) atomicExch(status, (int32_t)RKV_ERR_TIMEOUT);
+        if (tid == 0 && *ring.abort_flag) atomicExch(&header->status, (int32_t)RKV_ERR_TIMEOUT);
     }
 }
 
@@ -942,7 +988,7 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandS
 
 template <bool CB16, bool RB16>
 static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
-                          int grid_max, CandState* state, Partial* partials, int32_t* status,
+                          int grid_max, CandState* state, Partial* partials, WorkspaceHeader* header,
                           cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -955,19 +1001,19 @@ static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin,
     }
     // the grid is always the full resident grid: Partial rows are numbered by block
     verify_kernel<CB16, RB16><<<grid_max, kThreads, kSmemBytes, stream>>>(d_tensors, T, K, k_begin, k_end,
-                                                                         n_items, state, partials, status);
+                                                                         n_items, state, partials, header);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
 int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
                   const uint32_t variant_items[4], int grid, CandState* state, Partial* partials,
-                  int32_t* status, cudaStream_t stream) {
+                  WorkspaceHeader* header, cudaStream_t stream) {
     int rc = RKV_OK;
     for (int v = 0; v < 4 && rc == RKV_OK; ++v) {
         const uint32_t n = variant_items[v];
         if (!n) continue;
 #define RKV_LAUNCH(CB, RB) \
-    launch_variant<CB, RB>(d_tensors, T, K, k_begin, k_end, n, grid, state, partials, status, stream)
+    launch_variant<CB, RB>(d_tensors, T, K, k_begin, k_end, n, grid, state, partials, header, stream)
         switch (v) {
             case 0: rc = RKV_LAUNCH(false, false); break;
             case 1: rc = RKV_LAUNCH(false, true); break;
