@@ -56,16 +56,19 @@ struct __align__(16) WarpRec {
 };
 static_assert(sizeof(WarpRec) == 32, "WarpRec layout");
 
-// Per candidate of the part, refreshed from global memory at the start of an item.
+// Per candidate of the part, rebuilt from the published state at the start of an item.
+// With (te, te_tile) the published maximum of |c - r| and the tile it was found in, an
+// element can still be the FIRST maximum only if it is larger, or equal and in a tile at or
+// before te_tile.  For the item's tile that is one comparison against te_x:
+//     te_x = tile <= te_tile ? (largest float below te) : te          (-1 if nothing published)
+// tq_x is the same for the relative error.
 struct __align__(16) Hint {
-    float te; uint32_t te_tile;      // published maximum of |c - r| and its tile (-1 / 0 if none)
-    float tq; uint32_t tq_tile;      // same for the relative error
-    float tq_pred;                   // largest float below tq (-1 when tq <= 0)
+    float te_x;
+    float tq_x;
     uint32_t settled;                // bit0: known to differ from element 0; bit1: from the input
-    uint32_t first;                  // storage bits of the candidate's element 0
-    uint32_t pad;
+    uint32_t first;                  // element 0 of the candidate as an fp32 bit pattern
 };
-static_assert(sizeof(Hint) == 32, "Hint layout");
+static_assert(sizeof(Hint) == 16, "Hint layout");
 
 constexpr int kOffFull = 0;                                   // kStages mbarriers
 constexpr int kOffEmpty = kOffFull + 8 * kStages;
@@ -511,29 +514,25 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
     const bool lane_gen = R.general || !(s < kInf);
     // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
     uint32_t cnt = 0;
-    if (__any_sync(kFullMask, m > R.thr_min)) {
+    const bool any_over = __any_sync(kFullMask, m > R.thr_min);
+    if (any_over) {
 #pragma unroll
         for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
     }
-    // can one of these elements be the first maximum?  (te, te_tile) is a published
-    // maximum: an element equal to it in a later tile, or anything smaller, cannot.
-    bool rare = (m > h.te) || (m == h.te && tile <= h.te_tile) || lane_gen;
-    // Relative error.  fl(e/|r|) > tq implies e > tq*|r| >= RD(tq*|r|); fl(e/|r|) >= tq
-    // implies the same with the float below tq; a tie only matters at or before the hint's
-    // tile.  First a test on the thread's largest e and smallest non-zero |r|; only if that
-    // passes somewhere in the warp, the same test element by element (errors proportional to
-    // |r|, as in an all-zero output, pass the first test everywhere).
-    {
-        const float tqx = tile <= h.tq_tile ? h.tq_pred : h.tq;
-        if (__any_sync(kFullMask, m > __fmul_rd(tqx, R.minarp))) {
-            bool hit = false;
+    // Can one of these elements be the first maximum?  See Hint.
+    bool rare = (m > h.te_x) || lane_gen;
+    // Relative error.  fl(e/|r|) > t implies e > t*|r| >= RD(t*|r|) for a representable
+    // t >= 0.  First a test on the thread's largest e and smallest non-zero |r|; only if
+    // that passes somewhere in the warp, the same test element by element (errors
+    // proportional to |r|, as in an all-zero output, pass the first test everywhere).
+    if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
+        bool hit = false;
 #pragma unroll
-            for (int j = 0; j < E; ++j) {
-                const float ar = fabsf(R.r[j]);
-                hit |= (ar != 0.0f) && (e[j] > __fmul_rd(tqx, ar));
-            }
-            rare |= hit;
+        for (int j = 0; j < E; ++j) {
+            const float ar = fabsf(R.r[j]);
+            hit |= (ar != 0.0f) && (e[j] > __fmul_rd(h.tq_x, ar));
         }
+        rare |= hit;
     }
 
     const bool any_gen = __any_sync(kFullMask, lane_gen);
@@ -612,7 +611,7 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
         for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
         if (lane == 0) rec->sum += (double)sf;
     }
-    {
+    if (any_over || any_gen) {
         const uint32_t tot = __reduce_add_sync(kFullMask, cnt);
         if (lane == 0 && tot) rec->n_over += tot;
     }
@@ -704,6 +703,16 @@ __device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D,
     }
 }
 
+// Published (maximum, tile) -> the threshold an element of `tile` has to exceed to
+// be able to become the first maximum (see Hint).
+__device__ __forceinline__ float hint_threshold(unsigned long long key, uint32_t tile) {
+    if (!(key >> 32)) return -1.0f;
+    const uint32_t bits = (uint32_t)(key >> 32) - 1u;
+    const uint32_t at_tile = ~(uint32_t)key;
+    if (tile > at_tile) return __uint_as_float(bits);
+    return bits ? __uint_as_float(bits - 1u) : -1.0f;       // the float below; below +0 anything goes
+}
+
 template <bool CB16, bool RB16>
 __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tensors, int T, int K, int k_begin,
                                               int k_end, uint32_t n_items, CandState* __restrict__ state,
@@ -726,7 +735,8 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
     }
 
-    uint32_t n_used = 0;            // ring items consumed so far (same order as the producer issues)
+    // next ring stage to consume and the parity of its current use (same order as the producer issues)
+    uint32_t cstage = 0, cphase = 0;
     uint32_t ord = 0;               // items this block has started
     int cur_t = -1, cur_k0 = 0, cur_kc = 0;
     uint32_t cur_part = 0xFFFFFFFFu, cur_slot = 0;
@@ -736,8 +746,8 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         // The next item announces itself in the first ring stage it uses (which stays full
         // until it is consumed below).  All consumers agree on stopping: at the producer's
         // end mark, or when any thread of the block has given up on a wait.
-        const uint32_t s0 = n_used % kStages, ph0 = (n_used / kStages) & 1u;
-        const bool got = mbar_wait(ring.full0 + 8 * s0, ph0, ring.abort_flag);
+        const uint32_t s0 = cstage;
+        const bool got = mbar_wait(ring.full0 + 8 * s0, cphase, ring.abort_flag);
         const uint32_t id = got ? ids[s0] : kNoItem;
         if (consumer_sync_or((id == kNoItem || id >= n_items || *ring.abort_flag) ? 1u : 0u)) break;
         Item it;
@@ -762,17 +772,12 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         }
         // refresh the hints of this part from the published state
         if (tid < kc) {
-            const CandState* s = st_t + k0 + tid;
-            const unsigned long long he = __ldcg(&s->hint_e), hq = __ldcg(&s->hint_q);
+            const CandState* sc = st_t + k0 + tid;
             Hint h;
-            h.te = (he >> 32) ? __uint_as_float((uint32_t)(he >> 32) - 1u) : -1.0f;
-            h.te_tile = (he >> 32) ? ~(uint32_t)he : 0u;
-            h.tq = (hq >> 32) ? __uint_as_float((uint32_t)(hq >> 32) - 1u) : -1.0f;
-            h.tq_tile = (hq >> 32) ? ~(uint32_t)hq : 0u;
-            h.tq_pred = h.tq > 0.0f ? __uint_as_float(__float_as_uint(h.tq) - 1u) : -1.0f;
-            h.settled = __ldcg(&s->mismatch);
+            h.te_x = hint_threshold(__ldcg(&sc->hint_e), it.tile);
+            h.tq_x = hint_threshold(__ldcg(&sc->hint_q), it.tile);
+            h.settled = __ldcg(&sc->mismatch);
             h.first = ld_elem_bits(ptrs[tid], CB16 ? RKV_BF16 : RKV_F32, 0);
-            h.pad = 0;
             H[tid] = h;
         }
         if (tid == kPartK) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
@@ -781,12 +786,12 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         RefRegs R;
         uint32_t rb[E];
         if (D.ref_src == RKV_SRC_POINTER) {
-            const uint32_t s = n_used % kStages, ph = (n_used / kStages) & 1u;
-            mbar_wait(ring.full0 + 8 * s, ph, ring.abort_flag);
+            const uint32_t s = cstage;
+            mbar_wait(ring.full0 + 8 * s, cphase, ring.abort_flag);
             load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)s * kStageBytes, tid);
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
-            ++n_used;
+            if (++cstage == (uint32_t)kStages) { cstage = 0; cphase ^= 1u; }
         } else {
             load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, tid);
         }
@@ -821,9 +826,9 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
 
         // ---- every candidate of the part ----------------------------------------------
         for (int kk = 0; kk < kc; ++kk) {
-            const uint32_t s = n_used % kStages, ph = (n_used / kStages) & 1u;
+            const uint32_t s = cstage;
             const Hint h = H[kk];
-            mbar_wait(ring.full0 + 8 * s, ph, ring.abort_flag);
+            mbar_wait(ring.full0 + 8 * s, cphase, ring.abort_flag);
             const unsigned char* stage = stages + (size_t)s * kStageBytes;
             uint32_t w[NW];
 #pragma unroll
@@ -833,7 +838,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
-            ++n_used;
+            if (++cstage == (uint32_t)kStages) { cstage = 0; cphase ^= 1u; }
             if (len != (uint32_t)kTileElems) {
                 // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
                 // elements behind them come from global memory; positions past the end of the
