@@ -334,6 +334,9 @@ struct RefRegs {
     float thr_min;     // smallest threshold of the thread's elements
     float minarp;      // smallest non-zero |r|, +inf if all are zero
     bool general;      // a non-finite reference value: element-by-element rule
+    // used with bf16 candidates only:
+    bool warp_has_zero;  // some thread of the warp holds a reference value of exactly 0
+    float atol, rtol;
 };
 
 // The comparison rule for one element, every case included.
@@ -451,7 +454,7 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
         for (int j = 0; j < E; ++j)
             if (elem_off<VEC>(j, tid) >= len) rb[j] = 0u;
     }
-    bool nonfinite = false;
+    bool nonfinite = false, has_zero = false;
     uint32_t mn = 0xFFFFFFFFu;
     float tmin = kInf;
 #pragma unroll
@@ -461,11 +464,17 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
         R.r[j] = __uint_as_float(rb[j]);
         R.thr[j] = __fadd_rn(D.atol, __fmul_rn(D.rtol, __uint_as_float(ab)));
         tmin = fminf(tmin, R.thr[j]);
+        has_zero |= ab == 0u;
         mn = min(mn, ab - 1u);       // |r| orders like its bits; zero wraps to the top
     }
     R.thr_min = tmin;
     R.minarp = mn == 0xFFFFFFFFu ? kInf : __uint_as_float(mn + 1u);
     R.general = nonfinite;
+    if (CB16) {
+        R.warp_has_zero = __any_sync(kFullMask, mn == 0xFFFFFFFFu || has_zero);
+        R.atol = D.atol;
+        R.rtol = D.rtol;
+    }
 }
 
 __device__ __forceinline__ unsigned long long hint_key(float v, uint32_t tile) {
@@ -512,27 +521,62 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
 
     // a NaN or an infinity anywhere makes the sum non-finite
     const bool lane_gen = R.general || !(s < kInf);
-    // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
-    uint32_t cnt = 0;
-    const bool any_over = __any_sync(kFullMask, m > R.thr_min);
-    if (any_over) {
-#pragma unroll
-        for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
-    }
     // Can one of these elements be the first maximum?  See Hint.
     bool rare = (m > h.te_x) || lane_gen;
     // Relative error.  fl(e/|r|) > t implies e > t*|r| >= RD(t*|r|) for a representable
     // t >= 0.  First a test on the thread's largest e and smallest non-zero |r|; only if
     // that passes somewhere in the warp, the same test element by element (errors
-    // proportional to |r|, as in an all-zero output, pass the first test everywhere).
-    if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
-        bool hit = false;
+    // proportional to |r|, as in an all-zero output or a bf16 rounding, pass the first
+    // test everywhere).
+    //
+    // Over tolerance.  m <= thr_min means e_j <= m <= thr_min <= thr_j for every element:
+    // none over.  That test, too, is weak for errors proportional to |r|, the normal case
+    // for bf16 outputs.  There, while the published relative maximum is at most rtol, the
+    // element-by-element relative test covers it: thr_j = fl(atol + fl(rtol*|r_j|)) >=
+    // RD(t*|r_j|) for 0 <= t <= rtol, so an element over tolerance is a hit of that test
+    // (where r_j = 0 the test is e_j > atol).  fp32 keeps the plain form: the extra
+    // registers cost it more than the saved counting brings.
+    uint32_t cnt = 0;
+    bool any_over;
+    if constexpr (!CB16) {
+        any_over = __any_sync(kFullMask, m > R.thr_min);
+        if (any_over) {
 #pragma unroll
-        for (int j = 0; j < E; ++j) {
-            const float ar = fabsf(R.r[j]);
-            hit |= (ar != 0.0f) && (e[j] > __fmul_rd(h.tq_x, ar));
+            for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
         }
-        rare |= hit;
+        if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
+            bool hit = false;
+#pragma unroll
+            for (int j = 0; j < E; ++j) {
+                const float ar = fabsf(R.r[j]);
+                hit |= (ar != 0.0f) && (e[j] > __fmul_rd(h.tq_x, ar));
+            }
+            rare |= hit;
+        }
+    } else {
+        bool maybe_over = m > R.thr_min;
+        if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
+            const bool rel_covers = h.tq_x >= 0.0f && h.tq_x <= R.rtol;
+            bool hit = false, zover = false;
+            if (R.warp_has_zero) {
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const float ar = fabsf(R.r[j]);
+                    if (ar != 0.0f) hit |= e[j] > __fmul_rd(h.tq_x, ar);
+                    else zover |= e[j] > R.atol;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < E; ++j) hit |= e[j] > __fmul_rd(h.tq_x, fabsf(R.r[j]));
+            }
+            if (rel_covers) maybe_over = hit || zover;
+            rare |= hit;
+        }
+        any_over = __any_sync(kFullMask, maybe_over);
+        if (any_over) {
+#pragma unroll
+            for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
+        }
     }
 
     const bool any_gen = __any_sync(kFullMask, lane_gen);
