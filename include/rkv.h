@@ -273,7 +273,9 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
 
 /*
  * Host-only planning helper (no CUDA call): how the work of one tensor is cut.
- * The tensor is cut into *n_tiles tiles of *tile_elems elements.  One work item is
+ * The tensor is cut into *n_tiles tiles of *tile_elems elements (a thread of the
+ * verification kernel owns 64 bytes of each candidate tile: 3584 fp32 or 7168 bf16
+ * elements per tile).  One work item is
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
  * part past them.  A large tensor has two groups of items: the first *warm_tiles
@@ -283,10 +285,11 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * remaining tiles, with *parts_main parts of at most 64 candidates, skip nearly
  * all rare-path work.  A smaller tensor has one group: *warm_tiles == *n_tiles
  * and *parts_main == 0.  Part p of P covers candidates [p*K/P, (p+1)*K/P).
- *   num_sms   SM count of the device
- * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, null), UNSUPPORTED (n >= 2^40).
+ *   cand_dtype  RKV_F32 | RKV_BF16 (storage type of the candidates)
+ *   num_sms     SM count of the device
+ * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, bad dtype, null), UNSUPPORTED (n >= 2^40).
  */
-int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t *tile_elems, uint32_t *n_tiles,
+int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t *tile_elems, uint32_t *n_tiles,
                    uint32_t *warm_tiles, uint32_t *parts_warm, uint32_t *parts_main);
 
 /* Releases the library-owned scratch and staging buffers of all devices. */

@@ -14,11 +14,12 @@ namespace rkv {
 // planning
 // ----------------------------------------------------------------------------
 
-// How one tensor is cut: tiles of kTileElems elements; a large tensor's first
+// How one tensor is cut: tiles of tile_elems(cand_dtype) elements; a large tensor's first
 // kWarmTiles tiles form the warm-up group (see DevTensor).
-static int plan_one(uint64_t n, uint32_t* n_tiles, uint32_t* warm_tiles) {
+static int plan_one(uint64_t n, int cand_dtype, uint32_t* n_tiles, uint32_t* warm_tiles) {
     if (n == 0 || n >= kMaxN) return RKV_ERR_INVALID_ARG;
-    const uint64_t tiles = (n + kTileElems - 1) / kTileElems;
+    const uint64_t te = tile_elems(cand_dtype);
+    const uint64_t tiles = (n + te - 1) / te;
     if (tiles > 0x3FFFFFFFull) return RKV_ERR_UNSUPPORTED;
     *n_tiles = (uint32_t)tiles;
     *warm_tiles = tiles >= (uint64_t)kWarmMinTiles ? (uint32_t)kWarmTiles : (uint32_t)tiles;
@@ -87,7 +88,7 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
     uint64_t rows = 0, total_items[4] = {0, 0, 0, 0};
     for (int t = 0; t < T; ++t) {
         uint32_t tiles, warm;
-        const int rc = plan_one(tensors[t].n, &tiles, &warm);
+        const int rc = plan_one(tensors[t].n, tensors[t].cand_dtype, &tiles, &warm);
         if (rc != RKV_OK) return rc;
         plan->n_tiles[t] = tiles;
         plan->warm_tiles[t] = warm;
@@ -257,15 +258,16 @@ int rkv_set_stream(void* cuda_stream) {
     return RKV_OK;
 }
 
-int rkv_plan_items(uint64_t n, int K, int num_sms, uint32_t* tile_elems, uint32_t* n_tiles,
+int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t* tile_elems_out, uint32_t* n_tiles,
                    uint32_t* warm_tiles, uint32_t* parts_warm, uint32_t* parts_main) {
-    if (!tile_elems || !n_tiles || !warm_tiles || !parts_warm || !parts_main) return RKV_ERR_INVALID_ARG;
+    if (!tile_elems_out || !n_tiles || !warm_tiles || !parts_warm || !parts_main) return RKV_ERR_INVALID_ARG;
+    if (!dtype_ok(cand_dtype)) return RKV_ERR_INVALID_ARG;
     if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
     if (K < 1 || num_sms < 1 || num_sms > (1 << 20)) return RKV_ERR_INVALID_ARG;
-    const int rc = plan_one(n, n_tiles, warm_tiles);
+    const int rc = plan_one(n, cand_dtype, n_tiles, warm_tiles);
     if (rc != RKV_OK) return rc;
     const uint32_t grid = (uint32_t)(num_sms * kBlocksPerSm);
-    *tile_elems = kTileElems;
+    *tile_elems_out = tile_elems(cand_dtype);
     *parts_warm = part_count(*warm_tiles, (uint32_t)K, grid);
     *parts_main = *warm_tiles < *n_tiles ? part_count(*n_tiles - *warm_tiles, (uint32_t)K, grid) : 0u;
     return RKV_OK;

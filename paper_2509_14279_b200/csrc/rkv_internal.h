@@ -14,9 +14,13 @@ constexpr int kConsumerWarps = 7;                    // warps that compare
 constexpr int kConsumers = kConsumerWarps * 32;      // 224 threads
 constexpr int kThreads = kConsumers + 32;            // + one warp that issues the bulk copies = 256
 constexpr int kBlocksPerSm = 2;                      // resident verification blocks per SM
-constexpr int kElemsPerThread = 16;                  // elements of a tile one thread owns
-constexpr int kTileElems = kConsumers * kElemsPerThread;   // 3584 elements per tile
-constexpr int kStageBytes = kTileElems * 4;          // one ring stage holds a tile of fp32
+constexpr int kStageBytes = kConsumers * 64;         // a ring stage: 64 bytes of a candidate per thread
+// A thread owns 64 bytes of each candidate tile: 16 fp32 or 32 bf16 elements.
+constexpr int kTileElemsF32 = kStageBytes / 4;       // 3584 elements per tile of fp32 candidates
+constexpr int kTileElemsBF16 = kStageBytes / 2;      // 7168 elements per tile of bf16 candidates
+__host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
+    return cand_dtype == RKV_BF16 ? kTileElemsBF16 : kTileElemsF32;
+}
 constexpr int kStages = 6;                           // ring depth (bulk copies in flight)
 constexpr int kPartK = 64;                           // candidates a block tracks at a time
 constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
@@ -73,7 +77,7 @@ struct DevTensor {
     // part_count() parts per group.
     // Items of the tensors of one storage variant are numbered consecutively, all A
     // groups before all B groups; blocks take them in this order (see WorkspaceHeader).
-    uint32_t n_tiles;       // ceil(n / kTileElems)
+    uint32_t n_tiles;       // ceil(n / tile_elems(cand_dtype))
     uint32_t warm_tiles;    // tiles in group A (== n_tiles when there is no group B)
     uint32_t n_slots;       // Partial rows of this tensor: one per block of the grid
     uint32_t slot_base;     // first Partial row (K entries per row) of this tensor

@@ -39,7 +39,6 @@ namespace rkv {
 namespace {
 
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
-constexpr int E = kElemsPerThread;
 constexpr float kInf = __builtin_huge_valf();
 enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the producer's "no more items" mark
 
@@ -72,7 +71,7 @@ static_assert(sizeof(Hint) == 16, "Hint layout");
 
 constexpr int kOffFull = 0;                                   // kStages mbarriers
 constexpr int kOffEmpty = kOffFull + 8 * kStages;
-constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
+constexpr int kOffAbort = kOffEmpty + 8 * kStages;         // uint32
 constexpr int kOffRefState = kOffAbort + 16;                  // 2 x uint32 settled bits of the reference (item parity)
 constexpr int kOffIds = kOffRefState + 8;                     // kStages x uint32: item id that starts in a stage
 constexpr int kOffPtrC = 256;                                 // consumer copy of the pointers
@@ -83,6 +82,19 @@ constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpR
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
 static_assert(kOffPtrC >= kOffIds + 4 * kStages, "layout");
 static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
+
+// Geometry of a tile.  A thread owns 64 bytes of each candidate tile, so a candidate tile
+// always fills exactly one ring stage: 16 fp32 elements or 32 bf16 elements.  Their
+// reference values stay in registers for the whole item.  With fp32 candidates the
+// tolerance thresholds do too; with bf16 candidates they are recomputed in the rare case
+// that needs them (see process_candidate_b16).
+template <bool CB16>
+struct Geo {
+    static constexpr int E = CB16 ? 32 : 16;            // elements per thread
+    static constexpr int VEC = CB16 ? 8 : 4;            // elements per 16-byte piece
+    static constexpr int NW = 16;                       // 32-bit words per thread and candidate tile
+    static constexpr int kTile = kConsumers * E;        // elements per tile
+};
 
 // ----------------------------------------------------------------------------
 // small PTX helpers
@@ -228,6 +240,8 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
                                               const Ring& ring, WorkspaceHeader* header) {
     constexpr uint32_t CSZ = CB16 ? 2 : 4, RSZ = RB16 ? 2 : 4;
     constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
+    constexpr uint32_t kTile = Geo<CB16>::kTile;
+    constexpr uint32_t kRefStages = (CB16 && !RB16) ? 2 : 1;      // an fp32 tile under bf16 candidates
     const int lane = threadIdx.x & 31;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrP);
     volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
@@ -275,12 +289,18 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
             cur_part = part_key;
         }
         if (lane == 0) {
-            const uint64_t start = (uint64_t)it.tile * kTileElems;
-            const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
+            const uint64_t start = (uint64_t)it.tile * kTile;
+            const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
             bool first = true;
             if (D.ref_src == RKV_SRC_POINTER) {
-                issue(reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ, (len * RSZ) & ~15u, true, id);
-                first = false;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ;
+                const uint32_t rbytes = (len * RSZ) & ~15u;
+                for (uint32_t rs = 0; rs < kRefStages; ++rs) {
+                    const uint32_t lo = rs * kStageBytes;
+                    const uint32_t b = rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u;
+                    issue(src + lo, b, first, id);
+                    first = false;
+                }
             }
             const uint32_t cbytes = (len * CSZ) & ~15u;
             for (int k = k0; k < k1; ++k) {
@@ -302,7 +322,7 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
     // A block that gave up must not retire with copies still landing in its shared
     // memory: wait (bounded) for the copies issued last.
     if (lane == 0 && *ring.abort_flag) {
-        const uint32_t pending = n_issued < (uint32_t)kStages ? n_issued : (uint32_t)kStages;
+        const uint32_t pending = n_issued < kStages ? n_issued : kStages;
         for (uint32_t i = 0; i < pending; ++i) {
             const uint32_t q = n_issued - 1 - i;
             const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
@@ -318,7 +338,7 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
 // ----------------------------------------------------------------------------
 // consumer side: per-thread view of a tile
 // ----------------------------------------------------------------------------
-// A thread owns E = 16 elements of the tile as NV vectors of VEC elements
+// A thread owns E elements of the tile (see Geo) as vectors of VEC elements
 // (one 16-byte piece of a candidate each): vector jv of thread tid is vector
 // jv * 224 + tid of the tile.  Element j = jv * VEC + i of the thread has the
 // tile offset below; offsets grow with j.
@@ -328,15 +348,25 @@ __device__ __forceinline__ uint32_t elem_off(int j, int tid) {
 }
 
 // What a thread keeps for the whole item.
-struct RefRegs {
-    float r[E];        // reference values
-    float thr[E];      // atol + rtol*|r|, product and sum each rounded
+template <bool CB16>
+struct RefRegs;
+
+template <>
+struct RefRegs<false> {
+    float r[16];       // reference values
+    float thr[16];     // atol + rtol*|r|, product and sum each rounded
     float thr_min;     // smallest threshold of the thread's elements
     float minarp;      // smallest non-zero |r|, +inf if all are zero
     bool general;      // a non-finite reference value: element-by-element rule
-    // used with bf16 candidates only:
-    bool warp_has_zero;  // some thread of the warp holds a reference value of exactly 0
-    float atol, rtol;
+};
+
+template <>
+struct RefRegs<true> {
+    float r[32];          // reference values
+    float atol, rtol;     // (thresholds are recomputed where they are needed)
+    float thr_min;        // smallest threshold of the thread's elements
+    bool general;         // a non-finite reference value: element-by-element rule
+    bool warp_has_zero;   // some thread of the warp holds a reference value of exactly 0
 };
 
 // The comparison rule for one element, every case included.
@@ -407,13 +437,22 @@ __device__ __forceinline__ uint32_t first_elem_bits(const void* ptr, int src, in
 }
 
 // Load (or regenerate) the thread's reference values for a tile and derive what
-// depends on them alone.  `stage` holds the bulk-copied part of the tile
-// (ref_copied elements); anything beyond comes from global memory.
+// depends on them alone.  The bulk-copied part of the tile sits in ring stage
+// `stage_a` (and, for an fp32 reference under bf16 candidates, continues in
+// `stage_b`); anything beyond comes from global memory.  `rb` returns all E values as
+// fp32 bit patterns (for the reference's own loophole flags); `ref_s` is the thread's
+// shared-memory home for them with bf16 candidates.
 template <bool CB16, bool RB16>
-__device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const DevTensor& D, uint64_t start,
-                                         uint32_t len, const unsigned char* stage, int tid) {
-    constexpr int VEC = CB16 ? 8 : 4;
-    const bool full = len == (uint32_t)kTileElems;
+__device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB16>::E], const DevTensor& D,
+                                         uint64_t start, uint32_t len, const unsigned char* stage_a,
+                                         const unsigned char* stage_b, int tid) {
+    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC;
+    constexpr uint32_t RSZ = RB16 ? 2 : 4;
+    const bool full = len == (uint32_t)Geo<CB16>::kTile;
+    // byte `b` of the reference tile in the ring
+    auto at = [&](uint32_t b) -> const unsigned char* {
+        return b < (uint32_t)kStageBytes ? stage_a + b : stage_b + (b - kStageBytes);
+    };
     if (D.ref_src == RKV_SRC_GENERATED) {
 #pragma unroll
         for (int g = 0; g < E / 4; ++g) {
@@ -428,22 +467,21 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
         for (int g = 0; g < E / 4; ++g) {
             const uint32_t off0 = elem_off<VEC>(4 * g, tid);
             if (RB16) {
-                const uint2 t = *reinterpret_cast<const uint2*>(stage + (size_t)off0 * 2);
+                const uint2 t = *reinterpret_cast<const uint2*>(at(off0 * 2));
                 rb[4 * g + 0] = t.x << 16; rb[4 * g + 1] = t.x & 0xFFFF0000u;
                 rb[4 * g + 2] = t.y << 16; rb[4 * g + 3] = t.y & 0xFFFF0000u;
             } else {
-                const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)off0 * 4);
+                const uint4 t = *reinterpret_cast<const uint4*>(at(off0 * 4));
                 rb[4 * g + 0] = t.x; rb[4 * g + 1] = t.y; rb[4 * g + 2] = t.z; rb[4 * g + 3] = t.w;
             }
         }
     } else {
-        constexpr uint32_t RSZ = RB16 ? 2 : 4;
         const uint32_t copied = ((len * RSZ) & ~15u) / RSZ;
 #pragma unroll
         for (int j = 0; j < E; ++j) {
             const uint32_t off = elem_off<VEC>(j, tid);
             uint32_t b = 0;
-            if (off < copied) b = ld_elem_bits(stage, RB16 ? RKV_BF16 : RKV_F32, off);
+            if (off < copied) b = ld_elem_bits(at(off * RSZ), RB16 ? RKV_BF16 : RKV_F32, 0);
             else if (off < len) b = ld_elem_bits(D.ref, RB16 ? RKV_BF16 : RKV_F32, start + off);
             rb[j] = b;
         }
@@ -454,6 +492,7 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
         for (int j = 0; j < E; ++j)
             if (elem_off<VEC>(j, tid) >= len) rb[j] = 0u;
     }
+    const float atol = D.atol, rtol = D.rtol;
     bool nonfinite = false, has_zero = false;
     uint32_t mn = 0xFFFFFFFFu;
     float tmin = kInf;
@@ -461,19 +500,24 @@ __device__ __forceinline__ void load_ref(RefRegs& R, uint32_t (&rb)[E], const De
     for (int j = 0; j < E; ++j) {
         const uint32_t ab = rb[j] & 0x7FFFFFFFu;
         nonfinite |= !bits_finite(rb[j]);
+        const float thr = __fadd_rn(atol, __fmul_rn(rtol, __uint_as_float(ab)));
         R.r[j] = __uint_as_float(rb[j]);
-        R.thr[j] = __fadd_rn(D.atol, __fmul_rn(D.rtol, __uint_as_float(ab)));
-        tmin = fminf(tmin, R.thr[j]);
-        has_zero |= ab == 0u;
-        mn = min(mn, ab - 1u);       // |r| orders like its bits; zero wraps to the top
+        tmin = fminf(tmin, thr);
+        if constexpr (CB16) {
+            has_zero |= ab == 0u;
+        } else {
+            R.thr[j] = thr;
+            mn = min(mn, ab - 1u);   // |r| orders like its bits; zero wraps to the top
+        }
     }
     R.thr_min = tmin;
-    R.minarp = mn == 0xFFFFFFFFu ? kInf : __uint_as_float(mn + 1u);
     R.general = nonfinite;
-    if (CB16) {
-        R.warp_has_zero = __any_sync(kFullMask, mn == 0xFFFFFFFFu || has_zero);
-        R.atol = D.atol;
-        R.rtol = D.rtol;
+    if constexpr (CB16) {
+        R.atol = atol;
+        R.rtol = rtol;
+        R.warp_has_zero = __any_sync(kFullMask, has_zero);
+    } else {
+        R.minarp = mn == 0xFFFFFFFFu ? kInf : __uint_as_float(mn + 1u);
     }
 }
 
@@ -488,6 +532,63 @@ __device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[NW], int j) {
     return (j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16);
 }
 
+// Loophole flags of one candidate tile, until a difference has been seen.
+template <bool CB16>
+__device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const Hint& h, Hint* h_smem,
+                                                CandState* st, const DevTensor& D, const void* cand_g,
+                                                uint64_t start, uint32_t len, uint32_t wanted_flags, int tid,
+                                                int lane) {
+    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
+    constexpr uint32_t CSZ = CB16 ? 2 : 4;
+    // `settled` is the one hint field other warps update while this warp reads it: take
+    // lane 0's copy so that the branch below is uniform across the warp.
+    const uint32_t need = wanted_flags & ~__shfl_sync(kFullMask, h.settled, 0);
+    if (need) {
+        uint32_t acc1 = 0, acc2 = 0;
+        const bool full = len == (uint32_t)Geo<CB16>::kTile;
+        if (full && (need & 1u)) {
+            const uint32_t f = CB16 ? (h.first >> 16) * 0x10001u : h.first;
+#pragma unroll
+            for (int i = 0; i < NW; ++i) acc1 |= w[i] ^ f;
+        }
+        if (full && (need & 2u) && D.input_src == RKV_SRC_POINTER) {
+            // the input has the candidates' dtype: compare the 16-byte pieces as stored
+            const uint4* in = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(D.input) +
+                                                             start * CSZ) + tid;
+#pragma unroll
+            for (int jv = 0; jv < E / VEC; ++jv) {
+                const uint4 t = __ldg(in + jv * kConsumers);
+                acc2 |= (w[4 * jv] ^ t.x) | (w[4 * jv + 1] ^ t.y) | (w[4 * jv + 2] ^ t.z) | (w[4 * jv + 3] ^ t.w);
+            }
+        } else if (!full || (need & 2u)) {
+            const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+#pragma unroll
+            for (int g = 0; g < E / 4; ++g) {
+                const uint32_t off0 = elem_off<VEC>(4 * g, tid);
+                uint32_t in[4] = {0, 0, 0, 0};
+                if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t off = off0 + i;
+                    if (off < len) {
+                        uint32_t cb = cand_bits<CB16, NW>(w, 4 * g + i);
+                        if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
+                        if (!full) acc1 |= cb ^ h.first;
+                        acc2 |= cb ^ in[i];
+                    }
+                }
+            }
+        }
+        uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
+                        (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
+        seen &= need;
+        if (lane == 0 && seen) {
+            atomicOr(&st->mismatch, seen);
+            atomicOr(&h_smem->settled, seen);
+        }
+    }
+}
+
 // One candidate tile against the thread's reference registers.
 //   w        the thread's 16-byte pieces of the candidate tile (from the ring)
 //   h        the candidate's hint entry (a snapshot; see the file header)
@@ -496,13 +597,13 @@ __device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[NW], int j) {
 //   cand_g   the candidate tensor in global memory (only the last < 16 bytes of a
 //            ragged tensor are read from there)
 template <bool CB16>
-__device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32_t (&w)[CB16 ? E / 2 : E],
+__device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const uint32_t (&w)[16],
                                                   const Hint& h, Hint* h_smem, WarpRec* rec, CandState* st,
                                                   const DevTensor& D, const void* cand_g, uint32_t tile,
                                                   uint64_t start, uint32_t len, uint32_t wanted_flags,
                                                   int tid, int lane) {
-    constexpr int VEC = CB16 ? 8 : 4;
-    constexpr int NW = CB16 ? E / 2 : E;
+    static_assert(!CB16, "bf16 candidates take process_candidate_b16");
+    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
     constexpr uint32_t CSZ = CB16 ? 2 : 4;
 
     // ---- common path ---------------------------------------------------------------
@@ -521,62 +622,27 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
 
     // a NaN or an infinity anywhere makes the sum non-finite
     const bool lane_gen = R.general || !(s < kInf);
+    // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
+    uint32_t cnt = 0;
+    const bool any_over = __any_sync(kFullMask, m > R.thr_min);
+    if (any_over) {
+#pragma unroll
+        for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
+    }
     // Can one of these elements be the first maximum?  See Hint.
     bool rare = (m > h.te_x) || lane_gen;
     // Relative error.  fl(e/|r|) > t implies e > t*|r| >= RD(t*|r|) for a representable
     // t >= 0.  First a test on the thread's largest e and smallest non-zero |r|; only if
     // that passes somewhere in the warp, the same test element by element (errors
-    // proportional to |r|, as in an all-zero output or a bf16 rounding, pass the first
-    // test everywhere).
-    //
-    // Over tolerance.  m <= thr_min means e_j <= m <= thr_min <= thr_j for every element:
-    // none over.  That test, too, is weak for errors proportional to |r|, the normal case
-    // for bf16 outputs.  There, while the published relative maximum is at most rtol, the
-    // element-by-element relative test covers it: thr_j = fl(atol + fl(rtol*|r_j|)) >=
-    // RD(t*|r_j|) for 0 <= t <= rtol, so an element over tolerance is a hit of that test
-    // (where r_j = 0 the test is e_j > atol).  fp32 keeps the plain form: the extra
-    // registers cost it more than the saved counting brings.
-    uint32_t cnt = 0;
-    bool any_over;
-    if constexpr (!CB16) {
-        any_over = __any_sync(kFullMask, m > R.thr_min);
-        if (any_over) {
+    // proportional to |r|, as in an all-zero output, pass the first test everywhere).
+    if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
+        bool hit = false;
 #pragma unroll
-            for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
+        for (int j = 0; j < E; ++j) {
+            const float ar = fabsf(R.r[j]);
+            hit |= (ar != 0.0f) && (e[j] > __fmul_rd(h.tq_x, ar));
         }
-        if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
-            bool hit = false;
-#pragma unroll
-            for (int j = 0; j < E; ++j) {
-                const float ar = fabsf(R.r[j]);
-                hit |= (ar != 0.0f) && (e[j] > __fmul_rd(h.tq_x, ar));
-            }
-            rare |= hit;
-        }
-    } else {
-        bool maybe_over = m > R.thr_min;
-        if (__any_sync(kFullMask, m > __fmul_rd(h.tq_x, R.minarp))) {
-            const bool rel_covers = h.tq_x >= 0.0f && h.tq_x <= R.rtol;
-            bool hit = false, zover = false;
-            if (R.warp_has_zero) {
-#pragma unroll
-                for (int j = 0; j < E; ++j) {
-                    const float ar = fabsf(R.r[j]);
-                    if (ar != 0.0f) hit |= e[j] > __fmul_rd(h.tq_x, ar);
-                    else zover |= e[j] > R.atol;
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < E; ++j) hit |= e[j] > __fmul_rd(h.tq_x, fabsf(R.r[j]));
-            }
-            if (rel_covers) maybe_over = hit || zover;
-            rare |= hit;
-        }
-        any_over = __any_sync(kFullMask, maybe_over);
-        if (any_over) {
-#pragma unroll
-            for (int j = 0; j < E; ++j) cnt += (e[j] > R.thr[j]) ? 1u : 0u;
-        }
+        rare |= hit;
     }
 
     const bool any_gen = __any_sync(kFullMask, lane_gen);
@@ -660,61 +726,198 @@ __device__ __forceinline__ void process_candidate(const RefRegs& R, const uint32
         if (lane == 0 && tot) rec->n_over += tot;
     }
 
-    // ---- loophole flags, until a difference has been seen ---------------------------
-    // `settled` is the one hint field other warps update while this warp reads it: take
-    // lane 0's copy so that the branch below is uniform across the warp.
-    const uint32_t need = wanted_flags & ~__shfl_sync(kFullMask, h.settled, 0);
-    if (need) {
-        uint32_t acc1 = 0, acc2 = 0;
-        const bool full = len == (uint32_t)kTileElems;
-        if (full && (need & 1u)) {
-            const uint32_t f = CB16 ? (h.first >> 16) * 0x10001u : h.first;
+    candidate_flags<CB16>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+}
+
+// c - r for the bf16 value c in the low (half = 0) or high 16 bits of x: the bf16 value
+// widened exactly, one fp32 subtraction rounded to nearest (a mixed-precision instruction
+// of sm_100).
+__device__ __forceinline__ float sub_bf16_f32(uint32_t x, int half, float r) {
+    float d;
+    if (half)
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+    else
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+    return d;
+}
+
+// One pass over a thread's 32 elements of a bf16 candidate tile: largest and summed
+// |c - r|, and the largest d_j = fma(-t, |r_j|, e_j) for the relative-error threshold t
+// (see process_candidate_b16).  HAS_ZERO: reference values of exactly 0 may occur; they
+// take no part in the relative error, and `zover` tells whether one of them has an error
+// above atol.
+template <bool HAS_ZERO>
+__device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t (&w)[16], float t, float& m_out,
+                                         float& s_out, float& dm_out, bool& zover_out) {
+    const float nt = -t;
+    float m = 0.0f, dm = -kInf;
+    float sg[8];
+    bool zover = false;
 #pragma unroll
-            for (int i = 0; i < NW; ++i) acc1 |= w[i] ^ f;
-        }
-        if (full && (need & 2u) && D.input_src == RKV_SRC_POINTER) {
-            // the input has the candidates' dtype: compare the 16-byte pieces as stored
-            const uint4* in = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(D.input) +
-                                                             start * CSZ) + tid;
+    for (int g = 0; g < 8; ++g) {
+        float e[4], d[4];
 #pragma unroll
-            for (int jv = 0; jv < E / VEC; ++jv) {
-                const uint4 t = __ldg(in + jv * kConsumers);
-                acc2 |= (w[4 * jv] ^ t.x) | (w[4 * jv + 1] ^ t.y) | (w[4 * jv + 2] ^ t.z) | (w[4 * jv + 3] ^ t.w);
+        for (int i = 0; i < 4; ++i) {
+            const int j = 4 * g + i;
+            e[i] = fabsf(sub_bf16_f32(w[j >> 1], j & 1, R.r[j]));
+            float ar = fabsf(R.r[j]);
+            if (HAS_ZERO) {
+                const bool z = ar == 0.0f;
+                zover |= z && e[i] > R.atol;
+                ar = z ? kInf : ar;          // d = -inf (t > 0), NaN (t = 0; max skips it), +inf (t < 0)
             }
-        } else if (!full || (need & 2u)) {
-            const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+            d[i] = __fmaf_rn(nt, ar, e[i]);
+        }
+        m = fmaxf(fmaxf(m, fmaxf(e[0], e[1])), fmaxf(e[2], e[3]));
+        dm = fmaxf(fmaxf(dm, fmaxf(d[0], d[1])), fmaxf(d[2], d[3]));
+        sg[g] = __fadd_rn(__fadd_rn(e[0], e[1]), __fadd_rn(e[2], e[3]));
+    }
+    m_out = m;
+    dm_out = dm;
+    zover_out = zover;
+    s_out = __fadd_rn(__fadd_rn(__fadd_rn(sg[0], sg[1]), __fadd_rn(sg[2], sg[3])),
+                      __fadd_rn(__fadd_rn(sg[4], sg[5]), __fadd_rn(sg[6], sg[7])));
+}
+
+// One tile of a bf16 candidate (32 elements per thread) against the thread's reference
+// registers.  Same results as process_candidate; the tests that keep the rare work rare
+// are arranged for errors proportional to |r|, the normal case of a rounded bf16 output,
+// against which a test on the thread's largest error is powerless.
+//
+// Relative error.  With t = h.tq_x, element j can be a first maximum only if
+// fl(e_j / |r_j|) > t, which implies e_j > t * |r_j| exactly (t is representable, rounding
+// is monotone).  d_j = fma(-t, |r_j|, e_j) has the sign of that exact difference, except
+// that a positive difference below the subnormal range rounds to zero; such a difference
+// needs e_j < 2^-100 (the product has 48 significant bits).  So the elements pass as a
+// whole when max_j d_j < 0, or = 0 with the thread's largest error 0 or at least 2^-100.
+// t < 0 says that nothing is published yet, or a tie at 0 could still win: no filtering.
+//
+// Over tolerance.  thr_j = fl(atol + fl(rtol * |r_j|)) >= fl(rtol * |r_j|), and a float
+// e_j above fl(P) is above P itself, so e_j > thr_j implies e_j > rtol * |r_j| >= t * |r_j|
+// whenever 0 <= t <= rtol: while the published relative maximum is at most rtol, an element
+// over tolerance also fails the test above (where r_j = 0 the test is e_j > atol).
+// Otherwise: m <= thr_min means e_j <= m <= thr_min <= thr_j for every element.
+__device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, const uint32_t (&w)[16],
+                                                      const Hint& h, Hint* h_smem, WarpRec* rec,
+                                                      CandState* st, const DevTensor& D, const void* cand_g,
+                                                      uint32_t tile, uint64_t start, uint32_t len,
+                                                      uint32_t wanted_flags, int tid, int lane) {
+    constexpr int VEC = 8;
+    constexpr float kTiny = 7.8886090522101181e-31f;      // 2^-100
+    // candidate element j as an fp32 bit pattern
+    auto cbits = [&](int j) -> uint32_t {
+        const uint32_t x = w[j >> 1];
+        return (j & 1) ? (x & 0xFFFF0000u) : (x << 16);
+    };
+
+    // ---- common path ---------------------------------------------------------------
+    float m, s, dm;
+    bool zover;
+    if (R.warp_has_zero) pass_b16<true>(R, w, h.tq_x, m, s, dm, zover);
+    else pass_b16<false>(R, w, h.tq_x, m, s, dm, zover);
+
+    const bool lane_gen = R.general || !(s < kInf);
+    const bool hit = dm > 0.0f || h.tq_x < 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
+    const bool rare = (m > h.te_x) || lane_gen || hit;
+    const bool rel_covers = h.tq_x >= 0.0f && h.tq_x <= R.rtol;
+    const bool maybe_over = rel_covers ? (hit || zover) : (m > R.thr_min);
+    uint32_t cnt = 0;
+    const bool any_over = __any_sync(kFullMask, maybe_over);
+    if (any_over) {
 #pragma unroll
-            for (int g = 0; g < E / 4; ++g) {
-                const uint32_t off0 = elem_off<VEC>(4 * g, tid);
-                uint32_t in[4] = {0, 0, 0, 0};
-                if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+        for (int j = 0; j < 32; ++j) {
+            const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
+            cnt += (e > __fadd_rn(R.atol, __fmul_rn(R.rtol, fabsf(R.r[j])))) ? 1u : 0u;
+        }
+    }
+
+    const bool any_gen = __any_sync(kFullMask, lane_gen);
+    if (__any_sync(kFullMask, rare)) {
+        // ---- locate maxima; general rule where needed ------------------------------
+        const float rec_q = rec->qmax;
+        LaneGen a;
+        a.n_over = cnt; a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
+        a.emax = -1.0f; a.eoff = 0xFFFFu; a.qmax = -1.0f; a.qoff = 0xFFFFu; a.sum = (double)s;
+        if (lane_gen) {
+            a.n_over = 0; a.sum = 0.0;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t off = off0 + i;
-                    if (off < len) {
-                        uint32_t cb = cand_bits<CB16, NW>(w, 4 * g + i);
-                        if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
-                        if (!full) acc1 |= cb ^ h.first;
-                        acc2 |= cb ^ in[i];
-                    }
+            for (int j = 0; j < 32; ++j) {
+                const uint32_t off = elem_off<VEC>(j, tid);
+                // (a ragged tile's tail was patched into w by the caller)
+                if (off < len) elem_general(a, cbits(j), __float_as_uint(R.r[j]), off, R.atol, R.rtol);
+            }
+            if (a.n_noncomp) atomicAdd(&st->n_noncomp, (unsigned long long)a.n_noncomp);
+            if (a.n_nan) atomicAdd(&st->n_nan, (unsigned long long)a.n_nan);
+            if (a.n_inf) atomicAdd(&st->n_inf, (unsigned long long)a.n_inf);
+            if (a.n_infmis) atomicAdd(&st->n_infmis, (unsigned long long)a.n_infmis);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
+                const uint32_t off = elem_off<VEC>(j, tid);
+                // (positions past the end of a ragged tile hold zeros and never count)
+                if (e > a.emax && off < len) { a.emax = e; a.eoff = off; }
+                const float ar = fabsf(R.r[j]);
+                // the warp's own record comes from earlier tiles: only a strictly larger
+                // quotient can replace it
+                if (ar != 0.0f && e > __fmul_rd(fmaxf(rec_q, a.qmax), ar)) {
+                    const float q = __fdiv_rn(e, ar);
+                    if (q > a.qmax) { a.qmax = q; a.qoff = off; }
                 }
             }
         }
-        uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
-                        (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
-        seen &= need;
-        if (lane == 0 && seen) {
-            atomicOr(&st->mismatch, seen);
-            atomicOr(&h_smem->settled, seen);
+        cnt = a.n_over;
+        // warp-wide first maximum: largest value, then smallest offset.  Non-negative
+        // floats (and the -1 sentinel) order like their bit patterns as signed ints.
+        const int eb = __float_as_int(a.emax);
+        const int ebm = __reduce_max_sync(kFullMask, eb);
+        const uint32_t eoff = __reduce_min_sync(kFullMask, eb == ebm ? a.eoff : 0xFFFFu);
+        const int qb = __float_as_int(a.qmax);
+        const int qbm = __reduce_max_sync(kFullMask, qb);
+        const uint32_t qoff = __reduce_min_sync(kFullMask, qb == qbm ? a.qoff : 0xFFFFu);
+        double sd = a.sum;
+        if (any_gen) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sd += __shfl_xor_sync(kFullMask, sd, off);
+        } else {
+            float sf = s;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+            sd = (double)sf;
         }
+        if (lane == 0) {
+            WarpRec r = *rec;
+            const float em = __int_as_float(ebm), qm = __int_as_float(qbm);
+            if (em > r.emax) {
+                r.emax = em; r.etile = tile; r.offs = (r.offs & 0xFFFF0000u) | eoff;
+                atomicMax(&st->hint_e, hint_key(em, tile));
+            }
+            if (qm > r.qmax) {
+                r.qmax = qm; r.qtile = tile; r.offs = (r.offs & 0x0000FFFFu) | (qoff << 16);
+                atomicMax(&st->hint_q, hint_key(qm, tile));
+            }
+            r.sum += sd;
+            *rec = r;
+        }
+    } else {
+        float sf = s;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+        if (lane == 0) rec->sum += (double)sf;
     }
+    if (any_over || any_gen) {
+        const uint32_t tot = __reduce_add_sync(kFullMask, cnt);
+        if (lane == 0 && tot) rec->n_over += tot;
+    }
+    candidate_flags<true>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
 }
 
 // Merge the warp records of every candidate of a part into the block's
 // Partial row and clear them.  Called by all consumer threads between two
 // consumer barriers.
 __device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D, int K, int k0, int kc,
-                                              uint32_t slot, Partial* __restrict__ partials, int tid) {
+                                              uint32_t slot, Partial* __restrict__ partials, int tid,
+                                              uint32_t tile_elems) {
     if (tid < kc) {
         Partial p;
         p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX; p.sum = 0.0;
@@ -725,11 +928,11 @@ __device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D,
             p.n_over += r.n_over;
             p.sum += r.sum;
             if (r.emax >= 0.0f) {
-                const uint64_t idx = (uint64_t)r.etile * kTileElems + (r.offs & 0xFFFFu);
+                const uint64_t idx = (uint64_t)r.etile * tile_elems + (r.offs & 0xFFFFu);
                 if (r.emax > p.emax || (r.emax == p.emax && idx < p.eidx)) { p.emax = r.emax; p.eidx = idx; }
             }
             if (r.qmax >= 0.0f) {
-                const uint64_t idx = (uint64_t)r.qtile * kTileElems + (r.offs >> 16);
+                const uint64_t idx = (uint64_t)r.qtile * tile_elems + (r.offs >> 16);
                 if (r.qmax > p.qmax || (r.qmax == p.qmax && idx < p.qidx)) { p.qmax = r.qmax; p.qidx = idx; }
             }
             r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
@@ -762,9 +965,10 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
                                               int k_end, uint32_t n_items, CandState* __restrict__ state,
                                               Partial* __restrict__ partials, unsigned char* smem,
                                               const Ring& ring) {
-    constexpr int VEC = CB16 ? 8 : 4;
+    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
     constexpr int NV = E / VEC;
-    constexpr int NW = CB16 ? E / 2 : E;
+    constexpr uint32_t kTile = Geo<CB16>::kTile;
+    constexpr int kRefStages = (CB16 && !RB16) ? 2 : 1;
     constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrC);
@@ -801,15 +1005,15 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
         const int kc = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count) - k0;
         const uint32_t part_key = (it.group << 31) | it.part;
-        const uint64_t start = (uint64_t)it.tile * kTileElems;
-        const uint32_t len = (uint32_t)min((uint64_t)kTileElems, D.n - start);
+        const uint64_t start = (uint64_t)it.tile * kTile;
+        const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
         const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
         CandState* st_t = state + (size_t)it.t * (size_t)(K + 1);
         Hint* H = hints + (ord & 1u) * kPartK;
 
         if (it.t != cur_t || part_key != cur_part) {
             consumer_sync();                      // every warp is done with the previous part
-            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid);
+            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
             if (tid < kc) ptrs[tid] = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
             cur_t = it.t; cur_part = part_key; cur_k0 = k0; cur_kc = kc;
             cur_slot = blockIdx.x;                // one Partial row per block and tensor
@@ -827,17 +1031,28 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         if (tid == kPartK) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
 
         // ---- the thread's reference values --------------------------------------------
-        RefRegs R;
+        RefRegs<CB16> R;
         uint32_t rb[E];
         if (D.ref_src == RKV_SRC_POINTER) {
-            const uint32_t s = cstage;
-            mbar_wait(ring.full0 + 8 * s, cphase, ring.abort_flag);
-            load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)s * kStageBytes, tid);
+            // the reference tile fills one ring stage, or two (fp32 under bf16 candidates)
+            const uint32_t sa = cstage, pha = cphase;
+            mbar_wait(ring.full0 + 8 * sa, pha, ring.abort_flag);
+            if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
+            uint32_t sb = sa;
+            if (kRefStages == 2) {
+                sb = cstage;
+                mbar_wait(ring.full0 + 8 * sb, cphase, ring.abort_flag);
+                if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
+            }
+            load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes,
+                                 stages + (size_t)sb * kStageBytes, tid);
             __syncwarp();
-            if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
-            if (++cstage == (uint32_t)kStages) { cstage = 0; cphase ^= 1u; }
+            if (lane == 0) {
+                mbar_arrive(ring.empty0 + 8 * sa);
+                if (kRefStages == 2) mbar_arrive(ring.empty0 + 8 * sb);
+            }
         } else {
-            load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, tid);
+            load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, nullptr, tid);
         }
         consumer_sync();                          // hints, pointers and cleared records are visible
 
@@ -882,8 +1097,8 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
-            if (++cstage == (uint32_t)kStages) { cstage = 0; cphase ^= 1u; }
-            if (len != (uint32_t)kTileElems) {
+            if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
+            if (len != kTile) {
                 // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
                 // elements behind them come from global memory; positions past the end of the
                 // tensor get 0 against a reference of 0 (see load_ref): no error, never over
@@ -901,12 +1116,16 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
                     }
                 }
             }
-            process_candidate<CB16>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
-                                    it.tile, start, len, wanted, tid, lane);
+            if constexpr (CB16)
+                process_candidate_b16(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+                                      it.tile, start, len, wanted, tid, lane);
+            else
+                process_candidate<false>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+                                         it.tile, start, len, wanted, tid, lane);
         }
     }
     consumer_sync();
-    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid);
+    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
 }
 
 // One kernel per storage variant (candidate dtype, stored reference dtype), so

@@ -35,6 +35,10 @@ INPUT_COPY = "input_copy"
 BF16_ULP = "bf16_ulp"      # c = r * (1 + 2^-8 u), u uniform in [-1,1): about one bf16 ulp
 
 FAULT_KINDS = (CORRUPT, NAN_AT, INF_AT, CONST, INPUT_COPY, ZEROS)
+# Faults that fail whatever the scale of the data.  A CORRUPT element (+delta) is within
+# tolerance where rtol * |r| exceeds delta, as on the 1e4-scaled distribution under the
+# bf16 tolerances.
+SCALE_FREE_FAULT_KINDS = (NAN_AT, INF_AT, CONST, INPUT_COPY, ZEROS)
 
 
 @dataclass

@@ -96,7 +96,7 @@ def test_several_tiles_per_block_in_one_part(cand_dtype):
 def test_large_tensor_with_a_warm_up_group(cand_dtype):
     """A tensor large enough to be cut into a leading group of tiles (verified first, by all
     blocks) and the rest: results must not depend on which group an element falls in."""
-    tile = 3584
+    tile = 7168               # the larger of the two tile sizes: both dtypes get a second group
     n = tile * 2100 + 77
     ref = oracle_gen_tensor(88, 0, oracle.STUDENT_T2, n, "f32")
     inp = oracle_gen_tensor(88, 2, oracle.STUDENT_T2, n, cand_dtype)
@@ -152,6 +152,47 @@ def test_bf16_combinations(cand_dtype, ref_dtype, n):
                        gen_inp=(31, 2, rkv.DIST_NORMAL),
                        ref_dtype=rkv.F32 if ref_dtype == "f32" else rkv.BF16)
     assert got_a.tobytes() == got_b.tobytes()
+
+
+@pytest.mark.parametrize("atol,rtol", [(1e-2, 1.6e-2), (0.0, 1.6e-2), (1e-2, 0.0), (0.0, 0.0)])
+def test_bf16_candidates_at_the_edges_of_the_skip_tests(atol, rtol):
+    """Errors proportional to |r| around rtol, reference zeros with errors around atol,
+    values so small that e - t*|r| underflows, exact copies, equal quotients in every
+    tile, quotients that overflow: everything the bf16 path decides from a sign test."""
+    n = 7168 * 5 + 100
+    bf = torch.bfloat16
+    ref = oracle_gen_tensor(77, 0, oracle.NORMAL, n, "f32")
+    inp = oracle_gen_tensor(77, 2, oracle.NORMAL, n, "bf16")
+    cands = [ref.to(bf)]
+    for k in (0.5, 0.99, 1.0, 1.01, 1.5):
+        cands.append((ref * (1.0 + 1.6e-2 * k)).to(bf))
+    c = ref.to(bf).clone(); c[30000] = (ref[30000] * 1.05).to(bf); cands.append(c)   # one element, late tile
+    c = ref.to(bf).clone(); c[17] = (ref[17] * 1.05).to(bf); cands.append(c)         # one element, first tile
+    check_case(ref, cands, atol, rtol, inp, where="proportional")
+
+    # reference zeros: errors just below, at and above atol there; elsewhere rounding only
+    sp = oracle_gen_tensor(78, 0, oracle.SPARSE90, n, "f32")
+    zi = torch.nonzero(sp == 0).flatten()
+    cands = [sp.to(bf)]
+    for v in (0.99e-2, 1e-2, 1.01e-2, 1e-30, 1.0):
+        c = sp.to(bf).clone(); c[zi[::97]] = torch.tensor(v).to(bf); cands.append(c)
+    c = sp.to(bf).clone(); c[zi[-1]] = 0.5; cands.append(c)
+    check_case(sp, cands, atol, rtol, inp, where="zeros")
+
+    # tiny magnitudes: products and differences in and below the subnormal range
+    for scale in (1e-30, 1e-36, 1e-38, 3e-41):
+        tiny = (ref * scale).contiguous()
+        cands = [tiny.to(bf), (tiny * 1.01).to(bf), (tiny * 1.02).to(bf), torch.zeros(n, dtype=bf)]
+        c = tiny.to(bf).clone(); c[20000] = 1e-20; cands.append(c)                    # quotient overflows
+        check_case(tiny, cands, atol, rtol, inp, where=f"tiny {scale}")
+
+    # a reference that bf16 holds exactly: exact copies, and the same quotient everywhere
+    rb = ref.to(bf).to(torch.float32)
+    cands = [rb.to(bf), (rb * 2.0).to(bf), (rb * 1.5).to(bf), (rb * 1.0078125).to(bf)]
+    c = rb.to(bf).clone(); c[n - 1] = (rb[n - 1] * 2.0).to(bf); cands.append(c)
+    c = rb.to(bf).clone(); c[0] = (rb[0] * 2.0).to(bf); cands.append(c)
+    check_case(rb, cands, atol, rtol, inp, where="exact")
+    check_case(rb.to(bf), cands, atol, rtol, inp, where="exact, bf16 reference", ref_dtype=None)
 
 
 def test_nonfinite_everywhere():
