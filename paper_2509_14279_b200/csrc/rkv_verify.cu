@@ -562,11 +562,17 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
             }
         } else if (!full || (need & 2u)) {
             const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+            // Regenerating the input is the expensive part.  A candidate that is no copy
+            // of it almost surely shows that in the first four elements of every thread,
+            // so the warp stops generating once a difference has been seen.
+            bool with_input = (need & 2u) != 0u;
 #pragma unroll
             for (int g = 0; g < E / 4; ++g) {
+                if (g == 1 && with_input) with_input = !__any_sync(kFullMask, acc2 != 0u);
+                if (full && !with_input) break;
                 const uint32_t off0 = elem_off<VEC>(4 * g, tid);
                 uint32_t in[4] = {0, 0, 0, 0};
-                if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+                if (with_input && off0 < len) input_group<CB16>(D, start, off0, len, in);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t off = off0 + i;
@@ -574,7 +580,7 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
                         uint32_t cb = cand_bits<CB16, NW>(w, 4 * g + i);
                         if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
                         if (!full) acc1 |= cb ^ h.first;
-                        acc2 |= cb ^ in[i];
+                        if (with_input) acc2 |= cb ^ in[i];
                     }
                 }
             }
