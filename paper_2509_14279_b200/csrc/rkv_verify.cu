@@ -116,6 +116,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
 }
 
+// Arrive from the threads for which `on` holds, as one predicated instruction (no branch).
+__device__ __forceinline__ void mbar_arrive_if(uint32_t mbar, bool on) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(mbar), "r"((uint32_t)on)
+        : "memory");
+}
+
 __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -628,6 +637,17 @@ __device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const 
 
     // a NaN or an infinity anywhere makes the sum non-finite
     const bool lane_gen = R.general || !(s < kInf);
+    // One vote settles the common case: nothing over tolerance, no possible first maximum,
+    // nothing non-finite (the tests are explained below).
+    if (!__any_sync(kFullMask, lane_gen || m > R.thr_min || m > h.te_x || m > __fmul_rd(h.tq_x, R.minarp))) {
+        float sf = s;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+        const double total = rec->sum + (double)sf;       // every lane computes it, one stores
+        if (lane == 0) rec->sum = total;
+        candidate_flags<CB16>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+        return;
+    }
     // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
     uint32_t cnt = 0;
     const bool any_over = __any_sync(kFullMask, m > R.thr_min);
@@ -796,7 +816,8 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
 // that a positive difference below the subnormal range rounds to zero; such a difference
 // needs e_j < 2^-100 (the product has 48 significant bits).  So the elements pass as a
 // whole when max_j d_j < 0, or = 0 with the thread's largest error 0 or at least 2^-100.
-// t < 0 says that nothing is published yet, or a tie at 0 could still win: no filtering.
+// A negative t says that nothing is published yet, or that a tie at 0 could still win;
+// the hint table holds -inf then, which makes every d_j with r_j != 0 equal +inf.
 //
 // Over tolerance.  thr_j = fl(atol + fl(rtol * |r_j|)) >= fl(rtol * |r_j|), and a float
 // e_j above fl(P) is above P itself, so e_j > thr_j implies e_j > rtol * |r_j| >= t * |r_j|
@@ -823,23 +844,30 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
     else pass_b16<false>(R, w, h.tq_x, m, s, dm, zover);
 
     const bool lane_gen = R.general || !(s < kInf);
-    const bool hit = dm > 0.0f || h.tq_x < 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
+    const bool hit = dm > 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
     const bool rare = (m > h.te_x) || lane_gen || hit;
     const bool rel_covers = h.tq_x >= 0.0f && h.tq_x <= R.rtol;
     const bool maybe_over = rel_covers ? (hit || zover) : (m > R.thr_min);
-    uint32_t cnt = 0;
-    const bool any_over = __any_sync(kFullMask, maybe_over);
-    if (any_over) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
-            cnt += (e > __fadd_rn(R.atol, __fmul_rn(R.rtol, fabsf(R.r[j])))) ? 1u : 0u;
-        }
-    }
 
-    const bool any_gen = __any_sync(kFullMask, lane_gen);
-    if (__any_sync(kFullMask, rare)) {
-        // ---- locate maxima; general rule where needed ------------------------------
+    if (!__any_sync(kFullMask, rare || maybe_over)) {
+        // nothing but the sum to record (every lane computes it, one stores)
+        float sf = s;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
+        const double total = rec->sum + (double)sf;
+        if (lane == 0) rec->sum = total;
+    } else {
+        uint32_t cnt = 0;
+        const bool any_over = __any_sync(kFullMask, maybe_over);
+        if (any_over) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
+                cnt += (e > __fadd_rn(R.atol, __fmul_rn(R.rtol, fabsf(R.r[j])))) ? 1u : 0u;
+            }
+        }
+        const bool any_gen = __any_sync(kFullMask, lane_gen);
+        // ---- locate maxima; general rule where needed ----------------------------------
         const float rec_q = rec->qmax;
         LaneGen a;
         a.n_over = cnt; a.n_noncomp = 0; a.n_nan = 0; a.n_inf = 0; a.n_infmis = 0;
@@ -856,7 +884,7 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
             if (a.n_nan) atomicAdd(&st->n_nan, (unsigned long long)a.n_nan);
             if (a.n_inf) atomicAdd(&st->n_inf, (unsigned long long)a.n_inf);
             if (a.n_infmis) atomicAdd(&st->n_infmis, (unsigned long long)a.n_infmis);
-        } else {
+        } else if (rare) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
@@ -891,6 +919,7 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
             for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
             sd = (double)sf;
         }
+        const uint32_t tot = (any_over || any_gen) ? __reduce_add_sync(kFullMask, cnt) : 0u;
         if (lane == 0) {
             WarpRec r = *rec;
             const float em = __int_as_float(ebm), qm = __int_as_float(qbm);
@@ -903,17 +932,9 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
                 atomicMax(&st->hint_q, hint_key(qm, tile));
             }
             r.sum += sd;
+            r.n_over += tot;
             *rec = r;
         }
-    } else {
-        float sf = s;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
-        if (lane == 0) rec->sum += (double)sf;
-    }
-    if (any_over || any_gen) {
-        const uint32_t tot = __reduce_add_sync(kFullMask, cnt);
-        if (lane == 0 && tot) rec->n_over += tot;
     }
     candidate_flags<true>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
 }
@@ -1030,6 +1051,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             Hint h;
             h.te_x = hint_threshold(__ldcg(&sc->hint_e), it.tile);
             h.tq_x = hint_threshold(__ldcg(&sc->hint_q), it.tile);
+            if (CB16 && h.tq_x < 0.0f) h.tq_x = -kInf;     // see process_candidate_b16
             h.settled = __ldcg(&sc->mismatch);
             h.first = ld_elem_bits(ptrs[tid], CB16 ? RKV_BF16 : RKV_F32, 0);
             H[tid] = h;
@@ -1053,10 +1075,8 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes,
                                  stages + (size_t)sb * kStageBytes, tid);
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(ring.empty0 + 8 * sa);
-                if (kRefStages == 2) mbar_arrive(ring.empty0 + 8 * sb);
-            }
+            mbar_arrive_if(ring.empty0 + 8 * sa, lane == 0);
+            if (kRefStages == 2) mbar_arrive_if(ring.empty0 + 8 * sb, lane == 0);
         } else {
             load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, nullptr, tid);
         }
@@ -1102,7 +1122,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
                 w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(ring.empty0 + 8 * s);
+            mbar_arrive_if(ring.empty0 + 8 * s, lane == 0);
             if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
             if (len != kTile) {
                 // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
