@@ -768,17 +768,15 @@ __device__ __forceinline__ float sub_bf16_f32(uint32_t x, int half, float r) {
 }
 
 // One pass over a thread's 32 elements of a bf16 candidate tile: largest and summed
-// |c - r|, and the largest d_j = fma(-t, |r_j|, e_j) for the relative-error threshold t
-// (see process_candidate_b16).  HAS_ZERO: reference values of exactly 0 may occur; they
-// take no part in the relative error, and `zover` tells whether one of them has an error
-// above atol.
+// e_j = |c_j - r_j|, and the largest d_j, where d_j = fma(-t, |r_j|, e_j) for the
+// relative-error threshold t (see process_candidate_b16).  HAS_ZERO: reference values of
+// exactly 0 may occur; they take no part in the relative error, and d_j = e_j - atol there,
+// positive exactly when the element is over tolerance.
 template <bool HAS_ZERO>
 __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t (&w)[16], float t, float& m_out,
-                                         float& s_out, float& dm_out, bool& zover_out) {
-    const float nt = -t;
+                                         float& s_out, float& dm_out) {
     float m = 0.0f, dm = -kInf;
     float sg[8];
-    bool zover = false;
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
         float e[4], d[4];
@@ -786,13 +784,9 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
         for (int i = 0; i < 4; ++i) {
             const int j = 4 * g + i;
             e[i] = fabsf(sub_bf16_f32(w[j >> 1], j & 1, R.r[j]));
-            float ar = fabsf(R.r[j]);
-            if (HAS_ZERO) {
-                const bool z = ar == 0.0f;
-                zover |= z && e[i] > R.atol;
-                ar = z ? kInf : ar;          // d = -inf (t > 0), NaN (t = 0; max skips it), +inf (t < 0)
-            }
-            d[i] = __fmaf_rn(nt, ar, e[i]);
+            const float ar = fabsf(R.r[j]);
+            if (HAS_ZERO && ar == 0.0f) d[i] = __fsub_rn(e[i], R.atol);
+            else d[i] = __fmaf_rn(-t, ar, e[i]);
         }
         m = fmaxf(fmaxf(m, fmaxf(e[0], e[1])), fmaxf(e[2], e[3]));
         dm = fmaxf(fmaxf(dm, fmaxf(d[0], d[1])), fmaxf(d[2], d[3]));
@@ -800,7 +794,6 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
     }
     m_out = m;
     dm_out = dm;
-    zover_out = zover;
     s_out = __fadd_rn(__fadd_rn(__fadd_rn(sg[0], sg[1]), __fadd_rn(sg[2], sg[3])),
                       __fadd_rn(__fadd_rn(sg[4], sg[5]), __fadd_rn(sg[6], sg[7])));
 }
@@ -822,7 +815,9 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
 // Over tolerance.  thr_j = fl(atol + fl(rtol * |r_j|)) >= fl(rtol * |r_j|), and a float
 // e_j above fl(P) is above P itself, so e_j > thr_j implies e_j > rtol * |r_j| >= t * |r_j|
 // whenever 0 <= t <= rtol: while the published relative maximum is at most rtol, an element
-// over tolerance also fails the test above (where r_j = 0 the test is e_j > atol).
+// over tolerance also fails the test above.  Where r_j = 0 the pass takes d_j = e_j - atol,
+// the over-tolerance test itself; that such an element also counts as a possible maximum
+// costs a look, not a result.
 // Otherwise: m <= thr_min means e_j <= m <= thr_min <= thr_j for every element.
 __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, const uint32_t (&w)[16],
                                                       const Hint& h, Hint* h_smem, WarpRec* rec,
@@ -839,15 +834,14 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
 
     // ---- common path ---------------------------------------------------------------
     float m, s, dm;
-    bool zover;
-    if (R.warp_has_zero) pass_b16<true>(R, w, h.tq_x, m, s, dm, zover);
-    else pass_b16<false>(R, w, h.tq_x, m, s, dm, zover);
+    if (R.warp_has_zero) pass_b16<true>(R, w, h.tq_x, m, s, dm);
+    else pass_b16<false>(R, w, h.tq_x, m, s, dm);
 
     const bool lane_gen = R.general || !(s < kInf);
     const bool hit = dm > 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
     const bool rare = (m > h.te_x) || lane_gen || hit;
     const bool rel_covers = h.tq_x >= 0.0f && h.tq_x <= R.rtol;
-    const bool maybe_over = rel_covers ? (hit || zover) : (m > R.thr_min);
+    const bool maybe_over = rel_covers ? hit : (m > R.thr_min);
 
     if (!__any_sync(kFullMask, rare || maybe_over)) {
         // nothing but the sum to record (every lane computes it, one stores)
