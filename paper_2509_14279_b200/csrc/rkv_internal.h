@@ -21,7 +21,7 @@ constexpr int kTileElemsBF16 = kStageBytes / 2;      // 7168 elements per tile o
 __host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
     return cand_dtype == RKV_BF16 ? kTileElemsBF16 : kTileElemsF32;
 }
-constexpr int kStages = 6;                           // ring depth (bulk copies in flight)
+constexpr int kStages = 5;                           // ring depth (bulk copies in flight)
 constexpr int kPartK = 64;                           // candidates a block tracks at a time
 constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
 constexpr int kWarmMinTiles = 2048;                  // tensors with fewer tiles have no warm-up group

@@ -1,33 +1,36 @@
 // Fused single-pass verification kernel and its finalize kernel (sm_100a).
 //
-// Work decomposition.  A tensor is cut into tiles of 3584 elements; the K
-// candidates into parts of at most 64.  A work item is (tensor, part, tile).
-// A persistent thread block takes items round robin.  It has two roles:
+// Work decomposition.  A tensor is cut into tiles of 14336 candidate bytes (3584 fp32 or
+// 7168 bf16 elements); the K candidates into parts of at most 64.  A work item is
+// (tensor, group, part, tile).  A persistent thread block starts with the item of its own
+// number and then draws further items from a ticket counter.  It has two roles:
 //
 //   * one producer warp: a single thread issues bulk asynchronous copies
 //     (cp.async.bulk, completion counted on an mbarrier) that bring, for the
 //     item, the reference tile and then the same tile of every candidate of the
 //     part into a ring of shared-memory stages.  Several stages are in flight,
 //     so the copies of later candidates overlap the comparison of earlier ones;
-//   * seven consumer warps: each thread owns 16 elements of the tile.  It keeps
-//     their reference values and tolerance thresholds IN REGISTERS for the
-//     whole item and meets every candidate tile as it lands in the ring.
+//   * seven consumer warps: each thread owns 64 bytes of every candidate tile (16 fp32
+//     or 32 bf16 elements).  It keeps their reference values (and, for fp32 candidates,
+//     the tolerance thresholds) IN REGISTERS for the whole item and meets every
+//     candidate tile as it lands in the ring.
 //
 // Candidate bytes are read from HBM exactly once; the reference once per part.
-// When the reference is "generated" the threads regenerate their 16 values from
+// When the reference is "generated" the threads regenerate their values from
 // the Philox stream instead of reading them (fused generate + verify).
 //
 // Per element the common path is one subtraction, one running maximum and one
-// addition.  Counting the elements over tolerance, locating maxima, dividing for
-// the relative error and everything about non-finite values sit behind
-// predicates evaluated once per thread, candidate and tile:
+// addition (bf16 candidates: one fused multiply-add and one more maximum, see
+// process_candidate_b16).  Counting the elements over tolerance, locating maxima,
+// dividing for the relative error and everything about non-finite values sit behind
+// tests evaluated once per thread, candidate and tile and one warp vote:
 //   m > min thr              some element may be over tolerance  -> count them
 //   !(sum < inf)             a non-finite value                  -> general rule
 //   m beats/ties the hint    a new maximum is possible           -> locate it
 // The hints are running maxima that all blocks publish in global memory with
 // their tile number.  A hint only ever lets a thread skip elements that cannot
-// be the first maximum (see consider_maxima), so results do not depend on when a
-// hint becomes visible.
+// be the first maximum (see Hint), so results do not depend on when a hint
+// becomes visible.
 //
 // Reductions are deterministic: integer sums, lexicographic (value descending,
 // index ascending) maxima, fixed-order floating-point sums.  No float atomics.
