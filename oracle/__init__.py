@@ -56,6 +56,29 @@ class Result(ctypes.Structure):
         return {name: getattr(self, name) for name, _ in self._fields_ if name != "pad"}
 
 
+class ScreenResult(ctypes.Structure):
+    _fields_ = [
+        ("flags", ctypes.c_uint32),
+        ("pad", ctypes.c_uint32),
+        ("n_values", ctypes.c_uint64),
+        ("n_nonfinite", ctypes.c_uint64),
+        ("argmax_seed_spread", ctypes.c_uint64),
+        ("mean", ctypes.c_double),
+        ("std", ctypes.c_double),
+        ("vmin", ctypes.c_float),
+        ("vmax", ctypes.c_float),
+        ("max_seed_spread", ctypes.c_float),
+        ("pad2", ctypes.c_uint32),
+    ]
+
+    def as_dict(self) -> dict:
+        return {name: getattr(self, name) for name, _ in self._fields_ if not name.startswith("pad")}
+
+
+SCREEN_NARROW_RANGE, SCREEN_LOW_STD, SCREEN_LOW_SEED_VARIATION = 1, 2, 4
+SCREEN_UNIFORM_AXIS0, SCREEN_UNIFORM_AXIS1, SCREEN_NONFINITE = 8, 16, 32
+
+
 def build(force: bool = False) -> str:
     """Compile ``liboracle.so`` next to the source with gcc; return its path."""
     stale = (not os.path.exists(_LIB)
@@ -109,6 +132,10 @@ def lib() -> ctypes.CDLL:
         L.orc_max_rel_filtered.restype = ctypes.c_float
         L.orc_joint_pass.argtypes = [ctypes.POINTER(Result), ctypes.c_int, ctypes.c_int, u32p]
         L.orc_joint_pass.restype = None
+        L.orc_screen.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_uint64,
+                                 ctypes.c_uint64, ctypes.c_int, ctypes.c_float, ctypes.c_double,
+                                 ctypes.c_float, ctypes.POINTER(ScreenResult)]
+        L.orc_screen.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -224,3 +251,19 @@ def joint_pass(verdicts) -> list:
     out = (ctypes.c_uint32 * K)()
     lib().orc_joint_pass(arr, K, T, out)
     return [int(x) for x in out]
+
+
+def screen(outs, range_lim: float = 0.01, std_lim: float = 0.01, spread_lim: float = 0.01) -> dict:
+    """Task-soundness screens over the reference outputs of S seeds (2-D arrays of one shape)."""
+    arrs = [np.ascontiguousarray(a) for a in outs]
+    rows, cols = arrs[0].shape
+    for a in arrs:
+        if a.shape != (rows, cols) or a.dtype != arrs[0].dtype:
+            raise ValueError("outputs differ in shape or dtype")
+    ptrs = (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    r = ScreenResult()
+    rc = lib().orc_screen(ptrs, len(arrs), rows, cols, _dtype_of(arrs[0].reshape(-1)), float(range_lim),
+                          float(std_lim), float(spread_lim), ctypes.byref(r))
+    if rc != 0:
+        raise ValueError("orc_screen: bad argument")
+    return r.as_dict()

@@ -351,3 +351,91 @@ void orc_joint_pass(const orc_result *results, int K, int T, uint32_t *joint_pas
         joint_pass[k] = ok;
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/* Task-soundness screens (App. A.1 "filtering criteria"): statistics of the  */
+/* reference outputs of one task over S seeds, and the exclusion flags.      */
+/* ------------------------------------------------------------------------- */
+int orc_screen(const void *const *outs, int S, uint64_t rows, uint64_t cols, int dtype,
+               float range_lim, double std_lim, float spread_lim, orc_screen_result *res)
+{
+    if (!outs || !res || S < 1 || rows < 1 || cols < 1) return -1;
+    if (dtype != ORC_F32 && dtype != ORC_BF16) return -1;
+    for (int s = 0; s < S; ++s) if (!outs[s]) return -1;
+    const uint64_t n = rows * cols;
+
+    /* range, count, mean: every finite value of every seed */
+    uint64_t n_fin = 0, n_nonfin = 0;
+    float vmin = INFINITY, vmax = -INFINITY;
+    double sum = 0.0;
+    for (int s = 0; s < S; ++s)
+        for (uint64_t i = 0; i < n; ++i) {
+            const uint32_t b = load_bits(outs[s], dtype, i);
+            if (!bits_is_finite(b)) { n_nonfin++; continue; }
+            const float x = bits_f32(b);
+            if (x < vmin) vmin = x;
+            if (x > vmax) vmax = x;
+            sum += (double)x;
+            n_fin++;
+        }
+    const double mean = n_fin ? sum / (double)n_fin : 0.0;
+    /* population standard deviation, second pass about the mean */
+    double ss = 0.0;
+    for (int s = 0; s < S; ++s)
+        for (uint64_t i = 0; i < n; ++i) {
+            const uint32_t b = load_bits(outs[s], dtype, i);
+            if (!bits_is_finite(b)) continue;
+            const double d = (double)bits_f32(b) - mean;
+            ss += d * d;
+        }
+    const double sd = n_fin ? sqrt(ss / (double)n_fin) : 0.0;
+
+    /* variation across seeds: per element the spread max_s - min_s (one fp32
+     * subtraction); elements with a non-finite value in some seed are left out */
+    float spread = -1.0f;
+    uint64_t arg = ORC_NO_INDEX;
+    if (S >= 2)
+        for (uint64_t i = 0; i < n; ++i) {
+            float lo = INFINITY, hi = -INFINITY;
+            int ok = 1;
+            for (int s = 0; s < S; ++s) {
+                const uint32_t b = load_bits(outs[s], dtype, i);
+                if (!bits_is_finite(b)) { ok = 0; break; }
+                const float x = bits_f32(b);
+                if (x < lo) lo = x;
+                if (x > hi) hi = x;
+            }
+            if (!ok) continue;
+            const float d = hi - lo;
+            if (d > spread) { spread = d; arg = i; }
+        }
+
+    /* uniformity along an axis: every slice along it repeats its first element bit for bit */
+    int uni0 = rows >= 2, uni1 = cols >= 2;
+    for (int s = 0; s < S; ++s)
+        for (uint64_t r = 0; r < rows; ++r)
+            for (uint64_t c = 0; c < cols; ++c) {
+                const uint32_t b = load_bits(outs[s], dtype, r * cols + c);
+                if (b != load_bits(outs[s], dtype, c)) uni0 = 0;          /* down column c */
+                if (b != load_bits(outs[s], dtype, r * cols)) uni1 = 0;   /* along row r   */
+            }
+
+    memset(res, 0, sizeof *res);
+    res->n_values = (uint64_t)S * n;
+    res->n_nonfinite = n_nonfin;
+    res->argmax_seed_spread = arg;
+    res->mean = mean;
+    res->std = sd;
+    res->vmin = vmin;
+    res->vmax = vmax;
+    res->max_seed_spread = spread;
+    uint32_t f = 0;
+    if (n_fin && vmin >= -range_lim && vmax <= range_lim) f |= ORC_SCREEN_NARROW_RANGE;
+    if (n_fin && sd < std_lim) f |= ORC_SCREEN_LOW_STD;
+    if (S >= 2 && arg != ORC_NO_INDEX && spread < spread_lim) f |= ORC_SCREEN_LOW_SEED_VARIATION;
+    if (uni0) f |= ORC_SCREEN_UNIFORM_AXIS0;
+    if (uni1) f |= ORC_SCREEN_UNIFORM_AXIS1;
+    if (n_nonfin) f |= ORC_SCREEN_NONFINITE;
+    res->flags = f;
+    return 0;
+}

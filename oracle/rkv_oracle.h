@@ -129,6 +129,46 @@ float orc_max_rel_filtered(const float *ref, const float *cand, uint64_t n, uint
 /* joint_pass[k] = AND over tensors t of (results[k*T + t].verdict == 0). */
 void orc_joint_pass(const orc_result *results, int K, int T, uint32_t *joint_pass);
 
+/* ---- task-soundness screens (App. A.1, the filtering criteria) -----------------------
+ * A task is unsound when its reference outputs, over S seeds, (1) all lie in a narrow range
+ * around zero, (2) have a small standard deviation, (3) are uniform along an axis, or
+ * (4) hardly change with the input seed.  The paper gives the thresholds (0.01) in words
+ * only; the readings taken here:
+ *   (1) every finite value v of every seed has -range_lim <= v <= range_lim;
+ *   (2) the population standard deviation of all finite values, pooled over the seeds
+ *       (fp64, two passes), is below std_lim;
+ *   (3) seen as rows x cols, every column (axis 0) or every row (axis 1) of every seed
+ *       repeats its first element bit for bit;
+ *   (4) the largest per-element spread max_s x_s[i] - min_s x_s[i] (one fp32 subtraction;
+ *       elements with a non-finite value in some seed are left out) is below spread_lim.
+ * Parity status: pinned by closed forms, by brute force in numpy on tiny tensors and by
+ * invariants; the readings above are this project's: parity unpinned for them. */
+enum {
+    ORC_SCREEN_NARROW_RANGE = 1u << 0,
+    ORC_SCREEN_LOW_STD = 1u << 1,
+    ORC_SCREEN_LOW_SEED_VARIATION = 1u << 2,
+    ORC_SCREEN_UNIFORM_AXIS0 = 1u << 3,
+    ORC_SCREEN_UNIFORM_AXIS1 = 1u << 4,
+    ORC_SCREEN_NONFINITE = 1u << 5
+};
+
+typedef struct orc_screen_result {
+    uint32_t flags;
+    uint32_t pad;
+    uint64_t n_values;            /* S * rows * cols */
+    uint64_t n_nonfinite;
+    uint64_t argmax_seed_spread;  /* first element with the largest spread; ORC_NO_INDEX if none */
+    double mean;                  /* of the finite values */
+    double std;
+    float vmin, vmax;             /* of the finite values; +inf / -inf when there is none */
+    float max_seed_spread;        /* -1 when S < 2 or no element is finite in every seed */
+    uint32_t pad2;
+} orc_screen_result;
+
+/* outs: S pointers to rows*cols elements of dtype each.  Returns 0, or -1 on a bad argument. */
+int orc_screen(const void *const *outs, int S, uint64_t rows, uint64_t cols, int dtype,
+               float range_lim, double std_lim, float spread_lim, orc_screen_result *res);
+
 #ifdef __cplusplus
 }
 #endif
