@@ -295,6 +295,72 @@ int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t *til
 /* Releases the library-owned scratch and staging buffers of all devices. */
 int rkv_release_cached(void);
 
+/* ------------------------------------------------------------------------------------
+ * Task-soundness screens (App. A.1, the filtering criteria): is a task fit to be a
+ * benchmark at all?  The paper excludes a task whose reference outputs (1) all lie
+ * between -0.01 and 0.01, (2) have a standard deviation below 0.01 across model and input
+ * seeds, (3) are uniform along their axes, or (4) vary by less than 0.01 across input
+ * seeds.  One streaming pass over the reference outputs of S seeds computes the
+ * statistics behind the four criteria; the limits are arguments (0.01 in the paper).
+ * The readings taken, the paper giving the criteria in words only:
+ *   (1) every finite value v of every seed has -range_lim <= v <= range_lim;
+ *   (2) the population standard deviation of all finite values, pooled over the seeds,
+ *       is below std_lim;
+ *   (3) seen as rows x cols (row-major), every column (axis 0) or every row (axis 1) of
+ *       every seed repeats its first element bit for bit;
+ *   (4) the largest per-element spread max_s x_s[i] - min_s x_s[i] (one fp32 subtraction;
+ *       elements that are not finite in some seed are left out) is below spread_lim.
+ * ------------------------------------------------------------------------------------ */
+enum rkv_screen_flag {
+    RKV_SCREEN_NARROW_RANGE = 1u << 0,
+    RKV_SCREEN_LOW_STD = 1u << 1,
+    RKV_SCREEN_LOW_SEED_VARIATION = 1u << 2,
+    RKV_SCREEN_UNIFORM_AXIS0 = 1u << 3,
+    RKV_SCREEN_UNIFORM_AXIS1 = 1u << 4,
+    RKV_SCREEN_NONFINITE = 1u << 5      /* informative: some value is NaN or infinite */
+};
+
+typedef struct rkv_screen_stats {
+    uint32_t flags;               /* rkv_screen_flag bits; bits 0..4 each exclude the task */
+    uint32_t reserved;
+    uint64_t n_values;            /* S * rows * cols */
+    uint64_t n_nonfinite;
+    uint64_t argmax_seed_spread;  /* first element with the largest spread; RKV_NO_INDEX if none */
+    double mean;                  /* of the finite values */
+    double std;                   /* population standard deviation of the finite values */
+    float vmin, vmax;             /* of the finite values (the sign of a zero is unspecified);
+                                     +inf / -inf when there is none */
+    float max_seed_spread;        /* -1 when S < 2 or no element is finite in every seed */
+    uint32_t reserved2;
+} rkv_screen_stats;               /* 64 bytes */
+
+/* Bytes of device workspace rkv_screen_outputs needs on the current device (0 without one). */
+size_t rkv_screen_workspace_bytes(void);
+
+/*
+ * Screens the reference outputs of one task.
+ *   outs         HOST array of S DEVICE pointers, each to rows*cols elements of dtype,
+ *                contiguous, row-major, 16-byte aligned; caller-owned, only read
+ *   S            number of seeds, 1 <= S <= 16 (with S == 1 criterion (4) is not evaluated)
+ *   rows, cols   the two-dimensional view the uniformity criterion is taken on (a tensor of
+ *                more dimensions is passed as leading dimension x the rest, or any other
+ *                split the caller cares about); rows*cols < 2^40
+ *   dtype        RKV_F32 | RKV_BF16
+ *   range_lim, std_lim, spread_lim   the limits of criteria (1), (2), (4), each >= 0
+ *   stats_out    DEVICE pointer to one rkv_screen_stats, written by the call's last kernel
+ *   workspace    DEVICE memory of at least rkv_screen_workspace_bytes(), 16-byte aligned;
+ *                contents need not be preserved or cleared between calls
+ *   cuda_stream  the stream (cudaStream_t) the two kernels are launched on; the call does
+ *                not synchronise
+ * mean and std are accumulated in fp64 in a fixed order (bit-reproducible on one device
+ * model); everything else is exact.
+ * Errors: INVALID_ARG (null, S < 1, rows or cols < 1, bad dtype, a negative or NaN limit),
+ * UNSUPPORTED (S > 16, rows*cols >= 2^40), ALIGNMENT, WORKSPACE (null or too small), CUDA.
+ */
+int rkv_screen_outputs(const void *const *outs, int S, uint64_t rows, uint64_t cols, int dtype,
+                       float range_lim, double std_lim, float spread_lim, rkv_screen_stats *stats_out,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

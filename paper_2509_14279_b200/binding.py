@@ -34,6 +34,14 @@ STATS_DTYPE = np.dtype([
     ("max_abs_err", "<f4"), ("max_rel_err", "<f4"), ("mean_abs_err", "<f4"), ("reserved", "<u4"),
 ])
 STATS_BYTES = STATS_DTYPE.itemsize
+
+SCREEN_DTYPE = np.dtype([
+    ("flags", "<u4"), ("reserved", "<u4"), ("n_values", "<u8"), ("n_nonfinite", "<u8"),
+    ("argmax_seed_spread", "<u8"), ("mean", "<f8"), ("std", "<f8"), ("vmin", "<f4"), ("vmax", "<f4"),
+    ("max_seed_spread", "<f4"), ("reserved2", "<u4")])
+SCREEN_BYTES = SCREEN_DTYPE.itemsize
+SCREEN_NARROW_RANGE, SCREEN_LOW_STD, SCREEN_LOW_SEED_VARIATION = 1, 2, 4
+SCREEN_UNIFORM_AXIS0, SCREEN_UNIFORM_AXIS1, SCREEN_NONFINITE = 8, 16, 32
 assert STATS_BYTES == 88
 
 
@@ -106,6 +114,11 @@ def lib() -> ctypes.CDLL:
         L.rkv_plan_items.argtypes = [u64, i32, i32, i32, u32p, u32p, u32p, u32p, u32p]
         L.rkv_release_cached.restype = i32
         L.rkv_release_cached.argtypes = []
+        L.rkv_screen_workspace_bytes.restype = ctypes.c_size_t
+        L.rkv_screen_workspace_bytes.argtypes = []
+        L.rkv_screen_outputs.restype = i32
+        L.rkv_screen_outputs.argtypes = [ctypes.POINTER(vp), i32, u64, u64, i32, f32, ctypes.c_double, f32,
+                                         vp, vp, ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -322,3 +335,35 @@ def verify_batch_host(ref: torch.Tensor, cands, atol: float, rtol: float) -> np.
 
 def release_cached() -> None:
     lib().rkv_release_cached()
+
+
+def screen_workspace_bytes() -> int:
+    return int(lib().rkv_screen_workspace_bytes())
+
+
+def screen_outputs(outs, range_lim: float = 0.01, std_lim: float = 0.01, spread_lim: float = 0.01,
+                   stats_out: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                   stream=None) -> tuple:
+    """rkv_screen_outputs: the task-soundness screens over the reference outputs of S seeds
+    (2-D tensors of one shape and dtype on the device).  Returns (stats, workspace): the
+    device buffer holding one rkv_screen_stats (uint8, 64 bytes) and the workspace used."""
+    S = len(outs)
+    rows, cols = outs[0].shape
+    for o in outs:
+        if tuple(o.shape) != (rows, cols) or o.dtype != outs[0].dtype or not o.is_contiguous():
+            raise ValueError("outputs must be contiguous and agree in shape and dtype")
+    dev = outs[0].device
+    if stats_out is None:
+        stats_out = torch.empty(SCREEN_BYTES, dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = torch.empty(screen_workspace_bytes(), dtype=torch.uint8, device=dev)
+    ptrs = (ctypes.c_void_p * S)(*[o.data_ptr() for o in outs])
+    _check(lib().rkv_screen_outputs(ptrs, S, int(rows), int(cols), _dtype_code(outs[0]), float(range_lim),
+                                    float(std_lim), float(spread_lim), ctypes.c_void_p(stats_out.data_ptr()),
+                                    ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                    ctypes.c_void_p(_stream_ptr(stream))), "rkv_screen_outputs")
+    return stats_out, workspace
+
+
+def screen_to_numpy(stats: torch.Tensor) -> np.ndarray:
+    return stats.detach().cpu().numpy().view(SCREEN_DTYPE)

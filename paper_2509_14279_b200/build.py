@@ -16,7 +16,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librkv.so")
-SOURCES = ["rkv_api.cu", "rkv_gen.cu", "rkv_verify.cu"]
+SOURCES = ["rkv_api.cu", "rkv_gen.cu", "rkv_verify.cu", "rkv_screen.cu"]
 HEADERS = ["rkv_internal.h", "rkv_philox.cuh"]
 
 NVCC_FLAGS = [
