@@ -22,10 +22,10 @@ namespace rkv {
 namespace {
 
 constexpr int kScreenThreads = 256;
-constexpr int kScreenBlocksPerSm = 4;         // fp32 outputs; bf16 (8 elements per vector) fits 3
+constexpr int kScreenBlocksPerSm = 3;         // resident blocks per SM, fp32 outputs
 constexpr int kScreenBlocksPerSmB16 = 3;
 constexpr int kScreenMaxSeeds = 16;
-constexpr int kPivotSample = 1024;
+constexpr int kPivotSample = 256;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr float kInfF = __builtin_huge_valf();
 
@@ -64,7 +64,7 @@ __device__ __forceinline__ uint32_t load_elem_bits(const void* p, uint64_t i) {
 
 struct Acc {
     double sum, sumsq;
-    unsigned long long n_fin, n_nonfin, arg;
+    unsigned long long n_fin, n_nonfin, arg;     // n_fin: values visited until the thread is done, then the finite ones
     float vmin, vmax, spread;
     uint32_t nonuniform;
 };
@@ -72,12 +72,9 @@ struct Acc {
 __device__ __forceinline__ void acc_value(Acc& a, uint32_t b, double pivot, float& lo, float& hi, bool& ok) {
     if (finite_bits(b)) {
         const float x = __uint_as_float(b);
-        a.vmin = fminf(a.vmin, x);
-        a.vmax = fmaxf(a.vmax, x);
         const double d = (double)x - pivot;
         a.sum += d;
         a.sumsq = fma(d, d, a.sumsq);
-        a.n_fin++;
         lo = fminf(lo, x);
         hi = fmaxf(hi, x);
     } else {
@@ -124,6 +121,7 @@ __device__ __forceinline__ void screen_element(const ScreenArgs& A, Acc& a, doub
     float lo = kInfF, hi = -kInfF;
     bool ok = true;
     const uint64_t r = i / A.cols, c = i - r * A.cols;
+    a.n_fin += (unsigned long long)A.S;
     for (int s = 0; s < A.S; ++s) {
         const uint32_t b = load_elem_bits<B16>(A.outs[s], i);
         acc_value(a, b, pivot, lo, hi, ok);
@@ -132,9 +130,73 @@ __device__ __forceinline__ void screen_element(const ScreenArgs& A, Acc& a, doub
             if (b != load_elem_bits<B16>(A.outs[s], r * A.cols)) a.nonuniform |= 2u;
         }
     }
+    a.vmin = fminf(a.vmin, lo);
+    a.vmax = fmaxf(a.vmax, hi);
     if (A.S >= 2 && ok) {
         const float d = fabsf(__fsub_rn(hi, lo));
         if (d > a.spread) { a.spread = d; a.arg = i; }
+    }
+}
+
+// N outputs (s0 .. s0+N-1) at one vector position: their loads are issued together, then one
+// test tells whether all N * VEC values are finite (x * 0 is a zero for a finite x and NaN
+// otherwise) and the branch-free path can run.
+template <bool B16, int N>
+__device__ __forceinline__ void screen_chunk(const ScreenArgs& A, Acc& a, double pivot, int s0, uint64_t v,
+                                             uint32_t need, uint64_t r, uint64_t c0,
+                                             float (&lo)[B16 ? 8 : 4], float (&hi)[B16 ? 8 : 4],
+                                             bool (&ok)[B16 ? 8 : 4]) {
+    constexpr int VEC = B16 ? 8 : 4;
+    uint4 q[N];
+#pragma unroll
+    for (int u = 0; u < N; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[s0 + u]) + v);
+    uint32_t b[N][VEC];
+#pragma unroll
+    for (int u = 0; u < N; ++u) {
+        const uint32_t wv[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+        for (int j = 0; j < VEC; ++j)
+            b[u][j] = B16 ? ((j & 1) ? (wv[j >> 1] & 0xFFFF0000u) : (wv[j >> 1] << 16)) : wv[j];
+    }
+    float chk = 0.0f;
+#pragma unroll
+    for (int u = 0; u < N; ++u)
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) chk = __fmaf_rn(__uint_as_float(b[u][j]), 0.0f, chk);
+    if (chk == 0.0f) {
+#pragma unroll
+        for (int u = 0; u < N; ++u)
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+                const float x = __uint_as_float(b[u][j]);
+                lo[j] = fminf(lo[j], x);
+                hi[j] = fmaxf(hi[j], x);
+                const double d = (double)x - pivot;
+                a.sum += d;
+                a.sumsq = fma(d, d, a.sumsq);
+            }
+    } else {
+#pragma unroll
+        for (int u = 0; u < N; ++u)
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) acc_value(a, b[u][j], pivot, lo[j], hi[j], ok[j]);
+    }
+    if (need) {
+#pragma unroll
+        for (int u = 0; u < N; ++u) {
+            if (need & 1u) {
+                // the same columns of row 0, as stored
+                const uint4 f = __ldg(reinterpret_cast<const uint4*>(A.outs[s0 + u]) + c0 / VEC);
+                if ((q[u].x ^ f.x) | (q[u].y ^ f.y) | (q[u].z ^ f.z) | (q[u].w ^ f.w)) a.nonuniform |= 1u;
+            }
+            if (need & 2u) {
+                const uint32_t first = load_elem_bits<B16>(A.outs[s0 + u], r * A.cols);
+                uint32_t diff = 0;
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) diff |= b[u][j] ^ first;
+                if (diff) a.nonuniform |= 2u;
+            }
+        }
     }
 }
 
@@ -150,11 +212,15 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
     if (warp == 0) {
         double ps = 0.0;
         uint32_t pc = 0;
-        const uint64_t m = A.n < (uint64_t)kPivotSample ? A.n : (uint64_t)kPivotSample;
-        for (uint64_t i = lane; i < m; i += 32) {
-            const uint32_t b = load_elem_bits<B16>(A.outs[0], i);
-            if (finite_bits(b)) { ps += (double)__uint_as_float(b); pc++; }
+        uint32_t pb[kPivotSample / 32];
+#pragma unroll
+        for (int t = 0; t < kPivotSample / 32; ++t) {       // independent loads, issued together
+            const uint64_t i = (uint64_t)(lane + 32 * t);
+            pb[t] = i < A.n ? load_elem_bits<B16>(A.outs[0], i) : 0x7FC00000u;
         }
+#pragma unroll
+        for (int t = 0; t < kPivotSample / 32; ++t)
+            if (finite_bits(pb[t])) { ps += (double)__uint_as_float(pb[t]); pc++; }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             ps += __shfl_xor_sync(kFull, ps, off);
@@ -177,6 +243,7 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
     if (vec_rows) {
         for (uint64_t v = (uint64_t)blockIdx.x * kScreenThreads + tid; v < nvec; v += stride) {
             const uint64_t i0 = v * VEC;
+            a.n_fin += (unsigned long long)(VEC * A.S);
             float lo[VEC], hi[VEC];
             bool ok[VEC];
 #pragma unroll
@@ -185,37 +252,19 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
             const uint32_t need = axes_wanted & ~a.nonuniform;
             uint64_t r = 0, c0 = 0;
             if (need) { r = i0 / A.cols; c0 = i0 - r * A.cols; }
-            // four outputs at a time, their loads issued together
-            for (int s0 = 0; s0 < A.S; s0 += 4) {
-                uint4 q4[4];
+            // the outputs in chunks of 8, 4, 3 (fp32 only), 2 and 1
+            int s0 = 0;
+            if (!B16) {
+                for (; A.S - s0 >= 8; s0 += 8) screen_chunk<B16, B16 ? 1 : 8>(A, a, pivot, s0, v, need, r, c0, lo, hi, ok);
+                if (A.S - s0 >= 4) { screen_chunk<B16, B16 ? 1 : 4>(A, a, pivot, s0, v, need, r, c0, lo, hi, ok); s0 += 4; }
+            }
+            if (!B16 && A.S - s0 == 3) { screen_chunk<B16, B16 ? 1 : 3>(A, a, pivot, s0, v, need, r, c0, lo, hi, ok); s0 += 3; }
+            for (; A.S - s0 >= 2; s0 += 2) screen_chunk<B16, 2>(A, a, pivot, s0, v, need, r, c0, lo, hi, ok);
+            if (A.S - s0 >= 1) screen_chunk<B16, 1>(A, a, pivot, s0, v, need, r, c0, lo, hi, ok);
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (s0 + u < A.S) q4[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[s0 + u]) + v);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (s0 + u >= A.S) break;
-                    const int s = s0 + u;
-                    const uint4 q = q4[u];
-                    const uint32_t wv[4] = {q.x, q.y, q.z, q.w};
-                    uint32_t b[VEC];
-#pragma unroll
-                    for (int j = 0; j < VEC; ++j)
-                        b[j] = B16 ? ((j & 1) ? (wv[j >> 1] & 0xFFFF0000u) : (wv[j >> 1] << 16)) : wv[j];
-#pragma unroll
-                    for (int j = 0; j < VEC; ++j) acc_value(a, b[j], pivot, lo[j], hi[j], ok[j]);
-                    if (need & 1u) {
-                        // the same columns of row 0, as stored
-                        const uint4 f = __ldg(reinterpret_cast<const uint4*>(A.outs[s]) + c0 / VEC);
-                        if ((q.x ^ f.x) | (q.y ^ f.y) | (q.z ^ f.z) | (q.w ^ f.w)) a.nonuniform |= 1u;
-                    }
-                    if (need & 2u) {
-                        const uint32_t first = load_elem_bits<B16>(A.outs[s], r * A.cols);
-                        uint32_t diff = 0;
-#pragma unroll
-                        for (int j = 0; j < VEC; ++j) diff |= b[j] ^ first;
-                        if (diff) a.nonuniform |= 2u;
-                    }
-                }
+            for (int j = 0; j < VEC; ++j) {
+                a.vmin = fminf(a.vmin, lo[j]);
+                a.vmax = fmaxf(a.vmax, hi[j]);
             }
             if (A.S >= 2) {
 #pragma unroll
@@ -235,6 +284,7 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
             screen_element<B16>(A, a, pivot, i, (axes_wanted & ~a.nonuniform) != 0u);
     }
     a.nonuniform &= axes_wanted;
+    a.n_fin -= a.n_nonfin;
 
     // ---- block reduction: fixed shuffle tree, then the warps in order ----------------------
 #pragma unroll
