@@ -278,19 +278,23 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * elements per tile).  One work item is
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
- * part past them.  A large tensor has two groups of items: the first *warm_tiles
+ * part past them.  A large tensor has three groups of items: the first *warm_tiles
  * tiles, with the candidates cut into *parts_warm parts (many small ones, so that
  * every resident block -- 2 per SM -- starts with one of these items), are
  * verified first; the running maxima and loophole flags they publish let the
- * remaining tiles, with *parts_main parts of at most 64 candidates, skip nearly
- * all rare-path work.  A smaller tensor has one group: *warm_tiles == *n_tiles
- * and *parts_main == 0.  Part p of P covers candidates [p*K/P, (p+1)*K/P).
+ * tiles after them, with *parts_main parts of at most 64 candidates, skip nearly
+ * all rare-path work; the last *tail_tiles tiles, with *parts_tail parts of at most
+ * 16 candidates, come last and even out the finishing times of the blocks.  A
+ * smaller tensor has one group: *warm_tiles == *n_tiles, *parts_main == 0,
+ * *tail_tiles == 0 and *parts_tail == 0.  Part p of P covers candidates
+ * [p*K/P, (p+1)*K/P).
  *   cand_dtype  RKV_F32 | RKV_BF16 (storage type of the candidates)
  *   num_sms     SM count of the device
  * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, bad dtype, null), UNSUPPORTED (n >= 2^40).
  */
 int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t *tile_elems, uint32_t *n_tiles,
-                   uint32_t *warm_tiles, uint32_t *parts_warm, uint32_t *parts_main);
+                   uint32_t *warm_tiles, uint32_t *parts_warm, uint32_t *parts_main, uint32_t *tail_tiles,
+                   uint32_t *parts_tail);
 
 /* Releases the library-owned scratch and staging buffers of all devices. */
 int rkv_release_cached(void);

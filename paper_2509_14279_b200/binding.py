@@ -111,7 +111,7 @@ def lib() -> ctypes.CDLL:
         L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
         u32p = ctypes.POINTER(ctypes.c_uint32)
         L.rkv_plan_items.restype = i32
-        L.rkv_plan_items.argtypes = [u64, i32, i32, i32, u32p, u32p, u32p, u32p, u32p]
+        L.rkv_plan_items.argtypes = [u64, i32, i32, i32, u32p, u32p, u32p, u32p, u32p, u32p, u32p]
         L.rkv_release_cached.restype = i32
         L.rkv_release_cached.argtypes = []
         L.rkv_screen_workspace_bytes.restype = ctypes.c_size_t
@@ -154,9 +154,9 @@ def set_stream(stream=None) -> None:
 
 
 def plan_items(n: int, K: int, num_sms: int, cand_dtype: int = F32) -> tuple:
-    """Host-only: (tile_elems, n_tiles, warm_tiles, parts_warm, parts_main) for a tensor of
-    n elements and K candidates."""
-    v = [ctypes.c_uint32() for _ in range(5)]
+    """Host-only: (tile_elems, n_tiles, warm_tiles, parts_warm, parts_main, tail_tiles, parts_tail)
+    for a tensor of n elements and K candidates."""
+    v = [ctypes.c_uint32() for _ in range(7)]
     _check(lib().rkv_plan_items(int(n), int(cand_dtype), int(K), int(num_sms), *[ctypes.byref(x) for x in v]),
            "rkv_plan_items")
     return tuple(int(x.value) for x in v)

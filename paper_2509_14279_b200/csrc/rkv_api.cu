@@ -27,12 +27,13 @@ static int plan_one(uint64_t n, int cand_dtype, uint32_t* n_tiles, uint32_t* war
 }
 
 // Work items of one tensor for a launch over k_count candidates.
-static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t k_count, uint32_t grid) {
+static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t tail_tiles, uint32_t tail_div,
+                         uint32_t k_count, uint32_t grid) {
     uint64_t items = 0;
-    const uint32_t groups[2] = {warm_tiles, n_tiles - warm_tiles};
-    for (int g = 0; g < 2; ++g) {
-        if (!groups[g]) continue;
-        items += (uint64_t)groups[g] * part_count(groups[g], k_count, grid);
+    for (uint32_t g = 0; g < 3; ++g) {
+        const uint32_t nt = group_tiles(g, n_tiles, warm_tiles, tail_tiles);
+        if (!nt) continue;
+        items += (uint64_t)nt * group_parts(g, nt, k_count, grid, tail_div);
     }
     return items;
 }
@@ -92,8 +93,12 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
         if (rc != RKV_OK) return rc;
         plan->n_tiles[t] = tiles;
         plan->warm_tiles[t] = warm;
+        const uint32_t tail = tail_tiles_of(tiles, warm, grid);
+        plan->tail_tiles[t] = tail;
+        const uint32_t tail_div = tensors[t].ref_src == RKV_SRC_GENERATED ? kTailDivGenerated : kTailDiv;
+        plan->tail_div[t] = tail_div;
         plan->variant[t] = variant_of(tensors[t]);
-        const uint64_t items = items_of(tiles, warm, (uint32_t)k_count, grid);
+        const uint64_t items = items_of(tiles, warm, tail, tail_div, (uint32_t)k_count, grid);
         total_items[plan->variant[t]] += items;
         if (total_items[plan->variant[t]] > 0x7FFFFFFFull) return RKV_ERR_UNSUPPORTED;
         plan->n_slots[t] = grid;                 // one Partial row per block
@@ -163,7 +168,7 @@ void fill_dev_tensor(DevTensor& d, const rkv_tensor_desc& s, const Plan& plan, i
     d.cand_dtype = s.cand_dtype; d.ref_dtype = s.ref_dtype;
     d.ref_src = s.ref_src; d.input_src = s.input_src;
     d.atol = s.atol; d.rtol = s.rtol;
-    d.n_tiles = plan.n_tiles[t]; d.warm_tiles = plan.warm_tiles[t];
+    d.n_tiles = plan.n_tiles[t]; d.warm_tiles = plan.warm_tiles[t]; d.tail_tiles = plan.tail_tiles[t]; d.tail_div = plan.tail_div[t];
     d.n_slots = plan.n_slots[t]; d.slot_base = plan.slot_base[t];
     d.variant = plan.variant[t];
 }
@@ -195,7 +200,7 @@ int launch_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k
     uint32_t items[4] = {0, 0, 0, 0};
     const uint32_t kcount = (uint32_t)(k_end - k_begin);
     for (int t = 0; t < T; ++t)
-        items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], kcount, plan.grid);
+        items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], plan.tail_tiles[t], plan.tail_div[t], kcount, plan.grid);
     (void)tensors;
     int rc = launch_verify(L.d_tensors, T, K, k_begin, k_end, items, (int)plan.grid, L.state, L.partials,
                            L.header, stream);
@@ -259,8 +264,10 @@ int rkv_set_stream(void* cuda_stream) {
 }
 
 int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t* tile_elems_out, uint32_t* n_tiles,
-                   uint32_t* warm_tiles, uint32_t* parts_warm, uint32_t* parts_main) {
-    if (!tile_elems_out || !n_tiles || !warm_tiles || !parts_warm || !parts_main) return RKV_ERR_INVALID_ARG;
+                   uint32_t* warm_tiles, uint32_t* parts_warm, uint32_t* parts_main, uint32_t* tail_tiles,
+                   uint32_t* parts_tail) {
+    if (!tile_elems_out || !n_tiles || !warm_tiles || !parts_warm || !parts_main || !tail_tiles || !parts_tail)
+        return RKV_ERR_INVALID_ARG;
     if (!dtype_ok(cand_dtype)) return RKV_ERR_INVALID_ARG;
     if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
     if (K < 1 || num_sms < 1 || num_sms > (1 << 20)) return RKV_ERR_INVALID_ARG;
@@ -268,8 +275,11 @@ int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t* til
     if (rc != RKV_OK) return rc;
     const uint32_t grid = (uint32_t)(num_sms * kBlocksPerSm);
     *tile_elems_out = tile_elems(cand_dtype);
-    *parts_warm = part_count(*warm_tiles, (uint32_t)K, grid);
-    *parts_main = *warm_tiles < *n_tiles ? part_count(*n_tiles - *warm_tiles, (uint32_t)K, grid) : 0u;
+    *tail_tiles = tail_tiles_of(*n_tiles, *warm_tiles, grid);
+    const uint32_t main_tiles = group_tiles(1, *n_tiles, *warm_tiles, *tail_tiles);
+    *parts_warm = group_parts(0, *warm_tiles, (uint32_t)K, grid, kTailDiv);
+    *parts_main = main_tiles ? group_parts(1, main_tiles, (uint32_t)K, grid, kTailDiv) : 0u;
+    *parts_tail = *tail_tiles ? group_parts(2, *tail_tiles, (uint32_t)K, grid, kTailDiv) : 0u;
     return RKV_OK;
 }
 

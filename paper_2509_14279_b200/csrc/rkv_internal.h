@@ -25,6 +25,8 @@ constexpr int kStages = 5;                           // ring depth (bulk copies 
 constexpr int kPartK = 64;                           // candidates a block tracks at a time
 constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
 constexpr int kWarmMinTiles = 2048;                  // tensors with fewer tiles have no warm-up group
+constexpr int kTailDiv = 4;                          // a tail item covers a quarter of a part's candidates ...
+constexpr int kTailDivGenerated = 2;                 // ... half, when every item regenerates its reference tile
 constexpr int kMaxTensors = 64;
 constexpr uint64_t kMaxN = 1ull << 40;
 
@@ -69,20 +71,25 @@ struct DevTensor {
     int32_t cand_dtype, ref_dtype;
     int32_t ref_src, input_src;
     float atol, rtol;
-    // Work items.  A large tensor has two groups of items: group A covers its first
+    // Work items.  A large tensor has three groups of items: group A covers its first
     // warm_tiles tiles with small candidate parts (so that all blocks take part), group B
-    // the remaining tiles with parts of up to kPartK candidates.  Group A runs first: the
-    // maxima and loophole flags it publishes let group B skip almost all rare-path work.
-    // Smaller tensors only have group A.  Within a group item = part * tiles + tile, with
-    // part_count() parts per group.
+    // the tiles after them with parts of up to kPartK candidates, group C its last
+    // tail_tiles tiles with parts a quarter that size.  Group A runs first: the maxima and
+    // loophole flags it publishes let the rest skip almost all rare-path work.  Group C runs
+    // last: its short items even out the finishing times of the blocks.  Smaller tensors
+    // only have group A.  Within a group item = part * tiles + tile, with group_parts()
+    // parts per group.
     // Items of the tensors of one storage variant are numbered consecutively, all A
-    // groups before all B groups; blocks take them in this order (see WorkspaceHeader).
+    // groups, then all B groups, then all C groups; blocks take them in this order (see
+    // WorkspaceHeader).
     uint32_t n_tiles;       // ceil(n / tile_elems(cand_dtype))
     uint32_t warm_tiles;    // tiles in group A (== n_tiles when there is no group B)
     uint32_t n_slots;       // Partial rows of this tensor: one per block of the grid
     uint32_t slot_base;     // first Partial row (K entries per row) of this tensor
     uint32_t variant;       // 2 * (candidates bf16) + (reference stored as bf16)
-    uint32_t reserved[3];
+    uint32_t tail_tiles;    // tiles in group C
+    uint32_t tail_div;      // group C cuts the candidates into this many times the parts of group B
+    uint32_t reserved;
 };
 
 struct WorkspaceHeader {
@@ -101,6 +108,8 @@ static_assert(sizeof(WorkspaceHeader) == 256, "header size");
 struct Plan {
     uint32_t n_tiles[kMaxTensors];
     uint32_t warm_tiles[kMaxTensors];
+    uint32_t tail_tiles[kMaxTensors];
+    uint32_t tail_div[kMaxTensors];
     uint32_t n_slots[kMaxTensors];
     uint32_t slot_base[kMaxTensors];
     uint32_t variant[kMaxTensors];
@@ -129,6 +138,25 @@ __host__ __device__ inline uint32_t part_count(uint32_t tiles, uint32_t k_count,
         if (want > parts) parts = want;
     }
     return parts > k_count ? k_count : parts;
+}
+
+// Tiles, first tile and candidate parts of group g (0: A, 1: B, 2: C) of a tensor.
+__host__ __device__ inline uint32_t group_tiles(uint32_t g, uint32_t n_tiles, uint32_t warm, uint32_t tail) {
+    return g == 0 ? warm : g == 1 ? n_tiles - warm - tail : tail;
+}
+__host__ __device__ inline uint32_t group_first_tile(uint32_t g, uint32_t n_tiles, uint32_t warm, uint32_t tail) {
+    return g == 0 ? 0u : g == 1 ? warm : n_tiles - tail;
+}
+__host__ __device__ inline uint32_t group_parts(uint32_t g, uint32_t tiles, uint32_t k_count, uint32_t grid,
+                                                uint32_t tail_div) {
+    if (g != 2) return part_count(tiles, k_count, grid);
+    const uint32_t parts = (k_count + kPartK - 1) / kPartK * tail_div;
+    return parts > k_count ? k_count : parts;
+}
+// Tiles in group C: half a tile per block, for tensors long enough that the blocks'
+// finishing times would otherwise differ by up to a whole item.
+__host__ __device__ inline uint32_t tail_tiles_of(uint32_t n_tiles, uint32_t warm, uint32_t grid) {
+    return (n_tiles - warm >= 4u * grid && grid >= 2u) ? grid / 2u : 0u;
 }
 
 __host__ __device__ inline uint32_t part_begin(uint32_t part, uint32_t parts, uint32_t k_count) {

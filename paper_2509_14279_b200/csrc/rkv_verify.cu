@@ -202,7 +202,7 @@ __device__ __forceinline__ uint32_t ld_elem_bits(const void* base, int dtype, ui
 // ----------------------------------------------------------------------------
 struct Item {
     int t;
-    uint32_t group;          // 0 = A (leading tiles, small parts), 1 = B
+    uint32_t group;          // 0 = A (leading tiles, small parts), 1 = B, 2 = C (last tiles, small parts)
     uint32_t part, tile;     // tile is the tensor-wide tile index
     uint32_t n_parts;        // candidate parts of this group
     uint32_t first_item;     // first item of this (tensor, group) in this launch
@@ -213,19 +213,19 @@ struct Item {
 __device__ __forceinline__ bool decode_item(const DevTensor* __restrict__ tensors, int T, uint32_t variant,
                                             uint32_t k_count, uint32_t id, Item& it) {
     uint32_t base = 0;
-    for (uint32_t g = 0; g < 2; ++g) {
+    for (uint32_t g = 0; g < 3; ++g) {
         for (int t = 0; t < T; ++t) {
             if (tensors[t].variant != variant) continue;
-            const uint32_t warm = tensors[t].warm_tiles;
-            const uint32_t nt = g == 0 ? warm : tensors[t].n_tiles - warm;
+            const uint32_t warm = tensors[t].warm_tiles, tail = tensors[t].tail_tiles;
+            const uint32_t nt = group_tiles(g, tensors[t].n_tiles, warm, tail);
             if (nt == 0) continue;
-            const uint32_t parts = part_count(nt, k_count, gridDim.x);
+            const uint32_t parts = group_parts(g, nt, k_count, gridDim.x, tensors[t].tail_div);
             const uint32_t cnt = nt * parts;
             if (id - base < cnt) {
                 it.t = t;
                 it.group = g;
                 it.part = (id - base) / nt;
-                it.tile = (id - base) % nt + (g == 0 ? 0u : warm);
+                it.tile = (id - base) % nt + group_first_tile(g, tensors[t].n_tiles, warm, tail);
                 it.n_parts = parts;
                 it.first_item = base;
                 it.n_items = cnt;
@@ -291,7 +291,7 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
         const uint32_t k_count = (uint32_t)(k_end - k_begin);
         const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
         const int k1 = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count);
-        const uint32_t part_key = (it.group << 31) | it.part;
+        const uint32_t part_key = (it.group << 30) | it.part;
         if (it.t != cur_t || part_key != cur_part) {
             __syncwarp();
             for (int k = k0 + lane; k < k1; k += 32)
@@ -1028,7 +1028,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         const uint32_t k_count = (uint32_t)(k_end - k_begin);
         const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
         const int kc = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count) - k0;
-        const uint32_t part_key = (it.group << 31) | it.part;
+        const uint32_t part_key = (it.group << 30) | it.part;
         const uint64_t start = (uint64_t)it.tile * kTile;
         const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
         const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;

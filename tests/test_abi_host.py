@@ -59,7 +59,7 @@ def test_stats_struct_is_88_bytes():
 def test_item_plan_properties(n, K, dtype):
     sms = 148
     grid = 2 * sms
-    tile, n_tiles, warm, parts_warm, parts_main = rkv.plan_items(n, K, sms, dtype)
+    tile, n_tiles, warm, parts_warm, parts_main, tail, parts_tail = rkv.plan_items(n, K, sms, dtype)
     assert tile == (3584 if dtype == rkv.F32 else 7168)
     assert (n_tiles - 1) * tile < n <= n_tiles * tile
     assert 1 <= warm <= n_tiles
@@ -71,8 +71,15 @@ def test_item_plan_properties(n, K, dtype):
         # a large tensor: a short warm-up group, then the fewest parts of at most 64
         assert warm * tile >= 60000 and warm * 100 < n_tiles
         assert parts_main == -(-K // 64)
+        # a long tensor ends with half a tile per block in parts a quarter that size
+        if n_tiles - warm >= 4 * grid:
+            assert tail == grid // 2 and parts_tail == min(K, 4 * parts_main)
+            assert -(-K // parts_tail) <= 16
+        else:
+            assert tail == 0 and parts_tail == 0
+        assert warm + tail < n_tiles
     else:
-        assert parts_main == 0
+        assert parts_main == 0 and tail == 0 and parts_tail == 0
 
 
 def test_item_plan_rejects_bad_arguments():
