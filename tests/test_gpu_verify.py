@@ -95,7 +95,8 @@ def test_several_tiles_per_block_in_one_part(cand_dtype):
 @pytest.mark.parametrize("cand_dtype", ["f32", "bf16"])
 def test_large_tensor_with_a_warm_up_group(cand_dtype):
     """A tensor large enough to be cut into a leading group of tiles (verified first, by all
-    blocks) and the rest: results must not depend on which group an element falls in."""
+    blocks), the bulk, and a tail group of short items (its last tiles, verified last): results
+    must not depend on which group an element falls in."""
     tile = 7168               # the larger of the two tile sizes: both dtypes get a second group
     n = tile * 2100 + 77
     ref = oracle_gen_tensor(88, 0, oracle.STUDENT_T2, n, "f32")
