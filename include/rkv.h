@@ -282,8 +282,7 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * tiles, with the candidates cut into *parts_warm parts (many small ones, so that
  * every resident block -- 2 per SM -- starts with one of these items), are
  * verified first; the running maxima and loophole flags they publish let the
- * tiles after them, with *parts_main parts of at most 64 candidates (128 for bf16
- * candidates against a regenerated reference; this helper reports the 64 case), skip nearly
+ * tiles after them, with *parts_main parts of at most 64 candidates, skip nearly
  * all rare-path work; the last *tail_tiles tiles, with *parts_tail parts of at most
  * 16 candidates, come last and even out the finishing times of the blocks.  A
  * smaller tensor has one group: *warm_tiles == *n_tiles, *parts_main == 0,

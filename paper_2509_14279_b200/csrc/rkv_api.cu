@@ -28,12 +28,12 @@ static int plan_one(uint64_t n, int cand_dtype, uint32_t* n_tiles, uint32_t* war
 
 // Work items of one tensor for a launch over k_count candidates.
 static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t tail_tiles, uint32_t tail_div,
-                         uint32_t part_max, uint32_t k_count, uint32_t grid) {
+                         uint32_t k_count, uint32_t grid) {
     uint64_t items = 0;
     for (uint32_t g = 0; g < 3; ++g) {
         const uint32_t nt = group_tiles(g, n_tiles, warm_tiles, tail_tiles);
         if (!nt) continue;
-        items += (uint64_t)nt * group_parts(g, nt, k_count, grid, tail_div, part_max);
+        items += (uint64_t)nt * group_parts(g, nt, k_count, grid, tail_div);
     }
     return items;
 }
@@ -97,11 +97,8 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
         plan->tail_tiles[t] = tail;
         const uint32_t tail_div = tensors[t].ref_src == RKV_SRC_GENERATED ? kTailDivGenerated : kTailDiv;
         plan->tail_div[t] = tail_div;
-        const uint32_t part_max = (tensors[t].cand_dtype == RKV_BF16 && tensors[t].ref_src == RKV_SRC_GENERATED)
-                                      ? (uint32_t)kPartKWide : (uint32_t)kPartK;
-        plan->part_max[t] = part_max;
         plan->variant[t] = variant_of(tensors[t]);
-        const uint64_t items = items_of(tiles, warm, tail, tail_div, part_max, (uint32_t)k_count, grid);
+        const uint64_t items = items_of(tiles, warm, tail, tail_div, (uint32_t)k_count, grid);
         total_items[plan->variant[t]] += items;
         if (total_items[plan->variant[t]] > 0x7FFFFFFFull) return RKV_ERR_UNSUPPORTED;
         plan->n_slots[t] = grid;                 // one Partial row per block
@@ -171,7 +168,7 @@ void fill_dev_tensor(DevTensor& d, const rkv_tensor_desc& s, const Plan& plan, i
     d.cand_dtype = s.cand_dtype; d.ref_dtype = s.ref_dtype;
     d.ref_src = s.ref_src; d.input_src = s.input_src;
     d.atol = s.atol; d.rtol = s.rtol;
-    d.n_tiles = plan.n_tiles[t]; d.warm_tiles = plan.warm_tiles[t]; d.tail_tiles = plan.tail_tiles[t]; d.tail_div = plan.tail_div[t]; d.part_max = plan.part_max[t];
+    d.n_tiles = plan.n_tiles[t]; d.warm_tiles = plan.warm_tiles[t]; d.tail_tiles = plan.tail_tiles[t]; d.tail_div = plan.tail_div[t];
     d.n_slots = plan.n_slots[t]; d.slot_base = plan.slot_base[t];
     d.variant = plan.variant[t];
 }
@@ -203,7 +200,7 @@ int launch_case(const rkv_tensor_desc* tensors, int T, int K, int k_begin, int k
     uint32_t items[4] = {0, 0, 0, 0};
     const uint32_t kcount = (uint32_t)(k_end - k_begin);
     for (int t = 0; t < T; ++t)
-        items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], plan.tail_tiles[t], plan.tail_div[t], plan.part_max[t], kcount, plan.grid);
+        items[plan.variant[t]] += (uint32_t)items_of(plan.n_tiles[t], plan.warm_tiles[t], plan.tail_tiles[t], plan.tail_div[t], kcount, plan.grid);
     (void)tensors;
     int rc = launch_verify(L.d_tensors, T, K, k_begin, k_end, items, (int)plan.grid, L.state, L.partials,
                            L.header, stream);
@@ -280,9 +277,9 @@ int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t* til
     *tile_elems_out = tile_elems(cand_dtype);
     *tail_tiles = tail_tiles_of(*n_tiles, *warm_tiles, grid);
     const uint32_t main_tiles = group_tiles(1, *n_tiles, *warm_tiles, *tail_tiles);
-    *parts_warm = group_parts(0, *warm_tiles, (uint32_t)K, grid, kTailDiv, kPartK);
-    *parts_main = main_tiles ? group_parts(1, main_tiles, (uint32_t)K, grid, kTailDiv, kPartK) : 0u;
-    *parts_tail = *tail_tiles ? group_parts(2, *tail_tiles, (uint32_t)K, grid, kTailDiv, kPartK) : 0u;
+    *parts_warm = group_parts(0, *warm_tiles, (uint32_t)K, grid, kTailDiv);
+    *parts_main = main_tiles ? group_parts(1, main_tiles, (uint32_t)K, grid, kTailDiv) : 0u;
+    *parts_tail = *tail_tiles ? group_parts(2, *tail_tiles, (uint32_t)K, grid, kTailDiv) : 0u;
     return RKV_OK;
 }
 

@@ -22,8 +22,7 @@ __host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
     return cand_dtype == RKV_BF16 ? kTileElemsBF16 : kTileElemsF32;
 }
 constexpr int kStages = 5;                           // ring depth (bulk copies in flight)
-constexpr int kPartK = 64;                           // candidates a block tracks at a time ...
-constexpr int kPartKWide = 128;                      // ... bf16 candidates against a regenerated reference (fewer regenerations)
+constexpr int kPartK = 64;                           // candidates a block tracks at a time
 constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
 constexpr int kWarmMinTiles = 2048;                  // tensors with fewer tiles have no warm-up group
 constexpr int kTailDiv = 4;                          // a tail item covers a quarter of a part's candidates ...
@@ -74,7 +73,7 @@ struct DevTensor {
     float atol, rtol;
     // Work items.  A large tensor has three groups of items: group A covers its first
     // warm_tiles tiles with small candidate parts (so that all blocks take part), group B
-    // the tiles after them with parts of up to part_max candidates, group C its last
+    // the tiles after them with parts of up to kPartK candidates, group C its last
     // tail_tiles tiles with parts a quarter that size.  Group A runs first: the maxima and
     // loophole flags it publishes let the rest skip almost all rare-path work.  Group C runs
     // last: its short items even out the finishing times of the blocks.  Smaller tensors
@@ -90,7 +89,7 @@ struct DevTensor {
     uint32_t variant;       // 2 * (candidates bf16) + (reference stored as bf16)
     uint32_t tail_tiles;    // tiles in group C
     uint32_t tail_div;      // group C cuts the candidates into this many times the parts of group B
-    uint32_t part_max;      // most candidates in a part: kPartK or kPartKWide
+    uint32_t reserved;
 };
 
 struct WorkspaceHeader {
@@ -111,7 +110,6 @@ struct Plan {
     uint32_t warm_tiles[kMaxTensors];
     uint32_t tail_tiles[kMaxTensors];
     uint32_t tail_div[kMaxTensors];
-    uint32_t part_max[kMaxTensors];
     uint32_t n_slots[kMaxTensors];
     uint32_t slot_base[kMaxTensors];
     uint32_t variant[kMaxTensors];
@@ -128,15 +126,13 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
 int current_num_sms(int* num_sms);   // RKV_ERR_CUDA without a device
 
 // Number of candidate parts for a group of `tiles` tiles in a launch over k_count
-// candidates: enough parts that none holds more than part_max candidates (kPartK, or
-// kPartKWide for bf16 candidates against a regenerated reference), and, when the
+// candidates: enough parts that none holds more than kPartK candidates, and, when the
 // group has fewer tiles than there are blocks, enough that every block gets an item
 // (tiles * parts >= grid where k_count allows).  Part p of `parts` covers the candidates
 // [p * k_count / parts, (p + 1) * k_count / parts): sizes differ by at most one.
 // The kernels and the host use this one rule.
-__host__ __device__ inline uint32_t part_count(uint32_t tiles, uint32_t k_count, uint32_t grid,
-                                               uint32_t part_max) {
-    uint32_t parts = (k_count + part_max - 1) / part_max;
+__host__ __device__ inline uint32_t part_count(uint32_t tiles, uint32_t k_count, uint32_t grid) {
+    uint32_t parts = (k_count + kPartK - 1) / kPartK;
     if (tiles < grid) {
         const uint32_t want = (grid + tiles - 1) / tiles;
         if (want > parts) parts = want;
@@ -152,9 +148,9 @@ __host__ __device__ inline uint32_t group_first_tile(uint32_t g, uint32_t n_tile
     return g == 0 ? 0u : g == 1 ? warm : n_tiles - tail;
 }
 __host__ __device__ inline uint32_t group_parts(uint32_t g, uint32_t tiles, uint32_t k_count, uint32_t grid,
-                                                uint32_t tail_div, uint32_t part_max) {
-    if (g != 2) return part_count(tiles, k_count, grid, part_max);
-    const uint32_t parts = (k_count + part_max - 1) / part_max * tail_div;
+                                                uint32_t tail_div) {
+    if (g != 2) return part_count(tiles, k_count, grid);
+    const uint32_t parts = (k_count + kPartK - 1) / kPartK * tail_div;
     return parts > k_count ? k_count : parts;
 }
 // Tiles in group C: half a tile per block, for tensors long enough that the blocks'

@@ -78,21 +78,13 @@ constexpr int kOffAbort = kOffEmpty + 8 * kStages;         // uint32
 constexpr int kOffRefState = kOffAbort + 16;                  // 2 x uint32 settled bits of the reference (item parity)
 constexpr int kOffIds = kOffRefState + 8;                     // kStages x uint32: item id that starts in a stage
 constexpr int kOffPtrC = 256;                                 // consumer copy of the pointers
+constexpr int kOffPtrP = kOffPtrC + kPartK * 8;               // producer copy
+constexpr int kOffHint = kOffPtrP + kPartK * 8;               // two tables (item parity)
+constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
+constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
+constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
 static_assert(kOffPtrC >= kOffIds + 4 * kStages, "layout");
-// The tables behind the pointers are sized for the most candidates a part can hold:
-// kPartK, or kPartKWide in the kernels for bf16 candidates.
-template <bool CB16>
-struct Lay {
-    static constexpr int kCap = CB16 ? kPartKWide : kPartK;
-    static constexpr int kOffPtrP = kOffPtrC + kCap * 8;               // producer copy
-    static constexpr int kOffHint = kOffPtrP + kCap * 8;               // two tables (item parity)
-    static constexpr int kOffRec = kOffHint + 2 * kCap * (int)sizeof(Hint);
-    static constexpr int kOffStage = (kOffRec + kConsumerWarps * kCap * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
-    static constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
-};
-static_assert(2 * (Lay<false>::kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
-static_assert(2 * (Lay<true>::kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
-static_assert(kPartKWide <= kConsumers, "one thread per candidate of a part");
+static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
 // Geometry of a tile.  A thread owns 64 bytes of each candidate tile, so a candidate tile
 // always fills exactly one ring stage: 16 fp32 elements or 32 bf16 elements.  Their
@@ -227,7 +219,7 @@ __device__ __forceinline__ bool decode_item(const DevTensor* __restrict__ tensor
             const uint32_t warm = tensors[t].warm_tiles, tail = tensors[t].tail_tiles;
             const uint32_t nt = group_tiles(g, tensors[t].n_tiles, warm, tail);
             if (nt == 0) continue;
-            const uint32_t parts = group_parts(g, nt, k_count, gridDim.x, tensors[t].tail_div, tensors[t].part_max);
+            const uint32_t parts = group_parts(g, nt, k_count, gridDim.x, tensors[t].tail_div);
             const uint32_t cnt = nt * parts;
             if (id - base < cnt) {
                 it.t = t;
@@ -263,7 +255,7 @@ __device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tens
     constexpr uint32_t kTile = Geo<CB16>::kTile;
     constexpr uint32_t kRefStages = (CB16 && !RB16) ? 2 : 1;      // an fp32 tile under bf16 candidates
     const int lane = threadIdx.x & 31;
-    const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + Lay<CB16>::kOffPtrP);
+    const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrP);
     volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
     uint32_t n_issued = 0;
     int cur_t = -1;
@@ -949,14 +941,14 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
 // consumer barriers.
 __device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D, int K, int k0, int kc,
                                               uint32_t slot, Partial* __restrict__ partials, int tid,
-                                              uint32_t tile_elems, int cap) {
+                                              uint32_t tile_elems) {
     if (tid < kc) {
         Partial p;
         p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX; p.sum = 0.0;
         p.emax = -1.0f; p.qmax = -1.0f; p.valid = 1u; p.reserved = 0u;
 #pragma unroll
         for (int wp = 0; wp < kConsumerWarps; ++wp) {
-            WarpRec& r = recs[wp * cap + tid];
+            WarpRec& r = recs[wp * kPartK + tid];
             p.n_over += r.n_over;
             p.sum += r.sum;
             if (r.emax >= 0.0f) {
@@ -1004,14 +996,13 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
     constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrC);
-    constexpr int kCap = Lay<CB16>::kCap;
-    Hint* hints = reinterpret_cast<Hint*>(smem + Lay<CB16>::kOffHint);
-    WarpRec* recs = reinterpret_cast<WarpRec*>(smem + Lay<CB16>::kOffRec);
+    Hint* hints = reinterpret_cast<Hint*>(smem + kOffHint);
+    WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
     volatile uint32_t* ref_state = reinterpret_cast<volatile uint32_t*>(smem + kOffRefState);
-    const unsigned char* stages = smem + Lay<CB16>::kOffStage;
+    const unsigned char* stages = smem + kOffStage;
 
     // clear the records once; flush_records leaves them cleared
-    for (int i = tid; i < kConsumerWarps * kCap; i += kConsumers) {
+    for (int i = tid; i < kConsumerWarps * kPartK; i += kConsumers) {
         WarpRec& r = recs[i];
         r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
     }
@@ -1042,11 +1033,11 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
         const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
         const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
         CandState* st_t = state + (size_t)it.t * (size_t)(K + 1);
-        Hint* H = hints + (ord & 1u) * kCap;
+        Hint* H = hints + (ord & 1u) * kPartK;
 
         if (it.t != cur_t || part_key != cur_part) {
             consumer_sync();                      // every warp is done with the previous part
-            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile, kCap);
+            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
             if (tid < kc) ptrs[tid] = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
             cur_t = it.t; cur_part = part_key; cur_k0 = k0; cur_kc = kc;
             cur_slot = blockIdx.x;                // one Partial row per block and tensor
@@ -1062,7 +1053,7 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
             h.first = ld_elem_bits(ptrs[tid], CB16 ? RKV_BF16 : RKV_F32, 0);
             H[tid] = h;
         }
-        if (tid == kConsumers - 1) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
+        if (tid == kPartK) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
 
         // ---- the thread's reference values --------------------------------------------
         RefRegs<CB16> R;
@@ -1149,15 +1140,15 @@ __device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tens
                 }
             }
             if constexpr (CB16)
-                process_candidate_b16(R, w, h, &H[kk], &recs[warp * kCap + kk], st_t + k0 + kk, D, ptrs[kk],
+                process_candidate_b16(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
                                       it.tile, start, len, wanted, tid, lane);
             else
-                process_candidate<false>(R, w, h, &H[kk], &recs[warp * kCap + kk], st_t + k0 + kk, D, ptrs[kk],
+                process_candidate<false>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
                                          it.tile, start, len, wanted, tid, lane);
         }
     }
     consumer_sync();
-    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile, kCap);
+    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
 }
 
 // One kernel per storage variant (candidate dtype, stored reference dtype), so
@@ -1172,7 +1163,7 @@ verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, 
     Ring ring;
     ring.full0 = smem_u32(smem + kOffFull);
     ring.empty0 = smem_u32(smem + kOffEmpty);
-    ring.stage0 = smem_u32(smem + Lay<CB16>::kOffStage);
+    ring.stage0 = smem_u32(smem + kOffStage);
     ring.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -1295,12 +1286,12 @@ static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin,
     if (cudaGetDevice(&dev) != cudaSuccess) return RKV_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(verify_kernel<CB16, RB16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Lay<CB16>::kSmemBytes) != cudaSuccess)
+                                 kSmemBytes) != cudaSuccess)
             return RKV_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     // the grid is always the full resident grid: Partial rows are numbered by block
-    verify_kernel<CB16, RB16><<<grid_max, kThreads, Lay<CB16>::kSmemBytes, stream>>>(d_tensors, T, K, k_begin, k_end,
+    verify_kernel<CB16, RB16><<<grid_max, kThreads, kSmemBytes, stream>>>(d_tensors, T, K, k_begin, k_end,
                                                                          n_items, state, partials, header);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
