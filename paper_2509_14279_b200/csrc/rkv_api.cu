@@ -1,4 +1,4 @@
-// Host side of librkv: argument validation, slab planning, workspace layout,
+// Host side of librkv: argument validation, work-item planning, workspace layout,
 // launches, and the host-buffer end-to-end form.  No torch types anywhere.
 #include <math.h>
 #include <string.h>

@@ -127,7 +127,7 @@ def test_large_tensor_with_a_warm_up_group(cand_dtype):
 
 
 @pytest.mark.parametrize("dist", oracle.DISTS)
-def test_every_distribution_several_slabs_per_block(dist):
+def test_every_distribution_several_tiles_per_block(dist):
     n = 296 * 128 * 3 + 77            # several tiles, ragged tail
     ref = oracle_gen_tensor(7, 0, dist, n, "f32")
     inp = oracle_gen_tensor(7, 2, dist, n, "f32")

@@ -49,7 +49,7 @@ def _assert_same(got, want, where):
 
 def test_static_scratch_form_matches_the_allocating_form_on_two_calls_in_a_row():
     atol, rtol = 1e-5, 1e-5
-    case_a = _case(700001, 24, seed=11)           # several slabs per block, ragged tail
+    case_a = _case(700001, 24, seed=11)           # several tiles per block, ragged tail
     case_b = _case(4099, 7, seed=12)              # a much smaller case reusing the same scratch
     case_c = _case(300007, 13, seed=13, dtype="bf16")
     want = [rkv.stats_to_numpy(rkv.verify_batch(r, c, atol, rtol)) for r, c in (case_a, case_b, case_c)]
