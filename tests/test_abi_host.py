@@ -187,3 +187,33 @@ def test_population_plans_are_seeded_and_cover_the_kinds():
     m = pop.plan_multi(128, (1 << 20, 4096, 4096), seed=3, fault_rate=0.1)
     assert len(m) == 128 and all(len(r) == 3 for r in m)
     assert all(sum(c.kind in pop.FAULT_KINDS for c in r) <= 1 for r in m)
+
+
+def test_screen_outputs_validates_before_any_cuda_call():
+    L = rkv.lib()
+    assert rkv.SCREEN_BYTES == 64
+    text = open(os.path.join(ROOT, "include", "rkv.h")).read()
+    assert "rkv_screen_stats;               /* 64 bytes */" in text
+
+    def call(ptr_values=(0x1000, 0x2000), S=None, rows=8, cols=8, dtype=0, lims=(0.01, 0.01, 0.01),
+             stats=0x9000, ws=0x4000, ws_bytes=1 << 30):
+        ptrs = (ctypes.c_void_p * max(1, len(ptr_values)))(*ptr_values)
+        return L.rkv_screen_outputs(ptrs, len(ptr_values) if S is None else S, rows, cols, dtype, lims[0],
+                                    lims[1], lims[2], ctypes.c_void_p(stats), ctypes.c_void_p(ws), ws_bytes, None)
+
+    assert call(S=0) == rkv.ERR_INVALID_ARG
+    assert call(rows=0) == rkv.ERR_INVALID_ARG
+    assert call(cols=0) == rkv.ERR_INVALID_ARG
+    assert call(dtype=2) == rkv.ERR_INVALID_ARG
+    assert call(stats=0) == rkv.ERR_INVALID_ARG
+    assert call(ptr_values=(0x1000, 0)) == rkv.ERR_INVALID_ARG
+    assert call(ptr_values=(0x1000, 0x2004)) == rkv.ERR_ALIGNMENT
+    assert call(ptr_values=tuple(0x1000 * (i + 1) for i in range(17))) == rkv.ERR_UNSUPPORTED
+    assert call(rows=1 << 20, cols=1 << 20) == rkv.ERR_UNSUPPORTED
+    assert call(lims=(-0.01, 0.01, 0.01)) == rkv.ERR_INVALID_ARG
+    assert call(lims=(0.01, float("nan"), 0.01)) == rkv.ERR_INVALID_ARG
+    assert call(lims=(0.01, 0.01, -1.0)) == rkv.ERR_INVALID_ARG
+    assert call(ws=0) == rkv.ERR_WORKSPACE
+    assert call(ws=0x4008) == rkv.ERR_ALIGNMENT
+    assert L.rkv_screen_outputs(None, 2, 8, 8, 0, 0.01, 0.01, 0.01, ctypes.c_void_p(0x9000),
+                                ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_INVALID_ARG
