@@ -341,3 +341,28 @@ def test_error_codes_on_device():
     with pytest.raises(rkv.RkvError) as e:
         rkv.verify_multi([d], 1)
     assert e.value.status == rkv.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_seeded_random_cases_match_the_oracle(case):
+    """Sizes, candidate counts, dtypes, distributions and tolerances drawn from a seeded
+    generator: every statistic of every candidate against the oracle."""
+    rng = np.random.default_rng([2509, case])
+    n = int(rng.choice([1, 2, 7, 33, 1000, 3583, 3584, 3585, 7168, 7169, 20000, 65537, 200003, 1048577]))
+    if case % 6 == 5:
+        n = int(rng.integers(1, 300000))
+    K = int(rng.choice([1, 2, 3, 12, 13, 31, 64, 65, 70]))
+    cand_dtype, ref_dtype = [("f32", "f32"), ("bf16", "f32"), ("bf16", "bf16"), ("f32", "bf16")][case % 4]
+    dist = int(rng.choice(oracle.DISTS))
+    atol, rtol = [(1e-5, 1e-5), (1e-2, 1.6e-2), (0.0, 1e-3), (1e-3, 0.0), (0.0, 0.0), (1.0, 1.0)][int(rng.integers(0, 6))]
+    with_input = bool(rng.integers(0, 2))
+    ref = oracle_gen_tensor(300 + case, 0, dist, n, ref_dtype)
+    inp = oracle_gen_tensor(300 + case, 2, dist, n, cand_dtype)
+    cands = build_case_cpu(mixed_plan(K, n, seed=case, bf16=(cand_dtype == "bf16")), ref, inp, cand_dtype)
+    where = f"case {case}: n={n} K={K} {cand_dtype}/{ref_dtype} dist={dist} tol=({atol},{rtol}) input={with_input}"
+    got, _ = check_case(ref, cands, atol, rtol, inp if with_input else None, where=where)
+    # the same bytes with reference (and input) regenerated on the device
+    got2, _ = run_gpu(ref, cands, atol, rtol, gen_ref=(300 + case, 0, dist),
+                      gen_inp=(300 + case, 2, dist) if with_input else None,
+                      ref_dtype=rkv.F32 if ref_dtype == "f32" else rkv.BF16)
+    assert got2.tobytes() == got.tobytes(), where
