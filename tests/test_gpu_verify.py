@@ -325,6 +325,22 @@ def test_host_buffer_form(dtype):
         assert_stats_equal(got[k], want[k], f"host k={k}")
 
 
+def test_host_buffer_form_on_a_tensor_with_all_three_item_groups():
+    """Chunks of candidates (16, then the rest) over a tensor long enough for the warm-up
+    and the tail group; a ragged last tile."""
+    n, K = 3584 * 2100 + 5, 20
+    ref = oracle_gen_tensor(8, 0, oracle.UNIFORM_PM1, n, "f32")
+    plan = mixed_plan(K, n, seed=8)
+    plan[17] = pop.Candidate(pop.CORRUPT, delta=1.0, indices=(n - 1,))
+    plan[3] = pop.Candidate(pop.NAN_AT, indices=(3584 * 2050 + 7,))
+    cands = build_case_cpu(plan, ref, ref, "f32")
+    got = rkv.verify_batch_host(ref, cands, ATOL, RTOL)
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], ATOL, RTOL)
+    for k in range(K):
+        assert_stats_equal(got[k], want[k], f"host, large k={k}")
+    assert int(got[17]["argmax_abs_err"]) == n - 1
+
+
 def test_error_codes_on_device():
     n = 1024
     ref = torch.zeros(n + 4, device="cuda")
