@@ -26,6 +26,12 @@
  * stream-ordered on the given stream and never synchronises it, except where a
  * function says so.  bf16 tensors are raw 16-bit patterns.  Tensors are flat,
  * contiguous, row-major; a shape is only a product.
+ *
+ * Stream capture.  Every verification call sends a small descriptor table from
+ * host memory that does not outlive the call, so none of them can be recorded
+ * into a CUDA graph: a call on a stream that is being captured enqueues nothing
+ * and returns RKV_ERR_UNSUPPORTED.  (rkv_gen_inputs* and rkv_screen_outputs pass
+ * everything by value.)
  */
 #ifndef RKV_H
 #define RKV_H
@@ -182,7 +188,8 @@ int rkv_gen_inputs_ex(uint64_t seed, uint64_t stream_id, int dist, uint64_t n,
  * Runs on the stream set by rkv_set_stream.  Uses a library-owned scratch
  * buffer that grows on demand (cudaMalloc on first use / growth: not safe
  * during stream capture; concurrent calls on different streams would share it,
- * so serialise them).  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ * so serialise them).  Errors: INVALID_ARG, UNSUPPORTED (also: the stream is
+ * being captured), ALIGNMENT, CUDA.
  */
 int rkv_verify_batch(const void *ref, const void *const *cands, int K, uint64_t n, int dtype,
                      float atol, float rtol, rkv_stats *stats_out);
@@ -200,8 +207,9 @@ int rkv_verify_batch(const void *ref, const void *const *cands, int K, uint64_t 
  * Nothing is allocated on the device.  The descriptors and pointer tables are
  * copied to the workspace with one cudaMemcpyAsync from pageable host memory and
  * the rest of the workspace is cleared with one cudaMemsetAsync.
- * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.  A device-side
- * timeout is reported by rkv_device_status.
+ * Errors: INVALID_ARG, UNSUPPORTED (also: cuda_stream is being captured),
+ * ALIGNMENT, WORKSPACE, CUDA.  A device-side timeout is reported by
+ * rkv_device_status.
  */
 int rkv_verify_multi(const rkv_tensor_desc *tensors, int T, int K, rkv_stats *stats_out,
                      uint32_t *joint_pass, void *workspace, size_t workspace_bytes,
@@ -218,7 +226,8 @@ size_t rkv_workspace_bytes(const rkv_tensor_desc *tensors, int T, int K);
 int rkv_device_status(const void *workspace, void *cuda_stream);
 
 /*
- * End-to-end form with HOST buffers: copies the reference and the candidates to
+ * End-to-end form with HOST buffers (plumbing around rkv_verify_batch, no passage of its
+ * own): copies the reference and the candidates to
  * the device in chunks (overlapped with verification on two streams), verifies,
  * copies the K results back and synchronises.  Pinned host buffers make the
  * copies asynchronous.  Allocates (and caches) device staging memory.
@@ -228,6 +237,24 @@ int rkv_device_status(const void *workspace, void *cuda_stream);
  */
 int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, int K, uint64_t n,
                           int dtype, float atol, float rtol, rkv_stats *stats_host);
+
+/*
+ * The general case with HOST buffers (plumbing around rkv_verify_multi, no passage of
+ * its own): the descriptors of rkv_verify_multi, except that tensors[t].cands is a HOST
+ * array of K HOST pointers and tensors[t].ref / tensors[t].input are HOST pointers
+ * (when their source is RKV_SRC_POINTER; a generated reference or input is regenerated
+ * on the device and nothing of it is copied).  References and inputs are copied once,
+ * the candidates in chunks of a few candidates of every tensor, two chunks in flight,
+ * each chunk verified while the next one travels; the results come back and the
+ * stream set by rkv_set_stream is synchronised.  Host pointers need no alignment;
+ * pinned buffers make the copies asynchronous.  Allocates (and caches) device staging
+ * memory: not for callers that cannot allocate.
+ *   stats_host  HOST, K*T rkv_stats, entry [k*T + t]
+ *   joint_host  HOST, K uint32 (1 = pass on all T tensors), may be NULL
+ * Errors: INVALID_ARG, UNSUPPORTED (T > 64, n >= 2^40, capturing stream), CUDA.
+ */
+int rkv_verify_multi_host(const rkv_tensor_desc *tensors, int T, int K, rkv_stats *stats_host,
+                          uint32_t *joint_host);
 
 /*
  * rkv_verify_batch with no allocation of any kind.  (The paper has no
@@ -256,7 +283,8 @@ int rkv_verify_batch_host(const void *ref_host, const void *const *cands_host, i
  *
  * First call on a device: looks up the array's device address once (with that
  * device current) and sets a kernel attribute.  Make that first call outside any
- * stream capture.
+ * stream capture.  (Like every verification call it returns RKV_ERR_UNSUPPORTED
+ * on a stream that is being captured: its table is sent from the host stack.)
  *
  * All calls on a device share the one array, and it keeps whatever the previous
  * call left there.  The library rewrites the status word and the tables and
@@ -272,7 +300,8 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
                             float atol, float rtol, rkv_stats *stats_out, void *cuda_stream);
 
 /*
- * Host-only planning helper (no CUDA call): how the work of one tensor is cut.
+ * Host-only planning helper (no CUDA call; plumbing, no passage of its own): how the
+ * work of one tensor is cut.
  * The tensor is cut into *n_tiles tiles of *tile_elems elements (a thread of the
  * verification kernel owns 64 bytes of each candidate tile: 3584 fp32 or 7168 bf16
  * elements per tile).  One work item is

@@ -107,6 +107,8 @@ def lib() -> ctypes.CDLL:
         L.rkv_device_status.argtypes = [vp, vp]
         L.rkv_verify_batch_host.restype = i32
         L.rkv_verify_batch_host.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
+        L.rkv_verify_multi_host.restype = i32
+        L.rkv_verify_multi_host.argtypes = [ctypes.POINTER(TensorDescC), i32, i32, vp, vp]
         L.rkv_verify_batch_static.restype = i32
         L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
         u32p = ctypes.POINTER(ctypes.c_uint32)
@@ -140,6 +142,43 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"rkv tensors are float32 or bfloat16, got {t.dtype}")
 
 
+def _require(t, what: str, device=None, dtype=None, numel=None, min_bytes=None) -> None:
+    """Check a tensor before its raw pointer crosses the C ABI (the library sees no sizes).
+
+    The candidates come from machine-written kernels, so a tensor of the wrong shape, dtype
+    or device is an ordinary failure here: it must raise on the host, not become a read
+    past the end of a buffer on the device."""
+    if not isinstance(t, torch.Tensor):
+        raise TypeError(f"{what}: expected a torch.Tensor, got {type(t).__name__}")
+    if device is not None:
+        if t.device.type != device.type or (device.type == "cuda" and device.index is not None
+                                            and t.device.index != device.index):
+            raise ValueError(f"{what}: on {t.device}, expected {device}")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{what}: dtype {t.dtype}, expected {dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{what}: not contiguous")
+    if numel is not None and t.numel() != numel:
+        raise ValueError(f"{what}: {t.numel()} elements, expected {numel}")
+    if min_bytes is not None and t.numel() * t.element_size() < min_bytes:
+        raise ValueError(f"{what}: {t.numel() * t.element_size()} bytes, needs at least {min_bytes}")
+
+
+def _require_case(ref, cands, what: str, stats_out=None, device_type: str = "cuda"):
+    """ref and every candidate: same device, same dtype, contiguous, n elements each."""
+    if len(cands) < 1:
+        raise ValueError(f"{what}: no candidates")
+    _require(ref, f"{what}: ref")
+    if ref.device.type != device_type:
+        raise ValueError(f"{what}: ref is on {ref.device}, expected a {device_type} tensor")
+    _dtype_code(ref)
+    for k, c in enumerate(cands):
+        _require(c, f"{what}: candidate {k}", device=ref.device, dtype=ref.dtype, numel=ref.numel())
+    if stats_out is not None:
+        _require(stats_out, f"{what}: stats_out", device=ref.device, dtype=torch.uint8,
+                 min_bytes=len(cands) * STATS_BYTES)
+
+
 def _stream_ptr(stream=None) -> int:
     s = torch.cuda.current_stream() if stream is None else stream
     return int(s.cuda_stream)
@@ -168,6 +207,8 @@ def gen_inputs(seed: int, dist: int, shape, dtype: torch.dtype = torch.float32,
     shape = tuple(int(s) for s in shape)
     if out is None:
         out = torch.empty(shape, dtype=dtype, device="cuda")
+    else:
+        _require(out, "gen_inputs: out", device=torch.device("cuda"), numel=int(np.prod(shape)))
     set_stream()
     arr = (ctypes.c_int64 * len(shape))(*shape)
     _check(lib().rkv_gen_inputs(int(seed), int(dist), arr, len(shape), _dtype_code(out),
@@ -180,6 +221,8 @@ def gen_inputs_ex(seed: int, stream_id: int, dist: int, n: int, first_elem: int 
                   stream=None) -> torch.Tensor:
     if out is None:
         out = torch.empty(int(n), dtype=dtype, device="cuda")
+    else:
+        _require(out, "gen_inputs_ex: out", device=torch.device("cuda"), min_bytes=int(n) * out.element_size())
     _check(lib().rkv_gen_inputs_ex(int(seed), int(stream_id), int(dist), int(n), int(first_elem),
                                    _dtype_code(out), ctypes.c_void_p(out.data_ptr()),
                                    ctypes.c_void_p(_stream_ptr(stream))), "rkv_gen_inputs_ex")
@@ -196,6 +239,7 @@ def verify_batch(ref: torch.Tensor, cands, atol: float, rtol: float,
     """rkv_verify_batch: K candidates against one reference, same dtype, no input tensor.
     Returns the device buffer of K rkv_stats (uint8, K*88 bytes)."""
     K = len(cands)
+    _require_case(ref, cands, "verify_batch", stats_out)
     n = ref.numel()
     if stats_out is None:
         stats_out = torch.empty(K * STATS_BYTES, dtype=torch.uint8, device=ref.device)
@@ -215,6 +259,7 @@ def verify_batch_static(ref: torch.Tensor, cands, atol: float, rtol: float,
     device memory when they verify (all memory already in their own pool, or no allocator
     calls allowed on this thread).  Calls share that array: do not overlap them on the GPU."""
     K = len(cands)
+    _require_case(ref, cands, "verify_batch_static", stats_out)
     ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cands])
     _check(lib().rkv_verify_batch_static(ctypes.c_void_p(ref.data_ptr()), ptrs, K, ref.numel(),
                                          _dtype_code(ref), float(atol), float(rtol),
@@ -238,10 +283,24 @@ class TensorDesc:
     ref_dtype: int | None = None      # for a generated reference; default fp32
     _keep: list = field(default_factory=list, repr=False)
 
-    def to_c(self) -> TensorDescC:
+    def to_c(self, where: str = "cuda") -> TensorDescC:
+        """The C descriptor; `where` is the device type every tensor must live on ("cuda" for
+        the device forms, "cpu" for the host-buffer form)."""
         d = TensorDescC()
         d.n = int(self.n)
         K = len(self.cands)
+        if K < 1:
+            raise ValueError("TensorDesc: no candidates")
+        first = self.cands[0]
+        _require(first, "TensorDesc: candidate 0", device=torch.device(where), numel=d.n)
+        for k, c in enumerate(self.cands):
+            _require(c, f"TensorDesc: candidate {k}", device=first.device, dtype=first.dtype, numel=d.n)
+        if self.ref is not None:
+            _require(self.ref, "TensorDesc: ref", device=first.device, numel=d.n)
+        elif self.ref_gen is None:
+            raise ValueError("TensorDesc: neither ref nor ref_gen given")
+        if self.input is not None:     # a copy is a bit copy: the input has the candidates' dtype
+            _require(self.input, "TensorDesc: input", device=first.device, dtype=first.dtype, numel=d.n)
         ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in self.cands])
         self._keep.append(ptrs)
         d.cands = ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p))
@@ -297,10 +356,20 @@ def verify_multi(tensors, K: int, workspace: torch.Tensor | None = None,
         if need == 0:
             raise RkvError(ERR_INVALID_ARG, "rkv_workspace_bytes")
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    else:
+        _require(workspace, "verify_multi: workspace", device=dev, dtype=torch.uint8)
     if stats_out is None:
         stats_out = torch.empty(K * T * STATS_BYTES, dtype=torch.uint8, device=dev)
+    else:
+        _require(stats_out, "verify_multi: stats_out", device=dev, dtype=torch.uint8,
+                 min_bytes=K * T * STATS_BYTES)
     if joint_pass is None:
         joint_pass = torch.empty(K, dtype=torch.int32, device=dev)
+    else:
+        _require(joint_pass, "verify_multi: joint_pass", device=dev, dtype=torch.int32, numel=K)
+    for t in tensors:
+        if len(t.cands) != K:
+            raise ValueError(f"verify_multi: a tensor has {len(t.cands)} candidates, K = {K}")
     _check(lib().rkv_verify_multi(arr, T, int(K), ctypes.c_void_p(stats_out.data_ptr()),
                                   ctypes.c_void_p(joint_pass.data_ptr()),
                                   ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
@@ -321,8 +390,8 @@ def device_status(workspace: torch.Tensor, stream=None) -> int:
 def verify_batch_host(ref: torch.Tensor, cands, atol: float, rtol: float) -> np.ndarray:
     """rkv_verify_batch_host: HOST tensors in, structured numpy stats out (synchronous)."""
     K = len(cands)
+    _require_case(ref, cands, "verify_batch_host", device_type="cpu")
     n = ref.numel()
-    assert ref.device.type == "cpu" and all(c.device.type == "cpu" for c in cands)
     out = np.zeros(K, dtype=STATS_DTYPE)
     ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cands])
     set_stream()
@@ -331,6 +400,23 @@ def verify_batch_host(ref: torch.Tensor, cands, atol: float, rtol: float) -> np.
                                        out.ctypes.data_as(ctypes.c_void_p)),
            "rkv_verify_batch_host")
     return out
+
+
+def verify_multi_host(tensors, K: int) -> tuple:
+    """rkv_verify_multi_host: TensorDescs over HOST tensors in, (structured numpy stats of
+    shape [K, T], joint_pass [K] uint32) out.  Synchronous."""
+    T = len(tensors)
+    arr = (TensorDescC * T)()
+    for i, t in enumerate(tensors):
+        if len(t.cands) != K:
+            raise ValueError(f"verify_multi_host: a tensor has {len(t.cands)} candidates, K = {K}")
+        arr[i] = t.to_c(where="cpu")
+    out = np.zeros((K, T), dtype=STATS_DTYPE)
+    joint = np.zeros(K, dtype=np.uint32)
+    set_stream()
+    _check(lib().rkv_verify_multi_host(arr, T, int(K), out.ctypes.data_as(ctypes.c_void_p),
+                                       joint.ctypes.data_as(ctypes.c_void_p)), "rkv_verify_multi_host")
+    return out, joint
 
 
 def release_cached() -> None:

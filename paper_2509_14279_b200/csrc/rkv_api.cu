@@ -38,6 +38,16 @@ static uint64_t items_of(uint32_t n_tiles, uint32_t warm_tiles, uint32_t tail_ti
     return items;
 }
 
+// The descriptor tables of a call travel to the device from host memory that dies with the
+// call.  A stream capture would record that copy with its host address and every replay of
+// the graph would read freed memory, so the verification entry points refuse a capturing
+// stream instead of enqueueing anything.
+int refuse_capture(cudaStream_t stream) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) { cudaGetLastError(); return RKV_ERR_CUDA; }
+    return st == cudaStreamCaptureStatusNone ? RKV_OK : RKV_ERR_UNSUPPORTED;
+}
+
 static bool finite_nonneg(float x) { return x >= 0.0f && x <= 3.402823466e38f; }
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static bool dtype_ok(int d) { return d == RKV_F32 || d == RKV_BF16; }
@@ -332,6 +342,8 @@ int rkv_verify_multi(const rkv_tensor_desc* tensors, int T, int K, rkv_stats* st
     rc = make_plan(tensors, T, K, K, sms, &plan);
     if (rc != RKV_OK) return rc;
     if (workspace_bytes < plan.total_bytes) return RKV_ERR_WORKSPACE;
+    rc = refuse_capture(reinterpret_cast<cudaStream_t>(cuda_stream));
+    if (rc != RKV_OK) return rc;
     return run_case(tensors, T, K, 0, K, true, true, plan, stats_out, joint_pass, workspace,
                     reinterpret_cast<cudaStream_t>(cuda_stream));
 }
@@ -352,6 +364,8 @@ int rkv_verify_batch(const void* ref, const void* const* cands, int K, uint64_t 
     if (rc != RKV_OK) return rc;
     Plan plan;
     rc = make_plan(&d, 1, K, K, sms, &plan);
+    if (rc != RKV_OK) return rc;
+    rc = refuse_capture(g_stream);
     if (rc != RKV_OK) return rc;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -374,32 +388,53 @@ int rkv_device_status(const void* workspace, void* cuda_stream) {
     return st;
 }
 
-int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, int K, uint64_t n,
-                          int dtype, float atol, float rtol, rkv_stats* stats_host) {
-    if (!ref_host || !cands_host || !stats_host || K < 1 || n < 1 || !dtype_ok(dtype) ||
-        !finite_nonneg(atol) || !finite_nonneg(rtol))
-        return RKV_ERR_INVALID_ARG;
-    if (n >= kMaxN) return RKV_ERR_UNSUPPORTED;
-    for (int k = 0; k < K; ++k)
-        if (!cands_host[k]) return RKV_ERR_INVALID_ARG;
+int rkv_verify_multi_host(const rkv_tensor_desc* tensors, int T, int K, rkv_stats* stats_host,
+                          uint32_t* joint_host) {
+    if (!tensors || !stats_host || T < 1 || K < 1) return RKV_ERR_INVALID_ARG;
+    if (T > kMaxTensors) return RKV_ERR_UNSUPPORTED;
+    for (int t = 0; t < T; ++t) {
+        const rkv_tensor_desc& d = tensors[t];
+        if (d.n < 1 || !dtype_ok(d.cand_dtype) || !dtype_ok(d.ref_dtype) || !finite_nonneg(d.atol) ||
+            !finite_nonneg(d.rtol) || !d.cands)
+            return RKV_ERR_INVALID_ARG;
+        if (d.n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+        if (d.ref_src == RKV_SRC_POINTER ? !d.ref : (d.ref_src != RKV_SRC_GENERATED || !dist_ok(d.ref_gen.dist)))
+            return RKV_ERR_INVALID_ARG;
+        if (d.input_src == RKV_SRC_POINTER ? !d.input
+                                           : (d.input_src == RKV_SRC_GENERATED ? !dist_ok(d.input_gen.dist)
+                                                                               : d.input_src != RKV_SRC_NONE))
+            return RKV_ERR_INVALID_ARG;
+        for (int k = 0; k < K; ++k)
+            if (!d.cands[k]) return RKV_ERR_INVALID_ARG;
+    }
     int sms = 0;
     int rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    rc = refuse_capture(g_stream);
     if (rc != RKV_OK) return rc;
     int dev = 0;
     cudaGetDevice(&dev);
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceCache& c = g_cache[dev & 63];
 
-    const size_t esz = dtype == RKV_BF16 ? 2 : 4;
-    const size_t tensor_bytes = ((size_t)n * esz + 255) / 256 * 256;
-    // candidates travel in chunks of kc tensors, two chunks in flight
-    size_t kc = (size_t(512) << 20) / tensor_bytes;
+    // staging layout: references and inputs | two buffers of kc candidates of every tensor | results
+    auto round256 = [](size_t b) { return (b + 255) / 256 * 256; };
+    auto esz = [](int dtype) { return (size_t)(dtype == RKV_BF16 ? 2 : 4); };
+    size_t fixed_bytes = 0, per_cand = 0;
+    for (int t = 0; t < T; ++t) {
+        const rkv_tensor_desc& d = tensors[t];
+        if (d.ref_src == RKV_SRC_POINTER) fixed_bytes += round256((size_t)d.n * esz(d.ref_dtype));
+        if (d.input_src == RKV_SRC_POINTER) fixed_bytes += round256((size_t)d.n * esz(d.cand_dtype));
+        per_cand += round256((size_t)d.n * esz(d.cand_dtype));
+    }
+    // candidates travel in chunks of kc, two chunks in flight
+    size_t kc = (size_t(512) << 20) / per_cand;
     if (kc < 1) kc = 1;
     if (kc > (size_t)K) kc = (size_t)K;
     if (kc > 16) kc = 16;
-    const size_t stats_bytes = ((size_t)K * sizeof(rkv_stats) + 255) / 256 * 256;
-    const size_t need = tensor_bytes * (1 + 2 * kc) + stats_bytes;
-    rc = ensure(&c.staging, &c.staging_bytes, need);
+    const size_t stats_bytes = round256((size_t)K * (size_t)T * sizeof(rkv_stats));
+    const size_t joint_bytes = round256((size_t)K * sizeof(uint32_t));
+    rc = ensure(&c.staging, &c.staging_bytes, fixed_bytes + 2 * kc * per_cand + stats_bytes + joint_bytes);
     if (rc != RKV_OK) return rc;
     for (int i = 0; i < 2; ++i) {
         if (!c.copy_stream[i] &&
@@ -411,29 +446,42 @@ int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, i
         }
     }
     unsigned char* base = reinterpret_cast<unsigned char*>(c.staging);
-    unsigned char* d_ref = base;
-    unsigned char* d_chunk[2] = {base + tensor_bytes, base + tensor_bytes * (1 + kc)};
-    rkv_stats* d_stats = reinterpret_cast<rkv_stats*>(base + tensor_bytes * (1 + 2 * kc));
+    unsigned char* d_chunk[2] = {base + fixed_bytes, base + fixed_bytes + kc * per_cand};
+    rkv_stats* d_stats = reinterpret_cast<rkv_stats*>(base + fixed_bytes + 2 * kc * per_cand);
+    uint32_t* d_joint = reinterpret_cast<uint32_t*>(base + fixed_bytes + 2 * kc * per_cand + stats_bytes);
 
-    // device pointers of every candidate: candidate k lives in slot k % kc of buffer (k / kc) % 2
-    std::vector<const void*> ptrs((size_t)K);
-    for (int k = 0; k < K; ++k)
-        ptrs[(size_t)k] = d_chunk[((size_t)k / kc) & 1] + ((size_t)k % kc) * tensor_bytes;
-    rkv_tensor_desc d;
-    memset(&d, 0, sizeof d);
-    d.n = n; d.ref = d_ref; d.cands = ptrs.data();
-    d.cand_dtype = dtype; d.ref_dtype = dtype;
-    d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
-    d.atol = atol; d.rtol = rtol;
+    // device-side descriptors: candidate k of tensor t lives in slot k % kc of buffer (k / kc) % 2
+    std::vector<rkv_tensor_desc> dd(tensors, tensors + T);
+    std::vector<const void*> ptrs((size_t)T * (size_t)K);
+    cudaStream_t main = g_stream;
+    bool fail = false;
+    size_t fixed_at = 0, tensor_at = 0;
+    for (int t = 0; t < T; ++t) {
+        rkv_tensor_desc& d = dd[(size_t)t];
+        if (d.ref_src == RKV_SRC_POINTER) {
+            const size_t b = (size_t)d.n * esz(d.ref_dtype);
+            fail |= cudaMemcpyAsync(base + fixed_at, tensors[t].ref, b, cudaMemcpyHostToDevice, main) != cudaSuccess;
+            d.ref = base + fixed_at;
+            fixed_at += round256(b);
+        }
+        if (d.input_src == RKV_SRC_POINTER) {
+            const size_t b = (size_t)d.n * esz(d.cand_dtype);
+            fail |= cudaMemcpyAsync(base + fixed_at, tensors[t].input, b, cudaMemcpyHostToDevice, main) != cudaSuccess;
+            d.input = base + fixed_at;
+            fixed_at += round256(b);
+        }
+        const size_t cb = round256((size_t)d.n * esz(d.cand_dtype));
+        for (int k = 0; k < K; ++k)
+            ptrs[(size_t)t * K + k] = d_chunk[((size_t)k / kc) & 1] + ((size_t)k % kc) * per_cand + tensor_at;
+        d.cands = ptrs.data() + (size_t)t * K;
+        tensor_at += cb;
+    }
     Plan plan;
-    rc = make_plan(&d, 1, K, (int)kc, sms, &plan);
+    rc = make_plan(dd.data(), T, K, (int)kc, sms, &plan);
     if (rc != RKV_OK) return rc;
     rc = ensure(&c.workspace, &c.workspace_bytes, plan.total_bytes);
     if (rc != RKV_OK) return rc;
 
-    cudaStream_t main = g_stream;
-    bool fail = false;
-    fail |= cudaMemcpyAsync(d_ref, ref_host, (size_t)n * esz, cudaMemcpyHostToDevice, main) != cudaSuccess;
     const int n_chunks = (int)(((size_t)K + kc - 1) / kc);
     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
         const int b = ch & 1;
@@ -442,23 +490,41 @@ int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, i
         // the buffer may be overwritten once the verification of chunk ch-2 is done
         if (ch >= 2) fail |= cudaStreamWaitEvent(c.copy_stream[b], c.consumed[b], 0) != cudaSuccess;
         for (int k = k0; k < k1; ++k)
-            fail |= cudaMemcpyAsync(const_cast<void*>(ptrs[(size_t)k]), cands_host[k], (size_t)n * esz,
-                                    cudaMemcpyHostToDevice, c.copy_stream[b]) != cudaSuccess;
+            for (int t = 0; t < T; ++t)
+                fail |= cudaMemcpyAsync(const_cast<void*>(ptrs[(size_t)t * K + k]), tensors[t].cands[k],
+                                        (size_t)tensors[t].n * esz(tensors[t].cand_dtype), cudaMemcpyHostToDevice,
+                                        c.copy_stream[b]) != cudaSuccess;
         fail |= cudaEventRecord(c.copied[b], c.copy_stream[b]) != cudaSuccess;
         fail |= cudaStreamWaitEvent(main, c.copied[b], 0) != cudaSuccess;
         if (fail) break;
-        rc = run_case(&d, 1, K, k0, k1, k1 == K, ch == 0, plan, d_stats, nullptr, c.workspace, main);
+        rc = run_case(dd.data(), T, K, k0, k1, k1 == K, ch == 0, plan, d_stats, d_joint, c.workspace, main);
         if (rc != RKV_OK) { fail = true; break; }
         fail |= cudaEventRecord(c.consumed[b], main) != cudaSuccess;
     }
-    if (!fail)
-        fail |= cudaMemcpyAsync(stats_host, d_stats, (size_t)K * sizeof(rkv_stats), cudaMemcpyDeviceToHost,
-                                main) != cudaSuccess;
+    if (!fail) {
+        fail |= cudaMemcpyAsync(stats_host, d_stats, (size_t)K * (size_t)T * sizeof(rkv_stats),
+                                cudaMemcpyDeviceToHost, main) != cudaSuccess;
+        if (joint_host)
+            fail |= cudaMemcpyAsync(joint_host, d_joint, (size_t)K * sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                                    main) != cudaSuccess;
+    }
     const bool sync_fail = cudaStreamSynchronize(main) != cudaSuccess;
     cudaStreamSynchronize(c.copy_stream[0]);
     cudaStreamSynchronize(c.copy_stream[1]);
     if (fail || sync_fail) { cudaGetLastError(); return rc != RKV_OK ? rc : RKV_ERR_CUDA; }
     return RKV_OK;
+}
+
+int rkv_verify_batch_host(const void* ref_host, const void* const* cands_host, int K, uint64_t n,
+                          int dtype, float atol, float rtol, rkv_stats* stats_host) {
+    if (!cands_host) return RKV_ERR_INVALID_ARG;
+    rkv_tensor_desc d;
+    memset(&d, 0, sizeof d);
+    d.n = n; d.ref = ref_host; d.cands = cands_host;
+    d.cand_dtype = dtype; d.ref_dtype = dtype;
+    d.ref_src = RKV_SRC_POINTER; d.input_src = RKV_SRC_NONE;
+    d.atol = atol; d.rtol = rtol;
+    return rkv_verify_multi_host(&d, 1, K, stats_host, nullptr);
 }
 
 // ----------------------------------------------------------------------------
@@ -523,6 +589,8 @@ int rkv_verify_batch_static(const void* ref, const void* const* cands, int K, ui
     rc = make_plan(&d, 1, K, K, sms, &plan);
     if (rc != RKV_OK) return rc;
     if (plan.total_bytes > kStaticScratchBytes) return RKV_ERR_UNSUPPORTED;
+    rc = refuse_capture(reinterpret_cast<cudaStream_t>(cuda_stream));
+    if (rc != RKV_OK) return rc;
     void* scratch = nullptr;
     rc = static_scratch_address(&scratch);
     if (rc != RKV_OK) return rc;

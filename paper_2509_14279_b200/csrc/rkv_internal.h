@@ -124,6 +124,7 @@ int validate_tensors(const rkv_tensor_desc* tensors, int T, int K);
 // k_count: candidates one launch covers (K, or the chunk length of the host-buffer form)
 int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num_sms, Plan* plan);
 int current_num_sms(int* num_sms);   // RKV_ERR_CUDA without a device
+int refuse_capture(cudaStream_t stream);   // RKV_ERR_UNSUPPORTED while `stream` is being captured
 
 // Number of candidate parts for a group of `tiles` tiles in a launch over k_count
 // candidates: enough parts that none holds more than kPartK candidates, and, when the

@@ -13,8 +13,11 @@ from paper_2509_14279_b200 import population as pop
 EXACT_FIELDS = ("verdict", "flags", "n_over_tol", "n_nan", "n_inf", "n_inf_mismatch",
                 "n_comparable", "argmax_abs_err", "argmax_rel_err")
 BITWISE_FLOAT_FIELDS = ("max_abs_err", "max_rel_err")
-# mean-error statistics: the GPU sums fp32 partial sums of <= 8 elements in fp64, the
-# oracle sums every element in fp64; the bound is 3 * 2^-24 relative, the bar is 1e-6
+# mean-error statistics: the oracle sums every element in fp64.  The GPU sums a thread's 16
+# (fp32 candidates) or 32 (16-bit candidates) errors of a tile in a balanced fp32 tree (4 or 5
+# levels), the 32 threads of a warp in 5 more fp32 levels, and everything above that in fp64.
+# All terms are non-negative, so the relative error is at most 9 or 10 roundings of 2^-24,
+# about 6e-7; the bar is 1e-6.
 MEAN_RTOL = 1e-6
 
 

@@ -217,3 +217,32 @@ def test_screen_outputs_validates_before_any_cuda_call():
     assert call(ws=0x4008) == rkv.ERR_ALIGNMENT
     assert L.rkv_screen_outputs(None, 2, 8, 8, 0, 0.01, 0.01, 0.01, ctypes.c_void_p(0x9000),
                                 ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_INVALID_ARG
+
+
+def test_binding_refuses_mismatched_tensors_before_the_c_call():
+    """A candidate of the wrong size, dtype or device, a strided view or too small a result
+    buffer must raise on the host: the C ABI sees pointers only and would read past the end."""
+    ref = torch.zeros(1024)
+    good = torch.zeros(1024)
+    with pytest.raises(ValueError, match="candidate 1.*1000 elements"):
+        rkv._require_case(ref, [good, torch.zeros(1000)], "t", device_type="cpu")
+    with pytest.raises(TypeError, match="candidate 0.*dtype"):
+        rkv._require_case(ref, [good.to(torch.bfloat16)], "t", device_type="cpu")
+    with pytest.raises(ValueError, match="not contiguous"):
+        rkv._require_case(ref, [torch.zeros(2048)[::2]], "t", device_type="cpu")
+    with pytest.raises(TypeError, match="float32 or bfloat16"):
+        rkv._require_case(ref.double(), [good.double()], "t", device_type="cpu")
+    with pytest.raises(ValueError, match="no candidates"):
+        rkv._require_case(ref, [], "t", device_type="cpu")
+    with pytest.raises(ValueError, match="stats_out.*needs at least"):
+        rkv._require_case(ref, [good, good], "t", stats_out=torch.zeros(100, dtype=torch.uint8), device_type="cpu")
+    rkv._require_case(ref, [good, good], "t", stats_out=torch.zeros(176, dtype=torch.uint8), device_type="cpu")
+    # the device forms refuse host tensors, the host form refuses nothing it should take
+    with pytest.raises(ValueError, match="expected a cuda tensor"):
+        rkv.verify_batch(ref, [good], 1e-5, 1e-5)
+    with pytest.raises(ValueError, match="expected a cuda tensor"):
+        rkv.verify_batch_static(ref, [good], 1e-5, 1e-5, torch.zeros(88, dtype=torch.uint8))
+    with pytest.raises(ValueError, match="expected cuda"):
+        rkv.TensorDesc(n=1024, cands=[good], atol=1e-5, rtol=1e-5, ref=ref).to_c()
+    with pytest.raises(TypeError):
+        rkv._require(3.0, "x")

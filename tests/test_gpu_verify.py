@@ -341,6 +341,35 @@ def test_host_buffer_form_on_a_tensor_with_all_three_item_groups():
     assert int(got[17]["argmax_abs_err"]) == n - 1
 
 
+def test_host_buffer_form_of_the_general_case():
+    """rkv_verify_multi_host: an fp32 tensor read from host memory (reference and input) next to
+    a bf16 tensor whose reference and input are regenerated on the device; more candidates than
+    one chunk holds, so the partial results carry over between the chunk launches."""
+    n32, n16, K = 3584 * 40 + 3, 7168 * 33 + 5, 37
+    ref32 = oracle_gen_tensor(21, 0, oracle.NORMAL, n32, "f32")
+    inp32 = oracle_gen_tensor(21, 2, oracle.NORMAL, n32, "f32")
+    ref16 = oracle_gen_tensor(21, 1 << 32, oracle.UNIFORM_PM1, n16, "f32")
+    inp16 = oracle_gen_tensor(21, (1 << 32) | 2, oracle.UNIFORM_PM1, n16, "bf16")
+    c32 = build_case_cpu(mixed_plan(K, n32, seed=31), ref32, inp32, "f32")
+    c16 = build_case_cpu(mixed_plan(K, n16, seed=32, bf16=True), ref16, inp16, "bf16")
+    c16 = c16[5:] + c16[:5]                 # faults of the two tensors fall on different candidates
+    descs = [
+        rkv.TensorDesc(n=n32, cands=c32, atol=1e-5, rtol=1e-5, ref=ref32, input=inp32),
+        rkv.TensorDesc(n=n16, cands=c16, atol=1e-2, rtol=1.6e-2,
+                       ref_gen=(21, 1 << 32, rkv.DIST_UNIFORM_PM1), input_gen=(21, (1 << 32) | 2, rkv.DIST_UNIFORM_PM1)),
+    ]
+    got, joint = rkv.verify_multi_host(descs, K)
+    verdicts = []
+    for k in range(K):
+        w0 = oracle.verify(pop.bits_numpy(ref32), pop.bits_numpy(c32[k]), 1e-5, 1e-5, input=pop.bits_numpy(inp32))
+        w1 = oracle.verify(pop.bits_numpy(ref16), pop.bits_numpy(c16[k]), 1e-2, 1.6e-2, input=pop.bits_numpy(inp16))
+        assert_stats_equal(got[k, 0], w0, f"host multi f32 k={k}")
+        assert_stats_equal(got[k, 1], w1, f"host multi bf16 k={k}")
+        verdicts.append([w0["verdict"], w1["verdict"]])
+    assert joint.tolist() == oracle.joint_pass(verdicts)
+    assert 0 < int(joint.sum()) < K
+
+
 def test_error_codes_on_device():
     n = 1024
     ref = torch.zeros(n + 4, device="cuda")
@@ -357,6 +386,42 @@ def test_error_codes_on_device():
     with pytest.raises(rkv.RkvError) as e:
         rkv.verify_multi([d], 1)
     assert e.value.status == rkv.ERR_INVALID_ARG
+
+
+def test_a_capturing_stream_is_refused_and_nothing_is_recorded():
+    """The descriptor tables travel from host memory that dies with the call, so a call on a
+    stream under capture must return UNSUPPORTED without enqueueing anything.  The capture is
+    ended without ever being replayed."""
+    n = 4096
+    ref = torch.zeros(n, device="cuda")
+    cands = [torch.zeros(n, device="cuda")]
+    d = rkv.TensorDesc(n=n, cands=cands, atol=1e-5, rtol=1e-5, ref=ref)
+    stats, joint, ws = rkv.verify_multi([d], 1)                       # buffers allocated outside the capture
+    rkv.verify_batch(ref, cands, 1e-5, 1e-5, stats_out=stats)         # grows the library's own scratch now
+    rkv.verify_batch_static(ref, cands, 1e-5, 1e-5, stats)            # first static call outside capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    seen = []
+    with torch.cuda.stream(side):
+        graph.capture_begin(capture_error_mode="thread_local")
+        try:
+            for call in (lambda: rkv.verify_multi([d], 1, workspace=ws, stats_out=stats, joint_pass=joint),
+                         lambda: rkv.verify_batch(ref, cands, 1e-5, 1e-5, stats_out=stats),
+                         lambda: rkv.verify_batch_static(ref, cands, 1e-5, 1e-5, stats)):
+                try:
+                    call()
+                    seen.append(rkv.OK)
+                except rkv.RkvError as e:
+                    seen.append(e.status)
+        finally:
+            graph.capture_end()
+    del graph
+    assert seen == [rkv.ERR_UNSUPPORTED] * 3
+    # the same calls work again once the capture has ended
+    rkv.verify_multi([d], 1, workspace=ws, stats_out=stats, joint_pass=joint)
+    assert rkv.device_status(ws) == rkv.OK
+    assert int(rkv.stats_to_numpy(stats)[0]["verdict"]) == 0
 
 
 @pytest.mark.parametrize("case", range(24))

@@ -7,7 +7,9 @@ device).  For them the library carries an entry point whose scratch is a fixed
 array inside the library image.  This test drives it through the C ABI and holds
 it to the results of rkv_verify_batch, the allocating form, on the same inputs:
 every integer and index field and both maxima bit for bit, the error sum and
-mean within the 1e-6 relative bar the other parity tests use.
+mean within the 1e-6 relative bar the other parity tests use -- and, so that two
+CUDA paths agreeing with each other cannot hide a common mistake, to the CPU
+oracle's results on the same bytes by the same rule.
 
 Two calls in a row share the scratch array (it is never cleared between calls),
 so the second call runs a *different* case than the first -- other sizes, other
@@ -21,8 +23,9 @@ import torch
 
 import oracle
 from paper_2509_14279_b200 import binding as rkv
-from rkv_testlib import (EXACT_FIELDS, BITWISE_FLOAT_FIELDS, MEAN_RTOL, build_case_cpu, f32_bits,
-                         mixed_plan, oracle_gen_tensor)
+from paper_2509_14279_b200 import population as pop
+from rkv_testlib import (EXACT_FIELDS, BITWISE_FLOAT_FIELDS, MEAN_RTOL, assert_stats_equal, build_case_cpu,
+                         f32_bits, mixed_plan, oracle_gen_tensor)
 
 pytestmark = pytest.mark.gpu
 
@@ -31,6 +34,12 @@ def _case(n, K, seed, dtype="f32"):
     ref = oracle_gen_tensor(seed, 0, oracle.NORMAL, n, dtype)
     cands = build_case_cpu(mixed_plan(K, n, seed=seed, bf16=dtype == "bf16"), ref, ref, dtype)
     return ref.cuda(), [c.cuda() for c in cands]
+
+
+def _oracle_rows(case, atol, rtol):
+    ref, cands = case
+    ref_np = pop.bits_numpy(ref)
+    return [oracle.verify(ref_np, pop.bits_numpy(c), atol, rtol) for c in cands]
 
 
 def _assert_same(got, want, where):
@@ -66,6 +75,12 @@ def test_static_scratch_form_matches_the_allocating_form_on_two_calls_in_a_row()
     _assert_same(rkv.stats_to_numpy(outs[3]), want[0], "first case again")
     # the static form is deterministic: the repeat is byte-identical to the first call
     assert rkv.stats_to_numpy(outs[3]).tobytes() == rkv.stats_to_numpy(outs[0]).tobytes()
+    # and every call against the oracle
+    for i, (case, name) in enumerate(zip((case_a, case_b, case_c, case_a),
+                                         ("first call", "second call", "third call (bf16)", "first case again"))):
+        got = rkv.stats_to_numpy(outs[i])
+        for k, w in enumerate(_oracle_rows(case, atol, rtol)):
+            assert_stats_equal(got[k], w, f"static form vs oracle, {name} k={k}")
 
 
 def test_static_scratch_form_rejects_what_does_not_fit():
