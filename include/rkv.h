@@ -50,10 +50,14 @@ typedef enum rkv_status {
     RKV_ERR_ALIGNMENT = -3,    /* a device pointer is not 16-byte aligned */
     RKV_ERR_WORKSPACE = -4,    /* workspace missing or smaller than rkv_workspace_bytes() */
     RKV_ERR_CUDA = -5,         /* a CUDA runtime call failed (no device, launch error, ...) */
-    RKV_ERR_TIMEOUT = -6       /* device side: a bounded wait on a bulk copy ran out */
+    RKV_ERR_TIMEOUT = -6,      /* device side: a bounded wait on a bulk copy ran out */
+    RKV_ERR_BOUNDS = -7        /* device side, debug build only: a range check failed (the access was skipped) */
 } rkv_status;
 
-enum { RKV_F32 = 0, RKV_BF16 = 1 };
+/* Element storage types.  fp16 (IEEE binary16) and bf16 tensors are raw 16-bit patterns;
+ * both are widened to fp32 exactly before anything is computed.  The generator produces
+ * fp32 and bf16 only: a reference or input that is regenerated on the fly cannot be fp16. */
+enum { RKV_F32 = 0, RKV_BF16 = 1, RKV_F16 = 2 };
 
 /* Value distributions of the input generator. */
 enum {
@@ -139,8 +143,9 @@ typedef struct rkv_tensor_desc {
     const void *const *cands;  /* HOST array of K DEVICE pointers, n elements of cand_dtype each */
     rkv_gen_spec ref_gen;      /* used when ref_src == GENERATED   */
     rkv_gen_spec input_gen;    /* used when input_src == GENERATED */
-    int32_t cand_dtype;        /* RKV_F32 | RKV_BF16 */
-    int32_t ref_dtype;         /* RKV_F32 | RKV_BF16; a generated reference is rounded to it */
+    int32_t cand_dtype;        /* RKV_F32 | RKV_BF16 | RKV_F16 */
+    int32_t ref_dtype;         /* RKV_F32 | RKV_BF16 | RKV_F16; a generated reference is rounded to it
+                                  (RKV_F32 or RKV_BF16 then) */
     int32_t ref_src;           /* RKV_SRC_POINTER | RKV_SRC_GENERATED */
     int32_t input_src;         /* RKV_SRC_NONE | RKV_SRC_POINTER | RKV_SRC_GENERATED; the input
                                   has the candidates' dtype (a copy is a bit copy) */
@@ -217,12 +222,42 @@ int rkv_verify_multi(const rkv_tensor_desc *tensors, int T, int K, rkv_stats *st
 
 /* Scratch bytes rkv_verify_multi needs for this case on the current device
  * (0 on an invalid argument).  Depends on n, the dtypes, T, K and the device's
- * SM count only. */
+ * SM count only: tables, 64 bytes per (tensor, candidate), 48 bytes * K per tensor and
+ * resident thread block (per tile, for a tensor of fewer tiles than blocks), and one
+ * double per (tile of 16 KiB of a candidate, candidate) for the error sums. */
 size_t rkv_workspace_bytes(const rkv_tensor_desc *tensors, int T, int K);
 
+/*
+ * Config sweep (listing "Linear config": the single_ and multi_ lists of input, init and
+ * shared settings; App. "Kernel Evaluation Environment": a kernel is correct iff it
+ * passes for ALL input sizes x initialisation settings x seeds).  C test cases, each with
+ * its own tensors (shapes, storage types, tolerances, stored or regenerated reference),
+ * the same K candidate kernels in every case; one launch over the items of all cases.
+ *   cases        HOST array of C case descriptors; cases[c].tensors is a HOST array of
+ *                cases[c].T rkv_tensor_desc (each with its HOST array of K DEVICE pointers)
+ *   C            1 <= C; the tensors of all cases together: at most 4096
+ *   stats_out    DEVICE, K * (sum of T) rkv_stats: case c starts at K * (T of the cases
+ *                before it); inside the case entry [k * T_c + t]
+ *   case_pass    DEVICE, C*K uint32, entry [c*K + k] = candidate k passed on every tensor
+ *                of case c; may be NULL
+ *   all_pass     DEVICE, K uint32 = AND over the cases (the paper's verdict); may be NULL
+ *   workspace    DEVICE, >= rkv_sweep_workspace_bytes(cases, C, K), 256-byte aligned
+ * Errors as rkv_verify_multi; a device-side timeout is reported by rkv_device_status.
+ */
+typedef struct rkv_case_desc {
+    const rkv_tensor_desc *tensors;   /* HOST */
+    int32_t T;                        /* 1 <= T <= 64 */
+    int32_t reserved;
+} rkv_case_desc;
+
+int rkv_verify_sweep(const rkv_case_desc *cases, int C, int K, rkv_stats *stats_out, uint32_t *case_pass,
+                     uint32_t *all_pass, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+size_t rkv_sweep_workspace_bytes(const rkv_case_desc *cases, int C, int K);
+
 /* Synchronises cuda_stream and returns the device-side status word the last
- * rkv_verify_multi on this workspace left (RKV_OK or RKV_ERR_TIMEOUT), or
- * RKV_ERR_CUDA. */
+ * rkv_verify_multi / rkv_verify_sweep on this workspace left (RKV_OK, RKV_ERR_TIMEOUT,
+ * or RKV_ERR_BOUNDS from a debug build), or RKV_ERR_CUDA. */
 int rkv_device_status(const void *workspace, void *cuda_stream);
 
 /*
@@ -276,10 +311,11 @@ int rkv_verify_multi_host(const rkv_tensor_desc *tensors, int T, int K, rkv_stat
  * and stats_out are the caller's; inputs are only read.
  *
  * Limits: K <= 256, and the scratch the case needs (rkv_workspace_bytes of the
- * single-tensor case: about 48 bytes * K * 2 * SM count, whatever n is) must fit
- * in 8 MiB; on a 148-SM part every K <= 256 fits.  A larger case is rejected
- * with RKV_ERR_UNSUPPORTED before anything is launched.  Other errors:
- * INVALID_ARG, ALIGNMENT, CUDA.
+ * single-tensor case: about 48 bytes * K * 2 * SM count plus 8 bytes * K per 16 KiB
+ * of a candidate) must fit in 8 MiB; on a 148-SM part that is e.g. K = 64 candidates
+ * of 2^24 fp32 elements, or K = 256 of 2^21.  A larger case is rejected with
+ * RKV_ERR_UNSUPPORTED before anything is launched.  Other errors: INVALID_ARG,
+ * ALIGNMENT, CUDA.
  *
  * First call on a device: looks up the array's device address once (with that
  * device current) and sets a kernel attribute.  Make that first call outside any
@@ -303,7 +339,7 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * Host-only planning helper (no CUDA call; plumbing, no passage of its own): how the
  * work of one tensor is cut.
  * The tensor is cut into *n_tiles tiles of *tile_elems elements (a thread of the
- * verification kernel owns 64 bytes of each candidate tile: 3584 fp32 or 7168 bf16
+ * verification kernel owns 64 bytes of each candidate tile: 4096 fp32 or 8192 16-bit
  * elements per tile).  One work item is
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
@@ -317,7 +353,7 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * smaller tensor has one group: *warm_tiles == *n_tiles, *parts_main == 0,
  * *tail_tiles == 0 and *parts_tail == 0.  Part p of P covers candidates
  * [p*K/P, (p+1)*K/P).
- *   cand_dtype  RKV_F32 | RKV_BF16 (storage type of the candidates)
+ *   cand_dtype  RKV_F32 | RKV_BF16 | RKV_F16 (storage type of the candidates)
  *   num_sms     SM count of the device
  * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, bad dtype, null), UNSUPPORTED (n >= 2^40).
  */

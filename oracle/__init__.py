@@ -21,7 +21,7 @@ _SRC = os.path.join(_HERE, "rkv_oracle.c")
 _HDR = os.path.join(_HERE, "rkv_oracle.h")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 NORMAL, UNIFORM_PM1, STUDENT_T2, SPARSE90, NORMAL_1E4 = range(5)
 DISTS = (NORMAL, UNIFORM_PM1, STUDENT_T2, SPARSE90, NORMAL_1E4)
 
@@ -118,6 +118,8 @@ def lib() -> ctypes.CDLL:
         L.orc_student_t2.restype = ctypes.c_float
         L.orc_bf16_rne.argtypes = [ctypes.c_float]
         L.orc_bf16_rne.restype = ctypes.c_uint16
+        L.orc_f16_to_f32_bits.argtypes = [ctypes.c_uint16]
+        L.orc_f16_to_f32_bits.restype = ctypes.c_uint32
         L.orc_gen_value.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int, ctypes.c_uint64]
         L.orc_gen_value.restype = ctypes.c_float
         L.orc_gen.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int, ctypes.c_uint64,
@@ -145,7 +147,9 @@ def _dtype_of(a: np.ndarray) -> int:
         return F32
     if a.dtype == np.uint16:
         return BF16
-    raise TypeError(f"oracle tensors are float32 or uint16 (bf16 bits), got {a.dtype}")
+    if a.dtype == np.float16:
+        return F16
+    raise TypeError(f"oracle tensors are float32, float16 or uint16 (bf16 bits), got {a.dtype}")
 
 
 def philox4x32_10(ctr, key) -> tuple:
@@ -196,6 +200,10 @@ def student_t2(w: int) -> float:
 
 def bf16_rne(x: float) -> int:
     return int(lib().orc_bf16_rne(ctypes.c_float(x)))
+
+
+def f16_to_f32_bits(h: int) -> int:
+    return int(lib().orc_f16_to_f32_bits(int(h) & 0xFFFF))
 
 
 def gen(seed: int, stream_id: int, dist: int, n: int, dtype: int = F32,

@@ -215,14 +215,38 @@ int orc_gen(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t fi
 /* Verification                                                             */
 /* ------------------------------------------------------------------------ */
 
+/* IEEE binary16 -> the fp32 bit pattern of the same value (every binary16 value is an
+ * fp32 value).  1 sign bit, 5 exponent bits (bias 15), 10 fraction bits. */
+uint32_t orc_f16_to_f32_bits(uint16_t h)
+{
+    const uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+    const uint32_t expo = (h >> 10) & 0x1Fu;
+    uint32_t frac = h & 0x3FFu;
+    if (expo == 0x1Fu)                              /* infinity or NaN: payload kept in the top bits */
+        return sign | 0x7F800000u | (frac << 13);
+    if (expo == 0) {
+        if (frac == 0) return sign;                 /* signed zero */
+        /* subnormal: value = frac * 2^-24; shift the leading one up to the hidden-bit position */
+        int e = -14;
+        while (!(frac & 0x400u)) { frac <<= 1; e--; }
+        frac &= 0x3FFu;
+        return sign | ((uint32_t)(e + 127) << 23) | (frac << 13);
+    }
+    return sign | ((expo - 15u + 127u) << 23) | (frac << 13);
+}
+
 /* Element q of a tensor as the fp32 bit pattern of its exact upcast
- * (bf16 -> fp32 appends sixteen zero bits). */
+ * (bf16 -> fp32 appends sixteen zero bits; fp16 -> fp32 re-biases the exponent). */
 static uint32_t load_bits(const void *p, int dtype, uint64_t q)
 {
     if (dtype == ORC_F32)
         return ((const uint32_t *)p)[q];
+    if (dtype == ORC_F16)
+        return orc_f16_to_f32_bits(((const uint16_t *)p)[q]);
     return (uint32_t)((const uint16_t *)p)[q] << 16;
 }
+
+static int dtype_known(int d) { return d == ORC_F32 || d == ORC_BF16 || d == ORC_F16; }
 
 static int bits_is_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
 static int bits_is_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
@@ -233,8 +257,8 @@ int orc_verify(const void *ref, int ref_dtype, const void *input, int input_dtyp
                orc_result *res)
 {
     if (!ref || !cand || !res || n == 0) return -1;
-    if ((ref_dtype | cand_dtype) & ~1) return -1;
-    if (input && (input_dtype & ~1)) return -1;
+    if (!dtype_known(ref_dtype) || !dtype_known(cand_dtype)) return -1;
+    if (input && !dtype_known(input_dtype)) return -1;
 
     uint64_t n_over = 0, n_nan = 0, n_inf = 0, n_inf_mis = 0, n_cmp = 0;
     uint64_t arg_abs = ORC_NO_INDEX, arg_rel = ORC_NO_INDEX;

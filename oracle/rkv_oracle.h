@@ -28,6 +28,7 @@
  *                       The *choice* of the five distributions, the counter /
  *                       stream layout and the bf16 rounding of generated values
  *                       are this project's definitions: parity unpinned.
+ *   orc_f16_to_f32_bits pinned: all 65536 patterns against numpy's float16 -> float32.
  *   orc_verify          comparison rule pinned by brute force on tiny tensors,
  *                       by torch.isclose on finite data, and by invariants.
  *                       The flag -> verdict policy, the n == 1 rule and the
@@ -43,8 +44,9 @@
 extern "C" {
 #endif
 
-/* element storage types */
-enum { ORC_F32 = 0, ORC_BF16 = 1 };
+/* element storage types (the paper's kernels dispatch half precision too, listing
+ * "MaxPool2d backward": 16-bit outputs are widened exactly and compared in fp32) */
+enum { ORC_F32 = 0, ORC_BF16 = 1, ORC_F16 = 2 };
 
 /* value distributions */
 enum {
@@ -103,6 +105,7 @@ void orc_box_muller(uint32_t w0, uint32_t w1, float *z_even, float *z_odd);
 float orc_uniform_pm1(uint32_t w);
 float orc_student_t2(uint32_t w);
 uint16_t orc_bf16_rne(float x);
+uint32_t orc_f16_to_f32_bits(uint16_t h);              /* exact widening of IEEE binary16 */
 /* array forms of the two scalar routines, for exhaustive pins */
 void orc_log_unit_range(uint32_t k_first, uint32_t count, float *out);
 void orc_sincos_turn_range(uint32_t k_first, uint32_t count, float *s, float *c);

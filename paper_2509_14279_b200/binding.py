@@ -15,11 +15,13 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "librkv.so")
+# RKV_LIB selects another build of the same library (the range-checked debug build,
+# `python -m paper_2509_14279_b200.build --debug-bounds`, writes librkv_dbg.so)
+LIB_PATH = os.environ.get("RKV_LIB") or os.path.join(_PKG, "librkv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = (
-    0, -1, -2, -3, -4, -5, -6)
-F32, BF16 = 0, 1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = (
+    0, -1, -2, -3, -4, -5, -6, -7)
+F32, BF16, F16 = 0, 1, 2
 DIST_NORMAL, DIST_UNIFORM_PM1, DIST_STUDENT_T2, DIST_SPARSE90, DIST_NORMAL_1E4 = range(5)
 SRC_NONE, SRC_POINTER, SRC_GENERATED = 0, 1, 2
 FAIL_TOL, FAIL_NAN, FAIL_INF_MISMATCH, FAIL_LOOPHOLE_CONST, FAIL_LOOPHOLE_COPY = 1, 2, 4, 8, 16
@@ -73,6 +75,10 @@ class TensorDescC(ctypes.Structure):
     ]
 
 
+class CaseDescC(ctypes.Structure):
+    _fields_ = [("tensors", ctypes.POINTER(TensorDescC)), ("T", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 _lib = None
 
 
@@ -109,6 +115,14 @@ def lib() -> ctypes.CDLL:
         L.rkv_verify_batch_host.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp]
         L.rkv_verify_multi_host.restype = i32
         L.rkv_verify_multi_host.argtypes = [ctypes.POINTER(TensorDescC), i32, i32, vp, vp]
+        L.rkv_verify_sweep.restype = i32
+        L.rkv_verify_sweep.argtypes = [ctypes.POINTER(CaseDescC), i32, i32, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.rkv_sweep_workspace_bytes.restype = ctypes.c_size_t
+        L.rkv_sweep_workspace_bytes.argtypes = [ctypes.POINTER(CaseDescC), i32, i32]
+        L.rkv_debug_fault_drill.restype = i32
+        L.rkv_debug_fault_drill.argtypes = [ctypes.c_uint, ctypes.c_ulonglong]
+        L.rkv_debug_bounds_build.restype = i32
+        L.rkv_debug_bounds_build.argtypes = []
         L.rkv_verify_batch_static.restype = i32
         L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
         u32p = ctypes.POINTER(ctypes.c_uint32)
@@ -139,7 +153,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
-    raise TypeError(f"rkv tensors are float32 or bfloat16, got {t.dtype}")
+    if t.dtype == torch.float16:
+        return F16
+    raise TypeError(f"rkv tensors are float32, bfloat16 or float16, got {t.dtype}")
 
 
 def _require(t, what: str, device=None, dtype=None, numel=None, min_bytes=None) -> None:
@@ -375,6 +391,69 @@ def verify_multi(tensors, K: int, workspace: torch.Tensor | None = None,
                                   ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
                                   ctypes.c_void_p(_stream_ptr(stream))), "rkv_verify_multi")
     return stats_out, joint_pass, workspace
+
+
+def prepare_sweep(cases):
+    """Marshal the cases of a sweep once: `cases` is a list of lists of TensorDesc (one inner
+    list per test case).  Returns an opaque object to pass as ``descs=`` to verify_sweep."""
+    keep = []
+    arr = (CaseDescC * len(cases))()
+    for i, tensors in enumerate(cases):
+        ta = _desc_array(tensors)
+        keep.append(ta)
+        arr[i].tensors = ctypes.cast(ta, ctypes.POINTER(TensorDescC))
+        arr[i].T = len(tensors)
+    return (arr, keep)
+
+
+def verify_sweep(cases, K: int, workspace: torch.Tensor | None = None, stats_out: torch.Tensor | None = None,
+                 case_pass: torch.Tensor | None = None, all_pass: torch.Tensor | None = None, stream=None,
+                 descs=None):
+    """rkv_verify_sweep: C test cases (lists of TensorDesc), the same K candidates in each, one
+    launch.  Returns (stats, case_pass [C, K] int32, all_pass [K] int32, workspace); the stats of
+    case c start at K * (tensors of the cases before it) * 88 bytes, entry [k * T_c + t] inside."""
+    C = len(cases)
+    arr, keep = prepare_sweep(cases) if descs is None else descs
+    dev = cases[0][0].cands[0].device
+    n_t = sum(len(c) for c in cases)
+    for c in cases:
+        for t in c:
+            if len(t.cands) != K:
+                raise ValueError(f"verify_sweep: a tensor has {len(t.cands)} candidates, K = {K}")
+    if workspace is None:
+        need = int(lib().rkv_sweep_workspace_bytes(arr, C, int(K)))
+        if need == 0:
+            raise RkvError(ERR_INVALID_ARG, "rkv_sweep_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    else:
+        _require(workspace, "verify_sweep: workspace", device=dev, dtype=torch.uint8)
+    if stats_out is None:
+        stats_out = torch.empty(K * n_t * STATS_BYTES, dtype=torch.uint8, device=dev)
+    else:
+        _require(stats_out, "verify_sweep: stats_out", device=dev, dtype=torch.uint8, min_bytes=K * n_t * STATS_BYTES)
+    if case_pass is None:
+        case_pass = torch.empty((C, K), dtype=torch.int32, device=dev)
+    else:
+        _require(case_pass, "verify_sweep: case_pass", device=dev, dtype=torch.int32, numel=C * K)
+    if all_pass is None:
+        all_pass = torch.empty(K, dtype=torch.int32, device=dev)
+    else:
+        _require(all_pass, "verify_sweep: all_pass", device=dev, dtype=torch.int32, numel=K)
+    _check(lib().rkv_verify_sweep(arr, C, int(K), ctypes.c_void_p(stats_out.data_ptr()),
+                                  ctypes.c_void_p(case_pass.data_ptr()), ctypes.c_void_p(all_pass.data_ptr()),
+                                  ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                  ctypes.c_void_p(_stream_ptr(stream))), "rkv_verify_sweep")
+    return stats_out, case_pass, all_pass, workspace
+
+
+def debug_fault_drill(issue: int, wait_cycles: int) -> None:
+    """Test hook (not in rkv.h): the next verification call withholds block 0's issue-th bulk
+    copy and lets every bounded wait give up after wait_cycles clock cycles."""
+    _check(lib().rkv_debug_fault_drill(int(issue), int(wait_cycles)), "rkv_debug_fault_drill")
+
+
+def debug_bounds_build() -> bool:
+    return bool(lib().rkv_debug_bounds_build())
 
 
 def prepare(tensors):

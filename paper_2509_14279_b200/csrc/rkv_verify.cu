@@ -1,27 +1,32 @@
-// Fused single-pass verification kernel and its finalize kernel (sm_100a).
+// Fused single-pass verification kernel and its finalize kernels (sm_100a).
 //
-// Work decomposition.  A tensor is cut into tiles of 14336 candidate bytes (3584 fp32 or
-// 7168 bf16 elements); the K candidates into parts of at most 64.  A work item is
-// (tensor, group, part, tile).  A persistent thread block starts with the item of its own
-// number and then draws further items from a ticket counter.  It has two roles:
+// Work decomposition.  A tensor is cut into tiles of 16384 candidate bytes (4096 fp32 or
+// 8192 bf16 / fp16 elements); the K candidates into parts of at most 64.  A work item is
+// (tensor, group, part, tile); the items of every tensor of a call -- whatever its storage
+// types -- form one list (see Segment), and one launch of persistent thread blocks works
+// through it: a block starts with the item of its own number and then draws further items
+// from a ticket counter.  Items of fp32 candidates are bound by HBM, items of 16-bit
+// candidates by instruction issue; the list interleaves them, so that the two kinds overlap
+// on every SM instead of running one after the other.
 //
-//   * one producer warp: a single thread issues bulk asynchronous copies
-//     (cp.async.bulk, completion counted on an mbarrier) that bring, for the
-//     item, the reference tile and then the same tile of every candidate of the
-//     part into a ring of shared-memory stages.  Several stages are in flight,
-//     so the copies of later candidates overlap the comparison of earlier ones;
-//   * seven consumer warps: each thread owns 64 bytes of every candidate tile (16 fp32
-//     or 32 bf16 elements).  It keeps their reference values (and, for fp32 candidates,
-//     the tolerance thresholds) IN REGISTERS for the whole item and meets every
-//     candidate tile as it lands in the ring.
+// All eight warps of a block compare.  A thread owns 64 bytes of every candidate tile (16
+// fp32 or 32 16-bit elements); it keeps their reference values (and, for fp32 candidates,
+// the tolerance thresholds) IN REGISTERS for the whole item and meets every candidate tile
+// as it lands in a ring of shared-memory stages.  One lane of the last warp also feeds that
+// ring: between its own comparisons it issues the bulk asynchronous copies
+// (cp.async.bulk, completion counted on an mbarrier) that bring, for an item, the reference
+// tile and then the same tile of every candidate of the part.  It runs up to a ring's depth
+// ahead of the comparison, across item boundaries, so that copies are always in flight.  (A
+// warp that only issued copies would leave its scheduler half idle: with 128 registers a
+// thread, 16 warps fill an SM, and this way all 16 compare.)
 //
 // Candidate bytes are read from HBM exactly once; the reference once per part.
 // When the reference is "generated" the threads regenerate their values from
 // the Philox stream instead of reading them (fused generate + verify).
 //
 // Per element the common path is one subtraction, one running maximum and one
-// addition (bf16 candidates: one fused multiply-add and one more maximum, see
-// process_candidate_b16).  Counting the elements over tolerance, locating maxima,
+// addition (16-bit candidates: one fused multiply-add and one more maximum, see
+// process_candidate_16).  Counting the elements over tolerance, locating maxima,
 // dividing for the relative error and everything about non-finite values sit behind
 // tests evaluated once per thread, candidate and tile and one warp vote:
 //   m > min thr              some element may be over tolerance  -> count them
@@ -32,8 +37,11 @@
 // be the first maximum (see Hint), so results do not depend on when a hint
 // becomes visible.
 //
-// Reductions are deterministic: integer sums, lexicographic (value descending,
-// index ascending) maxima, fixed-order floating-point sums.  No float atomics.
+// Reductions are deterministic: integer sums; lexicographic (value descending, index
+// ascending) maxima; the error sum of a (tile, candidate) is a fixed tree over the tile's
+// elements and is stored per tile, and the finalize kernel adds the tile sums in tile
+// order -- whichever block verified whichever tile, the bits of the sum are the same.
+// No float atomics.
 #include "rkv_internal.h"
 #include "rkv_philox.cuh"
 
@@ -43,7 +51,26 @@ namespace {
 
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr float kInf = __builtin_huge_valf();
-enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the producer's "no more items" mark
+enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the issuer's "no more items" mark
+constexpr int kInfoRing = 8;                   // items in flight per block (> kStages: an item uses >= 1 stage)
+constexpr long long kWaitCycles = 2000000000LL;
+
+// ----------------------------------------------------------------------------
+// range checks of a debug build
+// ----------------------------------------------------------------------------
+// With RKV_DEBUG_BOUNDS every index into global memory and into the shared-memory tables
+// is checked before it is used; a violation records its site and value in the workspace
+// header, sets the status word and skips the access.  Nothing traps or asserts.
+#ifdef RKV_DEBUG_BOUNDS
+__device__ __noinline__ void bounds_fail(WorkspaceHeader* header, uint32_t site, unsigned long long value) {
+    if (atomicCAS(&header->bounds_site, 0u, site) == 0u) header->bounds_value = value;
+    atomicExch(&header->status, (int32_t)RKV_ERR_BOUNDS);
+}
+#define RKV_IN_BOUNDS(header, site, cond, value) \
+    ((cond) ? true : (bounds_fail((header), (site), (unsigned long long)(value)), false))
+#else
+#define RKV_IN_BOUNDS(header, site, cond, value) (true)
+#endif
 
 // ----------------------------------------------------------------------------
 // shared-memory layout (dynamic)
@@ -54,7 +81,7 @@ struct __align__(16) WarpRec {
     float qmax; uint32_t qtile;
     uint32_t offs;           // eoff | qoff << 16 : element offsets inside their tiles
     uint32_t n_over;
-    double sum;
+    double sum;              // of the current item's tile only
 };
 static_assert(sizeof(WarpRec) == 32, "WarpRec layout");
 
@@ -68,35 +95,69 @@ struct __align__(16) Hint {
     float te_x;
     float tq_x;
     uint32_t settled;                // bit0: known to differ from element 0; bit1: from the input
-    uint32_t first;                  // element 0 of the candidate as an fp32 bit pattern
+    uint32_t first;                  // element 0 of the candidate, storage bits
 };
 static_assert(sizeof(Hint) == 16, "Hint layout");
 
+// What the issuing lane tells the block about an item, before it arms the item's first stage.
+struct __align__(16) ItemInfo {
+    uint32_t id;             // kNoItem: no more items
+    uint32_t t;
+    uint32_t tile;           // tensor-wide tile index
+    uint32_t k0, kc;         // candidates [k0, k0 + kc) of the call
+    uint32_t reserved[3];
+};
+static_assert(sizeof(ItemInfo) == 32, "ItemInfo layout");
+
+// State of the issuing lane (only that lane touches it).
+struct __align__(16) IssuerState {
+    uint32_t n_issued;       // copies issued so far
+    uint32_t stage, phase;   // ring stage of the next copy and the parity its empty barrier must have passed
+    uint32_t pos, end, nref; // next copy of the current item: [0, nref) reference stages, [nref, end) candidates
+    uint32_t done;
+    uint32_t ord;            // items started so far
+    uint32_t cbytes, rbytes; // bytes copied per candidate tile / of the reference tile
+    uint32_t seg;            // segment the last item was found in
+    uint32_t next_id;        // the item after the current one (a ticket drawn one item ahead)
+    uint32_t drill;          // fault drill: number of the copy to withhold (0: none)
+    uint32_t reserved[3];
+    unsigned long long c_off;          // byte offset of the tile in every candidate
+    const unsigned char* ref_src;      // the tile in the stored reference
+};
+static_assert(sizeof(IssuerState) == 80, "IssuerState layout");
+
 constexpr int kOffFull = 0;                                   // kStages mbarriers
 constexpr int kOffEmpty = kOffFull + 8 * kStages;
-constexpr int kOffAbort = kOffEmpty + 8 * kStages;         // uint32
-constexpr int kOffRefState = kOffAbort + 16;                  // 2 x uint32 settled bits of the reference (item parity)
-constexpr int kOffIds = kOffRefState + 8;                     // kStages x uint32: item id that starts in a stage
-constexpr int kOffPtrC = 256;                                 // consumer copy of the pointers
-constexpr int kOffPtrP = kOffPtrC + kPartK * 8;               // producer copy
-constexpr int kOffHint = kOffPtrP + kPartK * 8;               // two tables (item parity)
+constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
+constexpr int kOffRefState = kOffAbort + 8;                   // 2 x uint32 settled bits of the reference (item parity)
+constexpr int kOffWaitLimit = kOffRefState + 8;               // long long: cycles a wait may take
+constexpr int kOffIssuer = 128;
+constexpr int kOffInfo = kOffIssuer + 96;
+constexpr int kOffPtrC = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);   // the comparing threads' copy of the pointers
+constexpr int kOffPtrP = kOffPtrC + kPartK * 8;                          // the issuer's copies, one per item in flight
+constexpr int kOffHint = kOffPtrP + kInfoRing * kPartK * 8;              // two tables (item parity)
 constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
-constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
+constexpr int kOffStage = (kOffRec + kWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
-static_assert(kOffPtrC >= kOffIds + 4 * kStages, "layout");
+static_assert(kOffWaitLimit + 8 <= kOffIssuer && sizeof(IssuerState) <= 96, "layout");
 static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
+// Candidate storage kinds the comparison is compiled for.
+enum : int { CK_F32 = 0, CK_BF16 = 1, CK_F16 = 2 };
+
 // Geometry of a tile.  A thread owns 64 bytes of each candidate tile, so a candidate tile
-// always fills exactly one ring stage: 16 fp32 elements or 32 bf16 elements.  Their
+// always fills exactly one ring stage: 16 fp32 elements or 32 16-bit elements.  Their
 // reference values stay in registers for the whole item.  With fp32 candidates the
-// tolerance thresholds do too; with bf16 candidates they are recomputed in the rare case
-// that needs them (see process_candidate_b16).
-template <bool CB16>
+// tolerance thresholds do too; with 16-bit candidates they are recomputed in the rare case
+// that needs them (see process_candidate_16).
+template <int CK>
 struct Geo {
-    static constexpr int E = CB16 ? 32 : 16;            // elements per thread
-    static constexpr int VEC = CB16 ? 8 : 4;            // elements per 16-byte piece
+    static constexpr bool C16 = CK != CK_F32;
+    static constexpr int E = C16 ? 32 : 16;             // elements per thread
+    static constexpr int VEC = C16 ? 8 : 4;             // elements per 16-byte piece
     static constexpr int NW = 16;                       // 32-bit words per thread and candidate tile
-    static constexpr int kTile = kConsumers * E;        // elements per tile
+    static constexpr int kTile = kThreads * E;          // elements per tile
+    static constexpr int DTYPE = CK == CK_F32 ? RKV_F32 : CK == CK_BF16 ? RKV_BF16 : RKV_F16;
 };
 
 // ----------------------------------------------------------------------------
@@ -140,24 +201,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
     return ok != 0;
 }
 
+// What every wait of a block shares: the flag that says "a wait ran out, drain" and the
+// number of clock cycles a wait may take.
+struct WaitCtl {
+    volatile uint32_t* abort_flag;
+    const volatile long long* limit;
+};
+
 // Bounded wait.  Returns false when the wait ran out (about a second) or when
 // another thread of the block has already given up; the block then drains: every
 // later wait returns at once, all barriers are still reached, and the status
 // word tells the host that the results are void.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t mbar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t mbar, uint32_t parity, WaitCtl ctl) {
     const long long t0 = clock64();
+    const long long limit = *ctl.limit;
     for (uint32_t spin = 0; spin < (1u << 26); ++spin) {
         if (mbar_try_wait(mbar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > 2000000000LL) break;
+        if (*ctl.abort_flag) return false;
+        if (clock64() - t0 > limit) break;
     }
-    *abort_flag = 1u;
+    *ctl.abort_flag = 1u;
     return false;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, WaitCtl ctl) {
     if (mbar_try_wait(mbar, parity)) return true;
-    return mbar_wait_slow(mbar, parity, abort_flag);
+    return mbar_wait_slow(mbar, parity, ctl);
 }
 
 // Bulk asynchronous copy global -> this block's shared memory; bytes is a
@@ -169,198 +238,191 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         : "memory");
 }
 
-// Barrier among the consumer threads only (the producer warp never joins).
-__device__ __forceinline__ void consumer_sync() {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
-}
-
-// The same barrier, returning whether any consumer thread passed a non-zero value.
-__device__ __forceinline__ bool consumer_sync_or(uint32_t v) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "barrier.red.or.pred q, 1, %2, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(out)
-        : "r"(v), "n"(kConsumers)
-        : "memory");
-    return out != 0;
+// Block barrier that also returns whether any thread passed a non-zero value.
+__device__ __forceinline__ bool block_sync_or(uint32_t v) {
+    return __syncthreads_or((int)v) != 0;
 }
 
 __device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
 __device__ __forceinline__ bool bits_inf(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
 __device__ __forceinline__ bool bits_nan(uint32_t b) { return (b & 0x7FFFFFFFu) > 0x7F800000u; }
 
+// 16 storage bits -> the fp32 bit pattern of the same value (exact for both kinds).
+__device__ __forceinline__ uint32_t upcast16(uint32_t raw, int dtype) {
+    if (dtype == RKV_BF16) return raw << 16;
+    float f;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((unsigned short)raw));
+    return __float_as_uint(f);
+}
+
+// Element i of a stored tensor as an fp32 bit pattern.
 __device__ __forceinline__ uint32_t ld_elem_bits(const void* base, int dtype, uint64_t i) {
-    if (dtype == RKV_BF16) return (uint32_t)reinterpret_cast<const uint16_t*>(base)[i] << 16;
-    return reinterpret_cast<const uint32_t*>(base)[i];
+    if (dtype == RKV_F32) return reinterpret_cast<const uint32_t*>(base)[i];
+    return upcast16(reinterpret_cast<const uint16_t*>(base)[i], dtype);
+}
+
+// Element i of a stored tensor, storage bits.
+__device__ __forceinline__ uint32_t ld_elem_raw(const void* base, int dtype, uint64_t i) {
+    if (dtype == RKV_F32) return reinterpret_cast<const uint32_t*>(base)[i];
+    return reinterpret_cast<const uint16_t*>(base)[i];
 }
 
 // ----------------------------------------------------------------------------
-// work items
+// what the kernel gets
 // ----------------------------------------------------------------------------
-struct Item {
-    int t;
-    uint32_t group;          // 0 = A (leading tiles, small parts), 1 = B, 2 = C (last tiles, small parts)
-    uint32_t part, tile;     // tile is the tensor-wide tile index
-    uint32_t n_parts;        // candidate parts of this group
-    uint32_t first_item;     // first item of this (tensor, group) in this launch
-    uint32_t n_items;        // items of this (tensor, group)
+struct Args {
+    const DevTensor* tensors;
+    const Segment* segments;
+    CandState* state;
+    Partial* partials;
+    double* sums;
+    WorkspaceHeader* header;
+    int T, K, k_begin, k_end;
+    uint32_t n_items, n_segments;
 };
 
-// Item `id` of this launch among the tensors of `variant`; false past the end.
-__device__ __forceinline__ bool decode_item(const DevTensor* __restrict__ tensors, int T, uint32_t variant,
-                                            uint32_t k_count, uint32_t id, Item& it) {
-    uint32_t base = 0;
-    for (uint32_t g = 0; g < 3; ++g) {
-        for (int t = 0; t < T; ++t) {
-            if (tensors[t].variant != variant) continue;
-            const uint32_t warm = tensors[t].warm_tiles, tail = tensors[t].tail_tiles;
-            const uint32_t nt = group_tiles(g, tensors[t].n_tiles, warm, tail);
-            if (nt == 0) continue;
-            const uint32_t parts = group_parts(g, nt, k_count, gridDim.x, tensors[t].tail_div);
-            const uint32_t cnt = nt * parts;
-            if (id - base < cnt) {
-                it.t = t;
-                it.group = g;
-                it.part = (id - base) / nt;
-                it.tile = (id - base) % nt + group_first_tile(g, tensors[t].n_tiles, warm, tail);
-                it.n_parts = parts;
-                it.first_item = base;
-                it.n_items = cnt;
-                return true;
-            }
-            base += cnt;
-        }
-    }
-    return false;
-}
-
 // ----------------------------------------------------------------------------
-// producer warp: feeds the ring
+// the issuing lane: feeds the ring
 // ----------------------------------------------------------------------------
 struct Ring {
     uint32_t full0, empty0;      // shared-memory addresses of the first full / empty mbarrier
     uint32_t stage0;             // shared-memory address of stage 0
-    volatile uint32_t* abort_flag;
+    WaitCtl ctl;
 };
 
-template <bool CB16, bool RB16>
-__device__ __forceinline__ void producer_loop(const DevTensor* __restrict__ tensors, int T, int k_begin,
-                                              int k_end, uint32_t n_items, unsigned char* smem,
-                                              const Ring& ring, WorkspaceHeader* header) {
-    constexpr uint32_t CSZ = CB16 ? 2 : 4, RSZ = RB16 ? 2 : 4;
-    constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
-    constexpr uint32_t kTile = Geo<CB16>::kTile;
-    constexpr uint32_t kRefStages = (CB16 && !RB16) ? 2 : 1;      // an fp32 tile under bf16 candidates
-    const int lane = threadIdx.x & 31;
-    const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrP);
-    volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
-    uint32_t n_issued = 0;
-    int cur_t = -1;
-    uint32_t cur_part = 0xFFFFFFFFu;
-
-    // mark: the id of the item that starts in this stage (kNoItem at the very end), else none
-    auto issue = [&](const unsigned char* src, uint32_t bytes, bool starts_item, uint32_t id) {
-        const uint32_t s = n_issued % kStages;
-        const uint32_t ph = (n_issued / kStages) & 1u;
-        // the stage is free once every consumer warp has released its previous use
-        mbar_wait(ring.empty0 + 8 * s, ph ^ 1u, ring.abort_flag);
-        if (starts_item) ids[s] = id;          // ordered before the arrive below
-        if (bytes) {
-            mbar_expect_tx(ring.full0 + 8 * s, bytes);
-            bulk_g2s(ring.stage0 + s * kStageBytes, src, bytes, ring.full0 + 8 * s);
-        } else {
-            mbar_arrive(ring.full0 + 8 * s);
+// Item `id` of the launch: which tensor, tile and candidates.  One lane runs this.
+__device__ __forceinline__ bool decode_item(const Args& A, uint32_t id, uint32_t& seg_cache, ItemInfo& info) {
+    if (id >= A.n_items) return false;
+    const uint32_t n_seg = A.n_segments;
+    uint32_t s = seg_cache;
+    if (!(s < n_seg && A.segments[s].first_id <= id && id < A.segments[s + 1].first_id)) {
+        uint32_t lo = 0, hi = n_seg;          // the segment with first_id <= id < next first_id
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (A.segments[mid].first_id <= id) lo = mid; else hi = mid;
         }
-        ++n_issued;
-    };
+        s = lo;
+        seg_cache = s;
+    }
+    const Segment sg = A.segments[s];
+    if (!RKV_IN_BOUNDS(A.header, 1, sg.tensor < (uint32_t)A.T && sg.group < 3u, sg.tensor)) return false;
+    const DevTensor& D = A.tensors[sg.tensor];
+    const uint32_t local = sg.first_local + (id - sg.first_id);
+    const uint32_t nt = group_tiles(sg.group, D.n_tiles, D.warm_tiles, D.tail_tiles);
+    const uint32_t parts = D.parts[sg.group];
+    const uint32_t part = local / nt;
+    if (!RKV_IN_BOUNDS(A.header, 2, nt > 0 && part < parts, local)) return false;
+    const uint32_t k_count = (uint32_t)(A.k_end - A.k_begin);
+    const uint32_t k0 = part_begin(part, parts, k_count);
+    info.id = id;
+    info.t = sg.tensor;
+    info.tile = local % nt + group_first_tile(sg.group, D.n_tiles, D.warm_tiles, D.tail_tiles);
+    info.k0 = (uint32_t)A.k_begin + k0;
+    info.kc = part_begin(part + 1, parts, k_count) - k0;
+    return true;
+}
 
-    // Every block starts with item blockIdx.x; after that lane 0 draws tickets, one ahead of
-    // the item it is issuing, so that the atomic's latency is never waited for.
-    uint32_t id = blockIdx.x;
+// Start the next item: draw a ticket for the one after it, decode, copy the part's pointers
+// into the item's table, publish the item's description.  At the end of the list the item
+// published is the end mark.
+__device__ __noinline__ void issuer_next_item(const Args& A, unsigned char* smem) {
+    IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
+    const uint32_t id = st->next_id;
+    const uint32_t slot = st->ord & (kInfoRing - 1);
+    // the ticket for the item after this one; its latency hides behind the set-up below
+    uint32_t ticket = 0;
+    if (id < A.n_items) ticket = atomicAdd(&A.header->next_ticket, 1u);
+    ItemInfo info;
+    info.id = kNoItem; info.t = 0; info.tile = 0; info.k0 = 0; info.kc = 0;
+    info.reserved[0] = info.reserved[1] = info.reserved[2] = 0;
+    uint32_t seg = st->seg;
+    st->pos = 0; st->nref = 0; st->end = 1; st->cbytes = 0; st->rbytes = 0;     // the end mark: one empty "copy"
+    if (decode_item(A, id, seg, info)) {
+        const DevTensor& D = A.tensors[info.t];
+        const uint32_t csz = elem_bytes(D.cand_dtype), rsz = elem_bytes(D.ref_dtype);
+        const uint32_t te = tile_elems(D.cand_dtype);
+        const uint64_t start = (uint64_t)info.tile * te;
+        const uint32_t len = (uint32_t)min((uint64_t)te, D.n - start);
+        st->cbytes = (len * csz) & ~15u;
+        st->c_off = start * csz;
+        uint32_t nref = 0;
+        if (D.ref_src == RKV_SRC_POINTER) {
+            nref = (te * rsz + kStageBytes - 1) / kStageBytes;
+            st->rbytes = (len * rsz) & ~15u;
+            st->ref_src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
+        }
+        st->nref = nref;
+        st->end = nref + info.kc;
+        const void** table = reinterpret_cast<const void**>(smem + kOffPtrP) + slot * kPartK;
+        for (uint32_t i = 0; i < info.kc; ++i) table[i] = D.cands[info.k0 + i];
+    } else {
+        st->done = 2u;                              // the end mark is the last thing to issue
+    }
+    st->seg = seg;
+    reinterpret_cast<ItemInfo*>(smem + kOffInfo)[slot] = info;
+    st->next_id = gridDim.x + ticket;
+}
+
+// Issue copies while ring stages are free; make sure copy number `need` has been issued
+// when this returns (waiting, bounded, for its stage if it has to).  Called by one lane.
+__device__ __forceinline__ void issuer_pump(const Args& A, unsigned char* smem, const Ring& ring, uint32_t need) {
+    IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
     for (;;) {
-        id = __shfl_sync(kFullMask, id, 0);
-        if (id >= n_items) break;
-        uint32_t next_id = 0;
-        if (lane == 0) next_id = gridDim.x + atomicAdd(&header->next_ticket, 1u);
-        Item it;
-        if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
-        const DevTensor& D = tensors[it.t];
-        const uint32_t k_count = (uint32_t)(k_end - k_begin);
-        const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
-        const int k1 = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count);
-        const uint32_t part_key = (it.group << 30) | it.part;
-        if (it.t != cur_t || part_key != cur_part) {
-            __syncwarp();
-            for (int k = k0 + lane; k < k1; k += 32)
-                ptrs[k - k0] = reinterpret_cast<const unsigned char*>(D.cands[k]);
-            __syncwarp();
-            cur_t = it.t;
-            cur_part = part_key;
+        if (st->done == 1u) return;
+        const uint32_t n = st->n_issued, s = st->stage, ph = st->phase;
+        // the stage is free once every warp has released its previous use
+        if (!mbar_try_wait(ring.empty0 + 8 * s, ph ^ 1u)) {
+            if ((int32_t)(n - need) > 0) return;                       // nobody is waiting for this copy yet
+            if (!mbar_wait_slow(ring.empty0 + 8 * s, ph ^ 1u, ring.ctl)) { st->done = 1u; return; }
         }
-        if (lane == 0) {
-            const uint64_t start = (uint64_t)it.tile * kTile;
-            const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
-            bool first = true;
-            if (D.ref_src == RKV_SRC_POINTER) {
-                const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * RSZ;
-                const uint32_t rbytes = (len * RSZ) & ~15u;
-                for (uint32_t rs = 0; rs < kRefStages; ++rs) {
-                    const uint32_t lo = rs * kStageBytes;
-                    const uint32_t b = rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u;
-                    issue(src + lo, b, first, id);
-                    first = false;
-                }
-            }
-            const uint32_t cbytes = (len * CSZ) & ~15u;
-            for (int k = k0; k < k1; ++k) {
-                issue(ptrs[k - k0] + start * CSZ, cbytes, first, id);
-                first = false;
-            }
+        if (st->pos == st->end) {
+            if (st->done == 2u || *ring.ctl.abort_flag) { st->done = 1u; return; }
+            issuer_next_item(A, smem);
+            st->ord += 1u;
         }
-        id = next_id;
-    }
-    if (lane == 0) {
-        issue(nullptr, 0u, true, kNoItem);                     // tell the consumers to stop
-        // the last block to get here clears the ticket counter for the next launch
-        __threadfence();
-        if (atomicAdd(&header->blocks_done, 1u) == gridDim.x - 1u) {
-            header->next_ticket = 0u;
-            header->blocks_done = 0u;
+        const uint32_t pos = st->pos;
+        const uint32_t full = ring.full0 + 8 * s;
+        const unsigned char* src;
+        uint32_t bytes;
+        if (pos < st->nref) {
+            const uint32_t lo = pos * kStageBytes;
+            bytes = st->rbytes > lo ? min(st->rbytes - lo, (uint32_t)kStageBytes) : 0u;
+            src = st->ref_src + lo;
+        } else {
+            const void* const* table = reinterpret_cast<const void* const*>(smem + kOffPtrP) +
+                                       ((st->ord - 1u) & (kInfoRing - 1)) * kPartK;
+            bytes = st->cbytes;
+            src = reinterpret_cast<const unsigned char*>(table[pos - st->nref]) + st->c_off;
         }
-    }
-    // A block that gave up must not retire with copies still landing in its shared
-    // memory: wait (bounded) for the copies issued last.
-    if (lane == 0 && *ring.abort_flag) {
-        const uint32_t pending = n_issued < kStages ? n_issued : kStages;
-        for (uint32_t i = 0; i < pending; ++i) {
-            const uint32_t q = n_issued - 1 - i;
-            const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
-            const long long t0 = clock64();
-            for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
-                if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
-                if (clock64() - t0 > 200000000LL) break;
-            }
+        // the fault drill of a test: arm the stage, withhold the copy
+        const bool withhold = n + 1u == st->drill;
+        if (bytes) {
+            mbar_expect_tx(full, bytes);
+            if (!withhold) bulk_g2s(ring.stage0 + s * kStageBytes, src, bytes, full);
+        } else {
+            mbar_arrive(full);
         }
+        st->pos = pos + 1u;
+        st->n_issued = n + 1u;
+        if (s + 1u == (uint32_t)kStages) { st->stage = 0u; st->phase = ph ^ 1u; }
+        else st->stage = s + 1u;
     }
 }
 
 // ----------------------------------------------------------------------------
-// consumer side: per-thread view of a tile
+// per-thread view of a tile
 // ----------------------------------------------------------------------------
 // A thread owns E elements of the tile (see Geo) as vectors of VEC elements
 // (one 16-byte piece of a candidate each): vector jv of thread tid is vector
-// jv * 224 + tid of the tile.  Element j = jv * VEC + i of the thread has the
+// jv * 256 + tid of the tile.  Element j = jv * VEC + i of the thread has the
 // tile offset below; offsets grow with j.
 template <int VEC>
 __device__ __forceinline__ uint32_t elem_off(int j, int tid) {
-    return (uint32_t)(((j / VEC) * kConsumers + tid) * VEC + (j % VEC));
+    return (uint32_t)(((j / VEC) * kThreads + tid) * VEC + (j % VEC));
 }
 
 // What a thread keeps for the whole item.
-template <bool CB16>
+template <bool C16>
 struct RefRegs;
 
 template <>
@@ -427,15 +489,14 @@ __device__ __forceinline__ void gen_group(uint64_t seed, uint64_t stream_id, int
 
 // Four consecutive elements of the input tensor as fp32 bit patterns (the input
 // has the candidates' dtype); elements at or beyond `len` come back as 0.
-template <bool CB16>
 __device__ __forceinline__ void input_group(const DevTensor& D, uint64_t start, uint32_t off0, uint32_t len,
                                             uint32_t out[4]) {
     if (D.input_src == RKV_SRC_GENERATED) {
-        gen_group(D.in_seed, D.in_stream, D.in_dist, start, off0, CB16, out);
+        gen_group(D.in_seed, D.in_stream, D.in_dist, start, off0, D.cand_dtype == RKV_BF16, out);
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            out[i] = (off0 + i < len) ? ld_elem_bits(D.input, CB16 ? RKV_BF16 : RKV_F32, start + off0 + i) : 0u;
+            out[i] = (off0 + i < len) ? ld_elem_bits(D.input, D.cand_dtype, start + off0 + i) : 0u;
     }
 }
 
@@ -450,17 +511,18 @@ __device__ __forceinline__ uint32_t first_elem_bits(const void* ptr, int src, in
 
 // Load (or regenerate) the thread's reference values for a tile and derive what
 // depends on them alone.  The bulk-copied part of the tile sits in ring stage
-// `stage_a` (and, for an fp32 reference under bf16 candidates, continues in
+// `stage_a` (and, for an fp32 reference under 16-bit candidates, continues in
 // `stage_b`); anything beyond comes from global memory.  `rb` returns all E values as
-// fp32 bit patterns (for the reference's own loophole flags); `ref_s` is the thread's
-// shared-memory home for them with bf16 candidates.
-template <bool CB16, bool RB16>
-__device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB16>::E], const DevTensor& D,
+// fp32 bit patterns (for the reference's own loophole flags).
+template <int CK>
+__device__ __forceinline__ void load_ref(RefRegs<Geo<CK>::C16>& R, uint32_t (&rb)[Geo<CK>::E], const DevTensor& D,
                                          uint64_t start, uint32_t len, const unsigned char* stage_a,
                                          const unsigned char* stage_b, int tid) {
-    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC;
-    constexpr uint32_t RSZ = RB16 ? 2 : 4;
-    const bool full = len == (uint32_t)Geo<CB16>::kTile;
+    constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC;
+    constexpr bool C16 = Geo<CK>::C16;
+    const int rdt = D.ref_dtype;
+    const uint32_t rsz = elem_bytes(rdt);
+    const bool full = len == (uint32_t)Geo<CK>::kTile;
     // byte `b` of the reference tile in the ring
     auto at = [&](uint32_t b) -> const unsigned char* {
         return b < (uint32_t)kStageBytes ? stage_a + b : stage_b + (b - kStageBytes);
@@ -469,8 +531,7 @@ __device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB
 #pragma unroll
         for (int g = 0; g < E / 4; ++g) {
             uint32_t v[4];
-            gen_group(D.ref_seed, D.ref_stream, D.ref_dist, start, elem_off<VEC>(4 * g, tid),
-                      D.ref_dtype == RKV_BF16, v);
+            gen_group(D.ref_seed, D.ref_stream, D.ref_dist, start, elem_off<VEC>(4 * g, tid), rdt == RKV_BF16, v);
 #pragma unroll
             for (int i = 0; i < 4; ++i) rb[4 * g + i] = v[i];
         }
@@ -478,23 +539,23 @@ __device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB
 #pragma unroll
         for (int g = 0; g < E / 4; ++g) {
             const uint32_t off0 = elem_off<VEC>(4 * g, tid);
-            if (RB16) {
+            if (rdt != RKV_F32) {
                 const uint2 t = *reinterpret_cast<const uint2*>(at(off0 * 2));
-                rb[4 * g + 0] = t.x << 16; rb[4 * g + 1] = t.x & 0xFFFF0000u;
-                rb[4 * g + 2] = t.y << 16; rb[4 * g + 3] = t.y & 0xFFFF0000u;
+                rb[4 * g + 0] = upcast16(t.x & 0xFFFFu, rdt); rb[4 * g + 1] = upcast16(t.x >> 16, rdt);
+                rb[4 * g + 2] = upcast16(t.y & 0xFFFFu, rdt); rb[4 * g + 3] = upcast16(t.y >> 16, rdt);
             } else {
                 const uint4 t = *reinterpret_cast<const uint4*>(at(off0 * 4));
                 rb[4 * g + 0] = t.x; rb[4 * g + 1] = t.y; rb[4 * g + 2] = t.z; rb[4 * g + 3] = t.w;
             }
         }
     } else {
-        const uint32_t copied = ((len * RSZ) & ~15u) / RSZ;
+        const uint32_t copied = ((len * rsz) & ~15u) / rsz;
 #pragma unroll
         for (int j = 0; j < E; ++j) {
             const uint32_t off = elem_off<VEC>(j, tid);
             uint32_t b = 0;
-            if (off < copied) b = ld_elem_bits(at(off * RSZ), RB16 ? RKV_BF16 : RKV_F32, 0);
-            else if (off < len) b = ld_elem_bits(D.ref, RB16 ? RKV_BF16 : RKV_F32, start + off);
+            if (off < copied) b = ld_elem_bits(at(off * rsz), rdt, 0);
+            else if (off < len) b = ld_elem_bits(D.ref, rdt, start + off);
             rb[j] = b;
         }
     }
@@ -515,7 +576,7 @@ __device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB
         const float thr = __fadd_rn(atol, __fmul_rn(rtol, __uint_as_float(ab)));
         R.r[j] = __uint_as_float(rb[j]);
         tmin = fminf(tmin, thr);
-        if constexpr (CB16) {
+        if constexpr (C16) {
             has_zero |= ab == 0u;
         } else {
             R.thr[j] = thr;
@@ -524,7 +585,7 @@ __device__ __forceinline__ void load_ref(RefRegs<CB16>& R, uint32_t (&rb)[Geo<CB
     }
     R.thr_min = tmin;
     R.general = nonfinite;
-    if constexpr (CB16) {
+    if constexpr (C16) {
         R.atol = atol;
         R.rtol = rtol;
         R.warp_has_zero = __any_sync(kFullMask, has_zero);
@@ -537,29 +598,31 @@ __device__ __forceinline__ unsigned long long hint_key(float v, uint32_t tile) {
     return ((unsigned long long)(__float_as_uint(v) + 1u) << 32) | (unsigned long long)(~tile);
 }
 
-// Candidate bits of element j of the thread, as an fp32 pattern.
-template <bool CB16, int NW>
-__device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[NW], int j) {
-    if (!CB16) return w[j];
-    return (j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16);
+// Candidate element j of the thread as an fp32 bit pattern.
+template <int CK>
+__device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[16], int j) {
+    if constexpr (CK == CK_F32) return w[j];
+    else if constexpr (CK == CK_BF16) return (j & 1) ? (w[j >> 1] & 0xFFFF0000u) : (w[j >> 1] << 16);
+    else return upcast16((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu), RKV_F16);
 }
 
 // Loophole flags of one candidate tile, until a difference has been seen.
-template <bool CB16>
+template <int CK>
 __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const Hint& h, Hint* h_smem,
                                                 CandState* st, const DevTensor& D, const void* cand_g,
                                                 uint64_t start, uint32_t len, uint32_t wanted_flags, int tid,
                                                 int lane) {
-    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
-    constexpr uint32_t CSZ = CB16 ? 2 : 4;
+    constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC, NW = Geo<CK>::NW, DT = Geo<CK>::DTYPE;
+    constexpr bool C16 = Geo<CK>::C16;
+    constexpr uint32_t CSZ = C16 ? 2 : 4;
     // `settled` is the one hint field other warps update while this warp reads it: take
     // lane 0's copy so that the branch below is uniform across the warp.
     const uint32_t need = wanted_flags & ~__shfl_sync(kFullMask, h.settled, 0);
     if (need) {
         uint32_t acc1 = 0, acc2 = 0;
-        const bool full = len == (uint32_t)Geo<CB16>::kTile;
+        const bool full = len == (uint32_t)Geo<CK>::kTile;
         if (full && (need & 1u)) {
-            const uint32_t f = CB16 ? (h.first >> 16) * 0x10001u : h.first;
+            const uint32_t f = C16 ? h.first * 0x10001u : h.first;
 #pragma unroll
             for (int i = 0; i < NW; ++i) acc1 |= w[i] ^ f;
         }
@@ -569,11 +632,12 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
                                                              start * CSZ) + tid;
 #pragma unroll
             for (int jv = 0; jv < E / VEC; ++jv) {
-                const uint4 t = __ldg(in + jv * kConsumers);
+                const uint4 t = __ldg(in + jv * kThreads);
                 acc2 |= (w[4 * jv] ^ t.x) | (w[4 * jv + 1] ^ t.y) | (w[4 * jv + 2] ^ t.z) | (w[4 * jv + 3] ^ t.w);
             }
         } else if (!full || (need & 2u)) {
             const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+            const uint32_t first_up = C16 ? upcast16(h.first, DT) : h.first;
             // Regenerating the input is the expensive part.  A candidate that is no copy
             // of it almost surely shows that in the first four elements of every thread,
             // so the warp stops generating once a difference has been seen.
@@ -584,14 +648,14 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
                 if (full && !with_input) break;
                 const uint32_t off0 = elem_off<VEC>(4 * g, tid);
                 uint32_t in[4] = {0, 0, 0, 0};
-                if (with_input && off0 < len) input_group<CB16>(D, start, off0, len, in);
+                if (with_input && off0 < len) input_group(D, start, off0, len, in);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t off = off0 + i;
                     if (off < len) {
-                        uint32_t cb = cand_bits<CB16, NW>(w, 4 * g + i);
-                        if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
-                        if (!full) acc1 |= cb ^ h.first;
+                        uint32_t cb = cand_bits<CK>(w, 4 * g + i);
+                        if (off >= copied) cb = ld_elem_bits(cand_g, DT, start + off);
+                        if (!full) acc1 |= cb ^ first_up;
                         if (with_input) acc2 |= cb ^ in[i];
                     }
                 }
@@ -607,28 +671,27 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
     }
 }
 
-// One candidate tile against the thread's reference registers.
+// One tile of an fp32 candidate against the thread's reference registers.
 //   w        the thread's 16-byte pieces of the candidate tile (from the ring)
 //   h        the candidate's hint entry (a snapshot; see the file header)
 //   rec      the warp's running result for this candidate (shared memory; lane 0 writes)
 //   st       the candidate's global state
 //   cand_g   the candidate tensor in global memory (only the last < 16 bytes of a
 //            ragged tensor are read from there)
-template <bool CB16>
-__device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const uint32_t (&w)[16],
-                                                  const Hint& h, Hint* h_smem, WarpRec* rec, CandState* st,
-                                                  const DevTensor& D, const void* cand_g, uint32_t tile,
-                                                  uint64_t start, uint32_t len, uint32_t wanted_flags,
-                                                  int tid, int lane) {
-    static_assert(!CB16, "bf16 candidates take process_candidate_b16");
-    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
-    constexpr uint32_t CSZ = CB16 ? 2 : 4;
+__device__ __forceinline__ void process_candidate_32(const RefRegs<false>& R, const uint32_t (&w)[16],
+                                                     const Hint& h, Hint* h_smem, WarpRec* rec, CandState* st,
+                                                     const DevTensor& D, const void* cand_g, uint32_t tile,
+                                                     uint64_t start, uint32_t len, uint32_t wanted_flags,
+                                                     int tid, int lane) {
+    constexpr int CK = CK_F32;
+    constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC;
+    constexpr uint32_t CSZ = 4;
 
     // ---- common path ---------------------------------------------------------------
     float e[E];
 #pragma unroll
     for (int j = 0; j < E; ++j)
-        e[j] = fabsf(__fsub_rn(__uint_as_float(cand_bits<CB16, NW>(w, j)), R.r[j]));
+        e[j] = fabsf(__fsub_rn(__uint_as_float(w[j]), R.r[j]));
     float m = fmaxf(fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])), fmaxf(fmaxf(e[4], e[5]), fmaxf(e[6], e[7])));
     m = fmaxf(m, fmaxf(fmaxf(fmaxf(e[8], e[9]), fmaxf(e[10], e[11])),
                        fmaxf(fmaxf(e[12], e[13]), fmaxf(e[14], e[15]))));
@@ -646,9 +709,8 @@ __device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const 
         float sf = s;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
-        const double total = rec->sum + (double)sf;       // every lane computes it, one stores
-        if (lane == 0) rec->sum = total;
-        candidate_flags<CB16>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+        if (lane == 0) rec->sum = (double)sf;
+        candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
         return;
     }
     // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
@@ -688,8 +750,8 @@ __device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const 
             for (int j = 0; j < E; ++j) {
                 const uint32_t off = elem_off<VEC>(j, tid);
                 if (off < len) {
-                    uint32_t cb = cand_bits<CB16, NW>(w, j);
-                    if (off >= copied) cb = ld_elem_bits(cand_g, CB16 ? RKV_BF16 : RKV_F32, start + off);
+                    uint32_t cb = w[j];
+                    if (off >= copied) cb = ld_elem_bits(cand_g, RKV_F32, start + off);
                     elem_general(a, cb, __float_as_uint(R.r[j]), off, D.atol, D.rtol);
                 }
             }
@@ -741,43 +803,51 @@ __device__ __forceinline__ void process_candidate(const RefRegs<CB16>& R, const 
                 r.qmax = qm; r.qtile = tile; r.offs = (r.offs & 0x0000FFFFu) | (qoff << 16);
                 atomicMax(&st->hint_q, hint_key(qm, tile));
             }
-            r.sum += sd;
+            r.sum = sd;
             *rec = r;
         }
     } else {
         float sf = s;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
-        if (lane == 0) rec->sum += (double)sf;
+        if (lane == 0) rec->sum = (double)sf;
     }
     if (any_over || any_gen) {
         const uint32_t tot = __reduce_add_sync(kFullMask, cnt);
         if (lane == 0 && tot) rec->n_over += tot;
     }
 
-    candidate_flags<CB16>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+    candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
 }
 
-// c - r for the bf16 value c in the low (half = 0) or high 16 bits of x: the bf16 value
+// c - r for the 16-bit value c in the low (half = 0) or high 16 bits of x: the value
 // widened exactly, one fp32 subtraction rounded to nearest (a mixed-precision instruction
 // of sm_100).
-__device__ __forceinline__ float sub_bf16_f32(uint32_t x, int half, float r) {
+template <int CK>
+__device__ __forceinline__ float sub16_f32(uint32_t x, int half, float r) {
     float d;
-    if (half)
-        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
-    else
-        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+    if constexpr (CK == CK_BF16) {
+        if (half)
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+        else
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+    } else {
+        if (half)
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.f16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+        else
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.f16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(x), "f"(r));
+    }
     return d;
 }
 
-// One pass over a thread's 32 elements of a bf16 candidate tile: largest and summed
+// One pass over a thread's 32 elements of a 16-bit candidate tile: largest and summed
 // e_j = |c_j - r_j|, and the largest d_j, where d_j = fma(-t, |r_j|, e_j) for the
-// relative-error threshold t (see process_candidate_b16).  HAS_ZERO: reference values of
+// relative-error threshold t (see process_candidate_16).  HAS_ZERO: reference values of
 // exactly 0 may occur; they take no part in the relative error, and d_j = e_j - atol there,
 // positive exactly when the element is over tolerance.
-template <bool HAS_ZERO>
-__device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t (&w)[16], float t, float& m_out,
-                                         float& s_out, float& dm_out) {
+template <int CK, bool HAS_ZERO>
+__device__ __forceinline__ void pass_16(const RefRegs<true>& R, const uint32_t (&w)[16], float t, float& m_out,
+                                        float& s_out, float& dm_out) {
     float m = 0.0f, dm = -kInf;
     float sg[8];
 #pragma unroll
@@ -786,7 +856,7 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int j = 4 * g + i;
-            e[i] = fabsf(sub_bf16_f32(w[j >> 1], j & 1, R.r[j]));
+            e[i] = fabsf(sub16_f32<CK>(w[j >> 1], j & 1, R.r[j]));
             const float ar = fabsf(R.r[j]);
             if (HAS_ZERO && ar == 0.0f) d[i] = __fsub_rn(e[i], R.atol);
             else d[i] = __fmaf_rn(-t, ar, e[i]);
@@ -801,10 +871,10 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
                       __fadd_rn(__fadd_rn(sg[4], sg[5]), __fadd_rn(sg[6], sg[7])));
 }
 
-// One tile of a bf16 candidate (32 elements per thread) against the thread's reference
-// registers.  Same results as process_candidate; the tests that keep the rare work rare
-// are arranged for errors proportional to |r|, the normal case of a rounded bf16 output,
-// against which a test on the thread's largest error is powerless.
+// One tile of a bf16 or fp16 candidate (32 elements per thread) against the thread's
+// reference registers.  Same results as process_candidate_32; the tests that keep the rare
+// work rare are arranged for errors proportional to |r|, the normal case of a rounded
+// 16-bit output, against which a test on the thread's largest error is powerless.
 //
 // Relative error.  With t = h.tq_x, element j can be a first maximum only if
 // fl(e_j / |r_j|) > t, which implies e_j > t * |r_j| exactly (t is representable, rounding
@@ -822,23 +892,19 @@ __device__ __forceinline__ void pass_b16(const RefRegs<true>& R, const uint32_t 
 // the over-tolerance test itself; that such an element also counts as a possible maximum
 // costs a look, not a result.
 // Otherwise: m <= thr_min means e_j <= m <= thr_min <= thr_j for every element.
-__device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, const uint32_t (&w)[16],
-                                                      const Hint& h, Hint* h_smem, WarpRec* rec,
-                                                      CandState* st, const DevTensor& D, const void* cand_g,
-                                                      uint32_t tile, uint64_t start, uint32_t len,
-                                                      uint32_t wanted_flags, int tid, int lane) {
+template <int CK>
+__device__ __forceinline__ void process_candidate_16(const RefRegs<true>& R, const uint32_t (&w)[16],
+                                                     const Hint& h, Hint* h_smem, WarpRec* rec,
+                                                     CandState* st, const DevTensor& D, const void* cand_g,
+                                                     uint32_t tile, uint64_t start, uint32_t len,
+                                                     uint32_t wanted_flags, int tid, int lane) {
     constexpr int VEC = 8;
     constexpr float kTiny = 7.8886090522101181e-31f;      // 2^-100
-    // candidate element j as an fp32 bit pattern
-    auto cbits = [&](int j) -> uint32_t {
-        const uint32_t x = w[j >> 1];
-        return (j & 1) ? (x & 0xFFFF0000u) : (x << 16);
-    };
 
     // ---- common path ---------------------------------------------------------------
     float m, s, dm;
-    if (R.warp_has_zero) pass_b16<true>(R, w, h.tq_x, m, s, dm);
-    else pass_b16<false>(R, w, h.tq_x, m, s, dm);
+    if (R.warp_has_zero) pass_16<CK, true>(R, w, h.tq_x, m, s, dm);
+    else pass_16<CK, false>(R, w, h.tq_x, m, s, dm);
 
     const bool lane_gen = R.general || !(s < kInf);
     const bool hit = dm > 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
@@ -847,19 +913,18 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
     const bool maybe_over = rel_covers ? hit : (m > R.thr_min);
 
     if (!__any_sync(kFullMask, rare || maybe_over)) {
-        // nothing but the sum to record (every lane computes it, one stores)
+        // nothing but the sum to record
         float sf = s;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
-        const double total = rec->sum + (double)sf;
-        if (lane == 0) rec->sum = total;
+        if (lane == 0) rec->sum = (double)sf;
     } else {
         uint32_t cnt = 0;
         const bool any_over = __any_sync(kFullMask, maybe_over);
         if (any_over) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
+                const float e = fabsf(__fsub_rn(__uint_as_float(cand_bits<CK>(w, j)), R.r[j]));
                 cnt += (e > __fadd_rn(R.atol, __fmul_rn(R.rtol, fabsf(R.r[j])))) ? 1u : 0u;
             }
         }
@@ -875,7 +940,7 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
             for (int j = 0; j < 32; ++j) {
                 const uint32_t off = elem_off<VEC>(j, tid);
                 // (a ragged tile's tail was patched into w by the caller)
-                if (off < len) elem_general(a, cbits(j), __float_as_uint(R.r[j]), off, R.atol, R.rtol);
+                if (off < len) elem_general(a, cand_bits<CK>(w, j), __float_as_uint(R.r[j]), off, R.atol, R.rtol);
             }
             if (a.n_noncomp) atomicAdd(&st->n_noncomp, (unsigned long long)a.n_noncomp);
             if (a.n_nan) atomicAdd(&st->n_nan, (unsigned long long)a.n_nan);
@@ -884,7 +949,7 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
         } else if (rare) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                const float e = fabsf(__fsub_rn(__uint_as_float(cbits(j)), R.r[j]));
+                const float e = fabsf(__fsub_rn(__uint_as_float(cand_bits<CK>(w, j)), R.r[j]));
                 const uint32_t off = elem_off<VEC>(j, tid);
                 // (positions past the end of a ragged tile hold zeros and never count)
                 if (e > a.emax && off < len) { a.emax = e; a.eoff = off; }
@@ -928,49 +993,67 @@ __device__ __forceinline__ void process_candidate_b16(const RefRegs<true>& R, co
                 r.qmax = qm; r.qtile = tile; r.offs = (r.offs & 0x0000FFFFu) | (qoff << 16);
                 atomicMax(&st->hint_q, hint_key(qm, tile));
             }
-            r.sum += sd;
+            r.sum = sd;
             r.n_over += tot;
             *rec = r;
         }
     }
-    candidate_flags<true>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+    candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
 }
 
-// Merge the warp records of every candidate of a part into the block's
-// Partial row and clear them.  Called by all consumer threads between two
-// consumer barriers.
-__device__ __forceinline__ void flush_records(WarpRec* recs, const DevTensor& D, int K, int k0, int kc,
-                                              uint32_t slot, Partial* __restrict__ partials, int tid,
-                                              uint32_t tile_elems) {
+// The error sums of the item just finished: for every candidate of its part, the warps'
+// tile sums added in warp order, stored in the (tile, candidate) slot, and cleared.
+// Called by all threads between two block barriers.
+__device__ __forceinline__ void flush_sums(WarpRec* recs, const Args& A, const DevTensor& D, uint32_t tile, int k0,
+                                           int kc, int tid) {
+    if (tid < kc) {
+        double s = 0.0;
+#pragma unroll
+        for (int wp = 0; wp < kWarps; ++wp) {
+            WarpRec& r = recs[wp * kPartK + tid];
+            s += r.sum;
+            r.sum = 0.0;
+        }
+        const unsigned long long at = D.sum_base + (unsigned long long)tile * (unsigned long long)A.K +
+                                      (unsigned long long)(k0 + tid);
+        if (RKV_IN_BOUNDS(A.header, 3, tile < D.n_tiles && k0 + tid < A.K, at)) A.sums[at] = s;
+    }
+}
+
+// Merge the warp records of every candidate of a part into the Partial row and clear
+// them.  Called by all threads between two block barriers.
+__device__ __forceinline__ void flush_records(WarpRec* recs, const Args& A, const DevTensor& D, int k0, int kc,
+                                              uint32_t slot, int tid, uint32_t tile_elems_) {
     if (tid < kc) {
         Partial p;
-        p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX; p.sum = 0.0;
-        p.emax = -1.0f; p.qmax = -1.0f; p.valid = 1u; p.reserved = 0u;
+        p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX;
+        p.emax = -1.0f; p.qmax = -1.0f; p.valid = 1u; p.reserved[0] = p.reserved[1] = p.reserved[2] = 0u;
 #pragma unroll
-        for (int wp = 0; wp < kConsumerWarps; ++wp) {
+        for (int wp = 0; wp < kWarps; ++wp) {
             WarpRec& r = recs[wp * kPartK + tid];
             p.n_over += r.n_over;
-            p.sum += r.sum;
             if (r.emax >= 0.0f) {
-                const uint64_t idx = (uint64_t)r.etile * tile_elems + (r.offs & 0xFFFFu);
+                const uint64_t idx = (uint64_t)r.etile * tile_elems_ + (r.offs & 0xFFFFu);
                 if (r.emax > p.emax || (r.emax == p.emax && idx < p.eidx)) { p.emax = r.emax; p.eidx = idx; }
             }
             if (r.qmax >= 0.0f) {
-                const uint64_t idx = (uint64_t)r.qtile * tile_elems + (r.offs >> 16);
+                const uint64_t idx = (uint64_t)r.qtile * tile_elems_ + (r.offs >> 16);
                 if (r.qmax > p.qmax || (r.qmax == p.qmax && idx < p.qidx)) { p.qmax = r.qmax; p.qidx = idx; }
             }
-            r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
+            r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0;
         }
-        // the block may have written this slot before (group A, then group B): merge
-        Partial* dst = &partials[((size_t)D.slot_base + slot) * (size_t)K + (size_t)(k0 + tid)];
-        const Partial old = *dst;
-        if (old.valid) {
-            p.n_over += old.n_over;
-            p.sum = old.sum + p.sum;
-            if (old.emax > p.emax || (old.emax == p.emax && old.eidx < p.eidx)) { p.emax = old.emax; p.eidx = old.eidx; }
-            if (old.qmax > p.qmax || (old.qmax == p.qmax && old.qidx < p.qidx)) { p.qmax = old.qmax; p.qidx = old.qidx; }
+        if (RKV_IN_BOUNDS(A.header, 4, slot < D.n_slots && k0 + tid < A.K, slot)) {
+            // the slot may have been written before (another group, or an earlier launch of a
+            // chunked call): merge
+            Partial* dst = &A.partials[((size_t)D.slot_base + slot) * (size_t)A.K + (size_t)(k0 + tid)];
+            const Partial old = *dst;
+            if (old.valid) {
+                p.n_over += old.n_over;
+                if (old.emax > p.emax || (old.emax == p.emax && old.eidx < p.eidx)) { p.emax = old.emax; p.eidx = old.eidx; }
+                if (old.qmax > p.qmax || (old.qmax == p.qmax && old.qidx < p.qidx)) { p.qmax = old.qmax; p.qidx = old.qidx; }
+            }
+            *dst = p;
         }
-        *dst = p;
     }
 }
 
@@ -984,207 +1067,267 @@ __device__ __forceinline__ float hint_threshold(unsigned long long key, uint32_t
     return bits ? __uint_as_float(bits - 1u) : -1.0f;       // the float below; below +0 anything goes
 }
 
-template <bool CB16, bool RB16>
-__device__ __forceinline__ void consumer_loop(const DevTensor* __restrict__ tensors, int T, int K, int k_begin,
-                                              int k_end, uint32_t n_items, CandState* __restrict__ state,
-                                              Partial* __restrict__ partials, unsigned char* smem,
-                                              const Ring& ring) {
-    constexpr int E = Geo<CB16>::E, VEC = Geo<CB16>::VEC, NW = Geo<CB16>::NW;
+// What a block carries from item to item.
+struct BlockState {
+    uint32_t cstage, cphase;     // next ring stage to consume and the parity of its current use
+    uint32_t ccount;             // stages consumed so far (= the number of the next copy to wait for)
+    uint32_t ord;                // items this block has started
+    bool is_issuer;              // this warp's lane 0 issues the copies
+};
+
+// Wait for the next ring stage; the issuing lane first makes sure its copy is on the way.
+__device__ __forceinline__ bool wait_stage(const Args& A, unsigned char* smem, const Ring& ring, BlockState& B,
+                                           int lane, uint32_t& stage_out) {
+    if (B.is_issuer) {
+        if (lane == 0) issuer_pump(A, smem, ring, B.ccount);
+        __syncwarp();
+    }
+    stage_out = B.cstage;
+    return mbar_wait(ring.full0 + 8 * B.cstage, B.cphase, ring.ctl);
+}
+
+__device__ __forceinline__ void advance_stage(BlockState& B) {
+    B.ccount += 1u;
+    if (++B.cstage == (uint32_t)kStages) { B.cstage = 0; B.cphase ^= 1u; }
+}
+
+// One item: every candidate of the part against the tile's reference values.
+template <int CK>
+__device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, const Ring& ring, BlockState& B,
+                                         const ItemInfo& it, const DevTensor& D) {
+    constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC, NW = Geo<CK>::NW;
     constexpr int NV = E / VEC;
-    constexpr uint32_t kTile = Geo<CB16>::kTile;
-    constexpr int kRefStages = (CB16 && !RB16) ? 2 : 1;
-    constexpr uint32_t kVariant = (CB16 ? 2u : 0u) + (RB16 ? 1u : 0u);
+    constexpr bool C16 = Geo<CK>::C16;
+    constexpr uint32_t kTile = Geo<CK>::kTile;
+    constexpr uint32_t CSZ = C16 ? 2 : 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrC);
-    Hint* hints = reinterpret_cast<Hint*>(smem + kOffHint);
+    Hint* H = reinterpret_cast<Hint*>(smem + kOffHint) + (B.ord & 1u) * kPartK;
     WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
     volatile uint32_t* ref_state = reinterpret_cast<volatile uint32_t*>(smem + kOffRefState);
     const unsigned char* stages = smem + kOffStage;
 
-    // clear the records once; flush_records leaves them cleared
-    for (int i = tid; i < kConsumerWarps * kPartK; i += kConsumers) {
-        WarpRec& r = recs[i];
-        r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
+    const int k0 = (int)it.k0, kc = (int)it.kc;
+    const uint64_t start = (uint64_t)it.tile * kTile;
+    const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
+    const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
+    CandState* st_t = A.state + D.state_base;
+
+    // the part's pointers and hints, from the published state
+    if (tid < kc) {
+        const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
+        ptrs[tid] = p;
+        const CandState* sc = st_t + k0 + tid;
+        Hint h;
+        h.te_x = hint_threshold(__ldcg(&sc->hint_e), it.tile);
+        h.tq_x = hint_threshold(__ldcg(&sc->hint_q), it.tile);
+        if (C16 && h.tq_x < 0.0f) h.tq_x = -kInf;     // see process_candidate_16
+        h.settled = __ldcg(&sc->mismatch);
+        h.first = ld_elem_raw(p, Geo<CK>::DTYPE, 0);
+        H[tid] = h;
     }
+    if (tid == kPartK) ref_state[B.ord & 1u] = __ldcg(&st_t[A.K].mismatch);
 
-    // next ring stage to consume and the parity of its current use (same order as the producer issues)
-    uint32_t cstage = 0, cphase = 0;
-    uint32_t ord = 0;               // items this block has started
-    int cur_t = -1, cur_k0 = 0, cur_kc = 0;
-    uint32_t cur_part = 0xFFFFFFFFu, cur_slot = 0;
-
-    volatile uint32_t* ids = reinterpret_cast<volatile uint32_t*>(smem + kOffIds);
-    for (;; ++ord) {
-        // The next item announces itself in the first ring stage it uses (which stays full
-        // until it is consumed below).  All consumers agree on stopping: at the producer's
-        // end mark, or when any thread of the block has given up on a wait.
-        const uint32_t s0 = cstage;
-        const bool got = mbar_wait(ring.full0 + 8 * s0, cphase, ring.abort_flag);
-        const uint32_t id = got ? ids[s0] : kNoItem;
-        if (consumer_sync_or((id == kNoItem || id >= n_items || *ring.abort_flag) ? 1u : 0u)) break;
-        Item it;
-        if (!decode_item(tensors, T, kVariant, (uint32_t)(k_end - k_begin), id, it)) break;
-        const DevTensor& D = tensors[it.t];
-        const uint32_t k_count = (uint32_t)(k_end - k_begin);
-        const int k0 = k_begin + (int)part_begin(it.part, it.n_parts, k_count);
-        const int kc = k_begin + (int)part_begin(it.part + 1, it.n_parts, k_count) - k0;
-        const uint32_t part_key = (it.group << 30) | it.part;
-        const uint64_t start = (uint64_t)it.tile * kTile;
-        const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
-        const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
-        CandState* st_t = state + (size_t)it.t * (size_t)(K + 1);
-        Hint* H = hints + (ord & 1u) * kPartK;
-
-        if (it.t != cur_t || part_key != cur_part) {
-            consumer_sync();                      // every warp is done with the previous part
-            if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
-            if (tid < kc) ptrs[tid] = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
-            cur_t = it.t; cur_part = part_key; cur_k0 = k0; cur_kc = kc;
-            cur_slot = blockIdx.x;                // one Partial row per block and tensor
+    // ---- the thread's reference values --------------------------------------------
+    RefRegs<C16> R;
+    uint32_t rb[E];
+    if (D.ref_src == RKV_SRC_POINTER) {
+        // the reference tile fills one ring stage, or two (fp32 under 16-bit candidates)
+        const bool two = (kTile * elem_bytes(D.ref_dtype)) > (uint32_t)kStageBytes;
+        uint32_t sa, sb;
+        wait_stage(A, smem, ring, B, lane, sa);
+        advance_stage(B);
+        sb = sa;
+        if (two) {
+            wait_stage(A, smem, ring, B, lane, sb);
+            advance_stage(B);
         }
-        // refresh the hints of this part from the published state
-        if (tid < kc) {
-            const CandState* sc = st_t + k0 + tid;
-            Hint h;
-            h.te_x = hint_threshold(__ldcg(&sc->hint_e), it.tile);
-            h.tq_x = hint_threshold(__ldcg(&sc->hint_q), it.tile);
-            if (CB16 && h.tq_x < 0.0f) h.tq_x = -kInf;     // see process_candidate_b16
-            h.settled = __ldcg(&sc->mismatch);
-            h.first = ld_elem_bits(ptrs[tid], CB16 ? RKV_BF16 : RKV_F32, 0);
-            H[tid] = h;
-        }
-        if (tid == kPartK) ref_state[ord & 1u] = __ldcg(&st_t[K].mismatch);
+        load_ref<CK>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes, stages + (size_t)sb * kStageBytes, tid);
+        __syncwarp();
+        mbar_arrive_if(ring.empty0 + 8 * sa, lane == 0);
+        if (two) mbar_arrive_if(ring.empty0 + 8 * sb, lane == 0);
+    } else {
+        load_ref<CK>(R, rb, D, start, len, nullptr, nullptr, tid);
+    }
+    __syncthreads();                          // hints, pointers and cleared records are visible
 
-        // ---- the thread's reference values --------------------------------------------
-        RefRegs<CB16> R;
-        uint32_t rb[E];
-        if (D.ref_src == RKV_SRC_POINTER) {
-            // the reference tile fills one ring stage, or two (fp32 under bf16 candidates)
-            const uint32_t sa = cstage, pha = cphase;
-            mbar_wait(ring.full0 + 8 * sa, pha, ring.abort_flag);
-            if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
-            uint32_t sb = sa;
-            if (kRefStages == 2) {
-                sb = cstage;
-                mbar_wait(ring.full0 + 8 * sb, cphase, ring.abort_flag);
-                if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
-            }
-            load_ref<CB16, RB16>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes,
-                                 stages + (size_t)sb * kStageBytes, tid);
-            __syncwarp();
-            mbar_arrive_if(ring.empty0 + 8 * sa, lane == 0);
-            if (kRefStages == 2) mbar_arrive_if(ring.empty0 + 8 * sb, lane == 0);
-        } else {
-            load_ref<CB16, RB16>(R, rb, D, start, len, nullptr, nullptr, tid);
-        }
-        consumer_sync();                          // hints, pointers and cleared records are visible
-
-        // reference flags (constant / copy of the input), until a difference has been seen
-        {
-            const uint32_t need = wanted & ~ref_state[ord & 1u];
-            if (need) {
-                const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed,
-                                                         D.ref_stream, D.ref_dist);
-                uint32_t acc1 = 0, acc2 = 0;
+    // reference flags (constant / copy of the input), until a difference has been seen
+    {
+        const uint32_t need = wanted & ~ref_state[B.ord & 1u];
+        if (need) {
+            const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed,
+                                                     D.ref_stream, D.ref_dist);
+            uint32_t acc1 = 0, acc2 = 0;
 #pragma unroll
-                for (int g = 0; g < E / 4; ++g) {
-                    const uint32_t off0 = elem_off<VEC>(4 * g, tid);
-                    uint32_t in[4] = {0, 0, 0, 0};
-                    if ((need & 2u) && off0 < len) input_group<CB16>(D, start, off0, len, in);
+            for (int g = 0; g < E / 4; ++g) {
+                const uint32_t off0 = elem_off<VEC>(4 * g, tid);
+                uint32_t in[4] = {0, 0, 0, 0};
+                if ((need & 2u) && off0 < len) input_group(D, start, off0, len, in);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if (off0 + i < len) {
-                            acc1 |= rb[4 * g + i] ^ r_first;
-                            acc2 |= rb[4 * g + i] ^ in[i];
-                        }
-                    }
-                }
-                uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
-                                (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
-                seen &= need;
-                if (lane == 0 && seen) atomicOr(&st_t[K].mismatch, seen);
-            }
-        }
-
-        // ---- every candidate of the part ----------------------------------------------
-        for (int kk = 0; kk < kc; ++kk) {
-            const uint32_t s = cstage;
-            const Hint h = H[kk];
-            mbar_wait(ring.full0 + 8 * s, cphase, ring.abort_flag);
-            const unsigned char* stage = stages + (size_t)s * kStageBytes;
-            uint32_t w[NW];
-#pragma unroll
-            for (int jv = 0; jv < NV; ++jv) {
-                const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kConsumers + tid) * 16);
-                w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
-            }
-            __syncwarp();
-            mbar_arrive_if(ring.empty0 + 8 * s, lane == 0);
-            if (++cstage == kStages) { cstage = 0; cphase ^= 1u; }
-            if (len != kTile) {
-                // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
-                // elements behind them come from global memory; positions past the end of the
-                // tensor get 0 against a reference of 0 (see load_ref): no error, never over
-                // tolerance, excluded from the relative error, and never the first maximum,
-                // because their offsets are larger than every real element's.
-                constexpr uint32_t CSZ = CB16 ? 2 : 4;
-                const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
-#pragma unroll
-                for (int j = 0; j < E; ++j) {
-                    const uint32_t off = elem_off<VEC>(j, tid);
-                    if (off >= copied) {
-                        const uint32_t cb = off < len ? ld_elem_bits(ptrs[kk], CB16 ? RKV_BF16 : RKV_F32, start + off) : 0u;
-                        if (!CB16) w[j] = cb;
-                        else w[j >> 1] = (j & 1) ? ((w[j >> 1] & 0x0000FFFFu) | cb) : ((w[j >> 1] & 0xFFFF0000u) | (cb >> 16));
+                for (int i = 0; i < 4; ++i) {
+                    if (off0 + i < len) {
+                        acc1 |= rb[4 * g + i] ^ r_first;
+                        acc2 |= rb[4 * g + i] ^ in[i];
                     }
                 }
             }
-            if constexpr (CB16)
-                process_candidate_b16(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
-                                      it.tile, start, len, wanted, tid, lane);
-            else
-                process_candidate<false>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
-                                         it.tile, start, len, wanted, tid, lane);
+            uint32_t seen = (__any_sync(kFullMask, acc1 != 0u) ? 1u : 0u) |
+                            (__any_sync(kFullMask, acc2 != 0u) ? 2u : 0u);
+            seen &= need;
+            if (lane == 0 && seen) atomicOr(&st_t[A.K].mismatch, seen);
         }
     }
-    consumer_sync();
-    if (cur_t >= 0) flush_records(recs, tensors[cur_t], K, cur_k0, cur_kc, cur_slot, partials, tid, kTile);
+
+    // ---- every candidate of the part ----------------------------------------------
+    for (int kk = 0; kk < kc; ++kk) {
+        const Hint h = H[kk];
+        uint32_t s;
+        wait_stage(A, smem, ring, B, lane, s);
+        const unsigned char* stage = stages + (size_t)s * kStageBytes;
+        uint32_t w[NW];
+#pragma unroll
+        for (int jv = 0; jv < NV; ++jv) {
+            const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kThreads + tid) * 16);
+            w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
+        }
+        __syncwarp();
+        mbar_arrive_if(ring.empty0 + 8 * s, lane == 0);
+        advance_stage(B);
+        if (len != kTile) {
+            // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
+            // elements behind them come from global memory; positions past the end of the
+            // tensor get 0 against a reference of 0 (see load_ref): no error, never over
+            // tolerance, excluded from the relative error, and never the first maximum,
+            // because their offsets are larger than every real element's.
+            const uint32_t copied = ((len * CSZ) & ~15u) / CSZ;
+#pragma unroll
+            for (int j = 0; j < E; ++j) {
+                const uint32_t off = elem_off<VEC>(j, tid);
+                if (off >= copied) {
+                    const uint32_t cb = off < len ? ld_elem_raw(ptrs[kk], Geo<CK>::DTYPE, start + off) : 0u;
+                    if (!C16) w[j] = cb;
+                    else w[j >> 1] = (j & 1) ? ((w[j >> 1] & 0x0000FFFFu) | (cb << 16)) : ((w[j >> 1] & 0xFFFF0000u) | cb);
+                }
+            }
+        }
+        if constexpr (C16)
+            process_candidate_16<CK>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+                                     it.tile, start, len, wanted, tid, lane);
+        else
+            process_candidate_32(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+                                 it.tile, start, len, wanted, tid, lane);
+    }
 }
 
-// One kernel per storage variant (candidate dtype, stored reference dtype), so
-// that each gets its own register allocation.  A launch handles the items of
-// every tensor of its variant; `n_items` counts them.
-template <bool CB16, bool RB16>
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
-verify_kernel(const DevTensor* __restrict__ tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
-              CandState* __restrict__ state, Partial* __restrict__ partials, WorkspaceHeader* header) {
+// Persistent blocks, kBlocksPerSm per SM.
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Args A) {
     extern __shared__ __align__(1024) unsigned char smem[];
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     Ring ring;
     ring.full0 = smem_u32(smem + kOffFull);
     ring.empty0 = smem_u32(smem + kOffEmpty);
     ring.stage0 = smem_u32(smem + kOffStage);
-    ring.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
+    ring.ctl.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
+    ring.ctl.limit = reinterpret_cast<const volatile long long*>(smem + kOffWaitLimit);
+    WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(ring.full0 + 8 * s, 1);                    // the producer's arrive + its bytes
-            mbar_init(ring.empty0 + 8 * s, kConsumerWarps);      // one release per consumer warp
+            mbar_init(ring.full0 + 8 * s, 1);             // the issuer's arrive + the copy's bytes
+            mbar_init(ring.empty0 + 8 * s, kWarps);       // one release per warp
         }
-        *ring.abort_flag = 0u;
+        *ring.ctl.abort_flag = 0u;
+        const unsigned long long lim = A.header->drill_issue ? A.header->drill_wait_cycles : 0ull;
+        *reinterpret_cast<volatile long long*>(smem + kOffWaitLimit) = lim ? (long long)lim : kWaitCycles;
+        IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
+        st->n_issued = 0; st->stage = 0; st->phase = 0; st->pos = 0; st->end = 0; st->nref = 0; st->done = 0;
+        st->ord = 0; st->cbytes = 0; st->rbytes = 0; st->seg = 0; st->c_off = 0; st->ref_src = nullptr;
+        st->next_id = blockIdx.x;             // every block starts with the item of its own number
+        st->drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // clear the records once; the flushes leave them cleared
+    for (int i = tid; i < kWarps * kPartK; i += kThreads) {
+        WarpRec& r = recs[i];
+        r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
+    }
     __syncthreads();
-    if (tid >= kConsumers) {
-        producer_loop<CB16, RB16>(tensors, T, k_begin, k_end, n_items, smem, ring, header);
-    } else {
-        consumer_loop<CB16, RB16>(tensors, T, K, k_begin, k_end, n_items, state, partials, smem, ring);
-        if (tid == 0 && *ring.abort_flag) atomicExch(&header->status, (int32_t)RKV_ERR_TIMEOUT);
+
+    BlockState B;
+    B.cstage = 0; B.cphase = 0; B.ccount = 0; B.ord = 0;
+    B.is_issuer = warp == kWarps - 1;
+    const ItemInfo* infos = reinterpret_cast<const ItemInfo*>(smem + kOffInfo);
+
+    int cur_t = -1, cur_k0 = 0, cur_kc = 0;
+    uint32_t cur_slot = 0, cur_tile = 0, cur_te = 0;
+    for (;; ++B.ord) {
+        // The next item announces itself before its first ring stage is armed (that stage stays
+        // full until it is consumed in run_item).  All threads agree on stopping: at the
+        // issuer's end mark, or when any thread of the block has given up on a wait.
+        uint32_t s0;
+        const bool got = wait_stage(A, smem, ring, B, lane, s0);
+        ItemInfo it = infos[B.ord & (kInfoRing - 1)];
+        if (!got) it.id = kNoItem;
+        if (block_sync_or((it.id == kNoItem || *ring.ctl.abort_flag) ? 1u : 0u)) break;
+        if (!RKV_IN_BOUNDS(A.header, 5, it.t < (uint32_t)A.T && it.kc >= 1u && it.kc <= (uint32_t)kPartK &&
+                                            it.k0 + it.kc <= (uint32_t)A.K, it.t))
+            break;
+        const DevTensor& D = A.tensors[it.t];
+        // every warp is done with the previous item: its sums, and, when the tensor or the
+        // candidates change, its records
+        if (cur_t >= 0) {
+            flush_sums(recs, A, A.tensors[cur_t], cur_tile, cur_k0, cur_kc, tid);
+            if ((int)it.t != cur_t || (int)it.k0 != cur_k0 || (int)it.kc != cur_kc ||
+                (A.tensors[cur_t].slot_by_tile && it.tile != cur_tile))
+                flush_records(recs, A, A.tensors[cur_t], cur_k0, cur_kc, cur_slot, tid, cur_te);
+        }
+        cur_t = (int)it.t; cur_k0 = (int)it.k0; cur_kc = (int)it.kc; cur_tile = it.tile;
+        cur_slot = D.slot_by_tile ? it.tile : blockIdx.x;
+        cur_te = tile_elems(D.cand_dtype);
+        // (the stage waited for above is consumed inside run_item: it holds the item's reference
+        // tile or its first candidate)
+        switch (D.cand_dtype) {
+            case RKV_F32: run_item<CK_F32>(A, smem, ring, B, it, D); break;
+            case RKV_BF16: run_item<CK_BF16>(A, smem, ring, B, it, D); break;
+            default: run_item<CK_F16>(A, smem, ring, B, it, D); break;
+        }
+    }
+    __syncthreads();
+    if (cur_t >= 0) {
+        flush_sums(recs, A, A.tensors[cur_t], cur_tile, cur_k0, cur_kc, tid);
+        flush_records(recs, A, A.tensors[cur_t], cur_k0, cur_kc, cur_slot, tid, cur_te);
+    }
+    if (tid == 0 && *ring.ctl.abort_flag) atomicExch(&A.header->status, (int32_t)RKV_ERR_TIMEOUT);
+
+    if (B.is_issuer && lane == 0) {
+        IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
+        // the last block to get here clears the ticket counter for the next launch
+        __threadfence();
+        if (atomicAdd(&A.header->blocks_done, 1u) == gridDim.x - 1u) {
+            A.header->next_ticket = 0u;
+            A.header->blocks_done = 0u;
+        }
+        // A block that gave up must not retire with copies still landing in its shared
+        // memory: wait (bounded) for the copies issued last.
+        if (*ring.ctl.abort_flag) {
+            const uint32_t n_issued = st->n_issued;
+            const uint32_t pending = n_issued < (uint32_t)kStages ? n_issued : (uint32_t)kStages;
+            for (uint32_t i = 0; i < pending; ++i) {
+                const uint32_t q = n_issued - 1 - i;
+                const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
+                const long long t0 = clock64();
+                for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+                    if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
+                    if (clock64() - t0 > 200000000LL) break;
+                }
+            }
+        }
     }
 }
 
 // ----------------------------------------------------------------------------
 // finalize: merge the per-block partials of each (candidate, tensor) in a fixed
-// order, derive flags and verdict, and the joint verdict over tensors
+// order, add the tile sums in tile order, derive flags and verdict; then the joint
+// verdicts over the tensors of a case and over the cases
 // ----------------------------------------------------------------------------
 constexpr int kFinThreads = 128;
 
@@ -1202,125 +1345,125 @@ __device__ __forceinline__ void wide_merge(Wide& a, const Wide& b) {
     a.sum += b.sum;
 }
 
+// One block per (tensor, candidate).
 __global__ void __launch_bounds__(kFinThreads)
 finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandState* __restrict__ state,
-                const Partial* __restrict__ partials, rkv_stats* __restrict__ stats_out,
-                uint32_t* __restrict__ joint_pass) {
+                const Partial* __restrict__ partials, const double* __restrict__ sums,
+                rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ fail) {
     __shared__ Wide red[kFinThreads];
-    const int k = blockIdx.x, tid = threadIdx.x;
-    uint32_t all_pass = 1;
-    for (int t = 0; t < T; ++t) {
-        const DevTensor D = tensors[t];
-        Wide w;
-        w.n_over = 0; w.sum = 0.0;
-        w.emax = -1.0f; w.qmax = -1.0f; w.eidx = RKV_NO_INDEX; w.qidx = RKV_NO_INDEX;
-        for (uint32_t s = tid; s < D.n_slots; s += kFinThreads) {
-            const Partial p = partials[((size_t)D.slot_base + s) * (size_t)K + (size_t)k];
-            if (!p.valid) continue;
-            Wide b;
-            b.n_over = p.n_over; b.sum = p.sum;
-            b.emax = p.emax; b.eidx = p.eidx; b.qmax = p.qmax; b.qidx = p.qidx;
-            wide_merge(w, b);
-        }
-        red[tid] = w;
-        __syncthreads();
-        for (int off = kFinThreads / 2; off > 0; off >>= 1) {
-            if (tid < off) {
-                Wide a = red[tid];
-                wide_merge(a, red[tid + off]);
-                red[tid] = a;
-            }
-            __syncthreads();
-        }
-        if (tid == 0) {
-            const Wide r = red[0];
-            const CandState cs = state[(size_t)t * (size_t)(K + 1) + (size_t)k];
-            const uint32_t ref_mismatch = state[(size_t)t * (size_t)(K + 1) + (size_t)K].mismatch;
-            rkv_stats st;
-            st.n_over_tol = r.n_over;
-            st.n_nan = cs.n_nan;
-            st.n_inf = cs.n_inf;
-            st.n_inf_mismatch = cs.n_infmis;
-            st.n_comparable = D.n - cs.n_noncomp;
-            st.argmax_abs_err = r.emax < 0.0f ? RKV_NO_INDEX : r.eidx;
-            st.argmax_rel_err = r.qmax < 0.0f ? RKV_NO_INDEX : r.qidx;
-            st.sum_abs_err = r.sum;
-            st.max_abs_err = r.emax < 0.0f ? 0.0f : r.emax;
-            st.max_rel_err = r.qmax < 0.0f ? 0.0f : r.qmax;
-            st.mean_abs_err = st.n_comparable ? (float)(r.sum / (double)st.n_comparable) : 0.0f;
-            st.reserved = 0;
-            const bool has_in = D.input_src != RKV_SRC_NONE;
-            uint32_t flags = 0;
-            if (!(cs.mismatch & 1u)) flags |= RKV_FLAG_CAND_CONST;
-            if (has_in && !(cs.mismatch & 2u)) flags |= RKV_FLAG_CAND_COPY_OF_INPUT;
-            if (!(ref_mismatch & 1u)) flags |= RKV_FLAG_REF_CONST;
-            if (has_in && !(ref_mismatch & 2u)) flags |= RKV_FLAG_REF_COPY_OF_INPUT;
-            if (cs.n_nan) flags |= RKV_FLAG_HAS_NAN;
-            if (cs.n_inf) flags |= RKV_FLAG_HAS_INF;
-            uint32_t verdict = 0;
-            if (r.n_over) verdict |= RKV_FAIL_TOL;
-            if (cs.n_nan) verdict |= RKV_FAIL_NAN;
-            if (cs.n_infmis) verdict |= RKV_FAIL_INF_MISMATCH;
-            if ((flags & RKV_FLAG_CAND_CONST) && !(flags & RKV_FLAG_REF_CONST) && D.n > 1)
-                verdict |= RKV_FAIL_LOOPHOLE_CONST;
-            if ((flags & RKV_FLAG_CAND_COPY_OF_INPUT) && !(flags & RKV_FLAG_REF_COPY_OF_INPUT))
-                verdict |= RKV_FAIL_LOOPHOLE_COPY;
-            st.flags = flags;
-            st.verdict = verdict;
-            stats_out[(size_t)k * T + t] = st;
-            if (verdict) all_pass = 0;
+    const int t = blockIdx.x / K, k = blockIdx.x % K, tid = threadIdx.x;
+    if (t >= T) return;
+    const DevTensor D = tensors[t];
+    Wide w;
+    w.n_over = 0; w.sum = 0.0;
+    w.emax = -1.0f; w.qmax = -1.0f; w.eidx = RKV_NO_INDEX; w.qidx = RKV_NO_INDEX;
+    for (uint32_t s = tid; s < D.n_slots; s += kFinThreads) {
+        const Partial p = partials[((size_t)D.slot_base + s) * (size_t)K + (size_t)k];
+        if (!p.valid) continue;
+        Wide b;
+        b.n_over = p.n_over; b.sum = 0.0;
+        b.emax = p.emax; b.eidx = p.eidx; b.qmax = p.qmax; b.qidx = p.qidx;
+        wide_merge(w, b);
+    }
+    // tile sums: thread i adds tiles i, i + 128, ... in that order; the tree below is fixed
+    for (uint32_t tile = tid; tile < D.n_tiles; tile += kFinThreads)
+        w.sum += sums[D.sum_base + (unsigned long long)tile * (unsigned long long)K + (unsigned long long)k];
+    red[tid] = w;
+    __syncthreads();
+    for (int off = kFinThreads / 2; off > 0; off >>= 1) {
+        if (tid < off) {
+            Wide a = red[tid];
+            wide_merge(a, red[tid + off]);
+            red[tid] = a;
         }
         __syncthreads();
     }
-    if (tid == 0 && joint_pass) joint_pass[k] = all_pass;
+    if (tid == 0) {
+        const Wide r = red[0];
+        const CandState cs = state[(size_t)D.state_base + (size_t)k];
+        const uint32_t ref_mismatch = state[(size_t)D.state_base + (size_t)K].mismatch;
+        rkv_stats st;
+        st.n_over_tol = r.n_over;
+        st.n_nan = cs.n_nan;
+        st.n_inf = cs.n_inf;
+        st.n_inf_mismatch = cs.n_infmis;
+        st.n_comparable = D.n - cs.n_noncomp;
+        st.argmax_abs_err = r.emax < 0.0f ? RKV_NO_INDEX : r.eidx;
+        st.argmax_rel_err = r.qmax < 0.0f ? RKV_NO_INDEX : r.qidx;
+        st.sum_abs_err = r.sum;
+        st.max_abs_err = r.emax < 0.0f ? 0.0f : r.emax;
+        st.max_rel_err = r.qmax < 0.0f ? 0.0f : r.qmax;
+        st.mean_abs_err = st.n_comparable ? (float)(r.sum / (double)st.n_comparable) : 0.0f;
+        st.reserved = 0;
+        const bool has_in = D.input_src != RKV_SRC_NONE;
+        uint32_t flags = 0;
+        if (!(cs.mismatch & 1u)) flags |= RKV_FLAG_CAND_CONST;
+        if (has_in && !(cs.mismatch & 2u)) flags |= RKV_FLAG_CAND_COPY_OF_INPUT;
+        if (!(ref_mismatch & 1u)) flags |= RKV_FLAG_REF_CONST;
+        if (has_in && !(ref_mismatch & 2u)) flags |= RKV_FLAG_REF_COPY_OF_INPUT;
+        if (cs.n_nan) flags |= RKV_FLAG_HAS_NAN;
+        if (cs.n_inf) flags |= RKV_FLAG_HAS_INF;
+        uint32_t verdict = 0;
+        if (r.n_over) verdict |= RKV_FAIL_TOL;
+        if (cs.n_nan) verdict |= RKV_FAIL_NAN;
+        if (cs.n_infmis) verdict |= RKV_FAIL_INF_MISMATCH;
+        if ((flags & RKV_FLAG_CAND_CONST) && !(flags & RKV_FLAG_REF_CONST) && D.n > 1)
+            verdict |= RKV_FAIL_LOOPHOLE_CONST;
+        if ((flags & RKV_FLAG_CAND_COPY_OF_INPUT) && !(flags & RKV_FLAG_REF_COPY_OF_INPUT))
+            verdict |= RKV_FAIL_LOOPHOLE_COPY;
+        st.flags = flags;
+        st.verdict = verdict;
+        stats_out[D.out_base + (unsigned long long)k * D.out_stride] = st;
+        if (verdict) atomicOr(&fail[(size_t)D.case_index * (size_t)K + (size_t)k], 1u);
+    }
+}
+
+// case_pass[c][k] = candidate k passed on every tensor of case c; all_pass[k] = on every case.
+__global__ void joint_kernel(const uint32_t* __restrict__ fail, int K, uint32_t n_cases,
+                             uint32_t* __restrict__ case_pass, uint32_t* __restrict__ all_pass) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    uint32_t all = 1u;
+    for (uint32_t c = 0; c < n_cases; ++c) {
+        const uint32_t ok = fail[(size_t)c * (size_t)K + (size_t)k] ? 0u : 1u;
+        if (case_pass) case_pass[(size_t)c * (size_t)K + (size_t)k] = ok;
+        all &= ok;
+    }
+    if (all_pass) all_pass[k] = all;
 }
 
 }  // namespace
 
-template <bool CB16, bool RB16>
-static int launch_variant(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end, uint32_t n_items,
-                          int grid_max, CandState* state, Partial* partials, WorkspaceHeader* header,
-                          cudaStream_t stream) {
+int launch_verify(const Layout& L, int T, int K, int k_begin, int k_end, uint32_t n_items, uint32_t n_segments,
+                  int grid, cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return RKV_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(verify_kernel<CB16, RB16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
             return RKV_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    // the grid is always the full resident grid: Partial rows are numbered by block
-    verify_kernel<CB16, RB16><<<grid_max, kThreads, kSmemBytes, stream>>>(d_tensors, T, K, k_begin, k_end,
-                                                                         n_items, state, partials, header);
+    Args A;
+    A.tensors = L.d_tensors; A.segments = L.d_segments; A.state = L.state; A.partials = L.partials;
+    A.sums = L.sums; A.header = L.header;
+    A.T = T; A.K = K; A.k_begin = k_begin; A.k_end = k_end; A.n_items = n_items; A.n_segments = n_segments;
+    // the grid is always the full resident grid: Partial rows of large tensors are numbered by block
+    verify_kernel<<<grid, kThreads, kSmemBytes, stream>>>(A);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
-int launch_verify(const DevTensor* d_tensors, int T, int K, int k_begin, int k_end,
-                  const uint32_t variant_items[4], int grid, CandState* state, Partial* partials,
-                  WorkspaceHeader* header, cudaStream_t stream) {
-    int rc = RKV_OK;
-    for (int v = 0; v < 4 && rc == RKV_OK; ++v) {
-        const uint32_t n = variant_items[v];
-        if (!n) continue;
-#define RKV_LAUNCH(CB, RB) \
-    launch_variant<CB, RB>(d_tensors, T, K, k_begin, k_end, n, grid, state, partials, header, stream)
-        switch (v) {
-            case 0: rc = RKV_LAUNCH(false, false); break;
-            case 1: rc = RKV_LAUNCH(false, true); break;
-            case 2: rc = RKV_LAUNCH(true, false); break;
-            default: rc = RKV_LAUNCH(true, true); break;
-        }
-#undef RKV_LAUNCH
+int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,
+                    uint32_t* all_pass, cudaStream_t stream) {
+    finalize_kernel<<<(unsigned)T * (unsigned)K, kFinThreads, 0, stream>>>(L.d_tensors, T, K, L.state, L.partials,
+                                                                          L.sums, stats_out, L.fail);
+    if (cudaGetLastError() != cudaSuccess) return RKV_ERR_CUDA;
+    if (case_pass || all_pass) {
+        joint_kernel<<<(K + 127) / 128, 128, 0, stream>>>(L.fail, K, n_cases, case_pass, all_pass);
+        if (cudaGetLastError() != cudaSuccess) return RKV_ERR_CUDA;
     }
-    return rc;
-}
-
-int launch_finalize(const DevTensor* d_tensors, int T, int K, const CandState* state,
-                    const Partial* partials, rkv_stats* stats_out, uint32_t* joint_pass,
-                    cudaStream_t stream) {
-    finalize_kernel<<<K, kFinThreads, 0, stream>>>(d_tensors, T, K, state, partials, stats_out, joint_pass);
-    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+    return RKV_OK;
 }
 
 }  // namespace rkv

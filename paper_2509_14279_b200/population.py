@@ -194,7 +194,7 @@ def plan_multi(K: int, numels: tuple, seed: int, fault_rate: float) -> list:
 
 
 def _torch_dtype(name: str) -> torch.dtype:
-    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[name]
 
 
 def materialize(cand: Candidate, ref: torch.Tensor, inp: torch.Tensor | None,
@@ -244,7 +244,7 @@ def materialize(cand: Candidate, ref: torch.Tensor, inp: torch.Tensor | None,
 
 
 def bits_numpy(t: torch.Tensor) -> np.ndarray:
-    """A CPU tensor as the numpy array the oracle takes (bf16 -> uint16 bits)."""
+    """A CPU tensor as the numpy array the oracle takes (bf16 -> uint16 bits, fp16 -> float16)."""
     t = t.detach().cpu().contiguous().reshape(-1)
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16)

@@ -45,7 +45,7 @@ def oracle_case(ref_np, cands_np, atol, rtol, input_np=None) -> list:
 
 
 def torch_dtype(code: str):
-    return {"f32": torch.float32, "bf16": torch.bfloat16}[code]
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[code]
 
 
 def oracle_gen_tensor(seed, stream, dist, n, dtype: str) -> torch.Tensor:

@@ -38,11 +38,11 @@ def test_library_exports_every_declared_symbol():
 def test_version_and_status_strings():
     assert rkv.version() >= 100
     seen = set()
-    for code in range(0, -7, -1):
+    for code in range(0, -8, -1):
         s = rkv.status_string(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 7
+    assert len(seen) == 8
     assert rkv.status_string(-99) == "unknown status"
 
 
@@ -54,13 +54,13 @@ def test_stats_struct_is_88_bytes():
 
 
 @pytest.mark.parametrize("K", [1, 2, 8, 63, 64, 65, 128, 256, 1000])
-@pytest.mark.parametrize("n", [1, 127, 3584, 3585, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
-@pytest.mark.parametrize("dtype", [rkv.F32, rkv.BF16])
+@pytest.mark.parametrize("n", [1, 127, 4096, 4097, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
+@pytest.mark.parametrize("dtype", [rkv.F32, rkv.BF16, rkv.F16])
 def test_item_plan_properties(n, K, dtype):
     sms = 148
     grid = 2 * sms
     tile, n_tiles, warm, parts_warm, parts_main, tail, parts_tail = rkv.plan_items(n, K, sms, dtype)
-    assert tile == (3584 if dtype == rkv.F32 else 7168)
+    assert tile == (4096 if dtype == rkv.F32 else 8192)
     assert (n_tiles - 1) * tile < n <= n_tiles * tile
     assert 1 <= warm <= n_tiles
     assert 1 <= parts_warm <= K and -(-K // parts_warm) <= 64
@@ -123,7 +123,8 @@ def test_verify_multi_validates_before_any_cuda_call():
         (dict(atol=float("nan")), rkv.ERR_INVALID_ARG),
         (dict(rtol=float("inf")), rkv.ERR_INVALID_ARG),
         (dict(atol=-1e-5), rkv.ERR_INVALID_ARG),
-        (dict(cand_dtype=2), rkv.ERR_INVALID_ARG),
+        (dict(cand_dtype=3), rkv.ERR_INVALID_ARG),
+        (dict(ref_src=2, ref_dtype=2), rkv.ERR_UNSUPPORTED),      # no fp16 rounding in the generator
         (dict(ref_dtype=-1), rkv.ERR_INVALID_ARG),
         (dict(ref_src=0), rkv.ERR_INVALID_ARG),
         (dict(ref_src=2, ref_dist=9), rkv.ERR_INVALID_ARG),
@@ -144,6 +145,40 @@ def test_verify_multi_validates_before_any_cuda_call():
                                       ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_UNSUPPORTED
     assert rkv.lib().rkv_verify_multi(None, 1, 1, ctypes.c_void_p(0x3000), None,
                                       ctypes.c_void_p(0x4000), 1 << 30, None) == rkv.ERR_INVALID_ARG
+
+
+def test_sweep_validates_before_any_cuda_call():
+    L = rkv.lib()
+    d, keep = _desc()
+    arr = (rkv.TensorDescC * 1)(d)
+
+    def call(cases, C, K=1, stats=0x3000, ws=0x4000, ws_bytes=1 << 30):
+        return L.rkv_verify_sweep(cases, C, K, ctypes.c_void_p(stats), None, None, ctypes.c_void_p(ws), ws_bytes, None)
+
+    one = (rkv.CaseDescC * 1)()
+    one[0].tensors = ctypes.cast(arr, ctypes.POINTER(rkv.TensorDescC))
+    one[0].T = 1
+    assert call(None, 1) == rkv.ERR_INVALID_ARG
+    assert call(one, 0) == rkv.ERR_INVALID_ARG
+    assert call(one, 1, K=0) == rkv.ERR_INVALID_ARG
+    assert call(one, 1, stats=0) == rkv.ERR_INVALID_ARG
+    assert call(one, 1, ws=0) == rkv.ERR_WORKSPACE
+    assert call(one, 1, ws=0x4010) == rkv.ERR_ALIGNMENT
+    one[0].T = 0
+    assert call(one, 1) == rkv.ERR_INVALID_ARG
+    one[0].T = 65
+    assert call(one, 1) == rkv.ERR_UNSUPPORTED
+    one[0].T = 1
+    many = (rkv.CaseDescC * 4097)()
+    for i in range(4097):
+        many[i].tensors = ctypes.cast(arr, ctypes.POINTER(rkv.TensorDescC))
+        many[i].T = 1
+    assert call(many, 4097) == rkv.ERR_UNSUPPORTED                 # more than 4096 tensors over all cases
+    bad, keep2 = _desc(ref=0x1004)
+    arr2 = (rkv.TensorDescC * 1)(bad)
+    one[0].tensors = ctypes.cast(arr2, ctypes.POINTER(rkv.TensorDescC))
+    assert call(one, 1) == rkv.ERR_ALIGNMENT
+    assert L.rkv_sweep_workspace_bytes(None, 1, 1) == 0
 
 
 def test_gen_and_batch_validate_before_any_cuda_call():
@@ -230,7 +265,7 @@ def test_binding_refuses_mismatched_tensors_before_the_c_call():
         rkv._require_case(ref, [good.to(torch.bfloat16)], "t", device_type="cpu")
     with pytest.raises(ValueError, match="not contiguous"):
         rkv._require_case(ref, [torch.zeros(2048)[::2]], "t", device_type="cpu")
-    with pytest.raises(TypeError, match="float32 or bfloat16"):
+    with pytest.raises(TypeError, match="float32, bfloat16 or float16"):
         rkv._require_case(ref.double(), [good.double()], "t", device_type="cpu")
     with pytest.raises(ValueError, match="no candidates"):
         rkv._require_case(ref, [], "t", device_type="cpu")

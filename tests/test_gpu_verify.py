@@ -81,12 +81,12 @@ def test_many_candidates_cross_the_merge_chunk_and_hint_limits(K):
 def test_several_tiles_per_block_in_one_part(cand_dtype):
     """More tiles than resident blocks: a block meets the same candidates tile after tile,
     carries its running maxima over, and uses the maxima other blocks have published."""
-    n = 3584 * 296 * 2 + 3584 * 40 + 1234
+    n = 4096 * 296 * 2 + 4096 * 40 + 1234
     ref = oracle_gen_tensor(77, 0, oracle.NORMAL, n, "f32")
     inp = oracle_gen_tensor(77, 2, oracle.NORMAL, n, cand_dtype)
     plan = mixed_plan(12, n, seed=77, bf16=cand_dtype == "bf16")
     # equal maxima far apart: the first index must win across blocks and tiles
-    plan.append(pop.Candidate(pop.CORRUPT, delta=1.0, indices=(n - 5, n // 2, 3584 * 300 + 17)))
+    plan.append(pop.Candidate(pop.CORRUPT, delta=1.0, indices=(n - 5, n // 2, 4096 * 300 + 17)))
     cands = build_case_cpu(plan, ref, inp, cand_dtype)
     tol = (1e-5, 1e-5) if cand_dtype == "f32" else (1e-2, 1.6e-2)
     check_case(ref, cands, tol[0], tol[1], inp, where=f"multi-tile {cand_dtype}")
@@ -97,7 +97,7 @@ def test_large_tensor_with_a_warm_up_group(cand_dtype):
     """A tensor large enough to be cut into a leading group of tiles (verified first, by all
     blocks), the bulk, and a tail group of short items (its last tiles, verified last): results
     must not depend on which group an element falls in."""
-    tile = 7168               # the larger of the two tile sizes: both dtypes get a second group
+    tile = 8192               # the larger of the two tile sizes: both dtypes get a second group
     n = tile * 2100 + 77
     ref = oracle_gen_tensor(88, 0, oracle.STUDENT_T2, n, "f32")
     inp = oracle_gen_tensor(88, 2, oracle.STUDENT_T2, n, cand_dtype)
@@ -108,7 +108,7 @@ def test_large_tensor_with_a_warm_up_group(cand_dtype):
         pop.Candidate(pop.CORRUPT, delta=1.0, indices=(tile * 5 + 3, tile * 18 + 1, n - 2)),
         # the only error lies behind the leading group
         pop.Candidate(pop.CORRUPT, delta=1.0, indices=(tile * 1000 + 11,)),
-        pop.Candidate(pop.NAN_AT, indices=(tile * 17 + 3583,)),
+        pop.Candidate(pop.NAN_AT, indices=(tile * 17 + 4095,)),
         pop.Candidate(pop.INF_AT, indices=(n - 1,)),
         pop.Candidate(pop.INPUT_COPY),
         pop.Candidate(pop.CONST, value=0.5),
@@ -160,7 +160,7 @@ def test_bf16_candidates_at_the_edges_of_the_skip_tests(atol, rtol):
     """Errors proportional to |r| around rtol, reference zeros with errors around atol,
     values so small that e - t*|r| underflows, exact copies, equal quotients in every
     tile, quotients that overflow: everything the bf16 path decides from a sign test."""
-    n = 7168 * 5 + 100
+    n = 8192 * 5 + 100
     bf = torch.bfloat16
     ref = oracle_gen_tensor(77, 0, oracle.NORMAL, n, "f32")
     inp = oracle_gen_tensor(77, 2, oracle.NORMAL, n, "bf16")
@@ -328,11 +328,11 @@ def test_host_buffer_form(dtype):
 def test_host_buffer_form_on_a_tensor_with_all_three_item_groups():
     """Chunks of candidates (16, then the rest) over a tensor long enough for the warm-up
     and the tail group; a ragged last tile."""
-    n, K = 3584 * 2100 + 5, 20
+    n, K = 4096 * 2100 + 5, 20
     ref = oracle_gen_tensor(8, 0, oracle.UNIFORM_PM1, n, "f32")
     plan = mixed_plan(K, n, seed=8)
     plan[17] = pop.Candidate(pop.CORRUPT, delta=1.0, indices=(n - 1,))
-    plan[3] = pop.Candidate(pop.NAN_AT, indices=(3584 * 2050 + 7,))
+    plan[3] = pop.Candidate(pop.NAN_AT, indices=(4096 * 2050 + 7,))
     cands = build_case_cpu(plan, ref, ref, "f32")
     got = rkv.verify_batch_host(ref, cands, ATOL, RTOL)
     want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], ATOL, RTOL)
@@ -345,7 +345,7 @@ def test_host_buffer_form_of_the_general_case():
     """rkv_verify_multi_host: an fp32 tensor read from host memory (reference and input) next to
     a bf16 tensor whose reference and input are regenerated on the device; more candidates than
     one chunk holds, so the partial results carry over between the chunk launches."""
-    n32, n16, K = 3584 * 40 + 3, 7168 * 33 + 5, 37
+    n32, n16, K = 4096 * 40 + 3, 8192 * 33 + 5, 37
     ref32 = oracle_gen_tensor(21, 0, oracle.NORMAL, n32, "f32")
     inp32 = oracle_gen_tensor(21, 2, oracle.NORMAL, n32, "f32")
     ref16 = oracle_gen_tensor(21, 1 << 32, oracle.UNIFORM_PM1, n16, "f32")
@@ -429,7 +429,7 @@ def test_seeded_random_cases_match_the_oracle(case):
     """Sizes, candidate counts, dtypes, distributions and tolerances drawn from a seeded
     generator: every statistic of every candidate against the oracle."""
     rng = np.random.default_rng([2509, case])
-    n = int(rng.choice([1, 2, 7, 33, 1000, 3583, 3584, 3585, 7168, 7169, 20000, 65537, 200003, 1048577]))
+    n = int(rng.choice([1, 2, 7, 33, 1000, 4095, 4096, 4097, 8192, 8193, 20000, 65537, 200003, 1048577]))
     if case % 6 == 5:
         n = int(rng.integers(1, 300000))
     K = int(rng.choice([1, 2, 3, 12, 13, 31, 64, 65, 70]))

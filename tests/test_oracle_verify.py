@@ -324,3 +324,39 @@ def test_config1_population_verdicts():
     assert res[5]["verdict"] == FAIL_TOL | FAIL_LOOPHOLE_CONST
     assert res[6]["max_abs_err"] == 0.0
     assert res[7]["verdict"] == FAIL_TOL and res[7]["max_rel_err"] == pytest.approx(1e-3, rel=1e-3)
+
+
+def test_fp16_widening_is_exact_for_every_pattern():
+    """orc_f16_to_f32_bits against numpy's float16 -> float32 conversion, all 65536 patterns
+    (NaN payloads included: both keep the ten fraction bits in the top of the fp32 fraction)."""
+    h = np.arange(65536, dtype=np.uint16)
+    want = h.view(np.float16).astype(np.float32).view(np.uint32)
+    got = np.array([oracle.f16_to_f32_bits(int(x)) for x in h], dtype=np.uint32)
+    nan = np.isnan(h.view(np.float16))
+    assert np.array_equal(got[~nan], want[~nan])
+    # NaNs: same sign, exponent all ones, the half's payload bits kept (numpy may set the quiet bit)
+    assert np.all((got[nan] & 0x7F800000) == 0x7F800000) and np.all((got[nan] & 0x007FFFFF) != 0)
+    assert np.array_equal(got[nan] & 0x80000000, want[nan] & 0x80000000)
+    assert np.array_equal((got[nan] | 0x00400000), (want[nan] | 0x00400000))
+
+
+def test_fp16_candidates_follow_the_same_rule():
+    """An fp16 candidate is compared as its exact fp32 value: the result equals verifying the
+    widened candidate as an fp32 tensor (the flags compare storage bits, which the widening
+    keeps distinct)."""
+    rng = np.random.default_rng(16)
+    n = 4099
+    ref = rng.standard_normal(n).astype(np.float32)
+    c16 = (ref * (1 + rng.uniform(-1, 1, n) * 2.0 ** -11)).astype(np.float16)
+    c16[7] = np.float16(np.nan)
+    c16[100] = np.float16(np.inf)
+    c16[200] = np.float16(6.1e-5) * np.float16(0.01)          # a subnormal half
+    a = oracle.verify(ref, c16, 1e-3, 1e-3)
+    b = oracle.verify(ref, c16.astype(np.float32), 1e-3, 1e-3)
+    assert a == b
+    assert a["n_nan"] == 1 and a["n_inf"] == 1 and a["n_comparable"] == n - 2
+    # an fp16 reference and an fp16 input as well
+    r16 = ref.astype(np.float16)
+    a = oracle.verify(r16, c16, 1e-3, 1e-3, input=c16)
+    b = oracle.verify(r16.astype(np.float32), c16.astype(np.float32), 1e-3, 1e-3, input=c16.astype(np.float32))
+    assert a == b and a["flags"] & oracle.CAND_COPY_OF_INPUT
