@@ -380,6 +380,10 @@ int rkv_debug_bounds_build(void) {
 #endif
 }
 
+// Not part of the public interface: resident verification blocks per SM on the current
+// device (the kernel is written for kBlocksPerSm = 2).
+int rkv_debug_occupancy(void) { return verify_occupancy(); }
+
 int rkv_plan_items(uint64_t n, int cand_dtype, int K, int num_sms, uint32_t* tile_elems_out, uint32_t* n_tiles,
                    uint32_t* warm_tiles, uint32_t* parts_warm, uint32_t* parts_main, uint32_t* tail_tiles,
                    uint32_t* parts_tail) {

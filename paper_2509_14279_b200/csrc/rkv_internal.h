@@ -216,6 +216,7 @@ struct Layout {
 // kernels (rkv_verify.cu / rkv_gen.cu)
 int launch_verify(const Layout& L, int T, int K, int k_begin, int k_end, uint32_t n_items, uint32_t n_segments,
                   int grid, cudaStream_t stream);
+int verify_occupancy();   // resident verification blocks per SM on the current device
 int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,
                     uint32_t* all_pass, cudaStream_t stream);
 int launch_gen(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t first_elem,

@@ -12,13 +12,16 @@
 // All eight warps of a block compare.  A thread owns 64 bytes of every candidate tile (16
 // fp32 or 32 16-bit elements); it keeps their reference values (and, for fp32 candidates,
 // the tolerance thresholds) IN REGISTERS for the whole item and meets every candidate tile
-// as it lands in a ring of shared-memory stages.  One lane of the last warp also feeds that
-// ring: between its own comparisons it issues the bulk asynchronous copies
-// (cp.async.bulk, completion counted on an mbarrier) that bring, for an item, the reference
-// tile and then the same tile of every candidate of the part.  It runs up to a ring's depth
-// ahead of the comparison, across item boundaries, so that copies are always in flight.  (A
-// warp that only issued copies would leave its scheduler half idle: with 128 registers a
-// thread, 16 warps fill an SM, and this way all 16 compare.)
+// as it lands in a ring of shared-memory stages.  The ring is fed by whoever frees a stage:
+// a warp that has read its 2 KB of a stage counts itself off on the stage, and the warp that
+// counts off last issues, there and then, the bulk asynchronous copy (cp.async.bulk,
+// completion counted on an mbarrier) that refills the stage.  What to copy it reads from a
+// queue of copy descriptors -- for an item the reference tile, then the same tile of every
+// candidate of the part, then on to the next item -- that the block's last warp writes one
+// item ahead, while the other warps fetch the item's hints.  Issuing a copy is a dozen
+// instructions, a full ring of copies is always in flight, across item boundaries, and no
+// warp is set aside to issue them.  (With 128 registers a thread, 16 warps fill an SM; a
+// warp that only issued copies would leave its scheduler half idle.)
 //
 // Candidate bytes are read from HBM exactly once; the reference once per part.
 // When the reference is "generated" the threads regenerate their values from
@@ -52,7 +55,9 @@ namespace {
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr float kInf = __builtin_huge_valf();
 enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the issuer's "no more items" mark
-constexpr int kInfoRing = 8;                   // items in flight per block (> kStages: an item uses >= 1 stage)
+constexpr int kInfoRing = 16;                  // item descriptions kept per block (> kStages + 4: an item uses >= 1 stage)
+constexpr int kDescRing = 256;                 // copy descriptors kept per block (> two items of kPartK + 2 copies)
+constexpr uint32_t kLead = kStages + 2;        // descriptors are prepared this far past the end of the current item
 constexpr long long kWaitCycles = 2000000000LL;
 
 // ----------------------------------------------------------------------------
@@ -109,37 +114,44 @@ struct __align__(16) ItemInfo {
 };
 static_assert(sizeof(ItemInfo) == 32, "ItemInfo layout");
 
-// State of the issuing lane (only that lane touches it).
-struct __align__(16) IssuerState {
-    uint32_t n_issued;       // copies issued so far
-    uint32_t stage, phase;   // ring stage of the next copy and the parity its empty barrier must have passed
-    uint32_t pos, end, nref; // next copy of the current item: [0, nref) reference stages, [nref, end) candidates
-    uint32_t done;
-    uint32_t ord;            // items started so far
-    uint32_t cbytes, rbytes; // bytes copied per candidate tile / of the reference tile
-    uint32_t seg;            // segment the last item was found in
-    uint32_t next_id;        // the item after the current one (a ticket drawn one item ahead)
-    uint32_t drill;          // fault drill: number of the copy to withhold (0: none)
-    uint32_t reserved[3];
-    unsigned long long c_off;          // byte offset of the tile in every candidate
-    const unsigned char* ref_src;      // the tile in the stored reference
+// One bulk copy of the schedule: copy number j of a block goes to ring stage j % kStages.
+struct __align__(16) CopyDesc {
+    const unsigned char* src;
+    uint32_t bytes;          // 0: nothing to copy (an empty tile piece): the stage is armed and completes at once
+    uint32_t withhold;       // fault drill of a test: arm the stage, do not issue the copy
 };
-static_assert(sizeof(IssuerState) == 80, "IssuerState layout");
+static_assert(sizeof(CopyDesc) == 16, "CopyDesc layout");
+
+// The schedule of a block: which items it takes and the copies they need.  Lane 0 of the
+// preparing warp writes it; the warps that refill stages only read q_end.
+struct __align__(16) Schedule {
+    uint32_t q_end;          // copies described so far: numbers [0, q_end)
+    uint32_t ord;            // items described so far
+    uint32_t next_id;        // launch-wide id of the next item (a ticket drawn one item ahead)
+    uint32_t seg;            // segment the last item was found in
+    uint32_t done;           // the end of the item list has been reached
+    uint32_t drill;          // fault drill: number (1-based) of the copy to withhold, 0: none
+    uint32_t reserved[2];
+};
+static_assert(sizeof(Schedule) == 32, "Schedule layout");
 
 constexpr int kOffFull = 0;                                   // kStages mbarriers
-constexpr int kOffEmpty = kOffFull + 8 * kStages;
-constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
+constexpr int kOffRelease = kOffFull + 8 * kStages;           // kStages x uint32: warps that have read the stage
+constexpr int kOffIssued = kOffRelease + 4 * kStages;         // kStages x uint32: 1 + number of the last copy issued into the stage
+constexpr int kOffAbort = kOffIssued + 4 * kStages;           // uint32
 constexpr int kOffRefState = kOffAbort + 8;                   // 2 x uint32 settled bits of the reference (item parity)
 constexpr int kOffWaitLimit = kOffRefState + 8;               // long long: cycles a wait may take
-constexpr int kOffIssuer = 128;
-constexpr int kOffInfo = kOffIssuer + 96;
-constexpr int kOffPtrC = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);   // the comparing threads' copy of the pointers
-constexpr int kOffPtrP = kOffPtrC + kPartK * 8;                          // the issuer's copies, one per item in flight
-constexpr int kOffHint = kOffPtrP + kInfoRing * kPartK * 8;              // two tables (item parity)
+constexpr int kOffSchedule = 128;
+constexpr int kOffInfo = kOffSchedule + (int)sizeof(Schedule);
+constexpr int kOffDesc = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);
+constexpr int kOffPtrC = kOffDesc + kDescRing * (int)sizeof(CopyDesc);   // the part's candidate pointers
+constexpr int kOffHint = kOffPtrC + kPartK * 8;                          // two tables (item parity)
 constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
 constexpr int kOffStage = (kOffRec + kWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
-static_assert(kOffWaitLimit + 8 <= kOffIssuer && sizeof(IssuerState) <= 96, "layout");
+static_assert(kOffWaitLimit + 8 <= kOffSchedule, "layout");
+static_assert(kDescRing >= 2 * (kPartK + 2) + (int)kLead && (kDescRing & (kDescRing - 1)) == 0, "descriptor ring");
+static_assert(kInfoRing >= (int)kLead + 3 && (kInfoRing & (kInfoRing - 1)) == 0, "item ring");
 static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
 // Candidate storage kinds the comparison is compiled for.
@@ -199,6 +211,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
         : "r"(mbar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+
+// Count one more warp off a stage (release: the warp's reads of the stage come first;
+// acquire: the warp that counts off last may overwrite it).  Returns the count before.
+__device__ __forceinline__ uint32_t count_off(uint32_t addr) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(addr) : "memory");
+    return old;
 }
 
 // What every wait of a block shares: the flag that says "a wait ran out, drain" and the
@@ -285,8 +305,9 @@ struct Args {
 // the issuing lane: feeds the ring
 // ----------------------------------------------------------------------------
 struct Ring {
-    uint32_t full0, empty0;      // shared-memory addresses of the first full / empty mbarrier
-    uint32_t stage0;             // shared-memory address of stage 0
+    uint32_t full0;              // shared-memory address of the first full mbarrier
+    uint32_t release0;           // ... of the first release counter
+    uint32_t stage0;             // ... of stage 0
     WaitCtl ctl;
 };
 
@@ -322,90 +343,115 @@ __device__ __forceinline__ bool decode_item(const Args& A, uint32_t id, uint32_t
     return true;
 }
 
-// Start the next item: draw a ticket for the one after it, decode, copy the part's pointers
-// into the item's table, publish the item's description.  At the end of the list the item
-// published is the end mark.
-__device__ __noinline__ void issuer_next_item(const Args& A, unsigned char* smem) {
-    IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
-    const uint32_t id = st->next_id;
-    const uint32_t slot = st->ord & (kInfoRing - 1);
-    // the ticket for the item after this one; its latency hides behind the set-up below
-    uint32_t ticket = 0;
-    if (id < A.n_items) ticket = atomicAdd(&A.header->next_ticket, 1u);
-    ItemInfo info;
-    info.id = kNoItem; info.t = 0; info.tile = 0; info.k0 = 0; info.kc = 0;
-    info.reserved[0] = info.reserved[1] = info.reserved[2] = 0;
-    uint32_t seg = st->seg;
-    st->pos = 0; st->nref = 0; st->end = 1; st->cbytes = 0; st->rbytes = 0;     // the end mark: one empty "copy"
-    if (decode_item(A, id, seg, info)) {
-        const DevTensor& D = A.tensors[info.t];
-        const uint32_t csz = elem_bytes(D.cand_dtype), rsz = elem_bytes(D.ref_dtype);
-        const uint32_t te = tile_elems(D.cand_dtype);
-        const uint64_t start = (uint64_t)info.tile * te;
-        const uint32_t len = (uint32_t)min((uint64_t)te, D.n - start);
-        st->cbytes = (len * csz) & ~15u;
-        st->c_off = start * csz;
-        uint32_t nref = 0;
-        if (D.ref_src == RKV_SRC_POINTER) {
-            nref = (te * rsz + kStageBytes - 1) / kStageBytes;
-            st->rbytes = (len * rsz) & ~15u;
-            st->ref_src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
+// Describe further items, whole items at a time, until the copies described reach past copy
+// number `target` or the item list ends.  Per item: draw the ticket for the one after it,
+// decode, publish its description for the comparing threads, and queue its copies -- the
+// reference tile (one or two stages) and the tile of every candidate of the part.  The whole
+// warp calls this: lane 0 keeps the schedule, all lanes fetch the candidates' pointers (one
+// round trip to memory instead of one per candidate).
+__device__ __forceinline__ void prepare_items(const Args& A, unsigned char* smem, uint32_t target, int lane) {
+    Schedule* sc = reinterpret_cast<Schedule*>(smem + kOffSchedule);
+    CopyDesc* desc = reinterpret_cast<CopyDesc*>(smem + kOffDesc);
+    for (int guard = 0; guard < kInfoRing; ++guard) {
+        uint32_t go = 0;
+        if (lane == 0) go = (!sc->done && sc->q_end <= target) ? 1u : 0u;
+        if (!__shfl_sync(kFullMask, go, 0)) break;
+        uint32_t t = 0, k0 = 0, kc = 0, q = 0, cbytes = 0, off_lo = 0, off_hi = 0, ticket = 0;
+        if (lane == 0) {
+            const uint32_t id = sc->next_id;
+            // the ticket for the item after this one; its latency hides behind the decoding
+            if (id < A.n_items) ticket = atomicAdd(&A.header->next_ticket, 1u);
+            ItemInfo info;
+            info.id = kNoItem; info.t = 0; info.tile = 0; info.k0 = 0; info.kc = 0;
+            info.reserved[0] = info.reserved[1] = info.reserved[2] = 0;
+            uint32_t seg = sc->seg;
+            q = sc->q_end;
+            if (decode_item(A, id, seg, info)) {
+                const DevTensor& D = A.tensors[info.t];
+                const uint32_t csz = elem_bytes(D.cand_dtype), rsz = elem_bytes(D.ref_dtype);
+                const uint32_t te = tile_elems(D.cand_dtype);
+                const uint64_t start = (uint64_t)info.tile * te;
+                const uint32_t len = (uint32_t)min((uint64_t)te, D.n - start);
+                cbytes = (len * csz) & ~15u;
+                const uint64_t c_off = start * csz;
+                off_lo = (uint32_t)c_off; off_hi = (uint32_t)(c_off >> 32);
+                if (D.ref_src == RKV_SRC_POINTER) {
+                    const uint32_t nref = (te * rsz + kStageBytes - 1) / kStageBytes;
+                    const uint32_t rbytes = (len * rsz) & ~15u;
+                    const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
+                    for (uint32_t r = 0; r < nref; ++r, ++q) {
+                        const uint32_t lo = r * kStageBytes;
+                        CopyDesc d;
+                        d.src = src + lo;
+                        d.bytes = rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u;
+                        d.withhold = q + 1u == sc->drill ? 1u : 0u;
+                        desc[q & (kDescRing - 1)] = d;
+                    }
+                }
+                t = info.t; k0 = info.k0; kc = info.kc;
+            } else {
+                sc->done = 1u;                      // the description with kNoItem ends the block's list
+            }
+            sc->seg = seg;
+            reinterpret_cast<ItemInfo*>(smem + kOffInfo)[sc->ord & (kInfoRing - 1)] = info;
         }
-        st->nref = nref;
-        st->end = nref + info.kc;
-        const void** table = reinterpret_cast<const void**>(smem + kOffPtrP) + slot * kPartK;
-        for (uint32_t i = 0; i < info.kc; ++i) table[i] = D.cands[info.k0 + i];
-    } else {
-        st->done = 2u;                              // the end mark is the last thing to issue
+        t = __shfl_sync(kFullMask, t, 0);
+        k0 = __shfl_sync(kFullMask, k0, 0);
+        kc = __shfl_sync(kFullMask, kc, 0);
+        q = __shfl_sync(kFullMask, q, 0);
+        cbytes = __shfl_sync(kFullMask, cbytes, 0);
+        off_lo = __shfl_sync(kFullMask, off_lo, 0);
+        off_hi = __shfl_sync(kFullMask, off_hi, 0);
+        if (kc) {
+            const void* const* src = A.tensors[t].cands + k0;
+            const unsigned long long c_off = ((unsigned long long)off_hi << 32) | off_lo;
+            const uint32_t drill = sc->drill;
+            for (uint32_t i = (uint32_t)lane; i < kc; i += 32u) {
+                CopyDesc d;
+                d.src = reinterpret_cast<const unsigned char*>(src[i]) + c_off;
+                d.bytes = cbytes;
+                d.withhold = q + i + 1u == drill ? 1u : 0u;
+                desc[(q + i) & (kDescRing - 1)] = d;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence_block();
+            sc->q_end = q + kc;
+            sc->ord += 1u;
+            sc->next_id = gridDim.x + ticket;
+        }
+        __syncwarp();
     }
-    st->seg = seg;
-    reinterpret_cast<ItemInfo*>(smem + kOffInfo)[slot] = info;
-    st->next_id = gridDim.x + ticket;
 }
 
-// Issue copies while ring stages are free; make sure copy number `need` has been issued
-// when this returns (waiting, bounded, for its stage if it has to).  Called by one lane.
-__device__ __forceinline__ void issuer_pump(const Args& A, unsigned char* smem, const Ring& ring, uint32_t need) {
-    IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
-    for (;;) {
-        if (st->done == 1u) return;
-        const uint32_t n = st->n_issued, s = st->stage, ph = st->phase;
-        // the stage is free once every warp has released its previous use
-        if (!mbar_try_wait(ring.empty0 + 8 * s, ph ^ 1u)) {
-            if ((int32_t)(n - need) > 0) return;                       // nobody is waiting for this copy yet
-            if (!mbar_wait_slow(ring.empty0 + 8 * s, ph ^ 1u, ring.ctl)) { st->done = 1u; return; }
+// Issue copy number j of the block's schedule into its ring stage, if it has been described
+// (beyond the end of the item list nothing is).  One lane calls this.
+__device__ __forceinline__ void issue_copy(unsigned char* smem, const Ring& ring, uint32_t j, uint32_t s) {
+    const volatile Schedule* sc = reinterpret_cast<const volatile Schedule*>(smem + kOffSchedule);
+    if (j >= sc->q_end) return;
+    const CopyDesc d = reinterpret_cast<const CopyDesc*>(smem + kOffDesc)[j & (kDescRing - 1)];
+    const uint32_t full = ring.full0 + 8 * s;
+    reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s] = j + 1u;
+    if (d.bytes) {
+        mbar_expect_tx(full, d.bytes);
+        if (!d.withhold) bulk_g2s(ring.stage0 + s * kStageBytes, d.src, d.bytes, full);
+    } else {
+        mbar_arrive(full);
+    }
+}
+
+// A warp has read ring stage `s` for the stage use number `use` (uses are numbered in the
+// order the schedule fills the ring, so use j sits in stage j % kStages).  The warp that
+// counts off last refills the stage with copy number use + kStages.
+__device__ __forceinline__ void release_stage(unsigned char* smem, const Ring& ring, uint32_t s, uint32_t use,
+                                              int lane) {
+    __syncwarp();
+    if (lane == 0) {
+        if (count_off(ring.release0 + 4 * s) == (uint32_t)kWarps - 1u) {
+            reinterpret_cast<volatile uint32_t*>(smem + kOffRelease)[s] = 0u;
+            issue_copy(smem, ring, use + (uint32_t)kStages, s);
         }
-        if (st->pos == st->end) {
-            if (st->done == 2u || *ring.ctl.abort_flag) { st->done = 1u; return; }
-            issuer_next_item(A, smem);
-            st->ord += 1u;
-        }
-        const uint32_t pos = st->pos;
-        const uint32_t full = ring.full0 + 8 * s;
-        const unsigned char* src;
-        uint32_t bytes;
-        if (pos < st->nref) {
-            const uint32_t lo = pos * kStageBytes;
-            bytes = st->rbytes > lo ? min(st->rbytes - lo, (uint32_t)kStageBytes) : 0u;
-            src = st->ref_src + lo;
-        } else {
-            const void* const* table = reinterpret_cast<const void* const*>(smem + kOffPtrP) +
-                                       ((st->ord - 1u) & (kInfoRing - 1)) * kPartK;
-            bytes = st->cbytes;
-            src = reinterpret_cast<const unsigned char*>(table[pos - st->nref]) + st->c_off;
-        }
-        // the fault drill of a test: arm the stage, withhold the copy
-        const bool withhold = n + 1u == st->drill;
-        if (bytes) {
-            mbar_expect_tx(full, bytes);
-            if (!withhold) bulk_g2s(ring.stage0 + s * kStageBytes, src, bytes, full);
-        } else {
-            mbar_arrive(full);
-        }
-        st->pos = pos + 1u;
-        st->n_issued = n + 1u;
-        if (s + 1u == (uint32_t)kStages) { st->stage = 0u; st->phase = ph ^ 1u; }
-        else st->stage = s + 1u;
     }
 }
 
@@ -1072,16 +1118,10 @@ struct BlockState {
     uint32_t cstage, cphase;     // next ring stage to consume and the parity of its current use
     uint32_t ccount;             // stages consumed so far (= the number of the next copy to wait for)
     uint32_t ord;                // items this block has started
-    bool is_issuer;              // this warp's lane 0 issues the copies
 };
 
-// Wait for the next ring stage; the issuing lane first makes sure its copy is on the way.
-__device__ __forceinline__ bool wait_stage(const Args& A, unsigned char* smem, const Ring& ring, BlockState& B,
-                                           int lane, uint32_t& stage_out) {
-    if (B.is_issuer) {
-        if (lane == 0) issuer_pump(A, smem, ring, B.ccount);
-        __syncwarp();
-    }
+// Wait for the next ring stage.
+__device__ __forceinline__ bool wait_stage(const Ring& ring, const BlockState& B, uint32_t& stage_out) {
     stage_out = B.cstage;
     return mbar_wait(ring.full0 + 8 * B.cstage, B.cphase, ring.ctl);
 }
@@ -1113,6 +1153,13 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
     CandState* st_t = A.state + D.state_base;
 
+    // the last warp describes the copies that will be issued while this item is compared: up
+    // to kLead copies past the item's own (the item's copies were described one item ago)
+    if (warp == kWarps - 1) {
+        const uint32_t nref = D.ref_src == RKV_SRC_POINTER
+                                  ? (kTile * elem_bytes(D.ref_dtype) + kStageBytes - 1) / kStageBytes : 0u;
+        prepare_items(A, smem, B.ccount + nref + (uint32_t)kc - 1u + kLead, lane);
+    }
     // the part's pointers and hints, from the published state
     if (tid < kc) {
         const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
@@ -1135,17 +1182,17 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
         // the reference tile fills one ring stage, or two (fp32 under 16-bit candidates)
         const bool two = (kTile * elem_bytes(D.ref_dtype)) > (uint32_t)kStageBytes;
         uint32_t sa, sb;
-        wait_stage(A, smem, ring, B, lane, sa);
+        const uint32_t use_a = B.ccount;
+        wait_stage(ring, B, sa);
         advance_stage(B);
         sb = sa;
         if (two) {
-            wait_stage(A, smem, ring, B, lane, sb);
+            wait_stage(ring, B, sb);
             advance_stage(B);
         }
         load_ref<CK>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes, stages + (size_t)sb * kStageBytes, tid);
-        __syncwarp();
-        mbar_arrive_if(ring.empty0 + 8 * sa, lane == 0);
-        if (two) mbar_arrive_if(ring.empty0 + 8 * sb, lane == 0);
+        release_stage(smem, ring, sa, use_a, lane);
+        if (two) release_stage(smem, ring, sb, use_a + 1u, lane);
     } else {
         load_ref<CK>(R, rb, D, start, len, nullptr, nullptr, tid);
     }
@@ -1182,7 +1229,7 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     for (int kk = 0; kk < kc; ++kk) {
         const Hint h = H[kk];
         uint32_t s;
-        wait_stage(A, smem, ring, B, lane, s);
+        wait_stage(ring, B, s);
         const unsigned char* stage = stages + (size_t)s * kStageBytes;
         uint32_t w[NW];
 #pragma unroll
@@ -1190,8 +1237,7 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
             const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kThreads + tid) * 16);
             w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
         }
-        __syncwarp();
-        mbar_arrive_if(ring.empty0 + 8 * s, lane == 0);
+        release_stage(smem, ring, s, B.ccount, lane);
         advance_stage(B);
         if (len != kTile) {
             // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
@@ -1220,12 +1266,12 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
 }
 
 // Persistent blocks, kBlocksPerSm per SM.
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Args A) {
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __grid_constant__ Args A) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     Ring ring;
     ring.full0 = smem_u32(smem + kOffFull);
-    ring.empty0 = smem_u32(smem + kOffEmpty);
+    ring.release0 = smem_u32(smem + kOffRelease);
     ring.stage0 = smem_u32(smem + kOffStage);
     ring.ctl.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
     ring.ctl.limit = reinterpret_cast<const volatile long long*>(smem + kOffWaitLimit);
@@ -1233,16 +1279,16 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Ar
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(ring.full0 + 8 * s, 1);             // the issuer's arrive + the copy's bytes
-            mbar_init(ring.empty0 + 8 * s, kWarps);       // one release per warp
+            reinterpret_cast<volatile uint32_t*>(smem + kOffRelease)[s] = 0u;
+            reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s] = 0u;
         }
         *ring.ctl.abort_flag = 0u;
         const unsigned long long lim = A.header->drill_issue ? A.header->drill_wait_cycles : 0ull;
         *reinterpret_cast<volatile long long*>(smem + kOffWaitLimit) = lim ? (long long)lim : kWaitCycles;
-        IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
-        st->n_issued = 0; st->stage = 0; st->phase = 0; st->pos = 0; st->end = 0; st->nref = 0; st->done = 0;
-        st->ord = 0; st->cbytes = 0; st->rbytes = 0; st->seg = 0; st->c_off = 0; st->ref_src = nullptr;
-        st->next_id = blockIdx.x;             // every block starts with the item of its own number
-        st->drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
+        Schedule* sc = reinterpret_cast<Schedule*>(smem + kOffSchedule);
+        sc->q_end = 0; sc->ord = 0; sc->seg = 0; sc->done = 0; sc->reserved[0] = sc->reserved[1] = 0;
+        sc->next_id = blockIdx.x;             // every block starts with the item of its own number
+        sc->drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // clear the records once; the flushes leave them cleared
@@ -1251,22 +1297,25 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Ar
         r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
     }
     __syncthreads();
+    // describe the first item (and what follows it closely) and fill the ring
+    if (warp == kWarps - 1) {
+        prepare_items(A, smem, kLead, lane);
+        if (lane == 0)
+            for (uint32_t j = 0; j < (uint32_t)kStages; ++j) issue_copy(smem, ring, j, j);
+    }
+    __syncthreads();
 
     BlockState B;
     B.cstage = 0; B.cphase = 0; B.ccount = 0; B.ord = 0;
-    B.is_issuer = warp == kWarps - 1;
     const ItemInfo* infos = reinterpret_cast<const ItemInfo*>(smem + kOffInfo);
 
     int cur_t = -1, cur_k0 = 0, cur_kc = 0;
     uint32_t cur_slot = 0, cur_tile = 0, cur_te = 0;
     for (;; ++B.ord) {
-        // The next item announces itself before its first ring stage is armed (that stage stays
-        // full until it is consumed in run_item).  All threads agree on stopping: at the
-        // issuer's end mark, or when any thread of the block has given up on a wait.
-        uint32_t s0;
-        const bool got = wait_stage(A, smem, ring, B, lane, s0);
-        ItemInfo it = infos[B.ord & (kInfoRing - 1)];
-        if (!got) it.id = kNoItem;
+        // The item's description was written while the item before it was being set up.  All
+        // threads agree on stopping: at the end of the list, or when any thread of the block
+        // has given up on a wait.
+        const ItemInfo it = infos[B.ord & (kInfoRing - 1)];
         if (block_sync_or((it.id == kNoItem || *ring.ctl.abort_flag) ? 1u : 0u)) break;
         if (!RKV_IN_BOUNDS(A.header, 5, it.t < (uint32_t)A.T && it.kc >= 1u && it.kc <= (uint32_t)kPartK &&
                                             it.k0 + it.kc <= (uint32_t)A.K, it.t))
@@ -1283,8 +1332,6 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Ar
         cur_t = (int)it.t; cur_k0 = (int)it.k0; cur_kc = (int)it.kc; cur_tile = it.tile;
         cur_slot = D.slot_by_tile ? it.tile : blockIdx.x;
         cur_te = tile_elems(D.cand_dtype);
-        // (the stage waited for above is consumed inside run_item: it holds the item's reference
-        // tile or its first candidate)
         switch (D.cand_dtype) {
             case RKV_F32: run_item<CK_F32>(A, smem, ring, B, it, D); break;
             case RKV_BF16: run_item<CK_BF16>(A, smem, ring, B, it, D); break;
@@ -1298,8 +1345,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Ar
     }
     if (tid == 0 && *ring.ctl.abort_flag) atomicExch(&A.header->status, (int32_t)RKV_ERR_TIMEOUT);
 
-    if (B.is_issuer && lane == 0) {
-        IssuerState* st = reinterpret_cast<IssuerState*>(smem + kOffIssuer);
+    if (tid == 0) {
         // the last block to get here clears the ticket counter for the next launch
         __threadfence();
         if (atomicAdd(&A.header->blocks_done, 1u) == gridDim.x - 1u) {
@@ -1307,13 +1353,12 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const Ar
             A.header->blocks_done = 0u;
         }
         // A block that gave up must not retire with copies still landing in its shared
-        // memory: wait (bounded) for the copies issued last.
+        // memory: wait (bounded) for the copy issued last into each stage.
         if (*ring.ctl.abort_flag) {
-            const uint32_t n_issued = st->n_issued;
-            const uint32_t pending = n_issued < (uint32_t)kStages ? n_issued : (uint32_t)kStages;
-            for (uint32_t i = 0; i < pending; ++i) {
-                const uint32_t q = n_issued - 1 - i;
-                const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
+            for (uint32_t s = 0; s < (uint32_t)kStages; ++s) {
+                const uint32_t jp1 = reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s];
+                if (!jp1) continue;
+                const uint32_t ph = ((jp1 - 1u) / kStages) & 1u;
                 const long long t0 = clock64();
                 for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
                     if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
@@ -1452,6 +1497,17 @@ int launch_verify(const Layout& L, int T, int K, int k_begin, int k_end, uint32_
     // the grid is always the full resident grid: Partial rows of large tensors are numbered by block
     verify_kernel<<<grid, kThreads, kSmemBytes, stream>>>(A);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+// Resident blocks per SM the device grants the verification kernel (0 on error).
+int verify_occupancy() {
+    int n = 0;
+    if (cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_kernel, kThreads, kSmemBytes) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
 }
 
 int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,
