@@ -224,7 +224,7 @@ int rkv_verify_multi(const rkv_tensor_desc *tensors, int T, int K, rkv_stats *st
  * (0 on an invalid argument).  Depends on n, the dtypes, T, K and the device's
  * SM count only: tables, 64 bytes per (tensor, candidate), 48 bytes * K per tensor and
  * resident thread block (per tile, for a tensor of fewer tiles than blocks), and one
- * double per (tile of 16 KiB of a candidate, candidate) for the error sums. */
+ * double per (tile of 14 KiB of a candidate, candidate) for the error sums. */
 size_t rkv_workspace_bytes(const rkv_tensor_desc *tensors, int T, int K);
 
 /*
@@ -311,7 +311,7 @@ int rkv_verify_multi_host(const rkv_tensor_desc *tensors, int T, int K, rkv_stat
  * and stats_out are the caller's; inputs are only read.
  *
  * Limits: K <= 256, and the scratch the case needs (rkv_workspace_bytes of the
- * single-tensor case: about 48 bytes * K * 2 * SM count plus 8 bytes * K per 16 KiB
+ * single-tensor case: about 48 bytes * K * 2 * SM count plus 8 bytes * K per 14 KiB
  * of a candidate) must fit in 8 MiB; on a 148-SM part that is e.g. K = 64 candidates
  * of 2^24 fp32 elements, or K = 256 of 2^21.  A larger case is rejected with
  * RKV_ERR_UNSUPPORTED before anything is launched.  Other errors: INVALID_ARG,
@@ -339,7 +339,7 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * Host-only planning helper (no CUDA call; plumbing, no passage of its own): how the
  * work of one tensor is cut.
  * The tensor is cut into *n_tiles tiles of *tile_elems elements (a thread of the
- * verification kernel owns 64 bytes of each candidate tile: 4096 fp32 or 8192 16-bit
+ * verification kernel owns 64 bytes of each candidate tile: 3584 fp32 or 7168 16-bit
  * elements per tile).  One work item is
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the

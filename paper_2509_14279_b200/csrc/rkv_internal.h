@@ -12,13 +12,14 @@
 namespace rkv {
 
 // ---- verification kernel geometry ------------------------------------------------
-constexpr int kWarps = 8;                            // every warp compares; the last one also issues the bulk copies
-constexpr int kThreads = kWarps * 32;                // 256 threads
+constexpr int kConsumerWarps = 7;                    // warps that compare
+constexpr int kConsumers = kConsumerWarps * 32;      // 224 threads
+constexpr int kThreads = kConsumers + 32;            // + one warp that issues the bulk copies = 256
 constexpr int kBlocksPerSm = 2;                      // resident verification blocks per SM
-constexpr int kStageBytes = kThreads * 64;           // a ring stage: 64 bytes of a candidate per thread
+constexpr int kStageBytes = kConsumers * 64;         // a ring stage: 64 bytes of a candidate per thread
 // A thread owns 64 bytes of each candidate tile: 16 fp32 or 32 16-bit elements.
-constexpr int kTileElems32 = kStageBytes / 4;        // 4096 elements per tile of fp32 candidates
-constexpr int kTileElems16 = kStageBytes / 2;        // 8192 elements per tile of bf16 / fp16 candidates
+constexpr int kTileElems32 = kStageBytes / 4;        // 3584 elements per tile of fp32 candidates
+constexpr int kTileElems16 = kStageBytes / 2;        // 7168 elements per tile of bf16 / fp16 candidates
 __host__ __device__ constexpr bool is16(int dtype) { return dtype != RKV_F32; }
 __host__ __device__ constexpr uint32_t elem_bytes(int dtype) { return dtype == RKV_F32 ? 4u : 2u; }
 __host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
@@ -26,13 +27,12 @@ __host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
 }
 constexpr int kStages = 5;                           // ring depth (bulk copies in flight)
 constexpr int kPartK = 64;                           // candidates a block tracks at a time
-constexpr int kWarmTiles = 16;                       // leading tiles of a large tensor that are verified first
+constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
 constexpr int kWarmMinTiles = 2048;                  // tensors with fewer tiles have no warm-up group
 constexpr int kTailDiv = 4;                          // a tail item covers a quarter of a part's candidates ...
 constexpr int kTailDivGenerated = 2;                 // ... half, when every item regenerates its reference tile
 constexpr int kMaxTensors = 64;                      // rkv_verify_multi
 constexpr int kMaxSweepTensors = 4096;               // rkv_verify_sweep, over all its cases
-constexpr int kInterleaveRounds = 64;                // how finely the item lists of several tensors are interleaved
 constexpr uint64_t kMaxN = 1ull << 40;
 
 // Result of one thread block (or, for a small tensor, of one tile) for one (tensor,

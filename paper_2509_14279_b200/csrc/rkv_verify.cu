@@ -1,27 +1,26 @@
 // Fused single-pass verification kernel and its finalize kernels (sm_100a).
 //
-// Work decomposition.  A tensor is cut into tiles of 16384 candidate bytes (4096 fp32 or
-// 8192 bf16 / fp16 elements); the K candidates into parts of at most 64.  A work item is
+// Work decomposition.  A tensor is cut into tiles of 14336 candidate bytes (3584 fp32 or
+// 7168 bf16 / fp16 elements); the K candidates into parts of at most 64.  A work item is
 // (tensor, group, part, tile); the items of every tensor of a call -- whatever its storage
 // types -- form one list (see Segment), and one launch of persistent thread blocks works
 // through it: a block starts with the item of its own number and then draws further items
-// from a ticket counter.  Items of fp32 candidates are bound by HBM, items of 16-bit
-// candidates by instruction issue; the list interleaves them, so that the two kinds overlap
-// on every SM instead of running one after the other.
+// from a ticket counter.
 //
-// All eight warps of a block compare.  A thread owns 64 bytes of every candidate tile (16
-// fp32 or 32 16-bit elements); it keeps their reference values (and, for fp32 candidates,
-// the tolerance thresholds) IN REGISTERS for the whole item and meets every candidate tile
-// as it lands in a ring of shared-memory stages.  The ring is fed by whoever frees a stage:
-// a warp that has read its 2 KB of a stage counts itself off on the stage, and the warp that
-// counts off last issues, there and then, the bulk asynchronous copy (cp.async.bulk,
-// completion counted on an mbarrier) that refills the stage.  What to copy it reads from a
-// queue of copy descriptors -- for an item the reference tile, then the same tile of every
-// candidate of the part, then on to the next item -- that the block's last warp writes one
-// item ahead, while the other warps fetch the item's hints.  Issuing a copy is a dozen
-// instructions, a full ring of copies is always in flight, across item boundaries, and no
-// warp is set aside to issue them.  (With 128 registers a thread, 16 warps fill an SM; a
-// warp that only issued copies would leave its scheduler half idle.)
+// A block has two roles:
+//
+//   * one producer warp: it takes the block's items one after the other -- the ticket for the
+//     next one is drawn while the current one is being issued -- decodes them, publishes their
+//     description, fetches the part's candidate pointers (all 32 lanes, one round trip) and
+//     then one lane issues the bulk asynchronous copies (cp.async.bulk, completion counted on
+//     an mbarrier) that bring, for the item, the reference tile and then the same tile of
+//     every candidate of the part into a ring of shared-memory stages.  Several stages are in
+//     flight, across item boundaries, so the copies of later candidates overlap the
+//     comparison of earlier ones;
+//   * seven consumer warps: each thread owns 64 bytes of every candidate tile (16 fp32 or 32
+//     16-bit elements).  It keeps their reference values (and, for fp32 candidates, the
+//     tolerance thresholds) IN REGISTERS for the whole item and meets every candidate tile as
+//     it lands in the ring.
 //
 // Candidate bytes are read from HBM exactly once; the reference once per part.
 // When the reference is "generated" the threads regenerate their values from
@@ -55,9 +54,7 @@ namespace {
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr float kInf = __builtin_huge_valf();
 enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the issuer's "no more items" mark
-constexpr int kInfoRing = 16;                  // item descriptions kept per block (> kStages + 4: an item uses >= 1 stage)
-constexpr int kDescRing = 256;                 // copy descriptors kept per block (> two items of kPartK + 2 copies)
-constexpr uint32_t kLead = kStages + 2;        // descriptors are prepared this far past the end of the current item
+constexpr int kInfoRing = 16;                  // item descriptions kept per block (> kStages + 1: an item uses >= 1 stage)
 constexpr long long kWaitCycles = 2000000000LL;
 
 // ----------------------------------------------------------------------------
@@ -114,44 +111,21 @@ struct __align__(16) ItemInfo {
 };
 static_assert(sizeof(ItemInfo) == 32, "ItemInfo layout");
 
-// One bulk copy of the schedule: copy number j of a block goes to ring stage j % kStages.
-struct __align__(16) CopyDesc {
-    const unsigned char* src;
-    uint32_t bytes;          // 0: nothing to copy (an empty tile piece): the stage is armed and completes at once
-    uint32_t withhold;       // fault drill of a test: arm the stage, do not issue the copy
-};
-static_assert(sizeof(CopyDesc) == 16, "CopyDesc layout");
-
-// The schedule of a block: which items it takes and the copies they need.  Lane 0 of the
-// preparing warp writes it; the warps that refill stages only read q_end.
-struct __align__(16) Schedule {
-    uint32_t q_end;          // copies described so far: numbers [0, q_end)
-    uint32_t ord;            // items described so far
-    uint32_t next_id;        // launch-wide id of the next item (a ticket drawn one item ahead)
-    uint32_t seg;            // segment the last item was found in
-    uint32_t done;           // the end of the item list has been reached
-    uint32_t drill;          // fault drill: number (1-based) of the copy to withhold, 0: none
-    uint32_t reserved[2];
-};
-static_assert(sizeof(Schedule) == 32, "Schedule layout");
-
-constexpr int kOffFull = 0;                                   // kStages mbarriers
-constexpr int kOffRelease = kOffFull + 8 * kStages;           // kStages x uint32: warps that have read the stage
-constexpr int kOffIssued = kOffRelease + 4 * kStages;         // kStages x uint32: 1 + number of the last copy issued into the stage
-constexpr int kOffAbort = kOffIssued + 4 * kStages;           // uint32
+constexpr int kOffFull = 0;                                   // kStages mbarriers: the stage's copy has landed
+constexpr int kOffEmpty = kOffFull + 8 * kStages;             // kStages mbarriers: every consumer warp has read the stage
+constexpr int kOffAbort = kOffEmpty + 8 * kStages;            // uint32
 constexpr int kOffRefState = kOffAbort + 8;                   // 2 x uint32 settled bits of the reference (item parity)
 constexpr int kOffWaitLimit = kOffRefState + 8;               // long long: cycles a wait may take
-constexpr int kOffSchedule = 128;
-constexpr int kOffInfo = kOffSchedule + (int)sizeof(Schedule);
-constexpr int kOffDesc = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);
-constexpr int kOffPtrC = kOffDesc + kDescRing * (int)sizeof(CopyDesc);   // the part's candidate pointers
-constexpr int kOffHint = kOffPtrC + kPartK * 8;                          // two tables (item parity)
+constexpr int kOffInfo = 128;
+constexpr int kOffPtrC = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);   // consumer copy of the part's candidate pointers
+constexpr int kOffPtrP = kOffPtrC + kPartK * 8;                          // producer copy (it runs an item ahead)
+constexpr int kOffHint = kOffPtrP + kPartK * 8;                          // two tables (item parity)
 constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
-constexpr int kOffStage = (kOffRec + kWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
+constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
-static_assert(kOffWaitLimit + 8 <= kOffSchedule, "layout");
-static_assert(kDescRing >= 2 * (kPartK + 2) + (int)kLead && (kDescRing & (kDescRing - 1)) == 0, "descriptor ring");
-static_assert(kInfoRing >= (int)kLead + 3 && (kInfoRing & (kInfoRing - 1)) == 0, "item ring");
+static_assert(kOffWaitLimit + 8 <= kOffInfo && kOffWaitLimit % 8 == 0 && kOffEmpty % 8 == 0 && kOffInfo % 16 == 0 &&
+              kOffPtrC % 8 == 0 && kOffPtrP % 8 == 0 && kOffHint % 16 == 0 && kOffRec % 16 == 0, "layout");
+static_assert(kInfoRing > kStages + 1 && (kInfoRing & (kInfoRing - 1)) == 0, "item ring");
 static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM must fit");
 
 // Candidate storage kinds the comparison is compiled for.
@@ -168,7 +142,7 @@ struct Geo {
     static constexpr int E = C16 ? 32 : 16;             // elements per thread
     static constexpr int VEC = C16 ? 8 : 4;             // elements per 16-byte piece
     static constexpr int NW = 16;                       // 32-bit words per thread and candidate tile
-    static constexpr int kTile = kThreads * E;          // elements per tile
+    static constexpr int kTile = kConsumers * E;        // elements per tile
     static constexpr int DTYPE = CK == CK_F32 ? RKV_F32 : CK == CK_BF16 ? RKV_BF16 : RKV_F16;
 };
 
@@ -213,14 +187,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
     return ok != 0;
 }
 
-// Count one more warp off a stage (release: the warp's reads of the stage come first;
-// acquire: the warp that counts off last may overwrite it).  Returns the count before.
-__device__ __forceinline__ uint32_t count_off(uint32_t addr) {
-    uint32_t old;
-    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(addr) : "memory");
-    return old;
-}
-
 // What every wait of a block shares: the flag that says "a wait ran out, drain" and the
 // number of clock cycles a wait may take.
 struct WaitCtl {
@@ -258,9 +224,23 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         : "memory");
 }
 
-// Block barrier that also returns whether any thread passed a non-zero value.
-__device__ __forceinline__ bool block_sync_or(uint32_t v) {
-    return __syncthreads_or((int)v) != 0;
+// Barrier among the consumer threads only (the producer warp never joins).
+__device__ __forceinline__ void consumer_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+
+// The same barrier, returning whether any consumer thread passed a non-zero value.
+__device__ __forceinline__ bool consumer_sync_or(uint32_t v) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "barrier.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"(v), "n"(kConsumers)
+        : "memory");
+    return out != 0;
 }
 
 __device__ __forceinline__ bool bits_finite(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
@@ -305,8 +285,7 @@ struct Args {
 // the issuing lane: feeds the ring
 // ----------------------------------------------------------------------------
 struct Ring {
-    uint32_t full0;              // shared-memory address of the first full mbarrier
-    uint32_t release0;           // ... of the first release counter
+    uint32_t full0, empty0;      // shared-memory addresses of the first full / empty mbarrier
     uint32_t stage0;             // ... of stage 0
     WaitCtl ctl;
 };
@@ -343,116 +322,111 @@ __device__ __forceinline__ bool decode_item(const Args& A, uint32_t id, uint32_t
     return true;
 }
 
-// Describe further items, whole items at a time, until the copies described reach past copy
-// number `target` or the item list ends.  Per item: draw the ticket for the one after it,
-// decode, publish its description for the comparing threads, and queue its copies -- the
-// reference tile (one or two stages) and the tile of every candidate of the part.  The whole
-// warp calls this: lane 0 keeps the schedule, all lanes fetch the candidates' pointers (one
-// round trip to memory instead of one per candidate).
-__device__ __forceinline__ void prepare_items(const Args& A, unsigned char* smem, uint32_t target, int lane) {
-    Schedule* sc = reinterpret_cast<Schedule*>(smem + kOffSchedule);
-    CopyDesc* desc = reinterpret_cast<CopyDesc*>(smem + kOffDesc);
-    for (int guard = 0; guard < kInfoRing; ++guard) {
-        uint32_t go = 0;
-        if (lane == 0) go = (!sc->done && sc->q_end <= target) ? 1u : 0u;
-        if (!__shfl_sync(kFullMask, go, 0)) break;
-        uint32_t t = 0, k0 = 0, kc = 0, q = 0, cbytes = 0, off_lo = 0, off_hi = 0, ticket = 0;
+// The producer warp.  Per item: draw the ticket for the one after it (its latency hides
+// behind the rest), decode, fetch the part's candidate pointers with all lanes, publish the
+// item's description, then lane 0 issues the item's copies in ring order, each as soon as
+// every consumer warp has released the stage's previous use.
+__device__ __forceinline__ void producer_loop(const Args& A, unsigned char* smem, const Ring& ring) {
+    const int lane = threadIdx.x & 31;
+    const void** table = reinterpret_cast<const void**>(smem + kOffPtrP);
+    ItemInfo* infos = reinterpret_cast<ItemInfo*>(smem + kOffInfo);
+    const uint32_t drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
+    uint32_t n_issued = 0, stage = 0, phase = 0, seg = 0, ord = 0;
+
+    auto issue = [&](const unsigned char* src, uint32_t bytes) {
+        // the stage is free once every consumer warp has released its previous use
+        mbar_wait(ring.empty0 + 8 * stage, phase ^ 1u, ring.ctl);
+        const uint32_t full = ring.full0 + 8 * stage;
+        if (bytes) {
+            mbar_expect_tx(full, bytes);
+            // (the fault drill of a test: arm the stage, withhold the copy)
+            if (n_issued + 1u != drill) bulk_g2s(ring.stage0 + stage * kStageBytes, src, bytes, full);
+        } else {
+            mbar_arrive(full);
+        }
+        ++n_issued;
+        if (++stage == (uint32_t)kStages) { stage = 0; phase ^= 1u; }
+    };
+
+    uint32_t id = blockIdx.x;                 // every block starts with the item of its own number
+    for (;;) {
+        id = __shfl_sync(kFullMask, id, 0);
+        if (id >= A.n_items || *ring.ctl.abort_flag) break;
+        uint32_t next_id = 0, ok = 0;
+        ItemInfo info;
+        info.id = kNoItem; info.t = 0; info.tile = 0; info.k0 = 0; info.kc = 0;
+        info.reserved[0] = info.reserved[1] = info.reserved[2] = 0;
         if (lane == 0) {
-            const uint32_t id = sc->next_id;
-            // the ticket for the item after this one; its latency hides behind the decoding
-            if (id < A.n_items) ticket = atomicAdd(&A.header->next_ticket, 1u);
-            ItemInfo info;
-            info.id = kNoItem; info.t = 0; info.tile = 0; info.k0 = 0; info.kc = 0;
-            info.reserved[0] = info.reserved[1] = info.reserved[2] = 0;
-            uint32_t seg = sc->seg;
-            q = sc->q_end;
-            if (decode_item(A, id, seg, info)) {
-                const DevTensor& D = A.tensors[info.t];
-                const uint32_t csz = elem_bytes(D.cand_dtype), rsz = elem_bytes(D.ref_dtype);
-                const uint32_t te = tile_elems(D.cand_dtype);
-                const uint64_t start = (uint64_t)info.tile * te;
-                const uint32_t len = (uint32_t)min((uint64_t)te, D.n - start);
-                cbytes = (len * csz) & ~15u;
-                const uint64_t c_off = start * csz;
-                off_lo = (uint32_t)c_off; off_hi = (uint32_t)(c_off >> 32);
-                if (D.ref_src == RKV_SRC_POINTER) {
-                    const uint32_t nref = (te * rsz + kStageBytes - 1) / kStageBytes;
-                    const uint32_t rbytes = (len * rsz) & ~15u;
-                    const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
-                    for (uint32_t r = 0; r < nref; ++r, ++q) {
-                        const uint32_t lo = r * kStageBytes;
-                        CopyDesc d;
-                        d.src = src + lo;
-                        d.bytes = rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u;
-                        d.withhold = q + 1u == sc->drill ? 1u : 0u;
-                        desc[q & (kDescRing - 1)] = d;
-                    }
+            next_id = gridDim.x + atomicAdd(&A.header->next_ticket, 1u);
+            ok = decode_item(A, id, seg, info) ? 1u : 0u;
+        }
+        if (!__shfl_sync(kFullMask, ok, 0)) break;
+        const uint32_t t = __shfl_sync(kFullMask, info.t, 0);
+        const uint32_t k0 = __shfl_sync(kFullMask, info.k0, 0);
+        const uint32_t kc = __shfl_sync(kFullMask, info.kc, 0);
+        const DevTensor& D = A.tensors[t];
+        {
+            const void* const* src = D.cands + k0;
+            for (uint32_t i = (uint32_t)lane; i < kc; i += 32u) table[i] = src[i];
+        }
+        __syncwarp();
+        if (lane == 0) {
+            infos[ord & (kInfoRing - 1)] = info;      // ordered before the arrive of the item's first stage
+            const uint32_t csz = elem_bytes(D.cand_dtype), rsz = elem_bytes(D.ref_dtype);
+            const uint32_t te = tile_elems(D.cand_dtype);
+            const uint64_t start = (uint64_t)info.tile * te;
+            const uint32_t len = (uint32_t)min((uint64_t)te, D.n - start);
+            if (D.ref_src == RKV_SRC_POINTER) {
+                const uint32_t nref = (te * rsz + kStageBytes - 1) / kStageBytes;
+                const uint32_t rbytes = (len * rsz) & ~15u;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
+                for (uint32_t r = 0; r < nref; ++r) {
+                    const uint32_t lo = r * kStageBytes;
+                    issue(src + lo, rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u);
                 }
-                t = info.t; k0 = info.k0; kc = info.kc;
-            } else {
-                sc->done = 1u;                      // the description with kNoItem ends the block's list
             }
-            sc->seg = seg;
-            reinterpret_cast<ItemInfo*>(smem + kOffInfo)[sc->ord & (kInfoRing - 1)] = info;
-        }
-        t = __shfl_sync(kFullMask, t, 0);
-        k0 = __shfl_sync(kFullMask, k0, 0);
-        kc = __shfl_sync(kFullMask, kc, 0);
-        q = __shfl_sync(kFullMask, q, 0);
-        cbytes = __shfl_sync(kFullMask, cbytes, 0);
-        off_lo = __shfl_sync(kFullMask, off_lo, 0);
-        off_hi = __shfl_sync(kFullMask, off_hi, 0);
-        if (kc) {
-            const void* const* src = A.tensors[t].cands + k0;
-            const unsigned long long c_off = ((unsigned long long)off_hi << 32) | off_lo;
-            const uint32_t drill = sc->drill;
-            for (uint32_t i = (uint32_t)lane; i < kc; i += 32u) {
-                CopyDesc d;
-                d.src = reinterpret_cast<const unsigned char*>(src[i]) + c_off;
-                d.bytes = cbytes;
-                d.withhold = q + i + 1u == drill ? 1u : 0u;
-                desc[(q + i) & (kDescRing - 1)] = d;
-            }
+            const uint32_t cbytes = (len * csz) & ~15u;
+            const uint64_t c_off = start * csz;
+            for (uint32_t i = 0; i < kc; ++i)
+                issue(reinterpret_cast<const unsigned char*>(table[i]) + c_off, cbytes);
         }
         __syncwarp();
-        if (lane == 0) {
-            __threadfence_block();
-            sc->q_end = q + kc;
-            sc->ord += 1u;
-            sc->next_id = gridDim.x + ticket;
-        }
-        __syncwarp();
+        ++ord;
+        id = next_id;
     }
-}
-
-// Issue copy number j of the block's schedule into its ring stage, if it has been described
-// (beyond the end of the item list nothing is).  One lane calls this.
-__device__ __forceinline__ void issue_copy(unsigned char* smem, const Ring& ring, uint32_t j, uint32_t s) {
-    const volatile Schedule* sc = reinterpret_cast<const volatile Schedule*>(smem + kOffSchedule);
-    if (j >= sc->q_end) return;
-    const CopyDesc d = reinterpret_cast<const CopyDesc*>(smem + kOffDesc)[j & (kDescRing - 1)];
-    const uint32_t full = ring.full0 + 8 * s;
-    reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s] = j + 1u;
-    if (d.bytes) {
-        mbar_expect_tx(full, d.bytes);
-        if (!d.withhold) bulk_g2s(ring.stage0 + s * kStageBytes, d.src, d.bytes, full);
-    } else {
-        mbar_arrive(full);
-    }
-}
-
-// A warp has read ring stage `s` for the stage use number `use` (uses are numbered in the
-// order the schedule fills the ring, so use j sits in stage j % kStages).  The warp that
-// counts off last refills the stage with copy number use + kStages.
-__device__ __forceinline__ void release_stage(unsigned char* smem, const Ring& ring, uint32_t s, uint32_t use,
-                                              int lane) {
-    __syncwarp();
     if (lane == 0) {
-        if (count_off(ring.release0 + 4 * s) == (uint32_t)kWarps - 1u) {
-            reinterpret_cast<volatile uint32_t*>(smem + kOffRelease)[s] = 0u;
-            issue_copy(smem, ring, use + (uint32_t)kStages, s);
+        ItemInfo end;
+        end.id = kNoItem; end.t = 0; end.tile = 0; end.k0 = 0; end.kc = 0;
+        end.reserved[0] = end.reserved[1] = end.reserved[2] = 0;
+        infos[ord & (kInfoRing - 1)] = end;
+        issue(nullptr, 0u);                              // tell the consumers to stop
+        // the last block to get here clears the ticket counter for the next launch
+        __threadfence();
+        if (atomicAdd(&A.header->blocks_done, 1u) == gridDim.x - 1u) {
+            A.header->next_ticket = 0u;
+            A.header->blocks_done = 0u;
+        }
+        // A block that gave up must not retire with copies still landing in its shared
+        // memory: wait (bounded) for the copies issued last.
+        if (*ring.ctl.abort_flag) {
+            const uint32_t pending = n_issued < (uint32_t)kStages ? n_issued : (uint32_t)kStages;
+            for (uint32_t i = 0; i < pending; ++i) {
+                const uint32_t q = n_issued - 1 - i;
+                const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
+                const long long t0 = clock64();
+                for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+                    if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
+                    if (clock64() - t0 > 200000000LL) break;
+                }
+            }
         }
     }
+}
+
+// A consumer warp has read ring stage `s`: release it.
+__device__ __forceinline__ void release_stage(const Ring& ring, uint32_t s, int lane) {
+    __syncwarp();
+    mbar_arrive_if(ring.empty0 + 8 * s, lane == 0);
 }
 
 // ----------------------------------------------------------------------------
@@ -460,11 +434,11 @@ __device__ __forceinline__ void release_stage(unsigned char* smem, const Ring& r
 // ----------------------------------------------------------------------------
 // A thread owns E elements of the tile (see Geo) as vectors of VEC elements
 // (one 16-byte piece of a candidate each): vector jv of thread tid is vector
-// jv * 256 + tid of the tile.  Element j = jv * VEC + i of the thread has the
+// jv * 224 + tid of the tile.  Element j = jv * VEC + i of the thread has the
 // tile offset below; offsets grow with j.
 template <int VEC>
 __device__ __forceinline__ uint32_t elem_off(int j, int tid) {
-    return (uint32_t)(((j / VEC) * kThreads + tid) * VEC + (j % VEC));
+    return (uint32_t)(((j / VEC) * kConsumers + tid) * VEC + (j % VEC));
 }
 
 // What a thread keeps for the whole item.
@@ -678,7 +652,7 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
                                                              start * CSZ) + tid;
 #pragma unroll
             for (int jv = 0; jv < E / VEC; ++jv) {
-                const uint4 t = __ldg(in + jv * kThreads);
+                const uint4 t = __ldg(in + jv * kConsumers);
                 acc2 |= (w[4 * jv] ^ t.x) | (w[4 * jv + 1] ^ t.y) | (w[4 * jv + 2] ^ t.z) | (w[4 * jv + 3] ^ t.w);
             }
         } else if (!full || (need & 2u)) {
@@ -1049,13 +1023,13 @@ __device__ __forceinline__ void process_candidate_16(const RefRegs<true>& R, con
 
 // The error sums of the item just finished: for every candidate of its part, the warps'
 // tile sums added in warp order, stored in the (tile, candidate) slot, and cleared.
-// Called by all threads between two block barriers.
+// Called by all consumer threads between two consumer barriers.
 __device__ __forceinline__ void flush_sums(WarpRec* recs, const Args& A, const DevTensor& D, uint32_t tile, int k0,
                                            int kc, int tid) {
     if (tid < kc) {
         double s = 0.0;
 #pragma unroll
-        for (int wp = 0; wp < kWarps; ++wp) {
+        for (int wp = 0; wp < kConsumerWarps; ++wp) {
             WarpRec& r = recs[wp * kPartK + tid];
             s += r.sum;
             r.sum = 0.0;
@@ -1067,7 +1041,7 @@ __device__ __forceinline__ void flush_sums(WarpRec* recs, const Args& A, const D
 }
 
 // Merge the warp records of every candidate of a part into the Partial row and clear
-// them.  Called by all threads between two block barriers.
+// them.  Called by all consumer threads between two consumer barriers.
 __device__ __forceinline__ void flush_records(WarpRec* recs, const Args& A, const DevTensor& D, int k0, int kc,
                                               uint32_t slot, int tid, uint32_t tile_elems_) {
     if (tid < kc) {
@@ -1075,7 +1049,7 @@ __device__ __forceinline__ void flush_records(WarpRec* recs, const Args& A, cons
         p.n_over = 0; p.eidx = RKV_NO_INDEX; p.qidx = RKV_NO_INDEX;
         p.emax = -1.0f; p.qmax = -1.0f; p.valid = 1u; p.reserved[0] = p.reserved[1] = p.reserved[2] = 0u;
 #pragma unroll
-        for (int wp = 0; wp < kWarps; ++wp) {
+        for (int wp = 0; wp < kConsumerWarps; ++wp) {
             WarpRec& r = recs[wp * kPartK + tid];
             p.n_over += r.n_over;
             if (r.emax >= 0.0f) {
@@ -1153,13 +1127,6 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
     CandState* st_t = A.state + D.state_base;
 
-    // the last warp describes the copies that will be issued while this item is compared: up
-    // to kLead copies past the item's own (the item's copies were described one item ago)
-    if (warp == kWarps - 1) {
-        const uint32_t nref = D.ref_src == RKV_SRC_POINTER
-                                  ? (kTile * elem_bytes(D.ref_dtype) + kStageBytes - 1) / kStageBytes : 0u;
-        prepare_items(A, smem, B.ccount + nref + (uint32_t)kc - 1u + kLead, lane);
-    }
     // the part's pointers and hints, from the published state
     if (tid < kc) {
         const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
@@ -1182,7 +1149,6 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
         // the reference tile fills one ring stage, or two (fp32 under 16-bit candidates)
         const bool two = (kTile * elem_bytes(D.ref_dtype)) > (uint32_t)kStageBytes;
         uint32_t sa, sb;
-        const uint32_t use_a = B.ccount;
         wait_stage(ring, B, sa);
         advance_stage(B);
         sb = sa;
@@ -1191,12 +1157,12 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
             advance_stage(B);
         }
         load_ref<CK>(R, rb, D, start, len, stages + (size_t)sa * kStageBytes, stages + (size_t)sb * kStageBytes, tid);
-        release_stage(smem, ring, sa, use_a, lane);
-        if (two) release_stage(smem, ring, sb, use_a + 1u, lane);
+        release_stage(ring, sa, lane);
+        if (two) release_stage(ring, sb, lane);
     } else {
         load_ref<CK>(R, rb, D, start, len, nullptr, nullptr, tid);
     }
-    __syncthreads();                          // hints, pointers and cleared records are visible
+    consumer_sync();                          // hints, pointers and cleared records are visible
 
     // reference flags (constant / copy of the input), until a difference has been seen
     {
@@ -1234,10 +1200,10 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
         uint32_t w[NW];
 #pragma unroll
         for (int jv = 0; jv < NV; ++jv) {
-            const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kThreads + tid) * 16);
+            const uint4 t = *reinterpret_cast<const uint4*>(stage + (size_t)(jv * kConsumers + tid) * 16);
             w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
         }
-        release_stage(smem, ring, s, B.ccount, lane);
+        release_stage(ring, s, lane);
         advance_stage(B);
         if (len != kTile) {
             // Ragged last tile: the copy brought whole 16-byte pieces only.  The few
@@ -1265,58 +1231,30 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     }
 }
 
-// Persistent blocks, kBlocksPerSm per SM.
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __grid_constant__ Args A) {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    Ring ring;
-    ring.full0 = smem_u32(smem + kOffFull);
-    ring.release0 = smem_u32(smem + kOffRelease);
-    ring.stage0 = smem_u32(smem + kOffStage);
-    ring.ctl.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
-    ring.ctl.limit = reinterpret_cast<const volatile long long*>(smem + kOffWaitLimit);
+// The consumer warps: item after item, as the producer announces them.
+__device__ __forceinline__ void consumer_loop(const Args& A, unsigned char* smem, const Ring& ring) {
+    const int tid = threadIdx.x;
     WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(ring.full0 + 8 * s, 1);             // the issuer's arrive + the copy's bytes
-            reinterpret_cast<volatile uint32_t*>(smem + kOffRelease)[s] = 0u;
-            reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s] = 0u;
-        }
-        *ring.ctl.abort_flag = 0u;
-        const unsigned long long lim = A.header->drill_issue ? A.header->drill_wait_cycles : 0ull;
-        *reinterpret_cast<volatile long long*>(smem + kOffWaitLimit) = lim ? (long long)lim : kWaitCycles;
-        Schedule* sc = reinterpret_cast<Schedule*>(smem + kOffSchedule);
-        sc->q_end = 0; sc->ord = 0; sc->seg = 0; sc->done = 0; sc->reserved[0] = sc->reserved[1] = 0;
-        sc->next_id = blockIdx.x;             // every block starts with the item of its own number
-        sc->drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+    const ItemInfo* infos = reinterpret_cast<const ItemInfo*>(smem + kOffInfo);
     // clear the records once; the flushes leave them cleared
-    for (int i = tid; i < kWarps * kPartK; i += kThreads) {
+    for (int i = tid; i < kConsumerWarps * kPartK; i += kConsumers) {
         WarpRec& r = recs[i];
         r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
     }
-    __syncthreads();
-    // describe the first item (and what follows it closely) and fill the ring
-    if (warp == kWarps - 1) {
-        prepare_items(A, smem, kLead, lane);
-        if (lane == 0)
-            for (uint32_t j = 0; j < (uint32_t)kStages; ++j) issue_copy(smem, ring, j, j);
-    }
-    __syncthreads();
-
     BlockState B;
     B.cstage = 0; B.cphase = 0; B.ccount = 0; B.ord = 0;
-    const ItemInfo* infos = reinterpret_cast<const ItemInfo*>(smem + kOffInfo);
 
     int cur_t = -1, cur_k0 = 0, cur_kc = 0;
     uint32_t cur_slot = 0, cur_tile = 0, cur_te = 0;
     for (;; ++B.ord) {
-        // The item's description was written while the item before it was being set up.  All
-        // threads agree on stopping: at the end of the list, or when any thread of the block
-        // has given up on a wait.
-        const ItemInfo it = infos[B.ord & (kInfoRing - 1)];
-        if (block_sync_or((it.id == kNoItem || *ring.ctl.abort_flag) ? 1u : 0u)) break;
+        // The next item announces itself before its first ring stage is armed (that stage stays
+        // full until it is consumed in run_item).  All consumers agree on stopping: at the
+        // producer's end mark, or when any thread of the block has given up on a wait.
+        uint32_t s0;
+        const bool got = wait_stage(ring, B, s0);
+        ItemInfo it = infos[B.ord & (kInfoRing - 1)];
+        if (!got) it.id = kNoItem;
+        if (consumer_sync_or((it.id == kNoItem || *ring.ctl.abort_flag) ? 1u : 0u)) break;
         if (!RKV_IN_BOUNDS(A.header, 5, it.t < (uint32_t)A.T && it.kc >= 1u && it.kc <= (uint32_t)kPartK &&
                                             it.k0 + it.kc <= (uint32_t)A.K, it.t))
             break;
@@ -1332,41 +1270,45 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __
         cur_t = (int)it.t; cur_k0 = (int)it.k0; cur_kc = (int)it.kc; cur_tile = it.tile;
         cur_slot = D.slot_by_tile ? it.tile : blockIdx.x;
         cur_te = tile_elems(D.cand_dtype);
+        // (the stage waited for above is consumed inside run_item: it holds the item's reference
+        // tile or its first candidate)
         switch (D.cand_dtype) {
             case RKV_F32: run_item<CK_F32>(A, smem, ring, B, it, D); break;
             case RKV_BF16: run_item<CK_BF16>(A, smem, ring, B, it, D); break;
             default: run_item<CK_F16>(A, smem, ring, B, it, D); break;
         }
     }
-    __syncthreads();
+    consumer_sync();
     if (cur_t >= 0) {
         flush_sums(recs, A, A.tensors[cur_t], cur_tile, cur_k0, cur_kc, tid);
         flush_records(recs, A, A.tensors[cur_t], cur_k0, cur_kc, cur_slot, tid, cur_te);
     }
     if (tid == 0 && *ring.ctl.abort_flag) atomicExch(&A.header->status, (int32_t)RKV_ERR_TIMEOUT);
+}
 
+// Persistent blocks, kBlocksPerSm per SM.
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __grid_constant__ Args A) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x;
+    Ring ring;
+    ring.full0 = smem_u32(smem + kOffFull);
+    ring.empty0 = smem_u32(smem + kOffEmpty);
+    ring.stage0 = smem_u32(smem + kOffStage);
+    ring.ctl.abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kOffAbort);
+    ring.ctl.limit = reinterpret_cast<const volatile long long*>(smem + kOffWaitLimit);
     if (tid == 0) {
-        // the last block to get here clears the ticket counter for the next launch
-        __threadfence();
-        if (atomicAdd(&A.header->blocks_done, 1u) == gridDim.x - 1u) {
-            A.header->next_ticket = 0u;
-            A.header->blocks_done = 0u;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(ring.full0 + 8 * s, 1);                    // the producer's arrive + the copy's bytes
+            mbar_init(ring.empty0 + 8 * s, kConsumerWarps);      // one release per consumer warp
         }
-        // A block that gave up must not retire with copies still landing in its shared
-        // memory: wait (bounded) for the copy issued last into each stage.
-        if (*ring.ctl.abort_flag) {
-            for (uint32_t s = 0; s < (uint32_t)kStages; ++s) {
-                const uint32_t jp1 = reinterpret_cast<volatile uint32_t*>(smem + kOffIssued)[s];
-                if (!jp1) continue;
-                const uint32_t ph = ((jp1 - 1u) / kStages) & 1u;
-                const long long t0 = clock64();
-                for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
-                    if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
-                    if (clock64() - t0 > 200000000LL) break;
-                }
-            }
-        }
+        *ring.ctl.abort_flag = 0u;
+        const unsigned long long lim = A.header->drill_issue ? A.header->drill_wait_cycles : 0ull;
+        *reinterpret_cast<volatile long long*>(smem + kOffWaitLimit) = lim ? (long long)lim : kWaitCycles;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncthreads();
+    if (tid >= kConsumers) producer_loop(A, smem, ring);
+    else consumer_loop(A, smem, ring);
 }
 
 // ----------------------------------------------------------------------------

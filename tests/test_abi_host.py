@@ -54,13 +54,13 @@ def test_stats_struct_is_88_bytes():
 
 
 @pytest.mark.parametrize("K", [1, 2, 8, 63, 64, 65, 128, 256, 1000])
-@pytest.mark.parametrize("n", [1, 127, 4096, 4097, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
+@pytest.mark.parametrize("n", [1, 127, 3584, 3585, 4096, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
 @pytest.mark.parametrize("dtype", [rkv.F32, rkv.BF16, rkv.F16])
 def test_item_plan_properties(n, K, dtype):
     sms = 148
     grid = 2 * sms
     tile, n_tiles, warm, parts_warm, parts_main, tail, parts_tail = rkv.plan_items(n, K, sms, dtype)
-    assert tile == (4096 if dtype == rkv.F32 else 8192)
+    assert tile == (3584 if dtype == rkv.F32 else 7168)
     assert (n_tiles - 1) * tile < n <= n_tiles * tile
     assert 1 <= warm <= n_tiles
     assert 1 <= parts_warm <= K and -(-K // parts_warm) <= 64
