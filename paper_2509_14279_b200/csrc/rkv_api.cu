@@ -336,10 +336,10 @@ int rkv_set_stream(void* cuda_stream) {
 }
 
 // Not part of the public interface (rkv.h does not declare it): arms a fault drill for the
-// next verification call of this process.  Block 0 of that call's kernel arms the ring
-// stage of its issue-th copy (1-based) but withholds the copy, and every bounded wait of
+// next verification call of this process.  Block 0 of that call's kernel skips its issue-th
+// copy (1-based; the ring stage is neither armed nor filled), and every bounded wait of
 // the launch gives up after wait_cycles clock cycles instead of about a second.  Nothing
-// is in flight and nothing faults: the block times out, drains and reports
+// is in flight because of it and nothing faults: the block times out, drains and reports
 // RKV_ERR_TIMEOUT through the status word.  issue == 0 disarms.
 int rkv_debug_fault_drill(unsigned int issue, unsigned long long wait_cycles) {
     std::lock_guard<std::mutex> lock(g_mutex);

@@ -119,8 +119,8 @@ struct WorkspaceHeader {
     uint32_t blocks_done;
     uint32_t reserved2;
     // Fault drill (a test makes a bounded wait run out without any memory fault):
-    // when drill_issue != 0, block 0 arms the ring stage of its drill_issue-th copy without
-    // issuing the copy, and every wait gives up after drill_wait_cycles clock cycles.
+    // when drill_issue != 0, block 0 skips its drill_issue-th copy (the ring stage is neither
+    // armed nor filled), and every wait gives up after drill_wait_cycles clock cycles.
     uint32_t drill_issue;
     uint32_t reserved0;
     unsigned long long drill_wait_cycles;

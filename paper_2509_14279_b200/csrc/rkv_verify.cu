@@ -332,15 +332,20 @@ __device__ __forceinline__ void producer_loop(const Args& A, unsigned char* smem
     ItemInfo* infos = reinterpret_cast<ItemInfo*>(smem + kOffInfo);
     const uint32_t drill = blockIdx.x == 0u ? A.header->drill_issue : 0u;
     uint32_t n_issued = 0, stage = 0, phase = 0, seg = 0, ord = 0;
+    uint32_t withheld = 0xFFFFFFFFu;          // ring stage a fault drill left unarmed
 
     auto issue = [&](const unsigned char* src, uint32_t bytes) {
-        // the stage is free once every consumer warp has released its previous use
-        mbar_wait(ring.empty0 + 8 * stage, phase ^ 1u, ring.ctl);
+        // the stage is free once every consumer warp has released its previous use; once a
+        // wait of the block has run out nothing more is issued
+        if (!mbar_wait(ring.empty0 + 8 * stage, phase ^ 1u, ring.ctl)) return;
         const uint32_t full = ring.full0 + 8 * stage;
-        if (bytes) {
+        if (n_issued + 1u == drill) {
+            // the fault drill of a test: this stage is neither armed nor filled, so whoever waits
+            // for it runs into the wait limit; nothing is in flight because of it
+            withheld = stage;
+        } else if (bytes) {
             mbar_expect_tx(full, bytes);
-            // (the fault drill of a test: arm the stage, withhold the copy)
-            if (n_issued + 1u != drill) bulk_g2s(ring.stage0 + stage * kStageBytes, src, bytes, full);
+            bulk_g2s(ring.stage0 + stage * kStageBytes, src, bytes, full);
         } else {
             mbar_arrive(full);
         }
@@ -367,7 +372,8 @@ __device__ __forceinline__ void producer_loop(const Args& A, unsigned char* smem
         const DevTensor& D = A.tensors[t];
         {
             const void* const* src = D.cands + k0;
-            for (uint32_t i = (uint32_t)lane; i < kc; i += 32u) table[i] = src[i];
+            for (uint32_t i = (uint32_t)lane; i < kc; i += 32u)
+                if (RKV_IN_BOUNDS(A.header, 6, i < (uint32_t)kPartK && k0 + i < (uint32_t)A.K, k0 + i)) table[i] = src[i];
         }
         __syncwarp();
         if (lane == 0) {
@@ -382,11 +388,14 @@ __device__ __forceinline__ void producer_loop(const Args& A, unsigned char* smem
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(D.ref) + start * rsz;
                 for (uint32_t r = 0; r < nref; ++r) {
                     const uint32_t lo = r * kStageBytes;
-                    issue(src + lo, rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u);
+                    uint32_t b = rbytes > lo ? min(rbytes - lo, (uint32_t)kStageBytes) : 0u;
+                    if (b && !RKV_IN_BOUNDS(A.header, 7, start * rsz + lo + b <= D.n * rsz, start)) b = 0u;
+                    issue(src + lo, b);
                 }
             }
-            const uint32_t cbytes = (len * csz) & ~15u;
+            uint32_t cbytes = (len * csz) & ~15u;
             const uint64_t c_off = start * csz;
+            if (cbytes && !RKV_IN_BOUNDS(A.header, 8, c_off + cbytes <= D.n * csz && cbytes <= (uint32_t)kStageBytes, c_off)) cbytes = 0u;
             for (uint32_t i = 0; i < kc; ++i)
                 issue(reinterpret_cast<const unsigned char*>(table[i]) + c_off, cbytes);
         }
@@ -413,6 +422,7 @@ __device__ __forceinline__ void producer_loop(const Args& A, unsigned char* smem
             for (uint32_t i = 0; i < pending; ++i) {
                 const uint32_t q = n_issued - 1 - i;
                 const uint32_t s = q % kStages, ph = (q / kStages) & 1u;
+                if (s == withheld) continue;
                 const long long t0 = clock64();
                 for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
                     if (mbar_try_wait(ring.full0 + 8 * s, ph)) break;
@@ -1127,6 +1137,9 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
     CandState* st_t = A.state + D.state_base;
 
+    // (range checks of a debug build: the tile lies inside the tensor; the state, hint and
+    // record tables are indexed by k0 + kk < K and kk < kPartK, checked with the item)
+    if (!RKV_IN_BOUNDS(A.header, 9, start < D.n && it.tile < D.n_tiles, it.tile)) return;
     // the part's pointers and hints, from the published state
     if (tid < kc) {
         const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
@@ -1196,6 +1209,7 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
         const Hint h = H[kk];
         uint32_t s;
         wait_stage(ring, B, s);
+        if (!RKV_IN_BOUNDS(A.header, 10, s < (uint32_t)kStages, s)) s = 0;
         const unsigned char* stage = stages + (size_t)s * kStageBytes;
         uint32_t w[NW];
 #pragma unroll
@@ -1283,7 +1297,7 @@ __device__ __forceinline__ void consumer_loop(const Args& A, unsigned char* smem
         flush_sums(recs, A, A.tensors[cur_t], cur_tile, cur_k0, cur_kc, tid);
         flush_records(recs, A, A.tensors[cur_t], cur_k0, cur_kc, cur_slot, tid, cur_te);
     }
-    if (tid == 0 && *ring.ctl.abort_flag) atomicExch(&A.header->status, (int32_t)RKV_ERR_TIMEOUT);
+    if (tid == 0 && *ring.ctl.abort_flag) atomicCAS(&A.header->status, (int32_t)RKV_OK, (int32_t)RKV_ERR_TIMEOUT);
 }
 
 // Persistent blocks, kBlocksPerSm per SM.

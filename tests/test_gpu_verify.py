@@ -447,3 +447,79 @@ def test_seeded_random_cases_match_the_oracle(case):
                       gen_inp=(300 + case, 2, dist) if with_input else None,
                       ref_dtype=rkv.F32 if ref_dtype == "f32" else rkv.BF16)
     assert got2.tobytes() == got.tobytes(), where
+
+
+@pytest.mark.parametrize("cand_dtype,ref_dtype", [("f16", "f32"), ("f16", "f16"), ("f32", "f16"), ("bf16", "f16")])
+@pytest.mark.parametrize("n", [1, 9, 7168, 7169, 100003])
+def test_fp16_storage(cand_dtype, ref_dtype, n):
+    """Half-precision candidates and references (the paper's kernels dispatch half too): widened
+    exactly, compared by the same rule; flags compare storage bits."""
+    K = 13
+    ref = oracle_gen_tensor(40, 0, oracle.NORMAL, n, "f32").to(torch_dtype_of(ref_dtype))
+    inp = oracle_gen_tensor(40, 2, oracle.NORMAL, n, "f32").to(torch_dtype_of(cand_dtype))
+    plan = mixed_plan(K, n, seed=40 + n % 7, bf16=cand_dtype != "f32")
+    cands = build_case_cpu(plan, ref, inp, cand_dtype)
+    tol = (1e-2, 1.6e-2) if cand_dtype == "bf16" else (1e-3, 2e-3)
+    got, want = check_case(ref, cands, tol[0], tol[1], inp, where=f"fp16 {cand_dtype}/{ref_dtype} n={n}")
+    if n > 1:
+        assert any(int(g["verdict"]) == 0 for g in got) and any(int(g["verdict"]) != 0 for g in got)
+
+
+def torch_dtype_of(code):
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[code]
+
+
+def test_fp16_cannot_be_regenerated():
+    n = 1024
+    c = [torch.zeros(n, dtype=torch.float16, device="cuda")]
+    d = rkv.TensorDesc(n=n, cands=c, atol=1e-3, rtol=1e-3, ref=torch.zeros(n, device="cuda"), input_gen=(0, 2, 0))
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.verify_multi([d], 1)
+    assert e.value.status == rkv.ERR_UNSUPPORTED
+    d = rkv.TensorDesc(n=n, cands=c, atol=1e-3, rtol=1e-3, ref_gen=(0, 0, 0), ref_dtype=rkv.F16)
+    with pytest.raises(rkv.RkvError) as e:
+        rkv.verify_multi([d], 1)
+    assert e.value.status == rkv.ERR_UNSUPPORTED
+
+
+def test_error_sum_bits_do_not_depend_on_which_block_took_which_tile():
+    """A tensor of thousands of tiles (blocks draw tickets: which block verifies which tile
+    differs from run to run) with heavy-tailed errors spanning many binades.  The sum is stored
+    per tile and added in tile order, so every run gives the same bits; a second workspace and
+    the host-buffer form (other launches, other candidate chunks) give them too."""
+    n, K = 3584 * 2500 + 11, 5
+    ref = oracle_gen_tensor(50, 0, oracle.NORMAL, n, "f32")
+    noise = oracle_gen_tensor(50, 4, oracle.STUDENT_T2, n, "f32")
+    cands = [ref + noise * s for s in (1e-9, 1e-4, 1.0, 1e4, 1e-12)]
+    runs = [run_gpu(ref, cands, ATOL, RTOL)[0] for _ in range(4)]
+    for r in runs[1:]:
+        assert r.tobytes() == runs[0].tobytes()
+    host = rkv.verify_batch_host(ref, cands, ATOL, RTOL)
+    assert host.tobytes() == runs[0].tobytes()
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], ATOL, RTOL)
+    for k in range(K):
+        assert_stats_equal(runs[0][k], want[k], f"k={k}")
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
+    """Fault drill: block 0 skips its third copy -- the ring stage is neither armed nor filled,
+    so nothing is in flight because of it and nothing faults -- and every wait of that launch
+    gives up after about a millisecond.  The kernel must return, the status word must say TIMEOUT, and the next
+    ordinary call on the same workspace must match the oracle."""
+    n, K = 3584 * 700 + 5, 6
+    ref = oracle_gen_tensor(60, 0, oracle.NORMAL, n, "f32")
+    cands_cpu = build_case_cpu(mixed_plan(K, n, seed=60), ref, ref, "f32")
+    cands = [c.cuda() for c in cands_cpu]
+    d = rkv.TensorDesc(n=n, cands=cands, atol=ATOL, rtol=RTOL, ref=ref.cuda())
+    stats, joint, ws = rkv.verify_multi([d], K)
+    assert rkv.device_status(ws) == rkv.OK
+    rkv.debug_fault_drill(3, 2_000_000)
+    rkv.verify_multi([d], K, workspace=ws, stats_out=stats, joint_pass=joint)
+    assert rkv.device_status(ws) == rkv.ERR_TIMEOUT
+    # the drill applied to that one call only
+    rkv.verify_multi([d], K, workspace=ws, stats_out=stats, joint_pass=joint)
+    assert rkv.device_status(ws) == rkv.OK
+    got = rkv.stats_to_numpy(stats)
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands_cpu], ATOL, RTOL)
+    for k in range(K):
+        assert_stats_equal(got[k], want[k], f"after the drill k={k}")
