@@ -75,6 +75,21 @@ class ScreenResult(ctypes.Structure):
         return {name: getattr(self, name) for name, _ in self._fields_ if not name.startswith("pad")}
 
 
+class CrossResult(ctypes.Structure):
+    _fields_ = [
+        ("flags", ctypes.c_uint32),
+        ("pad", ctypes.c_uint32),
+        ("n_nonfinite", ctypes.c_uint64),
+        ("argmax_spread", ctypes.c_uint64),
+        ("max_spread", ctypes.c_float),
+        ("pad2", ctypes.c_uint32),
+    ]
+
+    def as_dict(self) -> dict:
+        return {name: getattr(self, name) for name, _ in self._fields_ if not name.startswith("pad")}
+
+
+CROSS_IDENTICAL, CROSS_WITHIN_TOL, CROSS_LOW_SPREAD, CROSS_NONFINITE = 1, 2, 4, 8
 SCREEN_NARROW_RANGE, SCREEN_LOW_STD, SCREEN_LOW_SEED_VARIATION = 1, 2, 4
 SCREEN_UNIFORM_AXIS0, SCREEN_UNIFORM_AXIS1, SCREEN_NONFINITE = 8, 16, 32
 
@@ -138,6 +153,12 @@ def lib() -> ctypes.CDLL:
                                  ctypes.c_uint64, ctypes.c_int, ctypes.c_float, ctypes.c_double,
                                  ctypes.c_float, ctypes.POINTER(ScreenResult)]
         L.orc_screen.restype = ctypes.c_int
+        L.orc_cross_seed.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_uint64, ctypes.c_int,
+                                     ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.POINTER(CrossResult)]
+        L.orc_cross_seed.restype = ctypes.c_int
+        L.orc_copy_of_inputs.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_void_p,
+                                         ctypes.c_uint64, ctypes.c_int, ctypes.POINTER(ctypes.c_uint32)]
+        L.orc_copy_of_inputs.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -275,3 +296,34 @@ def screen(outs, range_lim: float = 0.01, std_lim: float = 0.01, spread_lim: flo
     if rc != 0:
         raise ValueError("orc_screen: bad argument")
     return r.as_dict()
+
+
+def cross_seed(outs, atol: float, rtol: float, spread_lim: float = 0.01) -> dict:
+    """Cross-seed variation of one candidate: outs[s] is its output for input seed s."""
+    arrs = [np.ascontiguousarray(a).reshape(-1) for a in outs]
+    for a in arrs:
+        if a.size != arrs[0].size or a.dtype != arrs[0].dtype:
+            raise ValueError("outputs differ in size or dtype")
+    ptrs = (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    r = CrossResult()
+    rc = lib().orc_cross_seed(ptrs, len(arrs), arrs[0].size, _dtype_of(arrs[0]), float(atol), float(rtol),
+                              float(spread_lim), ctypes.byref(r))
+    if rc != 0:
+        raise ValueError("orc_cross_seed: bad argument")
+    return r.as_dict()
+
+
+def copy_of_inputs(inputs, cand) -> int:
+    """Bit m set iff cand is a bit copy of inputs[m]."""
+    arrs = [np.ascontiguousarray(a).reshape(-1) for a in inputs]
+    c = np.ascontiguousarray(cand).reshape(-1)
+    for a in arrs:
+        if a.size != c.size or a.dtype != c.dtype:
+            raise ValueError("inputs and candidate differ in size or dtype")
+    ptrs = (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    m = ctypes.c_uint32()
+    rc = lib().orc_copy_of_inputs(ptrs, len(arrs), c.ctypes.data_as(ctypes.c_void_p), c.size, _dtype_of(c),
+                                  ctypes.byref(m))
+    if rc != 0:
+        raise ValueError("orc_copy_of_inputs: bad argument")
+    return int(m.value)

@@ -463,3 +463,77 @@ int orc_screen(const void *const *outs, int S, uint64_t rows, uint64_t cols, int
     res->flags = f;
     return 0;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Cross-seed variation of ONE candidate's outputs (Sec. 3: a loophole is an  */
+/* output with "insufficient variation across different seeds"; a kernel that */
+/* hard-codes its result ignores the input seed altogether).  outs[s] is the  */
+/* candidate's output for input seed s; seed 0 plays the reference.           */
+/* ------------------------------------------------------------------------- */
+int orc_cross_seed(const void *const *outs, int S, uint64_t n, int dtype, float atol, float rtol,
+                   float spread_lim, orc_cross_result *res)
+{
+    if (!outs || !res || S < 1 || n < 1 || !dtype_known(dtype)) return -1;
+    for (int s = 0; s < S; ++s) if (!outs[s]) return -1;
+
+    int identical = 1, within = 1;
+    uint64_t n_nonfin = 0, arg = ORC_NO_INDEX;
+    float spread = -1.0f;
+    for (uint64_t i = 0; i < n; ++i) {
+        const uint32_t b0 = load_bits(outs[0], dtype, i);
+        const float x0 = bits_f32(b0);
+        float lo = INFINITY, hi = -INFINITY;
+        int all_finite = 1;
+        for (int s = 0; s < S; ++s) {
+            const uint32_t b = load_bits(outs[s], dtype, i);
+            const float x = bits_f32(b);
+            if (b != b0) identical = 0;             /* the widening is one-to-one: storage bits differ */
+            if (!bits_is_finite(b)) all_finite = 0;
+            if (s > 0) {
+                /* the tolerance rule with seed 0's output on the right */
+                int close;
+                if (bits_is_finite(b) && bits_is_finite(b0))
+                    close = fabsf(x - x0) <= atol + (rtol * fabsf(x0));
+                else
+                    close = bits_is_inf(b) && b == b0;
+                if (!close) within = 0;
+            }
+            if (x < lo) lo = x;
+            if (x > hi) hi = x;
+        }
+        if (!all_finite) { n_nonfin++; continue; }
+        const float d = hi - lo;                    /* one fp32 subtraction */
+        if (d > spread) { spread = d; arg = i; }
+    }
+    memset(res, 0, sizeof *res);
+    res->n_nonfinite = n_nonfin;
+    res->argmax_spread = (S >= 2) ? arg : ORC_NO_INDEX;
+    res->max_spread = (S >= 2) ? spread : -1.0f;
+    uint32_t flags = 0;
+    if (S >= 2 && identical) flags |= ORC_CROSS_IDENTICAL;
+    if (S >= 2 && within) flags |= ORC_CROSS_WITHIN_TOL;
+    if (S >= 2 && spread >= 0.0f && spread < spread_lim) flags |= ORC_CROSS_LOW_SPREAD;
+    if (n_nonfin) flags |= ORC_CROSS_NONFINITE;
+    res->flags = flags;
+    return 0;
+}
+
+/* Which of the M input tensors (the operands a kernel receives: activations, weights,
+ * the incoming gradient ...) is the candidate output a bit copy of?  Bit m of the result is
+ * set iff every element of cand has the storage bits of inputs[m].  All tensors have n
+ * elements of dtype. */
+int orc_copy_of_inputs(const void *const *inputs, int M, const void *cand, uint64_t n, int dtype,
+                       uint32_t *mask)
+{
+    if (!inputs || !cand || !mask || M < 1 || M > 32 || n < 1 || !dtype_known(dtype)) return -1;
+    uint32_t m_out = 0;
+    for (int m = 0; m < M; ++m) {
+        if (!inputs[m]) return -1;
+        int same = 1;
+        for (uint64_t i = 0; i < n; ++i)
+            if (load_bits(cand, dtype, i) != load_bits(inputs[m], dtype, i)) { same = 0; break; }
+        if (same) m_out |= 1u << m;
+    }
+    *mask = m_out;
+    return 0;
+}

@@ -172,6 +172,42 @@ typedef struct orc_screen_result {
 int orc_screen(const void *const *outs, int S, uint64_t rows, uint64_t cols, int dtype,
                float range_lim, double std_lim, float spread_lim, orc_screen_result *res);
 
+/* ---- cross-seed variation of a candidate, copy of any input (Sec. 3, the loophole list:
+ * "insufficient output variation across different seeds", "hardcoding for specific input
+ * patterns"; App. A.1, criterion 4 read on a candidate's outputs instead of the task's).
+ * Readings taken, the paper giving no formula (parity unpinned for the readings; the
+ * arithmetic is pinned by whole-array numpy restatements and planted cases):
+ *   IDENTICAL    every seed's output has the storage bits of seed 0's output;
+ *   WITHIN_TOL   every seed's output is within atol + rtol*|x_0| of seed 0's output, element
+ *                by element, by the comparison rule of orc_verify (NaN never close, equal
+ *                infinities close);
+ *   LOW_SPREAD   the largest per-element spread max_s x_s[i] - min_s x_s[i] (one fp32
+ *                subtraction; elements not finite in some seed are left out) is below
+ *                spread_lim;
+ * with S == 1 nothing is flagged and max_spread is -1. */
+enum {
+    ORC_CROSS_IDENTICAL = 1u << 0,
+    ORC_CROSS_WITHIN_TOL = 1u << 1,
+    ORC_CROSS_LOW_SPREAD = 1u << 2,
+    ORC_CROSS_NONFINITE = 1u << 3
+};
+
+typedef struct orc_cross_result {
+    uint32_t flags;
+    uint32_t pad;
+    uint64_t n_nonfinite;       /* elements with a non-finite value in some seed */
+    uint64_t argmax_spread;     /* first element with the largest spread; ORC_NO_INDEX if none */
+    float max_spread;           /* -1 when S < 2 or no element is finite in every seed */
+    uint32_t pad2;
+} orc_cross_result;
+
+int orc_cross_seed(const void *const *outs, int S, uint64_t n, int dtype, float atol, float rtol,
+                   float spread_lim, orc_cross_result *res);
+
+/* Bit m of *mask: cand is a bit copy of inputs[m] (M <= 32 tensors of n elements of dtype). */
+int orc_copy_of_inputs(const void *const *inputs, int M, const void *cand, uint64_t n, int dtype,
+                       uint32_t *mask);
+
 #ifdef __cplusplus
 }
 #endif
