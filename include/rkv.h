@@ -430,6 +430,76 @@ int rkv_screen_outputs(const void *const *outs, int S, uint64_t rows, uint64_t c
                        float range_lim, double std_lim, float spread_lim, rkv_screen_stats *stats_out,
                        void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* ------------------------------------------------------------------------------------
+ * Two loophole checks that need no reference (Sec. 3, the loophole list: "insufficient
+ * output variation across different seeds", "hardcoding for specific input patterns";
+ * App. A.1, criterion 4 read on a candidate's outputs instead of the task's).
+ *
+ * Cross-seed variation.  A candidate kernel is run on S input seeds; a kernel that
+ * ignores its input (a hard-coded result) produces the same output every time.  With
+ * x_s[i] the candidate's output for seed s, widened to fp32, the readings taken (the paper
+ * gives no formula):
+ *   IDENTICAL    every x_s has the storage bits of x_0;
+ *   WITHIN_TOL   every x_s is within atol + rtol*|x_0| of x_0, element by element, by the
+ *                comparison rule of rkv_stats with x_0 as the reference (NaN never close,
+ *                equal infinities close);
+ *   LOW_SPREAD   the largest per-element spread max_s x_s[i] - min_s x_s[i] (one fp32
+ *                subtraction; elements not finite in some seed are left out) is below
+ *                spread_lim (0.01 in the paper's filtering criteria);
+ *   NONFINITE    informative: some element is NaN or infinite in some seed.
+ * With S == 1 none of the first three is set and max_spread is -1.
+ * ------------------------------------------------------------------------------------ */
+enum rkv_cross_flag {
+    RKV_CROSS_IDENTICAL = 1u << 0,
+    RKV_CROSS_WITHIN_TOL = 1u << 1,
+    RKV_CROSS_LOW_SPREAD = 1u << 2,
+    RKV_CROSS_NONFINITE = 1u << 3
+};
+
+typedef struct rkv_cross_stats {
+    uint32_t flags;             /* rkv_cross_flag bits */
+    uint32_t reserved;
+    uint64_t n_nonfinite;       /* elements with a non-finite value in some seed */
+    uint64_t argmax_spread;     /* first element with the largest spread; RKV_NO_INDEX if none */
+    float max_spread;           /* -1 when S < 2 or no element is finite in every seed */
+    uint32_t reserved2;
+} rkv_cross_stats;              /* 32 bytes */
+
+/* Bytes of device workspace rkv_cross_seed needs on the current device (0 on a bad argument
+ * or without a device). */
+size_t rkv_cross_workspace_bytes(int K, int S);
+
+/*
+ * Cross-seed variation of K candidates in one launch; every output byte is read once.
+ *   outs         HOST array of K*S DEVICE pointers, outs[k*S + s] = candidate k's output for
+ *                input seed s: n elements of dtype, contiguous, 16-byte aligned, only read
+ *   K, S         1 <= K <= 4096, 1 <= S <= 16
+ *   dtype        RKV_F32 | RKV_BF16 | RKV_F16
+ *   stats_out    DEVICE, K rkv_cross_stats
+ *   workspace    DEVICE, >= rkv_cross_workspace_bytes(K, S), 16-byte aligned
+ * Errors: INVALID_ARG, UNSUPPORTED (limits above, n >= 2^40, capturing stream), ALIGNMENT,
+ * WORKSPACE, CUDA.
+ */
+int rkv_cross_seed(const void *const *outs, int K, int S, uint64_t n, int dtype, float atol, float rtol,
+                   float spread_lim, rkv_cross_stats *stats_out, void *workspace, size_t workspace_bytes,
+                   void *cuda_stream);
+
+size_t rkv_copy_workspace_bytes(int K, int M);
+
+/*
+ * Copy of any input: a kernel receives several operands (activations, weights, the incoming
+ * gradient); an output that is a bit copy of one of them passes a value check whenever
+ * the reference happens to equal that operand, and is a pass-through either way.
+ *   inputs         HOST array of M DEVICE pointers (1 <= M <= 8), n elements of dtype each
+ *   cands          HOST array of K DEVICE pointers (1 <= K <= 4096), n elements of dtype each
+ *   copy_mask_out  DEVICE, K uint32: bit m set iff candidate k has the storage bytes of
+ *                  inputs[m] throughout (+0 and -0 differ)
+ * A candidate is compared with an operand until a difference has been seen; only true
+ * copies are read to the end.  Errors as rkv_cross_seed.
+ */
+int rkv_copy_of_inputs(const void *const *inputs, int M, const void *const *cands, int K, uint64_t n, int dtype,
+                       uint32_t *copy_mask_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

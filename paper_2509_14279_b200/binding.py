@@ -42,6 +42,10 @@ SCREEN_DTYPE = np.dtype([
     ("argmax_seed_spread", "<u8"), ("mean", "<f8"), ("std", "<f8"), ("vmin", "<f4"), ("vmax", "<f4"),
     ("max_seed_spread", "<f4"), ("reserved2", "<u4")])
 SCREEN_BYTES = SCREEN_DTYPE.itemsize
+CROSS_DTYPE = np.dtype([("flags", "<u4"), ("reserved", "<u4"), ("n_nonfinite", "<u8"), ("argmax_spread", "<u8"),
+                        ("max_spread", "<f4"), ("reserved2", "<u4")])
+CROSS_BYTES = CROSS_DTYPE.itemsize
+CROSS_IDENTICAL, CROSS_WITHIN_TOL, CROSS_LOW_SPREAD, CROSS_NONFINITE = 1, 2, 4, 8
 SCREEN_NARROW_RANGE, SCREEN_LOW_STD, SCREEN_LOW_SEED_VARIATION = 1, 2, 4
 SCREEN_UNIFORM_AXIS0, SCREEN_UNIFORM_AXIS1, SCREEN_NONFINITE = 8, 16, 32
 assert STATS_BYTES == 88
@@ -123,6 +127,15 @@ def lib() -> ctypes.CDLL:
         L.rkv_debug_fault_drill.argtypes = [ctypes.c_uint, ctypes.c_ulonglong]
         L.rkv_debug_bounds_build.restype = i32
         L.rkv_debug_bounds_build.argtypes = []
+        L.rkv_cross_workspace_bytes.restype = ctypes.c_size_t
+        L.rkv_cross_workspace_bytes.argtypes = [i32, i32]
+        L.rkv_cross_seed.restype = i32
+        L.rkv_cross_seed.argtypes = [ctypes.POINTER(vp), i32, i32, u64, i32, f32, f32, f32, vp, vp, ctypes.c_size_t, vp]
+        L.rkv_copy_workspace_bytes.restype = ctypes.c_size_t
+        L.rkv_copy_workspace_bytes.argtypes = [i32, i32]
+        L.rkv_copy_of_inputs.restype = i32
+        L.rkv_copy_of_inputs.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, u64, i32, vp, vp,
+                                         ctypes.c_size_t, vp]
         L.rkv_verify_batch_static.restype = i32
         L.rkv_verify_batch_static.argtypes = [vp, ctypes.POINTER(vp), i32, u64, i32, f32, f32, vp, vp]
         u32p = ctypes.POINTER(ctypes.c_uint32)
@@ -532,3 +545,59 @@ def screen_outputs(outs, range_lim: float = 0.01, std_lim: float = 0.01, spread_
 
 def screen_to_numpy(stats: torch.Tensor) -> np.ndarray:
     return stats.detach().cpu().numpy().view(SCREEN_DTYPE)
+
+
+def cross_seed(outs, atol: float, rtol: float, spread_lim: float = 0.01, stats_out: torch.Tensor | None = None,
+               workspace: torch.Tensor | None = None, stream=None) -> tuple:
+    """rkv_cross_seed: outs[k][s] is candidate k's output for input seed s (device tensors of one
+    size and dtype).  Returns (stats [K * 32 bytes, uint8], workspace)."""
+    K, S = len(outs), len(outs[0])
+    first = outs[0][0]
+    _require(first, "cross_seed: outs[0][0]", device=torch.device("cuda"))
+    code = _dtype_code(first)
+    for k, row in enumerate(outs):
+        if len(row) != S:
+            raise ValueError("cross_seed: every candidate needs the same number of seeds")
+        for s, t in enumerate(row):
+            _require(t, f"cross_seed: outs[{k}][{s}]", device=first.device, dtype=first.dtype, numel=first.numel())
+    dev = first.device
+    if workspace is None:
+        workspace = torch.empty(max(256, int(lib().rkv_cross_workspace_bytes(K, S))), dtype=torch.uint8, device=dev)
+    if stats_out is None:
+        stats_out = torch.empty(K * CROSS_BYTES, dtype=torch.uint8, device=dev)
+    else:
+        _require(stats_out, "cross_seed: stats_out", device=dev, dtype=torch.uint8, min_bytes=K * CROSS_BYTES)
+    ptrs = (ctypes.c_void_p * (K * S))(*[t.data_ptr() for row in outs for t in row])
+    _check(lib().rkv_cross_seed(ptrs, K, S, first.numel(), code, float(atol), float(rtol), float(spread_lim),
+                                ctypes.c_void_p(stats_out.data_ptr()), ctypes.c_void_p(workspace.data_ptr()),
+                                workspace.numel(), ctypes.c_void_p(_stream_ptr(stream))), "rkv_cross_seed")
+    return stats_out, workspace
+
+
+def cross_to_numpy(stats: torch.Tensor) -> np.ndarray:
+    return stats.detach().cpu().numpy().view(CROSS_DTYPE)
+
+
+def copy_of_inputs(inputs, cands, mask_out: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                   stream=None) -> tuple:
+    """rkv_copy_of_inputs: bit m of mask[k] is set iff candidate k is a bit copy of inputs[m].
+    Returns (mask [K] int32 on the device, workspace)."""
+    K, M = len(cands), len(inputs)
+    first = cands[0]
+    _require(first, "copy_of_inputs: candidate 0", device=torch.device("cuda"))
+    code = _dtype_code(first)
+    for i, t in enumerate(list(inputs) + list(cands)):
+        _require(t, f"copy_of_inputs: tensor {i}", device=first.device, dtype=first.dtype, numel=first.numel())
+    dev = first.device
+    if workspace is None:
+        workspace = torch.empty(max(256, int(lib().rkv_copy_workspace_bytes(K, M))), dtype=torch.uint8, device=dev)
+    if mask_out is None:
+        mask_out = torch.empty(K, dtype=torch.int32, device=dev)
+    else:
+        _require(mask_out, "copy_of_inputs: mask_out", device=dev, dtype=torch.int32, numel=K)
+    ip = (ctypes.c_void_p * M)(*[t.data_ptr() for t in inputs])
+    cp = (ctypes.c_void_p * K)(*[t.data_ptr() for t in cands])
+    _check(lib().rkv_copy_of_inputs(ip, M, cp, K, first.numel(), code, ctypes.c_void_p(mask_out.data_ptr()),
+                                    ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                    ctypes.c_void_p(_stream_ptr(stream))), "rkv_copy_of_inputs")
+    return mask_out, workspace

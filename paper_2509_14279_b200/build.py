@@ -23,7 +23,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librkv.so")
 LIB_DBG = os.path.join(PKG, "librkv_dbg.so")
-SOURCES = ["rkv_api.cu", "rkv_gen.cu", "rkv_verify.cu", "rkv_screen.cu"]
+SOURCES = ["rkv_api.cu", "rkv_gen.cu", "rkv_verify.cu", "rkv_screen.cu", "rkv_cross.cu"]
 HEADERS = ["rkv_internal.h", "rkv_philox.cuh"]
 
 NVCC_FLAGS = [

@@ -1,0 +1,370 @@
+// Two loophole checks on candidate outputs that need no reference (sm_100a):
+//
+//   * cross-seed variation: the outputs of K candidates for S input seeds, K * S tensors, in
+//     one launch.  For one vector position a thread visits the S outputs of its candidate in
+//     turn, so the per-element minimum and maximum across seeds, and seed 0's value, never
+//     leave registers; every output byte is read once.  Bound: HBM read bandwidth
+//     (K * S * n * element size bytes);
+//   * copy of any input: is a candidate's output a bit copy of one of the M operands the
+//     kernel received?  16-byte pieces are compared as stored; a block stops comparing
+//     against an operand as soon as any block has seen a difference, so only true copies are
+//     read to the end.
+//
+// Reductions are deterministic: integer sums, boolean ands, lexicographic (value descending,
+// index ascending) maxima, one partial per block merged in block order.
+#include <string.h>
+
+#include <vector>
+
+#include "rkv_internal.h"
+
+namespace rkv {
+
+namespace {
+
+constexpr int kCrossThreads = 256;
+constexpr int kCrossBlocksPerSm = 6;
+constexpr int kCrossMaxSeeds = 16;
+constexpr int kCopyMaxInputs = 8;
+constexpr int kCrossMaxK = 4096;
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+constexpr float kInfF = __builtin_huge_valf();
+
+__device__ __forceinline__ bool finite_bits(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
+__device__ __forceinline__ bool inf_bits(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
+
+// 16 storage bits -> the fp32 bit pattern of the same value.
+template <int DT>
+__device__ __forceinline__ uint32_t widen(uint32_t raw) {
+    if (DT == RKV_F32) return raw;
+    if (DT == RKV_BF16) return raw << 16;
+    float f;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"((unsigned short)raw));
+    return __float_as_uint(f);
+}
+
+struct __align__(16) CrossPartial {
+    unsigned long long arg;        // first element with the largest spread
+    unsigned long long n_nonfin;
+    float spread;                  // -1: none
+    uint32_t differs;              // bit0: some seed differs from seed 0 in bits; bit1: some seed is not within tolerance
+    uint32_t reserved[2];
+};
+static_assert(sizeof(CrossPartial) == 32, "CrossPartial layout");
+
+struct CrossAcc {
+    unsigned long long arg, n_nonfin;
+    float spread;
+    uint32_t differs;
+};
+
+__device__ __forceinline__ void merge(CrossAcc& a, const CrossAcc& b) {
+    if (b.spread > a.spread || (b.spread == a.spread && b.arg < a.arg)) { a.spread = b.spread; a.arg = b.arg; }
+    a.n_nonfin += b.n_nonfin;
+    a.differs |= b.differs;
+}
+
+// What one element position contributes, given its value in every seed so far.
+struct ElemState {
+    uint32_t b0;       // seed 0, widened bits
+    float lo, hi;
+    bool finite;
+};
+
+template <int DT>
+__device__ __forceinline__ void visit(ElemState& e, CrossAcc& a, uint32_t raw, uint32_t raw0, bool first,
+                                      float atol, float rtol) {
+    const uint32_t b = widen<DT>(raw);
+    const float x = __uint_as_float(b);
+    if (first) {
+        e.b0 = b; e.lo = x; e.hi = x; e.finite = finite_bits(b);
+        return;
+    }
+    if (raw != raw0) a.differs |= 1u;
+    const float x0 = __uint_as_float(e.b0);
+    bool close;
+    if (finite_bits(b) && finite_bits(e.b0))
+        close = fabsf(__fsub_rn(x, x0)) <= __fadd_rn(atol, __fmul_rn(rtol, fabsf(x0)));
+    else
+        close = inf_bits(b) && b == e.b0;
+    if (!close) a.differs |= 2u;
+    e.finite = e.finite && finite_bits(b);
+    // (min / max of a NaN leave the other operand: the element is left out anyway)
+    e.lo = fminf(e.lo, x);
+    e.hi = fmaxf(e.hi, x);
+}
+
+__device__ __forceinline__ void finish(const ElemState& e, CrossAcc& a, unsigned long long index) {
+    if (!e.finite) { a.n_nonfin++; return; }
+    const float d = __fsub_rn(e.hi, e.lo);
+    if (d > a.spread) { a.spread = d; a.arg = index; }       // ascending index: the first maximum stays
+}
+
+// grid = (blocks per candidate, K).  outs[k * S + s]: candidate k's output for input seed s.
+template <int DT>
+__global__ void __launch_bounds__(kCrossThreads)
+cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long long n, float atol, float rtol,
+                  CrossPartial* __restrict__ partials) {
+    constexpr int VEC = DT == RKV_F32 ? 4 : 8;
+    constexpr int CH = DT == RKV_F32 ? 8 : 4;            // outputs whose loads are issued together
+    const int k = blockIdx.y;
+    const void* const* mine = outs + (size_t)k * (size_t)S;
+    const unsigned long long n_vec = n / VEC;
+    CrossAcc a;
+    a.arg = RKV_NO_INDEX; a.n_nonfin = 0; a.spread = -1.0f; a.differs = 0;
+
+    for (unsigned long long v = (unsigned long long)blockIdx.x * kCrossThreads + threadIdx.x; v < n_vec;
+         v += (unsigned long long)gridDim.x * kCrossThreads) {
+        ElemState e[VEC];
+        uint32_t raw0[VEC];
+        for (int s0 = 0; s0 < S; s0 += CH) {
+            uint4 w[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c)
+                if (s0 + c < S) w[c] = __ldcs(reinterpret_cast<const uint4*>(mine[s0 + c]) + v);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                if (s0 + c >= S) break;
+                const uint32_t words[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                    const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
+                    if (s0 + c == 0) raw0[i] = raw;
+                    visit<DT>(e[i], a, raw, raw0[i], s0 + c == 0, atol, rtol);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) finish(e[i], a, v * VEC + i);
+    }
+    // the ragged end: fewer elements than a vector, one thread of the first block
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (unsigned long long i = n_vec * VEC; i < n; ++i) {
+            ElemState e;
+            uint32_t raw0 = 0;
+            for (int s = 0; s < S; ++s) {
+                const uint32_t raw = DT == RKV_F32 ? reinterpret_cast<const uint32_t*>(mine[s])[i]
+                                                   : reinterpret_cast<const unsigned short*>(mine[s])[i];
+                if (s == 0) raw0 = raw;
+                visit<DT>(e, a, raw, raw0, s == 0, atol, rtol);
+            }
+            finish(e, a, i);
+        }
+    }
+    // block reduction: shuffle tree, then the warps' results in warp order
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        CrossAcc b;
+        b.arg = __shfl_xor_sync(kFull, a.arg, off);
+        b.n_nonfin = __shfl_xor_sync(kFull, a.n_nonfin, off);
+        b.spread = __shfl_xor_sync(kFull, a.spread, off);
+        b.differs = __shfl_xor_sync(kFull, a.differs, off);
+        merge(a, b);
+    }
+    __shared__ CrossAcc warp_acc[kCrossThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_acc[threadIdx.x >> 5] = a;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CrossAcc t = warp_acc[0];
+        for (int w = 1; w < kCrossThreads / 32; ++w) merge(t, warp_acc[w]);
+        CrossPartial p;
+        p.arg = t.arg; p.n_nonfin = t.n_nonfin; p.spread = t.spread; p.differs = t.differs;
+        p.reserved[0] = p.reserved[1] = 0;
+        partials[(size_t)k * gridDim.x + blockIdx.x] = p;
+    }
+}
+
+__global__ void cross_finalize_kernel(const CrossPartial* __restrict__ partials, int K, int S, int blocks,
+                                      float spread_lim, rkv_cross_stats* __restrict__ stats_out) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    CrossAcc t;
+    t.arg = RKV_NO_INDEX; t.n_nonfin = 0; t.spread = -1.0f; t.differs = 0;
+    for (int b = 0; b < blocks; ++b) {
+        const CrossPartial p = partials[(size_t)k * blocks + b];
+        CrossAcc q;
+        q.arg = p.arg; q.n_nonfin = p.n_nonfin; q.spread = p.spread; q.differs = p.differs;
+        merge(t, q);
+    }
+    rkv_cross_stats st;
+    memset(&st, 0, sizeof st);
+    st.n_nonfinite = t.n_nonfin;
+    st.argmax_spread = S >= 2 ? t.arg : RKV_NO_INDEX;
+    st.max_spread = S >= 2 ? t.spread : -1.0f;
+    uint32_t flags = 0;
+    if (S >= 2 && !(t.differs & 1u)) flags |= RKV_CROSS_IDENTICAL;
+    if (S >= 2 && !(t.differs & 2u)) flags |= RKV_CROSS_WITHIN_TOL;
+    if (S >= 2 && t.spread >= 0.0f && t.spread < spread_lim) flags |= RKV_CROSS_LOW_SPREAD;
+    if (t.n_nonfin) flags |= RKV_CROSS_NONFINITE;
+    st.flags = flags;
+    stats_out[k] = st;
+}
+
+// ---- copy of any input ------------------------------------------------------------------
+// grid = (blocks per candidate, K).  differs[k]: bit m set once candidate k is known to
+// differ from input m.
+__global__ void __launch_bounds__(kCrossThreads)
+copy_any_kernel(const void* const* __restrict__ inputs, int M, const void* const* __restrict__ cands,
+                unsigned long long n_bytes, uint32_t* __restrict__ differs) {
+    const int k = blockIdx.y;
+    const unsigned char* c = reinterpret_cast<const unsigned char*>(cands[k]);
+    const uint32_t all = (1u << M) - 1u;
+    const unsigned long long n_vec = n_bytes / 16;
+    __shared__ uint32_t s_known;
+    uint32_t known = 0;                                  // inputs this block need not look at any more
+    uint32_t found = 0;                                  // differences this thread has seen
+    unsigned long long v = (unsigned long long)blockIdx.x * kCrossThreads + threadIdx.x;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kCrossThreads;
+    // the trip count is the same for every thread of the block: barriers inside the loop
+    const unsigned long long trips = (n_vec + stride - 1) / stride;
+    for (unsigned long long it = 0; it < trips; ++it, v += stride) {
+        if ((it & 7u) == 0u) {
+            // every eighth round: publish what this block has found, pick up what others have
+            const uint32_t warp_found = __reduce_or_sync(kFull, found);
+            if ((threadIdx.x & 31) == 0 && warp_found) atomicOr(&differs[k], warp_found);
+            found = 0;
+            __syncthreads();
+            if (threadIdx.x == 0) s_known = atomicOr(&differs[k], 0u);
+            __syncthreads();
+            known = s_known;
+            if (known == all) break;                     // block-uniform
+        }
+        if (v < n_vec) {
+            const uint4 cv = __ldcs(reinterpret_cast<const uint4*>(c) + v);
+            for (int m = 0; m < M; ++m) {
+                if ((known >> m) & 1u) continue;
+                const uint4 iv = __ldg(reinterpret_cast<const uint4*>(inputs[m]) + v);
+                if ((cv.x ^ iv.x) | (cv.y ^ iv.y) | (cv.z ^ iv.z) | (cv.w ^ iv.w)) found |= 1u << m;
+            }
+        }
+    }
+    // the bytes behind the last whole 16-byte piece
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (unsigned long long b = n_vec * 16; b < n_bytes; ++b)
+            for (int m = 0; m < M; ++m)
+                if (c[b] != reinterpret_cast<const unsigned char*>(inputs[m])[b]) found |= 1u << m;
+    }
+    if (found) atomicOr(&differs[k], found);
+}
+
+__global__ void copy_finalize_kernel(const uint32_t* __restrict__ differs, int K, int M, uint32_t* __restrict__ mask_out) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < K) mask_out[k] = ~differs[k] & ((1u << M) - 1u);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int blocks_per_candidate(uint64_t units, int K, int sms) {
+    uint64_t want = (units + kCrossThreads - 1) / kCrossThreads;
+    if (want < 1) want = 1;
+    uint64_t cap = ((uint64_t)sms * kCrossBlocksPerSm + (uint64_t)K - 1) / (uint64_t)K;
+    if (cap < 1) cap = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+}  // namespace
+}  // namespace rkv
+
+using namespace rkv;
+
+extern "C" {
+
+size_t rkv_cross_workspace_bytes(int K, int S) {
+    if (K < 1 || K > kCrossMaxK || S < 1 || S > kCrossMaxSeeds) return 0;
+    int sms = 0;
+    if (current_num_sms(&sms) != RKV_OK) return 0;
+    const size_t ptr_bytes = ((size_t)K * S * sizeof(void*) + 255) / 256 * 256;
+    // at most sms * kCrossBlocksPerSm + K blocks in all
+    return ptr_bytes + ((size_t)sms * kCrossBlocksPerSm + (size_t)K) * sizeof(CrossPartial);
+}
+
+int rkv_cross_seed(const void* const* outs, int K, int S, uint64_t n, int dtype, float atol, float rtol,
+                   float spread_lim, rkv_cross_stats* stats_out, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream) {
+    if (!outs || !stats_out || K < 1 || S < 1 || n < 1) return RKV_ERR_INVALID_ARG;
+    if (dtype != RKV_F32 && dtype != RKV_BF16 && dtype != RKV_F16) return RKV_ERR_INVALID_ARG;
+    if (!(atol >= 0.0f) || !(rtol >= 0.0f) || !(spread_lim >= 0.0f) || atol > 3.402823466e38f ||
+        rtol > 3.402823466e38f)
+        return RKV_ERR_INVALID_ARG;
+    if (K > kCrossMaxK || S > kCrossMaxSeeds || n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+    for (int i = 0; i < K * S; ++i) {
+        if (!outs[i]) return RKV_ERR_INVALID_ARG;
+        if (!aligned16(outs[i])) return RKV_ERR_ALIGNMENT;
+    }
+    if (!workspace) return RKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return RKV_ERR_ALIGNMENT;
+    int sms = 0;
+    int rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    if (workspace_bytes < rkv_cross_workspace_bytes(K, S)) return RKV_ERR_WORKSPACE;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    rc = refuse_capture(stream);                 // the pointer table travels from host memory of this call
+    if (rc != RKV_OK) return rc;
+    const size_t ptr_bytes = ((size_t)K * S * sizeof(void*) + 255) / 256 * 256;
+    const void** d_ptrs = reinterpret_cast<const void**>(workspace);
+    CrossPartial* partials = reinterpret_cast<CrossPartial*>(reinterpret_cast<unsigned char*>(workspace) + ptr_bytes);
+    if (cudaMemcpyAsync(d_ptrs, outs, (size_t)K * S * sizeof(void*), cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return RKV_ERR_CUDA;
+    }
+    const int vec = dtype == RKV_F32 ? 4 : 8;
+    const int blocks = blocks_per_candidate(n / vec, K, sms);
+    const dim3 grid((unsigned)blocks, (unsigned)K);
+    if (dtype == RKV_F32)
+        cross_seed_kernel<RKV_F32><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
+    else if (dtype == RKV_BF16)
+        cross_seed_kernel<RKV_BF16><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
+    else
+        cross_seed_kernel<RKV_F16><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
+    cross_finalize_kernel<<<(K + 127) / 128, 128, 0, stream>>>(partials, K, S, blocks, spread_lim, stats_out);
+    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+size_t rkv_copy_workspace_bytes(int K, int M) {
+    if (K < 1 || K > kCrossMaxK || M < 1 || M > kCopyMaxInputs) return 0;
+    return ((size_t)(K + M) * sizeof(void*) + 255) / 256 * 256 + (size_t)K * sizeof(uint32_t);
+}
+
+int rkv_copy_of_inputs(const void* const* inputs, int M, const void* const* cands, int K, uint64_t n, int dtype,
+                       uint32_t* copy_mask_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!inputs || !cands || !copy_mask_out || K < 1 || M < 1 || n < 1) return RKV_ERR_INVALID_ARG;
+    if (dtype != RKV_F32 && dtype != RKV_BF16 && dtype != RKV_F16) return RKV_ERR_INVALID_ARG;
+    if (K > kCrossMaxK || M > kCopyMaxInputs || n >= kMaxN) return RKV_ERR_UNSUPPORTED;
+    for (int m = 0; m < M; ++m) {
+        if (!inputs[m]) return RKV_ERR_INVALID_ARG;
+        if (!aligned16(inputs[m])) return RKV_ERR_ALIGNMENT;
+    }
+    for (int k = 0; k < K; ++k) {
+        if (!cands[k]) return RKV_ERR_INVALID_ARG;
+        if (!aligned16(cands[k])) return RKV_ERR_ALIGNMENT;
+    }
+    if (!workspace) return RKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return RKV_ERR_ALIGNMENT;
+    if (workspace_bytes < rkv_copy_workspace_bytes(K, M)) return RKV_ERR_WORKSPACE;
+    int sms = 0;
+    int rc = current_num_sms(&sms);
+    if (rc != RKV_OK) return rc;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    rc = refuse_capture(stream);
+    if (rc != RKV_OK) return rc;
+    const size_t ptr_bytes = ((size_t)(K + M) * sizeof(void*) + 255) / 256 * 256;
+    std::vector<const void*> table((size_t)(K + M));
+    for (int m = 0; m < M; ++m) table[(size_t)m] = inputs[m];
+    for (int k = 0; k < K; ++k) table[(size_t)(M + k)] = cands[k];
+    const void** d_ptrs = reinterpret_cast<const void**>(workspace);
+    uint32_t* differs = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(workspace) + ptr_bytes);
+    if (cudaMemcpyAsync(d_ptrs, table.data(), table.size() * sizeof(void*), cudaMemcpyHostToDevice, stream) !=
+            cudaSuccess ||
+        cudaMemsetAsync(differs, 0, (size_t)K * sizeof(uint32_t), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return RKV_ERR_CUDA;
+    }
+    const uint64_t n_bytes = n * (dtype == RKV_F32 ? 4u : 2u);
+    const int blocks = blocks_per_candidate(n_bytes / 16, K, sms);
+    copy_any_kernel<<<dim3((unsigned)blocks, (unsigned)K), kCrossThreads, 0, stream>>>(d_ptrs, M, d_ptrs + M, n_bytes,
+                                                                                      differs);
+    copy_finalize_kernel<<<(K + 127) / 128, 128, 0, stream>>>(differs, K, M, copy_mask_out);
+    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+}
+
+}  // extern "C"
