@@ -119,7 +119,8 @@ constexpr int kOffWaitLimit = kOffRefState + 8;               // long long: cycl
 constexpr int kOffInfo = 128;
 constexpr int kOffPtrC = kOffInfo + kInfoRing * (int)sizeof(ItemInfo);   // consumer copy of the part's candidate pointers
 constexpr int kOffPtrP = kOffPtrC + kPartK * 8;                          // producer copy (it runs an item ahead)
-constexpr int kOffHint = kOffPtrP + kPartK * 8;                          // two tables (item parity)
+constexpr int kOffFirst = kOffPtrP + kPartK * 8;                         // element 0 of the part's candidates, storage bits
+constexpr int kOffHint = kOffFirst + kPartK * 4;                         // two tables (item parity)
 constexpr int kOffRec = kOffHint + 2 * kPartK * (int)sizeof(Hint);
 constexpr int kOffStage = (kOffRec + kConsumerWarps * kPartK * (int)sizeof(WarpRec) + 1023) / 1024 * 1024;
 constexpr int kSmemBytes = kOffStage + kStages * kStageBytes;
@@ -1118,7 +1119,7 @@ __device__ __forceinline__ void advance_stage(BlockState& B) {
 // One item: every candidate of the part against the tile's reference values.
 template <int CK>
 __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, const Ring& ring, BlockState& B,
-                                         const ItemInfo& it, const DevTensor& D) {
+                                         const ItemInfo& it, const DevTensor& D, bool same_part) {
     constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC, NW = Geo<CK>::NW;
     constexpr int NV = E / VEC;
     constexpr bool C16 = Geo<CK>::C16;
@@ -1126,6 +1127,7 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     constexpr uint32_t CSZ = C16 ? 2 : 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned char** ptrs = reinterpret_cast<const unsigned char**>(smem + kOffPtrC);
+    uint32_t* firsts = reinterpret_cast<uint32_t*>(smem + kOffFirst);
     Hint* H = reinterpret_cast<Hint*>(smem + kOffHint) + (B.ord & 1u) * kPartK;
     WarpRec* recs = reinterpret_cast<WarpRec*>(smem + kOffRec);
     volatile uint32_t* ref_state = reinterpret_cast<volatile uint32_t*>(smem + kOffRefState);
@@ -1140,17 +1142,24 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     // (range checks of a debug build: the tile lies inside the tensor; the state, hint and
     // record tables are indexed by k0 + kk < K and kk < kPartK, checked with the item)
     if (!RKV_IN_BOUNDS(A.header, 9, start < D.n && it.tile < D.n_tiles, it.tile)) return;
-    // the part's pointers and hints, from the published state
+    // the part's pointers (kept while the block stays with the part) and hints, from the
+    // published state
     if (tid < kc) {
-        const unsigned char* p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
-        ptrs[tid] = p;
+        const unsigned char* p;
+        if (same_part) {
+            p = ptrs[tid];
+        } else {
+            p = reinterpret_cast<const unsigned char*>(D.cands[k0 + tid]);
+            ptrs[tid] = p;
+            firsts[tid] = ld_elem_raw(p, Geo<CK>::DTYPE, 0);
+        }
         const CandState* sc = st_t + k0 + tid;
         Hint h;
         h.te_x = hint_threshold(__ldcg(&sc->hint_e), it.tile);
         h.tq_x = hint_threshold(__ldcg(&sc->hint_q), it.tile);
         if (C16 && h.tq_x < 0.0f) h.tq_x = -kInf;     // see process_candidate_16
         h.settled = __ldcg(&sc->mismatch);
-        h.first = ld_elem_raw(p, Geo<CK>::DTYPE, 0);
+        h.first = firsts[tid];
         H[tid] = h;
     }
     if (tid == kPartK) ref_state[B.ord & 1u] = __ldcg(&st_t[A.K].mismatch);
@@ -1281,15 +1290,16 @@ __device__ __forceinline__ void consumer_loop(const Args& A, unsigned char* smem
                 (A.tensors[cur_t].slot_by_tile && it.tile != cur_tile))
                 flush_records(recs, A, A.tensors[cur_t], cur_k0, cur_kc, cur_slot, tid, cur_te);
         }
+        const bool same_part = (int)it.t == cur_t && (int)it.k0 == cur_k0 && (int)it.kc == cur_kc;
         cur_t = (int)it.t; cur_k0 = (int)it.k0; cur_kc = (int)it.kc; cur_tile = it.tile;
         cur_slot = D.slot_by_tile ? it.tile : blockIdx.x;
         cur_te = tile_elems(D.cand_dtype);
         // (the stage waited for above is consumed inside run_item: it holds the item's reference
         // tile or its first candidate)
         switch (D.cand_dtype) {
-            case RKV_F32: run_item<CK_F32>(A, smem, ring, B, it, D); break;
-            case RKV_BF16: run_item<CK_BF16>(A, smem, ring, B, it, D); break;
-            default: run_item<CK_F16>(A, smem, ring, B, it, D); break;
+            case RKV_F32: run_item<CK_F32>(A, smem, ring, B, it, D, same_part); break;
+            case RKV_BF16: run_item<CK_BF16>(A, smem, ring, B, it, D, same_part); break;
+            default: run_item<CK_F16>(A, smem, ring, B, it, D, same_part); break;
         }
     }
     consumer_sync();
