@@ -59,9 +59,10 @@ def parse_args(argv=None):
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "s1"],
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "s1", "x1", "w1"],
                     help="c1..c5: the verification workloads (c5, the large sweep, is the benchmark); "
-                         "s1: task-soundness screens (its own metric, not the benchmark)")
+                         "s1: task-soundness screens; x1: cross-seed variation check; w1: config sweep of 256 small "
+                         "cases (each its own metric, not the benchmark)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-workload", action="store_true")
@@ -757,13 +758,17 @@ def run_screen(args):
 def main():
     args = parse_args()
     relaunch_if_needed(args)
-    if args.workload == "s1":
+    if args.workload in ("s1", "x1", "w1"):
         if args.impl == "reference" or int(os.environ.get("WORLD_SIZE", "1")) > 1:
             if int(os.environ.get("RANK", "0")) == 0:
                 print(json.dumps({"impl": args.impl,
                                   "unavailable": f"workload {args.workload} runs on one GPU, native arm only"}))
             return
-        run_screen(args)
+        if args.workload == "s1":
+            run_screen(args)
+        else:
+            import bench_extra
+            (bench_extra.run_cross if args.workload == "x1" else bench_extra.run_sweep)(args, measured_peak, ClockSampler)
     elif args.impl == "reference":
         run_reference(args)
     else:

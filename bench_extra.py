@@ -1,0 +1,131 @@
+"""Bench workloads beside the headline (each its own metric, not the benchmark):
+
+x1  cross-seed variation check: K = 32 candidates x S = 4 input seeds of 2^22 fp32 elements
+    (2 GiB streamed per call, every byte once).
+w1  config sweep: 256 small test cases (the paper's listing shapes: batch 16/64/4 x features
+    128/4096/10, a scalar loss; fp32 / bf16 / fp16), K = 8 candidates, verified by ONE
+    rkv_verify_sweep call, against the same cases verified by 256 rkv_verify_multi calls.
+"""
+from __future__ import annotations
+
+import json
+import statistics
+import time
+
+
+def _events(fn, launches, torch):
+    ev = []
+    for _ in range(launches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        ev.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def run_cross(args, measured_peak, ClockSampler):
+    import torch
+
+    from paper_2509_14279_b200 import binding as rkv
+
+    torch.cuda.set_device(0)
+    K, S, n = 32, 4, 1 << 22
+    outs = []
+    for k in range(K):
+        row = [rkv.gen_inputs_ex(31 + k, s, rkv.DIST_NORMAL, n) for s in range(S)]
+        if k % 8 == 7:                       # a candidate that ignores its input
+            row = [row[0]] + [row[0].clone() for _ in range(S - 1)]
+        outs.append(row)
+    stats, ws = rkv.cross_seed(outs, 1e-5, 1e-5)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        rkv.cross_seed(outs, 1e-5, 1e-5, stats_out=stats, workspace=ws)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.15)
+    ms = _events(lambda: rkv.cross_seed(outs, 1e-5, 1e-5, stats_out=stats, workspace=ws), args.steps, torch)
+    clocks = sampler.stop()
+    del flush
+    nbytes = K * S * n * 4
+    mean = statistics.mean(ms)
+    peak, kind = measured_peak()
+    got = rkv.cross_to_numpy(stats)
+    ok = all(bool(int(g["flags"]) & rkv.CROSS_IDENTICAL) == (k % 8 == 7) for k, g in enumerate(got))
+    print(json.dumps({
+        "metric": "cross_seed_GBps", "value": round(nbytes / mean / 1e6, 2), "unit": "GB/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(mean, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"x1: cross-seed variation, K={K} candidates x S={S} seeds of {n} fp32 elements",
+                   "bytes_per_step": nbytes, "l2": "inputs larger than L2 (2 GiB per call)"},
+        "gpu_launches": 2 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "cross_seed_kernel", "achieved": round(nbytes / mean / 1e6, 1),
+                     "peak": peak, "peak_kind": f"of {kind}", "unit": "GB/s",
+                     "frac": round(nbytes / mean / 1e6 / peak, 4), "algorithmic_bytes_per_launch": nbytes,
+                     "avg_launch_ms": round(mean, 4), "median_launch_ms": round(statistics.median(ms), 4),
+                     "best_launch_ms": round(min(ms), 4), "traffic": None},
+        "clocks": clocks, "result_check": "ok" if ok else "UNEXPECTED"}), flush=True)
+
+
+def run_sweep(args, measured_peak, ClockSampler):
+    import torch
+
+    from paper_2509_14279_b200 import binding as rkv
+
+    torch.cuda.set_device(0)
+    K, C = 8, 256
+    shapes = [(16, 128), (64, 128), (4, 128), (16, 4096), (64, 4096), (4, 10), (64, 10), (1,)]
+    kinds = [torch.float32, torch.bfloat16, torch.float16]
+    cases, nbytes = [], 0
+    for c in range(C):
+        n = 1
+        for d in shapes[c % len(shapes)]:
+            n *= d
+        dt = kinds[c % 3]
+        ref = rkv.gen_inputs_ex(700 + c, 0, c % 5, n)
+        cands = [(ref * (1.0 + (1e-7 if k else 0.0))).to(dt) for k in range(K)]
+        tol = (1e-5, 1e-5) if dt == torch.float32 else (1e-2, 1.6e-2)
+        cases.append([rkv.TensorDesc(n=n, cands=cands, atol=tol[0], rtol=tol[1], ref=ref)])
+        nbytes += K * n * cands[0].element_size() + n * 4
+    descs = rkv.prepare_sweep(cases)
+    stats, cp, ap, ws = rkv.verify_sweep(cases, K, descs=descs)
+    singles = []
+    for t in cases:
+        arr = rkv.prepare(t)
+        s, j, w = rkv.verify_multi(t, K, descs=arr)
+        singles.append((t, arr, s, j, w))
+    torch.cuda.synchronize()
+
+    def one_launch():
+        rkv.verify_sweep(cases, K, workspace=ws, stats_out=stats, case_pass=cp, all_pass=ap, descs=descs)
+
+    def one_call_per_case():
+        for (t, arr, s, j, w) in singles:
+            rkv.verify_multi(t, K, workspace=w, stats_out=s, joint_pass=j, descs=arr)
+
+    for _ in range(max(args.warmup, 3)):
+        one_launch()
+        one_call_per_case()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.15)
+    steps = min(args.steps, 20)
+    ms_sweep = _events(one_launch, steps, torch)
+    ms_calls = _events(one_call_per_case, steps, torch)
+    clocks = sampler.stop()
+    a, b = statistics.mean(ms_sweep), statistics.mean(ms_calls)
+    ok = rkv.device_status(ws) == 0 and int(ap.sum().item()) == K
+    print(json.dumps({
+        "metric": "sweep_cases_per_s", "value": round(C / a * 1e3, 1), "unit": "cases/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(a, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 arithmetic on f32 / bf16 / fp16 candidates", "data": "synthetic",
+        "config": {"workload": f"w1: config sweep, {C} small cases (listing shapes), K={K} candidates, one launch",
+                   "bytes_per_step": nbytes, "l2": "the whole sweep fits in L2: a launch-latency workload"},
+        "gpu_launches": 3 * steps,
+        "one_launch": {"ms": round(a, 4), "median_ms": round(statistics.median(ms_sweep), 4), "best_ms": round(min(ms_sweep), 4),
+                       "GBps": round(nbytes / a / 1e6, 1)},
+        "one_call_per_case": {"ms": round(b, 4), "median_ms": round(statistics.median(ms_calls), 4),
+                              "best_ms": round(min(ms_calls), 4), "calls": C, "GBps": round(nbytes / b / 1e6, 1)},
+        "speedup_of_one_launch": round(b / a, 2), "clocks": clocks, "result_check": "ok" if ok else "UNEXPECTED"}),
+        flush=True)
