@@ -281,3 +281,49 @@ def test_binding_refuses_mismatched_tensors_before_the_c_call():
         rkv.TensorDesc(n=1024, cands=[good], atol=1e-5, rtol=1e-5, ref=ref).to_c()
     with pytest.raises(TypeError):
         rkv._require(3.0, "x")
+
+
+def test_cross_checks_validate_before_any_cuda_call():
+    L = rkv.lib()
+    assert rkv.CROSS_BYTES == 32
+    vp = ctypes.c_void_p
+
+    def cross(ptrs=(0x1000, 0x2000), K=1, S=2, n=64, dtype=0, atol=1e-5, rtol=1e-5, lim=0.01, stats=0x9000,
+              ws=0x4000, ws_bytes=1 << 30):
+        arr = (vp * max(1, len(ptrs)))(*ptrs)
+        return L.rkv_cross_seed(arr, K, S, n, dtype, atol, rtol, lim, vp(stats), vp(ws), ws_bytes, None)
+
+    assert cross(K=0) == rkv.ERR_INVALID_ARG
+    assert cross(S=0) == rkv.ERR_INVALID_ARG
+    assert cross(n=0) == rkv.ERR_INVALID_ARG
+    assert cross(dtype=3) == rkv.ERR_INVALID_ARG
+    assert cross(atol=-1.0) == rkv.ERR_INVALID_ARG
+    assert cross(rtol=float("nan")) == rkv.ERR_INVALID_ARG
+    assert cross(lim=-0.5) == rkv.ERR_INVALID_ARG
+    assert cross(stats=0) == rkv.ERR_INVALID_ARG
+    assert cross(S=17) == rkv.ERR_UNSUPPORTED
+    assert cross(K=4097) == rkv.ERR_UNSUPPORTED
+    assert cross(n=1 << 40) == rkv.ERR_UNSUPPORTED
+    assert cross(ptrs=(0x1000, 0)) == rkv.ERR_INVALID_ARG
+    assert cross(ptrs=(0x1000, 0x2004)) == rkv.ERR_ALIGNMENT
+    assert cross(ws=0) == rkv.ERR_WORKSPACE
+    assert L.rkv_cross_seed(None, 1, 2, 64, 0, 1e-5, 1e-5, 0.01, vp(0x9000), vp(0x4000), 1 << 30, None) == rkv.ERR_INVALID_ARG
+
+    def copy(inputs=(0x1000,), cands=(0x2000,), n=64, dtype=0, mask=0x9000, ws=0x4000, ws_bytes=1 << 30, M=None, K=None):
+        ia = (vp * max(1, len(inputs)))(*inputs)
+        ca = (vp * max(1, len(cands)))(*cands)
+        return L.rkv_copy_of_inputs(ia, len(inputs) if M is None else M, ca, len(cands) if K is None else K, n, dtype,
+                                    vp(mask), vp(ws), ws_bytes, None)
+
+    assert copy(M=0) == rkv.ERR_INVALID_ARG
+    assert copy(K=0) == rkv.ERR_INVALID_ARG
+    assert copy(n=0) == rkv.ERR_INVALID_ARG
+    assert copy(dtype=7) == rkv.ERR_INVALID_ARG
+    assert copy(mask=0) == rkv.ERR_INVALID_ARG
+    assert copy(inputs=(0x1000,) * 9) == rkv.ERR_UNSUPPORTED
+    assert copy(inputs=(0,)) == rkv.ERR_INVALID_ARG
+    assert copy(cands=(0x2008,)) == rkv.ERR_ALIGNMENT
+    assert copy(ws=0) == rkv.ERR_WORKSPACE
+    assert copy(ws_bytes=8) == rkv.ERR_WORKSPACE
+    assert L.rkv_copy_workspace_bytes(0, 1) == 0 and L.rkv_copy_workspace_bytes(4, 2) >= 4 * 4 + 6 * 8
+    assert L.rkv_cross_workspace_bytes(1, 17) == 0
