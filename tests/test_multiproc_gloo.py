@@ -72,3 +72,22 @@ def test_two_ranks_shard_the_candidates_and_agree(tmp_path, K):
         assert got[:K] == want
         assert got[K] == 10 + world - 1          # the slowest rank's time
         assert got[K + 1] == K                   # every candidate verified exactly once
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did(tmp_path):
+    """`bench.py --gpus 2` with WORLD_SIZE unset re-executes itself under torch.distributed.run with two
+    ranks on 127.0.0.1.  The reference arm runs on CPU: rank 0 prints the one JSON line with n_gpus = 2,
+    rank 1 exits 0 without work."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "1", "--workload", "c1"], env=env, capture_output=True, text=True,
+                       timeout=600, cwd=str(tmp_path))
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["value"] > 0
