@@ -640,7 +640,7 @@ __device__ __forceinline__ uint32_t cand_bits(const uint32_t (&w)[16], int j) {
 // Loophole flags of one candidate tile, until a difference has been seen.
 template <int CK>
 __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const Hint& h, Hint* h_smem,
-                                                CandState* st, const DevTensor& D, const void* cand_g,
+                                                CandState* st, const DevTensor& D, const unsigned char* const* cand_p,
                                                 uint64_t start, uint32_t len, uint32_t wanted_flags, int tid,
                                                 int lane) {
     constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC, NW = Geo<CK>::NW, DT = Geo<CK>::DTYPE;
@@ -685,7 +685,7 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
                     const uint32_t off = off0 + i;
                     if (off < len) {
                         uint32_t cb = cand_bits<CK>(w, 4 * g + i);
-                        if (off >= copied) cb = ld_elem_bits(cand_g, DT, start + off);
+                        if (off >= copied) cb = ld_elem_bits(*cand_p, DT, start + off);
                         if (!full) acc1 |= cb ^ first_up;
                         if (with_input) acc2 |= cb ^ in[i];
                     }
@@ -707,11 +707,11 @@ __device__ __forceinline__ void candidate_flags(const uint32_t (&w)[16], const H
 //   h        the candidate's hint entry (a snapshot; see the file header)
 //   rec      the warp's running result for this candidate (shared memory; lane 0 writes)
 //   st       the candidate's global state
-//   cand_g   the candidate tensor in global memory (only the last < 16 bytes of a
+//   cand_p   where the pointer to the candidate tensor in global memory is kept (only the last < 16 bytes of a
 //            ragged tensor are read from there)
 __device__ __forceinline__ void process_candidate_32(const RefRegs<false>& R, const uint32_t (&w)[16],
                                                      const Hint& h, Hint* h_smem, WarpRec* rec, CandState* st,
-                                                     const DevTensor& D, const void* cand_g, uint32_t tile,
+                                                     const DevTensor& D, const unsigned char* const* cand_p, uint32_t tile,
                                                      uint64_t start, uint32_t len, uint32_t wanted_flags,
                                                      int tid, int lane) {
     constexpr int CK = CK_F32;
@@ -741,7 +741,7 @@ __device__ __forceinline__ void process_candidate_32(const RefRegs<false>& R, co
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sf = __fadd_rn(sf, __shfl_xor_sync(kFullMask, sf, off));
         if (lane == 0) rec->sum = (double)sf;
-        candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+        candidate_flags<CK>(w, h, h_smem, st, D, cand_p, start, len, wanted_flags, tid, lane);
         return;
     }
     // m <= thr_min means e_j <= m <= thr_min <= thr_j for every element: none over
@@ -782,7 +782,7 @@ __device__ __forceinline__ void process_candidate_32(const RefRegs<false>& R, co
                 const uint32_t off = elem_off<VEC>(j, tid);
                 if (off < len) {
                     uint32_t cb = w[j];
-                    if (off >= copied) cb = ld_elem_bits(cand_g, RKV_F32, start + off);
+                    if (off >= copied) cb = ld_elem_bits(*cand_p, RKV_F32, start + off);
                     elem_general(a, cb, __float_as_uint(R.r[j]), off, D.atol, D.rtol);
                 }
             }
@@ -848,7 +848,7 @@ __device__ __forceinline__ void process_candidate_32(const RefRegs<false>& R, co
         if (lane == 0 && tot) rec->n_over += tot;
     }
 
-    candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+    candidate_flags<CK>(w, h, h_smem, st, D, cand_p, start, len, wanted_flags, tid, lane);
 }
 
 // c - r for the 16-bit value c in the low (half = 0) or high 16 bits of x: the value
@@ -926,7 +926,7 @@ __device__ __forceinline__ void pass_16(const RefRegs<true>& R, const uint32_t (
 template <int CK>
 __device__ __forceinline__ void process_candidate_16(const RefRegs<true>& R, const uint32_t (&w)[16],
                                                      const Hint& h, Hint* h_smem, WarpRec* rec,
-                                                     CandState* st, const DevTensor& D, const void* cand_g,
+                                                     CandState* st, const DevTensor& D, const unsigned char* const* cand_p,
                                                      uint32_t tile, uint64_t start, uint32_t len,
                                                      uint32_t wanted_flags, int tid, int lane) {
     constexpr int VEC = 8;
@@ -1029,7 +1029,7 @@ __device__ __forceinline__ void process_candidate_16(const RefRegs<true>& R, con
             *rec = r;
         }
     }
-    candidate_flags<CK>(w, h, h_smem, st, D, cand_g, start, len, wanted_flags, tid, lane);
+    candidate_flags<CK>(w, h, h_smem, st, D, cand_p, start, len, wanted_flags, tid, lane);
 }
 
 // The error sums of the item just finished: for every candidate of its part, the warps'
@@ -1101,7 +1101,6 @@ __device__ __forceinline__ float hint_threshold(unsigned long long key, uint32_t
 // What a block carries from item to item.
 struct BlockState {
     uint32_t cstage, cphase;     // next ring stage to consume and the parity of its current use
-    uint32_t ccount;             // stages consumed so far (= the number of the next copy to wait for)
     uint32_t ord;                // items this block has started
 };
 
@@ -1112,7 +1111,6 @@ __device__ __forceinline__ bool wait_stage(const Ring& ring, const BlockState& B
 }
 
 __device__ __forceinline__ void advance_stage(BlockState& B) {
-    B.ccount += 1u;
     if (++B.cstage == (uint32_t)kStages) { B.cstage = 0; B.cphase ^= 1u; }
 }
 
@@ -1246,10 +1244,10 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
             }
         }
         if constexpr (C16)
-            process_candidate_16<CK>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+            process_candidate_16<CK>(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, &ptrs[kk],
                                      it.tile, start, len, wanted, tid, lane);
         else
-            process_candidate_32(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, ptrs[kk],
+            process_candidate_32(R, w, h, &H[kk], &recs[warp * kPartK + kk], st_t + k0 + kk, D, &ptrs[kk],
                                  it.tile, start, len, wanted, tid, lane);
     }
 }
@@ -1265,7 +1263,7 @@ __device__ __forceinline__ void consumer_loop(const Args& A, unsigned char* smem
         r.emax = -1.0f; r.etile = 0; r.qmax = -1.0f; r.qtile = 0; r.offs = 0; r.n_over = 0; r.sum = 0.0;
     }
     BlockState B;
-    B.cstage = 0; B.cphase = 0; B.ccount = 0; B.ord = 0;
+    B.cstage = 0; B.cphase = 0; B.ord = 0;
 
     int cur_t = -1, cur_k0 = 0, cur_kc = 0;
     uint32_t cur_slot = 0, cur_tile = 0, cur_te = 0;
