@@ -117,7 +117,9 @@ typedef struct rkv_stats {
     uint64_t n_comparable;
     uint64_t argmax_abs_err;
     uint64_t argmax_rel_err;
-    double sum_abs_err;       /* sum of e over comparable elements        */
+    double sum_abs_err;       /* sum of e over comparable elements: fp32 within a tile of 14 KiB of
+                                 the candidate, fp64 above; within 1e-6 of a sequential fp64 sum,
+                                 and the same bits on every run (it is added in tile order)      */
     float max_abs_err;        /* 0 when nothing is comparable             */
     float max_rel_err;
     float mean_abs_err;       /* (float)(sum_abs_err / n_comparable), 0 if none */

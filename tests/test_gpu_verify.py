@@ -301,7 +301,7 @@ def test_runs_are_deterministic():
         assert a.tobytes() == b.tobytes()
 
 
-def test_north_star_two_call_form():
+def test_plain_two_call_form():
     shape = (256, 1024)
     ref = rkv.gen_inputs(0, rkv.DIST_NORMAL, shape)
     n = ref.numel()
