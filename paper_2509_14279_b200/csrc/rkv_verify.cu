@@ -1354,14 +1354,14 @@ __device__ __forceinline__ void wide_merge(Wide& a, const Wide& b) {
     a.sum += b.sum;
 }
 
-// One block per (tensor, candidate).
-__global__ void __launch_bounds__(kFinThreads)
-finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandState* __restrict__ state,
-                const Partial* __restrict__ partials, const double* __restrict__ sums,
-                rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ fail) {
-    __shared__ Wide red[kFinThreads];
-    const int t = blockIdx.x / K, k = blockIdx.x % K, tid = threadIdx.x;
-    if (t >= T) return;
+// The result of candidate k on tensor t, by one block; returns the verdict (in thread 0).
+__device__ __forceinline__ uint32_t finalize_one(Wide* red, const DevTensor* __restrict__ tensors, int t, int k, int K,
+                                                 const CandState* __restrict__ state,
+                                                 const Partial* __restrict__ partials,
+                                                 const double* __restrict__ sums,
+                                                 rkv_stats* __restrict__ stats_out) {
+    const int tid = threadIdx.x;
+    uint32_t verdict_out = 0;
     const DevTensor D = tensors[t];
     Wide w;
     w.n_over = 0; w.sum = 0.0;
@@ -1423,8 +1423,35 @@ finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandS
         st.flags = flags;
         st.verdict = verdict;
         stats_out[D.out_base + (unsigned long long)k * D.out_stride] = st;
-        if (verdict) atomicOr(&fail[(size_t)D.case_index * (size_t)K + (size_t)k], 1u);
+        verdict_out = verdict;
     }
+    __syncthreads();                  // `red` is free for the next tensor
+    return verdict_out;
+}
+
+// One block per (tensor, candidate); the verdicts of a case meet in its fail words (a sweep).
+__global__ void __launch_bounds__(kFinThreads)
+finalize_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandState* __restrict__ state,
+                const Partial* __restrict__ partials, const double* __restrict__ sums,
+                rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ fail) {
+    __shared__ Wide red[kFinThreads];
+    const int t = blockIdx.x / K, k = blockIdx.x % K;
+    if (t >= T) return;
+    const uint32_t verdict = finalize_one(red, tensors, t, k, K, state, partials, sums, stats_out);
+    if (threadIdx.x == 0 && verdict)
+        atomicOr(&fail[(size_t)tensors[t].case_index * (size_t)K + (size_t)k], 1u);
+}
+
+// One case: one block per candidate goes through the case's tensors and writes the joint verdict.
+__global__ void __launch_bounds__(kFinThreads)
+finalize_case_kernel(const DevTensor* __restrict__ tensors, int T, int K, const CandState* __restrict__ state,
+                     const Partial* __restrict__ partials, const double* __restrict__ sums,
+                     rkv_stats* __restrict__ stats_out, uint32_t* __restrict__ joint_pass) {
+    __shared__ Wide red[kFinThreads];
+    const int k = blockIdx.x;
+    uint32_t failed = 0;
+    for (int t = 0; t < T; ++t) failed |= finalize_one(red, tensors, t, k, K, state, partials, sums, stats_out);
+    if (threadIdx.x == 0 && joint_pass) joint_pass[k] = failed ? 0u : 1u;
 }
 
 // case_pass[c][k] = candidate k passed on every tensor of case c; all_pass[k] = on every case.
@@ -1476,6 +1503,12 @@ int verify_occupancy() {
 
 int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,
                     uint32_t* all_pass, cudaStream_t stream) {
+    if (n_cases == 1 && !case_pass && T <= kMaxTensors) {
+        // one case: no second kernel for the joint verdict
+        finalize_case_kernel<<<(unsigned)K, kFinThreads, 0, stream>>>(L.d_tensors, T, K, L.state, L.partials, L.sums,
+                                                                     stats_out, all_pass);
+        return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
+    }
     finalize_kernel<<<(unsigned)T * (unsigned)K, kFinThreads, 0, stream>>>(L.d_tensors, T, K, L.state, L.partials,
                                                                           L.sums, stats_out, L.fail);
     if (cudaGetLastError() != cudaSuccess) return RKV_ERR_CUDA;
