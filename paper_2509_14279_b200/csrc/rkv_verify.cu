@@ -53,7 +53,7 @@ namespace {
 
 constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 constexpr float kInf = __builtin_huge_valf();
-enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the issuer's "no more items" mark
+enum : uint32_t { kNoItem = 0xFFFFFFFFu };     // the producer's "no more items" mark
 constexpr int kInfoRing = 16;                  // item descriptions kept per block (> kStages + 1: an item uses >= 1 stage)
 constexpr long long kWaitCycles = 2000000000LL;
 
@@ -101,7 +101,7 @@ struct __align__(16) Hint {
 };
 static_assert(sizeof(Hint) == 16, "Hint layout");
 
-// What the issuing lane tells the block about an item, before it arms the item's first stage.
+// What the producer tells the consumers about an item, before it arms the item's first stage.
 struct __align__(16) ItemInfo {
     uint32_t id;             // kNoItem: no more items
     uint32_t t;
@@ -283,7 +283,7 @@ struct Args {
 };
 
 // ----------------------------------------------------------------------------
-// the issuing lane: feeds the ring
+// the producer warp: feeds the ring
 // ----------------------------------------------------------------------------
 struct Ring {
     uint32_t full0, empty0;      // shared-memory addresses of the first full / empty mbarrier
