@@ -28,7 +28,10 @@
 //
 // Per element the common path is one subtraction, one running maximum and one
 // addition (16-bit candidates: one fused multiply-add and one more maximum, see
-// process_candidate_16).  Counting the elements over tolerance, locating maxima,
+// process_candidate_16; whole tiles of 16-bit candidates are taken two candidates at a
+// time, straight from their ring stages, see pair_common_16: the waits, votes, warp
+// reductions and loop overhead of a step are then paid once per two candidates).
+// Counting the elements over tolerance, locating maxima,
 // dividing for the relative error and everything about non-finite values sit behind
 // tests evaluated once per thread, candidate and tile and one warp vote:
 //   m > min thr              some element may be over tolerance  -> count them
@@ -540,6 +543,22 @@ __device__ __forceinline__ uint32_t first_elem_bits(const void* ptr, int src, in
     return g[0];
 }
 
+// The thread's E elements of a tile of a generated tensor (distribution DIST), as fp32 bit
+// patterns; bf16 == true rounds them to bf16 first.
+template <int CK, int DIST>
+__device__ __forceinline__ void gen_thread_tile(uint64_t seed, uint64_t stream_id, uint64_t start, int tid, bool bf16,
+                                                uint32_t (&rb)[Geo<CK>::E]) {
+    constexpr int E = Geo<CK>::E, VEC = Geo<CK>::VEC;
+    const PhiloxKey key = philox_key(seed);
+#pragma unroll
+    for (int g = 0; g < E / 4; ++g) {
+        float v[4];
+        gen_block<DIST>((start + elem_off<VEC>(4 * g, tid)) >> 2, stream_id, key, v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rb[4 * g + i] = bf16 ? (bf16_rne_bits(v[i]) << 16) : __float_as_uint(v[i]);
+    }
+}
+
 // Load (or regenerate) the thread's reference values for a tile and derive what
 // depends on them alone.  The bulk-copied part of the tile sits in ring stage
 // `stage_a` (and, for an fp32 reference under 16-bit candidates, continues in
@@ -559,12 +578,14 @@ __device__ __forceinline__ void load_ref(RefRegs<Geo<CK>::C16>& R, uint32_t (&rb
         return b < (uint32_t)kStageBytes ? stage_a + b : stage_b + (b - kStageBytes);
     };
     if (D.ref_src == RKV_SRC_GENERATED) {
-#pragma unroll
-        for (int g = 0; g < E / 4; ++g) {
-            uint32_t v[4];
-            gen_group(D.ref_seed, D.ref_stream, D.ref_dist, start, elem_off<VEC>(4 * g, tid), rdt == RKV_BF16, v);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) rb[4 * g + i] = v[i];
+        // the distribution is chosen once, outside the loop over the thread's Philox blocks: the
+        // blocks are independent, and as straight-line code their long dependent chains overlap
+        switch (D.ref_dist) {
+            case 0: gen_thread_tile<CK, 0>(D.ref_seed, D.ref_stream, start, tid, rdt == RKV_BF16, rb); break;
+            case 1: gen_thread_tile<CK, 1>(D.ref_seed, D.ref_stream, start, tid, rdt == RKV_BF16, rb); break;
+            case 2: gen_thread_tile<CK, 2>(D.ref_seed, D.ref_stream, start, tid, rdt == RKV_BF16, rb); break;
+            case 3: gen_thread_tile<CK, 3>(D.ref_seed, D.ref_stream, start, tid, rdt == RKV_BF16, rb); break;
+            default: gen_thread_tile<CK, 4>(D.ref_seed, D.ref_stream, start, tid, rdt == RKV_BF16, rb); break;
         }
     } else if (full) {
 #pragma unroll
@@ -902,6 +923,99 @@ __device__ __forceinline__ void pass_16(const RefRegs<true>& R, const uint32_t (
                       __fadd_rn(__fadd_rn(sg[4], sg[5]), __fadd_rn(sg[6], sg[7])));
 }
 
+// Eight elements (one 16-byte piece) of each of two 16-bit candidates against reference
+// values r[0..8): the work of pass_16 for both, sharing |r_j| and the test for a reference
+// of zero.  acc = {m_a, dm_a, m_b, dm_b}; returns the two partial sums of the piece.
+template <int CK, bool HAS_ZERO>
+__device__ __forceinline__ void piece_16x2(const float* r, float atol, const uint4& a, const uint4& b, float ta,
+                                           float tb, float (&acc)[4], float& sum_a, float& sum_b) {
+    const uint32_t wa[4] = {a.x, a.y, a.z, a.w}, wb[4] = {b.x, b.y, b.z, b.w};
+    float sa[2], sb[2];
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        float ea[4], da[4], eb[4], db[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int j = 4 * g + i;
+            ea[i] = fabsf(sub16_f32<CK>(wa[j >> 1], j & 1, r[j]));
+            eb[i] = fabsf(sub16_f32<CK>(wb[j >> 1], j & 1, r[j]));
+            const float ar = fabsf(r[j]);
+            if (HAS_ZERO && ar == 0.0f) {
+                da[i] = __fsub_rn(ea[i], atol);
+                db[i] = __fsub_rn(eb[i], atol);
+            } else {
+                da[i] = __fmaf_rn(-ta, ar, ea[i]);
+                db[i] = __fmaf_rn(-tb, ar, eb[i]);
+            }
+        }
+        acc[0] = fmaxf(fmaxf(acc[0], fmaxf(ea[0], ea[1])), fmaxf(ea[2], ea[3]));
+        acc[1] = fmaxf(fmaxf(acc[1], fmaxf(da[0], da[1])), fmaxf(da[2], da[3]));
+        acc[2] = fmaxf(fmaxf(acc[2], fmaxf(eb[0], eb[1])), fmaxf(eb[2], eb[3]));
+        acc[3] = fmaxf(fmaxf(acc[3], fmaxf(db[0], db[1])), fmaxf(db[2], db[3]));
+        sa[g] = __fadd_rn(__fadd_rn(ea[0], ea[1]), __fadd_rn(ea[2], ea[3]));
+        sb[g] = __fadd_rn(__fadd_rn(eb[0], eb[1]), __fadd_rn(eb[2], eb[3]));
+    }
+    sum_a = __fadd_rn(sa[0], sa[1]);
+    sum_b = __fadd_rn(sb[0], sb[1]);
+}
+
+// Two whole tiles of 16-bit candidates straight from their ring stages (pa, pb: the thread's
+// first 16-byte piece of each), common case only.  The pieces are read one ahead of the
+// arithmetic; both stages are released once the last piece has been read.  Returns true when
+// neither candidate needs anything but its error sum recorded (then rec[0].sum and rec[1].sum
+// are written); false leaves both candidates to process_candidate_16.
+template <int CK, bool HAS_ZERO>
+__device__ __forceinline__ bool pair_common_16(const RefRegs<true>& R, const unsigned char* pa,
+                                               const unsigned char* pb, uint32_t empty_a, uint32_t empty_b,
+                                               const Hint& ha, const Hint& hb, WarpRec* rec, int lane) {
+    constexpr float kTiny = 7.8886090522101181e-31f;      // 2^-100
+    constexpr int kStep = kConsumers * 16;                // bytes from a thread's piece to its next one
+    float acc[4] = {0.0f, -kInf, 0.0f, -kInf};
+    float ca[4], cb[4];
+    uint4 a = *reinterpret_cast<const uint4*>(pa), b = *reinterpret_cast<const uint4*>(pb);
+#pragma unroll
+    for (int jv = 0; jv < 4; ++jv) {
+        uint4 an = a, bn = b;
+        if (jv < 3) {
+            an = *reinterpret_cast<const uint4*>(pa + (jv + 1) * kStep);
+            bn = *reinterpret_cast<const uint4*>(pb + (jv + 1) * kStep);
+        }
+        if (jv == 2) {
+            // every piece of both tiles has been read
+            __syncwarp();
+            mbar_arrive_if(empty_a, lane == 0);
+            mbar_arrive_if(empty_b, lane == 0);
+        }
+        piece_16x2<CK, HAS_ZERO>(&R.r[8 * jv], R.atol, a, b, ha.tq_x, hb.tq_x, acc, ca[jv], cb[jv]);
+        a = an; b = bn;
+    }
+    const float s_a = __fadd_rn(__fadd_rn(ca[0], ca[1]), __fadd_rn(ca[2], ca[3]));
+    const float s_b = __fadd_rn(__fadd_rn(cb[0], cb[1]), __fadd_rn(cb[2], cb[3]));
+    bool slow = R.general;
+    {
+        const float m = acc[0], dm = acc[1];
+        const bool hit = dm > 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
+        const bool rel_covers = ha.tq_x >= 0.0f && ha.tq_x <= R.rtol;
+        slow |= !(s_a < kInf) || (m > ha.te_x) || hit || (!rel_covers && m > R.thr_min);
+    }
+    {
+        const float m = acc[2], dm = acc[3];
+        const bool hit = dm > 0.0f || (dm == 0.0f && m != 0.0f && m < kTiny);
+        const bool rel_covers = hb.tq_x >= 0.0f && hb.tq_x <= R.rtol;
+        slow |= !(s_b < kInf) || (m > hb.te_x) || hit || (!rel_covers && m > R.thr_min);
+    }
+    if (__any_sync(kFullMask, slow)) return false;
+    // both warp sums with one butterfly: lanes 0..15 end up with candidate a's, lanes 16..31 with
+    // candidate b's; every level adds the same two values as the butterfly of one candidate
+    const bool up = (lane & 16) != 0;
+    const float keep = up ? s_b : s_a, give = up ? s_a : s_b;
+    float v = __fadd_rn(keep, __shfl_xor_sync(kFullMask, give, 16));
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) v = __fadd_rn(v, __shfl_xor_sync(kFullMask, v, off));
+    if ((lane & 15) == 0) rec[lane >> 4].sum = (double)v;
+    return true;
+}
+
 // One tile of a bf16 or fp16 candidate (32 elements per thread) against the thread's
 // reference registers.  Same results as process_candidate_32; the tests that keep the rare
 // work rare are arranged for errors proportional to |r|, the normal case of a rounded
@@ -1212,7 +1326,52 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     }
 
     // ---- every candidate of the part ----------------------------------------------
-    for (int kk = 0; kk < kc; ++kk) {
+    int kk = 0;
+    if constexpr (C16) {
+        // Whole tiles: two candidates per step while the common case holds.  The rare work
+        // reads the candidate's pieces again, from global memory (the stages are released).
+        if (len == kTile) {
+            for (; kk + 1 < kc; kk += 2) {
+                const Hint ha = H[kk], hb = H[kk + 1];
+                uint32_t sa, sb;
+                wait_stage(ring, B, sa);
+                advance_stage(B);
+                wait_stage(ring, B, sb);
+                advance_stage(B);
+                if (!RKV_IN_BOUNDS(A.header, 11, sa < (uint32_t)kStages && sb < (uint32_t)kStages, sa)) sa = sb = 0;
+                WarpRec* rec = &recs[warp * kPartK + kk];
+                const unsigned char* pa = stages + (size_t)sa * kStageBytes + (size_t)tid * 16;
+                const unsigned char* pb = stages + (size_t)sb * kStageBytes + (size_t)tid * 16;
+                const bool common =
+                    R.warp_has_zero
+                        ? pair_common_16<CK, true>(R, pa, pb, ring.empty0 + 8 * sa, ring.empty0 + 8 * sb, ha, hb, rec, lane)
+                        : pair_common_16<CK, false>(R, pa, pb, ring.empty0 + 8 * sa, ring.empty0 + 8 * sb, ha, hb, rec, lane);
+                const uint32_t settled = __shfl_sync(kFullMask, ha.settled & hb.settled, 0);
+                if (!common || (wanted & ~settled)) {
+#pragma unroll 1
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t w[NW];
+                        // (a whole tile: its kStageBytes lie inside the tensor)
+                        const uint4* gp = reinterpret_cast<const uint4*>(ptrs[kk + c] + start * CSZ) + tid;
+#pragma unroll
+                        for (int jv = 0; jv < NV; ++jv) {
+                            uint4 t = make_uint4(0u, 0u, 0u, 0u);
+                            if (RKV_IN_BOUNDS(A.header, 12, (start + kTile) * CSZ <= D.n * CSZ, start)) t = __ldcg(gp + jv * kConsumers);
+                            w[4 * jv + 0] = t.x; w[4 * jv + 1] = t.y; w[4 * jv + 2] = t.z; w[4 * jv + 3] = t.w;
+                        }
+                        const Hint h = c ? hb : ha;
+                        if (!common)
+                            process_candidate_16<CK>(R, w, h, &H[kk + c], rec + c, st_t + k0 + kk + c, D, &ptrs[kk + c],
+                                                     it.tile, start, len, wanted, tid, lane);
+                        else
+                            candidate_flags<CK>(w, h, &H[kk + c], st_t + k0 + kk + c, D, &ptrs[kk + c], start, len, wanted,
+                                                tid, lane);
+                    }
+                }
+            }
+        }
+    }
+    for (; kk < kc; ++kk) {
         const Hint h = H[kk];
         uint32_t s;
         wait_stage(ring, B, s);
