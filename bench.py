@@ -233,6 +233,9 @@ def build_case(W, dist_name: str, seed: int, rank: int = 0):
         plans.append(plan)
         del cands
     launches += 2                              # verify_kernel (one launch for all tensors) + finalize_case_kernel
+    if W.fused and any(n >= 2048 * (3584 if (W.cand_dtype == "f32" or (W.cand_dtype == "mixed" and t == 0)) else 7168)
+                       for t, n in enumerate(W.numels)):
+        launches += 1                          # copy_check_kernel: regenerated input, a tensor with a warm-up group
     return {"dist": dist_name, "seed": seed, "descs": descs, "gens": gens, "K": W.K, "plans": plans,
             "plan_last": plans[-1], "algo_bytes": algo_bytes, "launches": launches}
 
@@ -344,7 +347,7 @@ def time_workload_alone(name: str, rank: int, launches: int = 20):
         del c, ev
         torch.cuda.empty_cache()
     r = roofline_of(durs, statistics.mean(nbytes), name,
-                    "events bracket rkv_verify_multi: table upload + workspace clear + verify_kernel + finalize_case_kernel")
+                    "events bracket rkv_verify_multi: table upload + workspace clear + verify_kernel (+ copy_check_kernel with a regenerated input) + finalize_case_kernel")
     return {"workload": f"{W.name}: K={W.K}, shapes {list(W.shapes)}, cand {W.cand_dtype}, "
                         f"{len(W.dists)} distributions",
             "ms_per_call": r["avg_launch_ms"], "median_ms": r["median_launch_ms"], "best_ms": r["best_launch_ms"],
@@ -486,7 +489,7 @@ def run_native(args):
     launch_bytes = statistics.mean(b for (_, _, b) in events)
     roofline = roofline_of(durs, launch_bytes, args.workload,
                            "events bracket rkv_verify_multi: table upload + workspace clear + verify_kernel "
-                           "(one launch over every tensor and storage type) + finalize_case_kernel")
+                           "(one launch over every tensor and storage type) + copy_check_kernel (regenerated input) + finalize_case_kernel")
 
     checks = [verdict_check(c) for cases in sets for c in cases]
     pairs = [[f"{c['dist']}/seed {c['seed']}" for c in cases] for cases in sets]

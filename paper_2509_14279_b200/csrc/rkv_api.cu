@@ -142,6 +142,7 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
     plan->grid = grid;
     plan->T = T;
     plan->n_cases = n_cases;
+    plan->any_deferred = false;
     uint64_t rows = 0, sums = 0;
     for (int t = 0; t < T; ++t) {
         const rkv_tensor_desc& s = tensors[t];
@@ -168,6 +169,8 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
         d.sum_base = sums;
         sums += (uint64_t)d.n_tiles * (uint64_t)K;
         d.case_index = case_of ? case_of[t] : 0u;
+        d.defer_copy = (s.input_src == RKV_SRC_GENERATED && d.warm_tiles < d.n_tiles) ? 1u : 0u;
+        if (d.defer_copy) plan->any_deferred = true;
         d.out_base = out_base ? out_base[t] : (uint64_t)t;
         d.out_stride = out_stride ? out_stride[t] : (uint32_t)T;
     }
@@ -288,6 +291,10 @@ int run_case(const rkv_tensor_desc* tensors, int K, int k_begin, int k_end, bool
     }
     int rc = launch_verify(L, plan.T, K, k_begin, k_end, plan.n_items, plan.n_segments, (int)plan.grid, stream);
     if (rc != RKV_OK) return rc;
+    if (plan.any_deferred) {
+        rc = launch_copy_check(L, plan.T, K, k_begin, k_end, (int)plan.grid / kBlocksPerSm, stream);
+        if (rc != RKV_OK) return rc;
+    }
     if (finalize) rc = launch_finalize(L, plan.T, K, plan.n_cases, stats_out, case_pass, all_pass, stream);
     return rc;
 }

@@ -97,6 +97,12 @@ struct DevTensor {
     uint32_t state_base;    // first CandState of this tensor (K + 1 entries)
     uint32_t out_stride;    // rkv_stats index step from candidate k to k + 1 (tensors of the tensor's case)
     uint32_t case_index;    // the case this tensor belongs to (0 unless a sweep)
+    // 1: the input is regenerated and the tensor has tiles beyond its warm-up group.  The
+    // verification kernel then compares candidates with the input on the warm-up tiles only
+    // (which settles every candidate that is no copy); the few candidates still bit-equal to
+    // the input after them are compared over the whole tensor by copy_check_kernel.
+    uint32_t defer_copy;
+    uint32_t reserved0;
     uint64_t sum_base;      // first tile sum (n_tiles x K doubles, [tile][k]) of this tensor
     uint64_t out_base;      // rkv_stats index of candidate 0 of this tensor
 };
@@ -146,6 +152,7 @@ struct Plan {
     uint32_t grid = 0;                   // blocks per launch (num_sms * kBlocksPerSm)
     uint32_t n_items = 0;
     uint32_t n_cases = 1;
+    bool any_deferred = false;           // some tensor has defer_copy set: copy_check_kernel runs after verify_kernel
     size_t off_tensors = 0, off_segments = 0, off_ptrs = 0, off_fail = 0, off_state = 0, off_partials = 0,
            off_sums = 0;
     size_t upload_bytes = 0;             // header + descriptors + segments + pointer tables
@@ -217,6 +224,9 @@ struct Layout {
 int launch_verify(const Layout& L, int T, int K, int k_begin, int k_end, uint32_t n_items, uint32_t n_segments,
                   int grid, cudaStream_t stream);
 int verify_occupancy();   // resident verification blocks per SM on the current device
+// Candidates [k_begin, k_end) of every tensor with defer_copy set that are still bit-equal to the
+// regenerated input after the warm-up tiles: compared with it over the whole tensor.
+int launch_copy_check(const Layout& L, int T, int K, int k_begin, int k_end, int num_sms, cudaStream_t stream);
 int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,
                     uint32_t* all_pass, cudaStream_t stream);
 int launch_gen(uint64_t seed, uint64_t stream_id, int dist, uint64_t n, uint64_t first_elem,

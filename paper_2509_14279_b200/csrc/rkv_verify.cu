@@ -1248,7 +1248,11 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
     const int k0 = (int)it.k0, kc = (int)it.kc;
     const uint64_t start = (uint64_t)it.tile * kTile;
     const uint32_t len = (uint32_t)min((uint64_t)kTile, D.n - start);
-    const uint32_t wanted = D.input_src != RKV_SRC_NONE ? 3u : 1u;
+    // flags looked for: bit0 constant, bit1 copy of the input.  The reference is always checked for
+    // both; with defer_copy the candidates are compared with the (regenerated) input on the warm-up
+    // tiles only, and copy_check_kernel settles whoever is still bit-equal to it after them.
+    const uint32_t wanted_ref = D.input_src != RKV_SRC_NONE ? 3u : 1u;
+    const uint32_t wanted = (D.defer_copy && it.tile >= D.warm_tiles) ? 1u : wanted_ref;
     CandState* st_t = A.state + D.state_base;
 
     // (range checks of a debug build: the tile lies inside the tensor; the state, hint and
@@ -1300,7 +1304,7 @@ __device__ __forceinline__ void run_item(const Args& A, unsigned char* smem, con
 
     // reference flags (constant / copy of the input), until a difference has been seen
     {
-        const uint32_t need = wanted & ~ref_state[B.ord & 1u];
+        const uint32_t need = wanted_ref & ~ref_state[B.ord & 1u];
         if (need) {
             const uint32_t r_first = first_elem_bits(D.ref, D.ref_src, D.ref_dtype, D.ref_seed,
                                                      D.ref_stream, D.ref_dist);
@@ -1493,6 +1497,94 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __
 }
 
 // ----------------------------------------------------------------------------
+// copy check: candidates still bit-equal to a regenerated input after the warm-up tiles
+// ----------------------------------------------------------------------------
+// The whole grid compares one such candidate with the input, regenerated Philox block by
+// Philox block (one 16-byte piece of the candidate per thread and step), and stops at the
+// first difference any thread finds.  Only true copies are read to the end.
+constexpr int kCopyThreads = 256;
+
+template <int DIST, bool BF16>
+__device__ __forceinline__ void copy_check_scan(const DevTensor& D, const unsigned char* cand, CandState* st) {
+    const PhiloxKey key = philox_key(D.in_seed);
+    constexpr uint32_t kUnit = BF16 ? 8u : 4u;                 // elements per 16-byte piece
+    const uint64_t n_units = (D.n + kUnit - 1) / kUnit;
+    const uint64_t stride = (uint64_t)gridDim.x * kCopyThreads;
+    uint32_t it = 0;
+    for (uint64_t u = (uint64_t)blockIdx.x * kCopyThreads + threadIdx.x; u < n_units; u += stride, ++it) {
+        // somebody has found a difference: done (looked at every 8th step)
+        if ((it & 7u) == 7u && (__ldcg(&st->mismatch) & 2u)) return;
+        const uint64_t e0 = u * kUnit;
+        uint32_t g[8];
+        float v[4];
+        gen_block<DIST>(BF16 ? 2 * u : u, D.in_stream, key, v);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) g[q] = BF16 ? bf16_rne_bits(v[q]) : __float_as_uint(v[q]);
+        if (BF16) {
+            gen_block<DIST>(2 * u + 1, D.in_stream, key, v);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) g[4 + q] = bf16_rne_bits(v[q]);
+        }
+        uint32_t diff = 0;
+        if (e0 + kUnit <= D.n) {
+            const uint4 c = __ldcs(reinterpret_cast<const uint4*>(cand) + u);
+            if (BF16) diff = (c.x ^ (g[0] | (g[1] << 16))) | (c.y ^ (g[2] | (g[3] << 16))) |
+                             (c.z ^ (g[4] | (g[5] << 16))) | (c.w ^ (g[6] | (g[7] << 16)));
+            else diff = (c.x ^ g[0]) | (c.y ^ g[1]) | (c.z ^ g[2]) | (c.w ^ g[3]);
+        } else {
+#pragma unroll
+            for (uint32_t q = 0; q < kUnit; ++q)
+                if (e0 + q < D.n) diff |= ld_elem_raw(cand, BF16 ? RKV_BF16 : RKV_F32, e0 + q) ^ g[q];
+        }
+        if (diff) {
+            atomicOr(&st->mismatch, 2u);
+            return;
+        }
+    }
+}
+
+// Every block goes through the same (tensor, candidate) pairs, found 256 at a time by all its
+// threads at once (one global read per thread instead of one after the other), and takes its
+// share of each pair's pieces.
+__global__ void __launch_bounds__(kCopyThreads)
+copy_check_kernel(const DevTensor* __restrict__ tensors, int T, int k_begin, int k_end, CandState* state) {
+    __shared__ unsigned char t_flag[kCopyThreads], k_flag[kCopyThreads];
+    const int tid = threadIdx.x;
+    for (int t0 = 0; t0 < T; t0 += kCopyThreads) {
+        const int mine_t = (t0 + tid < T && tensors[t0 + tid].defer_copy) ? 1 : 0;
+        t_flag[tid] = (unsigned char)mine_t;
+        if (!__syncthreads_or(mine_t)) continue;
+        const int t_end = min(T - t0, kCopyThreads);
+        for (int ti = 0; ti < t_end; ++ti) {
+            if (!t_flag[ti]) continue;
+            const DevTensor& D = tensors[t0 + ti];
+            const bool b16 = D.cand_dtype == RKV_BF16;
+            for (int kb = k_begin; kb < k_end; kb += kCopyThreads) {
+                const int k = kb + tid;
+                const int mine_k = (k < k_end && !(__ldcg(&state[D.state_base + k].mismatch) & 2u)) ? 1 : 0;
+                __syncthreads();                       // the previous round's flags have been read
+                k_flag[tid] = (unsigned char)mine_k;
+                if (!__syncthreads_or(mine_k)) continue;
+                const int k_cnt = min(k_end - kb, kCopyThreads);
+                for (int ki = 0; ki < k_cnt; ++ki) {
+                    if (!k_flag[ki]) continue;
+                    CandState* st = state + D.state_base + kb + ki;
+                    const unsigned char* cand = reinterpret_cast<const unsigned char*>(D.cands[kb + ki]);
+                    switch (D.in_dist) {
+                        case 0: b16 ? copy_check_scan<0, true>(D, cand, st) : copy_check_scan<0, false>(D, cand, st); break;
+                        case 1: b16 ? copy_check_scan<1, true>(D, cand, st) : copy_check_scan<1, false>(D, cand, st); break;
+                        case 2: b16 ? copy_check_scan<2, true>(D, cand, st) : copy_check_scan<2, false>(D, cand, st); break;
+                        case 3: b16 ? copy_check_scan<3, true>(D, cand, st) : copy_check_scan<3, false>(D, cand, st); break;
+                        default: b16 ? copy_check_scan<4, true>(D, cand, st) : copy_check_scan<4, false>(D, cand, st); break;
+                    }
+                }
+            }
+        }
+        __syncthreads();                               // t_flag is rewritten by the next round
+    }
+}
+
+// ----------------------------------------------------------------------------
 // finalize: merge the per-block partials of each (candidate, tensor) in a fixed
 // order, add the tile sums in tile order, derive flags and verdict; then the joint
 // verdicts over the tensors of a case and over the cases
@@ -1658,6 +1750,12 @@ int verify_occupancy() {
         return 0;
     }
     return n;
+}
+
+int launch_copy_check(const Layout& L, int T, int K, int k_begin, int k_end, int num_sms, cudaStream_t stream) {
+    (void)K;
+    copy_check_kernel<<<(unsigned)num_sms * 3u, kCopyThreads, 0, stream>>>(L.d_tensors, T, k_begin, k_end, L.state);
+    return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
 int launch_finalize(const Layout& L, int T, int K, uint32_t n_cases, rkv_stats* stats_out, uint32_t* case_pass,

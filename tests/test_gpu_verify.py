@@ -523,3 +523,33 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_workspace_stays_usable
     want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands_cpu], ATOL, RTOL)
     for k in range(K):
         assert_stats_equal(got[k], want[k], f"after the drill k={k}")
+
+
+@pytest.mark.parametrize("dtype,tile", [("f32", 3584), ("bf16", 7168)])
+def test_copy_of_a_regenerated_input_on_a_tensor_with_a_warm_up_group(dtype, tile):
+    """Reference and input regenerated on the device, a tensor long enough to have a warm-up
+    group: the candidates are compared with the input on the warm-up tiles only, and whoever is
+    still bit-equal to it afterwards is compared over the whole tensor by the copy-check kernel.
+    A true copy must be flagged; copies that differ in one element (inside the warm-up tiles,
+    right behind them, in the middle, at the very end) must not."""
+    n = tile * 2048 + (1234 if dtype == "f32" else 77)
+    odt = "f32" if dtype == "f32" else "bf16"
+    ref = oracle_gen_tensor(5, 0, oracle.UNIFORM_PM1, n, "f32")
+    inp = oracle_gen_tensor(5, 2, oracle.UNIFORM_PM1, n, odt)
+    def copy_but(i):
+        c = inp.clone()
+        c[i] = 0.25 if float(c[i]) != 0.25 else 0.5
+        return c
+    cands = [inp.clone(), copy_but(3 * tile + 1), copy_but(18 * tile + 5), copy_but(n // 2 + 3), copy_but(n - 1),
+             pop.materialize(pop.Candidate(pop.REF_EXACT), ref, inp, dtype),
+             pop.materialize(pop.Candidate(pop.BF16_ULP if dtype == "bf16" else pop.NOISE, sigma=1e-7, noise_seed=9),
+                             ref, inp, dtype),
+             inp.clone()]
+    tol = (1e-5, 1e-5) if dtype == "f32" else (1e-2, 1.6e-2)
+    got, joint = run_gpu(ref, cands, tol[0], tol[1], gen_ref=(5, 0, rkv.DIST_UNIFORM_PM1),
+                         gen_inp=(5, 2, rkv.DIST_UNIFORM_PM1))
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], tol[0], tol[1], pop.bits_numpy(inp))
+    for k, w in enumerate(want):
+        assert_stats_equal(got[k], w, f"copy check {dtype} k={k}")
+    copy_flag = [bool(int(g["flags"]) & rkv.FLAG_CAND_COPY_OF_INPUT) for g in got]
+    assert copy_flag == [True, False, False, False, False, False, False, True]
