@@ -1500,40 +1500,44 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __
 // copy check: candidates still bit-equal to a regenerated input after the warm-up tiles
 // ----------------------------------------------------------------------------
 // The whole grid compares one such candidate with the input, regenerated Philox block by
-// Philox block (one 16-byte piece of the candidate per thread and step), and stops at the
+// Philox block (four elements of the candidate per thread and step), and stops at the
 // first difference any thread finds.  Only true copies are read to the end.
 constexpr int kCopyThreads = 256;
 
 template <int DIST, bool BF16>
 __device__ __forceinline__ void copy_check_scan(const DevTensor& D, const unsigned char* cand, CandState* st) {
     const PhiloxKey key = philox_key(D.in_seed);
-    constexpr uint32_t kUnit = BF16 ? 8u : 4u;                 // elements per 16-byte piece
-    const uint64_t n_units = (D.n + kUnit - 1) / kUnit;
+    // one Philox block = four elements per thread and step: 16 bytes of an fp32 candidate, 8 of a bf16 one
+    const uint64_t n_blocks = (D.n + 3u) >> 2;
     const uint64_t stride = (uint64_t)gridDim.x * kCopyThreads;
     uint32_t it = 0;
-    for (uint64_t u = (uint64_t)blockIdx.x * kCopyThreads + threadIdx.x; u < n_units; u += stride, ++it) {
+    for (uint64_t u = (uint64_t)blockIdx.x * kCopyThreads + threadIdx.x; u < n_blocks; u += stride, ++it) {
         // somebody has found a difference: done (looked at every 8th step)
         if ((it & 7u) == 7u && (__ldcg(&st->mismatch) & 2u)) return;
-        const uint64_t e0 = u * kUnit;
-        uint32_t g[8];
+        const uint64_t e0 = u << 2;
+        const bool whole = e0 + 4u <= D.n;
+        // the candidate's piece is asked for first: its latency hides behind the generation
+        uint4 c = make_uint4(0u, 0u, 0u, 0u);
+        if (whole) {
+            if (BF16) {
+                const uint2 h = __ldcs(reinterpret_cast<const uint2*>(cand) + u);
+                c.x = h.x; c.y = h.y;
+            } else {
+                c = __ldcs(reinterpret_cast<const uint4*>(cand) + u);
+            }
+        }
         float v[4];
-        gen_block<DIST>(BF16 ? 2 * u : u, D.in_stream, key, v);
+        gen_block<DIST>(u, D.in_stream, key, v);
+        uint32_t g[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) g[q] = BF16 ? bf16_rne_bits(v[q]) : __float_as_uint(v[q]);
-        if (BF16) {
-            gen_block<DIST>(2 * u + 1, D.in_stream, key, v);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) g[4 + q] = bf16_rne_bits(v[q]);
-        }
         uint32_t diff = 0;
-        if (e0 + kUnit <= D.n) {
-            const uint4 c = __ldcs(reinterpret_cast<const uint4*>(cand) + u);
-            if (BF16) diff = (c.x ^ (g[0] | (g[1] << 16))) | (c.y ^ (g[2] | (g[3] << 16))) |
-                             (c.z ^ (g[4] | (g[5] << 16))) | (c.w ^ (g[6] | (g[7] << 16)));
+        if (whole) {
+            if (BF16) diff = (c.x ^ (g[0] | (g[1] << 16))) | (c.y ^ (g[2] | (g[3] << 16)));
             else diff = (c.x ^ g[0]) | (c.y ^ g[1]) | (c.z ^ g[2]) | (c.w ^ g[3]);
         } else {
 #pragma unroll
-            for (uint32_t q = 0; q < kUnit; ++q)
+            for (uint32_t q = 0; q < 4u; ++q)
                 if (e0 + q < D.n) diff |= ld_elem_raw(cand, BF16 ? RKV_BF16 : RKV_F32, e0 + q) ^ g[q];
         }
         if (diff) {
