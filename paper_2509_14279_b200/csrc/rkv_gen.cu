@@ -23,8 +23,12 @@ gen_kernel(uint64_t seed, uint64_t stream_id, uint64_t first_block, uint64_t n, 
         const uint64_t e0 = u * kUnitElems;
         const bool full = e0 + kUnitElems <= n;
         if (!BF16) {
-            float v[4];
+            // two Philox blocks a step where the thread has two left (their dependent chains overlap)
+            const uint64_t u2 = u + stride;
+            const bool pair = u2 < n_units && (u2 + 1) * 4 <= n;
+            float v[4], v2[4];
             gen_block<DIST>(first_block + u, stream_id, key, v);
+            gen_block<DIST>(first_block + (pair ? u2 : u), stream_id, key, v2);    // (unconditional: one basic block)
             float* o = reinterpret_cast<float*>(out) + e0;
             if (full) {
                 *reinterpret_cast<float4*>(o) = make_float4(v[0], v[1], v[2], v[3]);
@@ -32,6 +36,10 @@ gen_kernel(uint64_t seed, uint64_t stream_id, uint64_t first_block, uint64_t n, 
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (e0 + q < n) o[q] = v[q];
+            }
+            if (pair) {
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + u2 * 4) = make_float4(v2[0], v2[1], v2[2], v2[3]);
+                u += stride;
             }
         } else {
             float v[8];
