@@ -100,9 +100,33 @@ __device__ __forceinline__ void finish(const ElemState& e, CrossAcc& a, unsigned
     if (d > a.spread) { a.spread = d; a.arg = index; }       // ascending index: the first maximum stays
 }
 
+// One vector position by the general rule (values that are not finite included).  Out of line: it
+// runs for the rare positions that hold a NaN or an infinity, and its registers stay out of the
+// kernel's count.
+template <int DT>
+__device__ __noinline__ CrossAcc general_position(const void* const* mine, int S, unsigned long long v, float atol,
+                                                  float rtol, CrossAcc a) {
+    constexpr int VEC = DT == RKV_F32 ? 4 : 8;
+    ElemState e[VEC];
+    uint32_t raw0[VEC];
+    for (int s = 0; s < S; ++s) {
+        const uint4 w = __ldcs(reinterpret_cast<const uint4*>(mine[s]) + v);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
+            if (s == 0) raw0[i] = raw;
+            visit<DT>(e[i], a, raw, raw0[i], s == 0, atol, rtol);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) finish(e[i], a, v * VEC + i);
+    return a;
+}
+
 // grid = (blocks per candidate, K).  outs[k * S + s]: candidate k's output for input seed s.
 template <int DT>
-__global__ void __launch_bounds__(kCrossThreads)
+__global__ void __launch_bounds__(kCrossThreads, 3)
 cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long long n, float atol, float rtol,
                   CrossPartial* __restrict__ partials) {
     constexpr int VEC = DT == RKV_F32 ? 4 : 8;
@@ -115,8 +139,16 @@ cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long lon
 
     for (unsigned long long v = (unsigned long long)blockIdx.x * kCrossThreads + threadIdx.x; v < n_vec;
          v += (unsigned long long)gridDim.x * kCrossThreads) {
-        ElemState e[VEC];
-        uint32_t raw0[VEC];
+        // Common case: every value of the position is finite.  Then "within tolerance of seed 0" is one
+        // subtraction and one comparison against a threshold kept from seed 0, "same bits" one
+        // exclusive-or per 32-bit word, and one fused multiply-add per value (x * 0 is NaN exactly for
+        // NaN and the infinities) tells afterwards whether the assumption held.  If it did not, the
+        // position is done again by the general rule.
+        float x0[VEC], thr[VEC], lo[VEC], hi[VEC];
+        uint32_t w0[4] = {0u, 0u, 0u, 0u};
+        uint32_t xacc = 0;
+        float chk = 0.0f;
+        bool far = false;
         for (int s0 = 0; s0 < S; s0 += CH) {
             uint4 w[CH];
 #pragma unroll
@@ -126,16 +158,42 @@ cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long lon
             for (int c = 0; c < CH; ++c) {
                 if (s0 + c >= S) break;
                 const uint32_t words[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+                if (s0 + c == 0) {
 #pragma unroll
-                for (int i = 0; i < VEC; ++i) {
-                    const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
-                    if (s0 + c == 0) raw0[i] = raw;
-                    visit<DT>(e[i], a, raw, raw0[i], s0 + c == 0, atol, rtol);
+                    for (int q = 0; q < 4; ++q) w0[q] = words[q];
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
+                        const float x = __uint_as_float(widen<DT>(raw));
+                        x0[i] = x; lo[i] = x; hi[i] = x;
+                        thr[i] = __fadd_rn(atol, __fmul_rn(rtol, fabsf(x)));
+                        chk = __fmaf_rn(x, 0.0f, chk);
+                    }
+                } else {
+                    xacc |= (words[0] ^ w0[0]) | (words[1] ^ w0[1]) | (words[2] ^ w0[2]) | (words[3] ^ w0[3]);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) {
+                        const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
+                        const float x = __uint_as_float(widen<DT>(raw));
+                        far |= !(fabsf(__fsub_rn(x, x0[i])) <= thr[i]);
+                        lo[i] = fminf(lo[i], x);
+                        hi[i] = fmaxf(hi[i], x);
+                        chk = __fmaf_rn(x, 0.0f, chk);
+                    }
                 }
             }
         }
+        if (chk == 0.0f) {
+            a.differs |= (xacc ? 1u : 0u) | (far ? 2u : 0u);
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) finish(e[i], a, v * VEC + i);
+            for (int i = 0; i < VEC; ++i) {
+                const float d = __fsub_rn(hi[i], lo[i]);
+                if (d > a.spread) { a.spread = d; a.arg = v * VEC + i; }       // ascending index: the first maximum stays
+            }
+            continue;
+        }
+        // ---- general rule (a NaN or an infinity somewhere in the position), out of line ----
+        a = general_position<DT>(mine, S, v, atol, rtol, a);
     }
     // the ragged end: fewer elements than a vector, one thread of the first block
     if (blockIdx.x == 0 && threadIdx.x == 0) {
