@@ -1505,45 +1505,48 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) verify_kernel(const __
 constexpr int kCopyThreads = 256;
 
 template <int DIST, bool BF16>
-__device__ __forceinline__ void copy_check_scan(const DevTensor& D, const unsigned char* cand, CandState* st) {
+__device__ __noinline__ void copy_check_scan(const DevTensor& D, const unsigned char* cand, CandState* st) {
     const PhiloxKey key = philox_key(D.in_seed);
     // one Philox block = four elements per thread and step: 16 bytes of an fp32 candidate, 8 of a bf16 one
-    const uint64_t n_blocks = (D.n + 3u) >> 2;
+    const uint64_t n = D.n, stream_id = D.in_stream;
+    const uint64_t n_whole = n >> 2;
     const uint64_t stride = (uint64_t)gridDim.x * kCopyThreads;
-    uint32_t it = 0;
-    for (uint64_t u = (uint64_t)blockIdx.x * kCopyThreads + threadIdx.x; u < n_blocks; u += stride, ++it) {
+    uint64_t u = (uint64_t)blockIdx.x * kCopyThreads + threadIdx.x;
+    while (u < n_whole) {
         // somebody has found a difference: done (looked at every 8th step)
-        if ((it & 7u) == 7u && (__ldcg(&st->mismatch) & 2u)) return;
-        const uint64_t e0 = u << 2;
-        const bool whole = e0 + 4u <= D.n;
-        // the candidate's piece is asked for first: its latency hides behind the generation
-        uint4 c = make_uint4(0u, 0u, 0u, 0u);
-        if (whole) {
+        if (__ldcg(&st->mismatch) & 2u) return;
+#pragma unroll 1
+        for (int j = 0; j < 8 && u < n_whole; ++j, u += stride) {
+            // the candidate's piece is asked for first: its latency hides behind the generation
+            uint4 c = make_uint4(0u, 0u, 0u, 0u);
             if (BF16) {
                 const uint2 h = __ldcs(reinterpret_cast<const uint2*>(cand) + u);
                 c.x = h.x; c.y = h.y;
             } else {
                 c = __ldcs(reinterpret_cast<const uint4*>(cand) + u);
             }
+            float v[4];
+            gen_block<DIST>(u, stream_id, key, v);
+            uint32_t diff;
+            if (BF16) diff = (c.x ^ (bf16_rne_bits(v[0]) | (bf16_rne_bits(v[1]) << 16))) |
+                             (c.y ^ (bf16_rne_bits(v[2]) | (bf16_rne_bits(v[3]) << 16)));
+            else diff = (c.x ^ __float_as_uint(v[0])) | (c.y ^ __float_as_uint(v[1])) |
+                        (c.z ^ __float_as_uint(v[2])) | (c.w ^ __float_as_uint(v[3]));
+            if (diff) {
+                atomicOr(&st->mismatch, 2u);
+                return;
+            }
         }
+    }
+    // the last one to three elements of a tensor whose length is no multiple of four
+    if ((n & 3u) && blockIdx.x == 0 && threadIdx.x == 0) {
         float v[4];
-        gen_block<DIST>(u, D.in_stream, key, v);
-        uint32_t g[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) g[q] = BF16 ? bf16_rne_bits(v[q]) : __float_as_uint(v[q]);
+        gen_block<DIST>(n_whole, stream_id, key, v);
         uint32_t diff = 0;
-        if (whole) {
-            if (BF16) diff = (c.x ^ (g[0] | (g[1] << 16))) | (c.y ^ (g[2] | (g[3] << 16)));
-            else diff = (c.x ^ g[0]) | (c.y ^ g[1]) | (c.z ^ g[2]) | (c.w ^ g[3]);
-        } else {
-#pragma unroll
-            for (uint32_t q = 0; q < 4u; ++q)
-                if (e0 + q < D.n) diff |= ld_elem_raw(cand, BF16 ? RKV_BF16 : RKV_F32, e0 + q) ^ g[q];
-        }
-        if (diff) {
-            atomicOr(&st->mismatch, 2u);
-            return;
-        }
+        for (uint32_t q = 0; q < (uint32_t)(n & 3u); ++q)
+            diff |= ld_elem_raw(cand, BF16 ? RKV_BF16 : RKV_F32, (n_whole << 2) + q) ^
+                    (BF16 ? bf16_rne_bits(v[q]) : __float_as_uint(v[q]));
+        if (diff) atomicOr(&st->mismatch, 2u);
     }
 }
 
