@@ -1,7 +1,8 @@
 // rkv_gen_inputs: counter-based multi-distribution input generator (sm_100a).
 //
-// One thread produces whole Philox blocks (four consecutive elements each) and
-// writes them with one 16-byte store: a block for fp32, two blocks for bf16.
+// One thread produces whole Philox blocks (four consecutive elements each), two a
+// step so that their dependent chains overlap: for bf16 the two blocks of one 16-byte
+// store, for fp32 the blocks of two 16-byte stores a grid stride apart.
 // Consecutive threads write consecutive 16-byte units, so a warp stores 512
 // contiguous bytes.  The kernel is ALU-bound (about 50 integer + fp32
 // instructions per element against 4 bytes written).
