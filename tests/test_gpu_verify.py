@@ -553,3 +553,35 @@ def test_copy_of_a_regenerated_input_on_a_tensor_with_a_warm_up_group(dtype, til
         assert_stats_equal(got[k], w, f"copy check {dtype} k={k}")
     copy_flag = [bool(int(g["flags"]) & rkv.FLAG_CAND_COPY_OF_INPUT) for g in got]
     assert copy_flag == [True, False, False, False, False, False, False, True]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+def test_two_candidates_per_step_fall_back_late_in_a_long_tensor(dtype):
+    """16-bit candidates of a tensor with a warm-up group are taken two per step once the
+    published maxima make the common case common.  Planted far behind the warm-up tiles: a new
+    largest error, a NaN, an infinity and a lone element over tolerance, each in another
+    candidate of a pair (and in both of one pair), so that the step has to give both candidates
+    to the one-by-one code, which reads their pieces again from global memory."""
+    tile = 7168
+    n = tile * 2100 + 13
+    ref = oracle_gen_tensor(8, 0, oracle.UNIFORM_PM1, n, "f32")
+    td = torch.bfloat16 if dtype == "bf16" else torch.float16
+    base = ref.to(td)
+    def planted(edits):
+        c = base.clone()
+        for i, v in edits:
+            c[i] = v
+        return c
+    late = tile * 2000
+    cands = [base.clone(), planted([(n - 5, 3.0)]),
+             planted([(late + 3, float("nan"))]), planted([(late + tile + 9, float("inf"))]),
+             planted([(late + 5 * tile + 1, 0.75), (late + 5 * tile + 2, -0.75)]), base.clone(),
+             planted([(late + 77, float(base[late + 77]) + 0.125)])]
+    atol, rtol = 1e-2, 1.6e-2
+    got, joint = run_gpu(ref, cands, atol, rtol)
+    want = oracle_case(pop.bits_numpy(ref), [pop.bits_numpy(c) for c in cands], atol, rtol)
+    for k, w in enumerate(want):
+        assert_stats_equal(got[k], w, f"late fallback {dtype} k={k}")
+        assert int(joint[k]) == int(w["verdict"] == 0)
+    assert int(got[1]["argmax_abs_err"]) == n - 5
+    assert [int(j) for j in joint] == [1, 0, 0, 0, 0, 1, 0]
