@@ -23,7 +23,7 @@ namespace rkv {
 namespace {
 
 constexpr int kCrossThreads = 256;
-constexpr int kCrossBlocksPerSm = 6;
+constexpr int kCrossBlocksPerSm = 24;      // blocks per SM the grid is sized for (about eight waves: measured best of 3 .. 48)
 constexpr int kCrossMaxSeeds = 16;
 constexpr int kCopyMaxInputs = 8;
 constexpr int kCrossMaxK = 4096;
