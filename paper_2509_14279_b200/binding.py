@@ -547,10 +547,16 @@ def screen_to_numpy(stats: torch.Tensor) -> np.ndarray:
     return stats.detach().cpu().numpy().view(SCREEN_DTYPE)
 
 
-def cross_seed(outs, atol: float, rtol: float, spread_lim: float = 0.01, stats_out: torch.Tensor | None = None,
-               workspace: torch.Tensor | None = None, stream=None) -> tuple:
-    """rkv_cross_seed: outs[k][s] is candidate k's output for input seed s (device tensors of one
-    size and dtype).  Returns (stats [K * 32 bytes, uint8], workspace)."""
+class CrossTable:
+    """The checked pointer table of one rkv_cross_seed call (see prepare_cross)."""
+
+    def __init__(self, ptrs, K, S, n, code, device, keep):
+        self.ptrs, self.K, self.S, self.n, self.code, self.device, self.keep = ptrs, K, S, n, code, device, keep
+
+
+def prepare_cross(outs) -> CrossTable:
+    """Check outs[k][s] (candidate k's output for input seed s: device tensors of one size and
+    dtype) once and marshal their addresses, for callers that repeat a call on the same tensors."""
     K, S = len(outs), len(outs[0])
     first = outs[0][0]
     _require(first, "cross_seed: outs[0][0]", device=torch.device("cuda"))
@@ -560,15 +566,24 @@ def cross_seed(outs, atol: float, rtol: float, spread_lim: float = 0.01, stats_o
             raise ValueError("cross_seed: every candidate needs the same number of seeds")
         for s, t in enumerate(row):
             _require(t, f"cross_seed: outs[{k}][{s}]", device=first.device, dtype=first.dtype, numel=first.numel())
-    dev = first.device
+    ptrs = (ctypes.c_void_p * (K * S))(*[t.data_ptr() for row in outs for t in row])
+    return CrossTable(ptrs, K, S, first.numel(), code, first.device, [list(row) for row in outs])
+
+
+def cross_seed(outs, atol: float, rtol: float, spread_lim: float = 0.01, stats_out: torch.Tensor | None = None,
+               workspace: torch.Tensor | None = None, stream=None, table: CrossTable | None = None) -> tuple:
+    """rkv_cross_seed: outs[k][s] is candidate k's output for input seed s (device tensors of one
+    size and dtype); with ``table`` (from prepare_cross on the same tensors) the checks and the
+    marshalling are not repeated.  Returns (stats [K * 32 bytes, uint8], workspace)."""
+    tb = table if table is not None else prepare_cross(outs)
+    K, S, dev = tb.K, tb.S, tb.device
     if workspace is None:
         workspace = torch.empty(max(256, int(lib().rkv_cross_workspace_bytes(K, S))), dtype=torch.uint8, device=dev)
     if stats_out is None:
         stats_out = torch.empty(K * CROSS_BYTES, dtype=torch.uint8, device=dev)
     else:
         _require(stats_out, "cross_seed: stats_out", device=dev, dtype=torch.uint8, min_bytes=K * CROSS_BYTES)
-    ptrs = (ctypes.c_void_p * (K * S))(*[t.data_ptr() for row in outs for t in row])
-    _check(lib().rkv_cross_seed(ptrs, K, S, first.numel(), code, float(atol), float(rtol), float(spread_lim),
+    _check(lib().rkv_cross_seed(tb.ptrs, K, S, tb.n, tb.code, float(atol), float(rtol), float(spread_lim),
                                 ctypes.c_void_p(stats_out.data_ptr()), ctypes.c_void_p(workspace.data_ptr()),
                                 workspace.numel(), ctypes.c_void_p(_stream_ptr(stream))), "rkv_cross_seed")
     return stats_out, workspace

@@ -4,7 +4,9 @@
 //     one launch.  For one vector position a thread visits the S outputs of its candidate in
 //     turn, so the per-element minimum and maximum across seeds, and seed 0's value, never
 //     leave registers; every output byte is read once.  Bound: HBM read bandwidth
-//     (K * S * n * element size bytes);
+//     (K * S * n * element size bytes).  Up to eight seeds take cross_seed_few_kernel (every seed's
+//     piece of a position in registers at once, eight 16-byte loads per thread in flight), more
+//     take cross_seed_kernel (batches of loads, per-element state carried between batches);
 //   * copy of any input: is a candidate's output a bit copy of one of the M operands the
 //     kernel received?  16-byte pieces are compared as stored; a block stops comparing
 //     against an operand as soon as any block has seen a difference, so only true copies are
@@ -28,7 +30,6 @@ constexpr int kCrossMaxSeeds = 16;
 constexpr int kCopyMaxInputs = 8;
 constexpr int kCrossMaxK = 4096;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
-constexpr float kInfF = __builtin_huge_valf();
 
 __device__ __forceinline__ bool finite_bits(uint32_t b) { return (b & 0x7F800000u) != 0x7F800000u; }
 __device__ __forceinline__ bool inf_bits(uint32_t b) { return (b & 0x7FFFFFFFu) == 0x7F800000u; }
@@ -124,6 +125,129 @@ __device__ __noinline__ CrossAcc general_position(const void* const* mine, int S
     return a;
 }
 
+// The end of both kernels: the ragged end of the tensor, then the block's partial.
+template <int DT>
+__device__ __forceinline__ void cross_block_end(CrossAcc a, const void* const* mine, int k, int S, unsigned long long n,
+                                                float atol, float rtol, CrossPartial* __restrict__ partials) {
+    constexpr int VEC = DT == RKV_F32 ? 4 : 8;
+    const unsigned long long n_vec = n / VEC;
+    // the ragged end: fewer elements than a vector, one thread of the first block
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (unsigned long long i = n_vec * VEC; i < n; ++i) {
+            ElemState e;
+            uint32_t raw0 = 0;
+            for (int s = 0; s < S; ++s) {
+                const uint32_t raw = DT == RKV_F32 ? reinterpret_cast<const uint32_t*>(mine[s])[i]
+                                                   : reinterpret_cast<const unsigned short*>(mine[s])[i];
+                if (s == 0) raw0 = raw;
+                visit<DT>(e, a, raw, raw0, s == 0, atol, rtol);
+            }
+            finish(e, a, i);
+        }
+    }
+    // block reduction: shuffle tree, then the warps' results in warp order
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        CrossAcc b;
+        b.arg = __shfl_xor_sync(kFull, a.arg, off);
+        b.n_nonfin = __shfl_xor_sync(kFull, a.n_nonfin, off);
+        b.spread = __shfl_xor_sync(kFull, a.spread, off);
+        b.differs = __shfl_xor_sync(kFull, a.differs, off);
+        merge(a, b);
+    }
+    __shared__ CrossAcc warp_acc[kCrossThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_acc[threadIdx.x >> 5] = a;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CrossAcc t = warp_acc[0];
+        for (int w = 1; w < kCrossThreads / 32; ++w) merge(t, warp_acc[w]);
+        CrossPartial p;
+        p.arg = t.arg; p.n_nonfin = t.n_nonfin; p.spread = t.spread; p.differs = t.differs;
+        p.reserved[0] = p.reserved[1] = 0;
+        partials[(size_t)k * gridDim.x + blockIdx.x] = p;
+    }
+}
+
+// One storage word -> element i of it, widened.
+template <int DT>
+__device__ __forceinline__ float elem_of(const uint4& w, int i) {
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    const uint32_t raw = DT == RKV_F32 ? words[i] : ((i & 1) ? words[i >> 1] >> 16 : words[i >> 1] & 0xFFFFu);
+    return __uint_as_float(widen<DT>(raw));
+}
+
+// S <= CH: every seed's piece of a position is in registers at once, so nothing is carried from
+// seed to seed but the loaded words themselves, and NP positions (one grid stride apart) have their
+// loads in flight together: CH * NP 16-byte loads per thread.  A seed slot beyond S repeats seed 0's
+// piece, which changes none of the results.  Same rule and same results as cross_seed_kernel.
+template <int DT, int CH, int NP, int MINB>
+__global__ void __launch_bounds__(kCrossThreads, MINB)
+cross_seed_few_kernel(const void* const* __restrict__ outs, int S, unsigned long long n, float atol, float rtol,
+                      CrossPartial* __restrict__ partials) {
+    constexpr int VEC = DT == RKV_F32 ? 4 : 8;
+    const int k = blockIdx.y;
+    const void* const* mine = outs + (size_t)k * (size_t)S;
+    const unsigned long long n_vec = n / VEC;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kCrossThreads;
+    CrossAcc a;
+    a.arg = RKV_NO_INDEX; a.n_nonfin = 0; a.spread = -1.0f; a.differs = 0;
+    const uint4* base[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) base[c] = reinterpret_cast<const uint4*>(mine[c < S ? c : 0]);
+
+    for (unsigned long long v = (unsigned long long)blockIdx.x * kCrossThreads + threadIdx.x; v < n_vec;
+         v += NP * stride) {
+        uint4 w[NP][CH];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const unsigned long long vp = v + (unsigned long long)p * stride;
+            if (vp < n_vec) {
+#pragma unroll
+                for (int c = 0; c < CH; ++c) w[p][c] = __ldcs(base[c] + vp);
+            }
+        }
+        // positions in ascending order, so that the first maximum stays
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const unsigned long long vp = v + (unsigned long long)p * stride;
+            if (vp >= n_vec) break;
+            uint32_t xacc = 0;
+#pragma unroll
+            for (int c = 1; c < CH; ++c)
+                xacc |= (w[p][c].x ^ w[p][0].x) | (w[p][c].y ^ w[p][0].y) | (w[p][c].z ^ w[p][0].z) | (w[p][c].w ^ w[p][0].w);
+            // (x * 0 is NaN exactly for NaN and the infinities: chk tells whether every value was finite)
+            float chk = 0.0f, best = -1.0f;
+            int best_i = 0;
+            bool far = false;
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) {
+                const float x0 = elem_of<DT>(w[p][0], i);
+                const float thr = __fadd_rn(atol, __fmul_rn(rtol, fabsf(x0)));
+                float lo = x0, hi = x0;
+                chk = __fmaf_rn(x0, 0.0f, chk);
+#pragma unroll
+                for (int c = 1; c < CH; ++c) {
+                    const float x = elem_of<DT>(w[p][c], i);
+                    far |= !(fabsf(__fsub_rn(x, x0)) <= thr);
+                    lo = fminf(lo, x);
+                    hi = fmaxf(hi, x);
+                    chk = __fmaf_rn(x, 0.0f, chk);
+                }
+                const float d = __fsub_rn(hi, lo);
+                if (d > best) { best = d; best_i = i; }
+            }
+            if (chk == 0.0f) {
+                a.differs |= (xacc ? 1u : 0u) | (far ? 2u : 0u);
+                if (best > a.spread) { a.spread = best; a.arg = vp * VEC + best_i; }
+            } else {
+                // a NaN or an infinity somewhere in the position: the general rule, out of line
+                a = general_position<DT>(mine, S, vp, atol, rtol, a);
+            }
+        }
+    }
+    cross_block_end<DT>(a, mine, k, S, n, atol, rtol, partials);
+}
+
 // grid = (blocks per candidate, K).  outs[k * S + s]: candidate k's output for input seed s.
 template <int DT>
 __global__ void __launch_bounds__(kCrossThreads, 3)
@@ -195,41 +319,7 @@ cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long lon
         // ---- general rule (a NaN or an infinity somewhere in the position), out of line ----
         a = general_position<DT>(mine, S, v, atol, rtol, a);
     }
-    // the ragged end: fewer elements than a vector, one thread of the first block
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (unsigned long long i = n_vec * VEC; i < n; ++i) {
-            ElemState e;
-            uint32_t raw0 = 0;
-            for (int s = 0; s < S; ++s) {
-                const uint32_t raw = DT == RKV_F32 ? reinterpret_cast<const uint32_t*>(mine[s])[i]
-                                                   : reinterpret_cast<const unsigned short*>(mine[s])[i];
-                if (s == 0) raw0 = raw;
-                visit<DT>(e, a, raw, raw0, s == 0, atol, rtol);
-            }
-            finish(e, a, i);
-        }
-    }
-    // block reduction: shuffle tree, then the warps' results in warp order
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        CrossAcc b;
-        b.arg = __shfl_xor_sync(kFull, a.arg, off);
-        b.n_nonfin = __shfl_xor_sync(kFull, a.n_nonfin, off);
-        b.spread = __shfl_xor_sync(kFull, a.spread, off);
-        b.differs = __shfl_xor_sync(kFull, a.differs, off);
-        merge(a, b);
-    }
-    __shared__ CrossAcc warp_acc[kCrossThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_acc[threadIdx.x >> 5] = a;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        CrossAcc t = warp_acc[0];
-        for (int w = 1; w < kCrossThreads / 32; ++w) merge(t, warp_acc[w]);
-        CrossPartial p;
-        p.arg = t.arg; p.n_nonfin = t.n_nonfin; p.spread = t.spread; p.differs = t.differs;
-        p.reserved[0] = p.reserved[1] = 0;
-        partials[(size_t)k * gridDim.x + blockIdx.x] = p;
-    }
+    cross_block_end<DT>(a, mine, k, S, n, atol, rtol, partials);
 }
 
 __global__ void cross_finalize_kernel(const CrossPartial* __restrict__ partials, int K, int S, int blocks,
@@ -368,12 +458,23 @@ int rkv_cross_seed(const void* const* outs, int K, int S, uint64_t n, int dtype,
     const int vec = dtype == RKV_F32 ? 4 : 8;
     const int blocks = blocks_per_candidate(n / vec, K, sms);
     const dim3 grid((unsigned)blocks, (unsigned)K);
-    if (dtype == RKV_F32)
-        cross_seed_kernel<RKV_F32><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
-    else if (dtype == RKV_BF16)
-        cross_seed_kernel<RKV_BF16><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
-    else
-        cross_seed_kernel<RKV_F16><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials);
+    // Up to eight seeds: all of a position's pieces in registers at once, eight 16-byte loads per thread in
+    // flight (three blocks per SM for fp32; the 16-bit forms unpack twice the values and get the registers
+    // of two blocks per SM, measured faster than three with spills).
+#define RKV_CROSS_FEW(DT, CH, NP, MINB) \
+    cross_seed_few_kernel<DT, CH, NP, MINB><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials)
+#define RKV_CROSS_BY_S(DT, MINB)                              \
+    do {                                                      \
+        if (S <= 2) RKV_CROSS_FEW(DT, 2, 4, MINB);            \
+        else if (S <= 4) RKV_CROSS_FEW(DT, 4, 2, MINB);       \
+        else if (S <= 8) RKV_CROSS_FEW(DT, 8, 1, MINB);       \
+        else cross_seed_kernel<DT><<<grid, kCrossThreads, 0, stream>>>(d_ptrs, S, n, atol, rtol, partials); \
+    } while (0)
+    if (dtype == RKV_F32) RKV_CROSS_BY_S(RKV_F32, 3);
+    else if (dtype == RKV_BF16) RKV_CROSS_BY_S(RKV_BF16, 2);
+    else RKV_CROSS_BY_S(RKV_F16, 2);
+#undef RKV_CROSS_BY_S
+#undef RKV_CROSS_FEW
     cross_finalize_kernel<<<(K + 127) / 128, 128, 0, stream>>>(partials, K, S, blocks, spread_lim, stats_out);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }

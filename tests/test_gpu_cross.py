@@ -43,7 +43,8 @@ KINDS = ["honest", "hardcoded", "ignores_input", "nearly_fixed", "one_element", 
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
-@pytest.mark.parametrize("n,S", [(1, 2), (5, 3), (1000, 1), (4099, 2), (65537, 4), (300001, 9), (1 << 20, 16)])
+@pytest.mark.parametrize("n,S", [(1, 2), (5, 3), (1000, 1), (4099, 2), (65537, 4), (70001, 6), (200003, 8), (300001, 9),
+                                 (1 << 20, 16)])
 def test_cross_seed_matches_the_oracle(dtype, n, S):
     outs = [_candidate_outputs(k, n, S, dtype, seed=7 + i) for i, k in enumerate(KINDS)]
     atol, rtol = (1e-5, 1e-5) if dtype == "f32" else (1e-2, 1.6e-2)
