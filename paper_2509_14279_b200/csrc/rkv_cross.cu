@@ -322,18 +322,31 @@ cross_seed_kernel(const void* const* __restrict__ outs, int S, unsigned long lon
     cross_block_end<DT>(a, mine, k, S, n, atol, rtol, partials);
 }
 
+// One warp per candidate: the lanes go through the blocks' partials in strides, then a shuffle tree
+// (the merge is associative and commutative: integer sums, ors, value-then-first-index maxima).
 __global__ void cross_finalize_kernel(const CrossPartial* __restrict__ partials, int K, int S, int blocks,
                                       float spread_lim, rkv_cross_stats* __restrict__ stats_out) {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= K) return;
+    const int k = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (k >= K) return;                                  // whole warps leave together
     CrossAcc t;
     t.arg = RKV_NO_INDEX; t.n_nonfin = 0; t.spread = -1.0f; t.differs = 0;
-    for (int b = 0; b < blocks; ++b) {
+    for (int b = lane; b < blocks; b += 32) {
         const CrossPartial p = partials[(size_t)k * blocks + b];
         CrossAcc q;
         q.arg = p.arg; q.n_nonfin = p.n_nonfin; q.spread = p.spread; q.differs = p.differs;
         merge(t, q);
     }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        CrossAcc q;
+        q.arg = __shfl_xor_sync(kFull, t.arg, off);
+        q.n_nonfin = __shfl_xor_sync(kFull, t.n_nonfin, off);
+        q.spread = __shfl_xor_sync(kFull, t.spread, off);
+        q.differs = __shfl_xor_sync(kFull, t.differs, off);
+        merge(t, q);
+    }
+    if (lane != 0) return;
     rkv_cross_stats st;
     memset(&st, 0, sizeof st);
     st.n_nonfinite = t.n_nonfin;
@@ -475,7 +488,7 @@ int rkv_cross_seed(const void* const* outs, int K, int S, uint64_t n, int dtype,
     else RKV_CROSS_BY_S(RKV_F16, 2);
 #undef RKV_CROSS_BY_S
 #undef RKV_CROSS_FEW
-    cross_finalize_kernel<<<(K + 127) / 128, 128, 0, stream>>>(partials, K, S, blocks, spread_lim, stats_out);
+    cross_finalize_kernel<<<(K + 3) / 4, 128, 0, stream>>>(partials, K, S, blocks, spread_lim, stats_out);
     return cudaGetLastError() == cudaSuccess ? RKV_OK : RKV_ERR_CUDA;
 }
 
