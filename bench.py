@@ -92,6 +92,37 @@ def kernel_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
+def generator_inst_per_elem():
+    """Lane-instructions per generated element and distribution, from the committed ncu count
+    (``profiles/gen_kernel_f32.md``); None once the generator's sources changed since."""
+    try:
+        h = hashlib.sha256()
+        for f in ("rkv_gen.cu", "rkv_philox.cuh"):
+            with open(os.path.join(ROOT, "paper_2509_14279_b200", "csrc", f), "rb") as fh:
+                h.update(fh.read())
+        rec, inst = {}, {}
+        with open(os.path.join(ROOT, "profiles", "gen_kernel_f32.md")) as fh:
+            for line in fh:
+                if line.startswith("- lane_inst_per_elem "):
+                    k, v = line[len("- lane_inst_per_elem "):].split(":", 1)
+                    inst[k.strip()] = float(v)
+                elif line.startswith("- kernel_source_hash:"):
+                    rec["hash"] = line.split(":", 1)[1].strip().strip("`")
+        return inst if rec.get("hash") == h.hexdigest()[:16] else None
+    except Exception:
+        return None
+
+
+def sm_max_mhz(index: int) -> float:
+    """clocks.max.sm of the device (read only), 1965 MHz if nvidia-smi does not answer."""
+    try:
+        r = subprocess.run(["nvidia-smi", "--query-gpu=clocks.max.sm", "--format=csv,noheader,nounits", "-i", str(index)],
+                           capture_output=True, text=True, timeout=20)
+        return float(r.stdout.strip().splitlines()[0])
+    except Exception:
+        return 1965.0
+
+
 def recorded_traffic(workload: str, algo_bytes: float):
     """DRAM bytes per launch of the dominant kernel, from the committed ncu summary
     (``profiles/verify_kernel_<workload>.md`` holds the measured DRAM bytes per
@@ -368,6 +399,10 @@ def time_generator(with_oracle: bool):
 
     n = 1 << 24
     peak, peak_kind = measured_peak()
+    inst = generator_inst_per_elem()
+    props = torch.cuda.get_device_properties(0)
+    # one warp instruction per scheduler and clock: SMs x 4 schedulers x 32 lanes x the SM clock
+    alu_peak = props.multi_processor_count * 4 * 32 * sm_max_mhz(0) * 1e6
     out = torch.empty(n, dtype=torch.float32, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     res = {}
@@ -388,10 +423,15 @@ def time_generator(with_oracle: bool):
         res[name] = {"gpu_elems_per_s": round(n / mean, 1), "us_per_launch": round(mean * 1e6, 2),
                      "best_us": round(min(durs) * 1e6, 2), "written_GBps": round(n * 4 / mean / 1e9, 1),
                      "frac": round(n * 4 / mean / 1e9 / peak, 4)}
+        if inst and name in inst:
+            res[name]["lane_inst_per_elem"] = inst[name]
+            res[name]["alu_frac"] = round(n / mean * inst[name] / alu_peak, 4)
     out_d = {"kernel": "gen_kernel", "bound": "alu", "elements": n, "dtype": "f32", "peak": peak,
-             "peak_kind": f"of {peak_kind}", "per_distribution": res,
+             "peak_kind": f"of {peak_kind}", "alu_peak_lane_inst_per_s": alu_peak, "per_distribution": res,
              "note": "frac = bytes written / event time / copy peak; the kernel is bound by its arithmetic "
-                     "(Philox rounds, polynomial log/sincos, IEEE divide and square root), not by the stores"}
+                     "(Philox rounds, polynomial log/sincos, IEEE divide and square root), not by the stores; "
+                     "alu_frac = elements/s x lane-instructions per element (ncu count, profiles/gen_kernel_f32.md) "
+                     "/ (SMs x 4 schedulers x 32 lanes x max SM clock)"}
     if with_oracle:
         import oracle
         n_o = 1 << 21

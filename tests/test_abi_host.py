@@ -281,6 +281,11 @@ def test_binding_refuses_mismatched_tensors_before_the_c_call():
         rkv.TensorDesc(n=1024, cands=[good], atol=1e-5, rtol=1e-5, ref=ref).to_c()
     with pytest.raises(TypeError):
         rkv._require(3.0, "x")
+    # the pointer table of the cross-seed check is refused the same way, before anything is marshalled
+    with pytest.raises(ValueError, match="on cpu, expected cuda"):
+        rkv.prepare_cross([[good, good]])
+    with pytest.raises(ValueError, match="on cpu, expected cuda"):
+        rkv.cross_seed([[good, good]], 1e-5, 1e-5)
 
 
 def test_cross_checks_validate_before_any_cuda_call():
