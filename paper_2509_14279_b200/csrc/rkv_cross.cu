@@ -176,6 +176,50 @@ __device__ __forceinline__ float elem_of(const uint4& w, int i) {
     return __uint_as_float(widen<DT>(raw));
 }
 
+// Two 16-bit values per 32-bit word at once.  Minimum and maximum select one of their operands, so
+// the packed forms give exactly the values the fp32 forms give on the widened operands.
+template <int DT>
+__device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    if (DT == RKV_BF16) asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    else asm("min.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+template <int DT>
+__device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    if (DT == RKV_BF16) asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    else asm("max.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// chk + x * 0 in both halves: stays a zero while every x is finite, NaN afterwards
+template <int DT>
+__device__ __forceinline__ uint32_t fma2_zero(uint32_t x, uint32_t chk) {
+    uint32_t d;
+    const uint32_t zero = 0u;
+    if (DT == RKV_BF16) asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(x), "r"(zero), "r"(chk));
+    else asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(x), "r"(zero), "r"(chk));
+    return d;
+}
+// x - r in fp32 with one rounding, x the low or high 16-bit value of a word (widening is exact, so
+// this is the fp32 subtraction of the widened value)
+template <int DT>
+__device__ __forceinline__ float sub_half_f32(uint32_t word, int half, float r) {
+    float d;
+    if (DT == RKV_BF16) {
+        if (half) asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(word), "f"(r));
+        else asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(word), "f"(r));
+    } else {
+        if (half) asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.f16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(word), "f"(r));
+        else asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.f16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(word), "f"(r));
+    }
+    return d;
+}
+template <int DT>
+__device__ __forceinline__ float half_of(uint32_t word, int half) {
+    return __uint_as_float(widen<DT>(half ? word >> 16 : word & 0xFFFFu));
+}
+
 // S <= CH: every seed's piece of a position is in registers at once, so nothing is carried from
 // seed to seed but the loaded words themselves, and NP positions (one grid stride apart) have their
 // loads in flight together: CH * NP 16-byte loads per thread.  A seed slot beyond S repeats seed 0's
@@ -219,6 +263,36 @@ cross_seed_few_kernel(const void* const* __restrict__ outs, int S, unsigned long
             float chk = 0.0f, best = -1.0f;
             int best_i = 0;
             bool far = false;
+            if (DT != RKV_F32) {
+                // 16-bit values two at a time: packed minimum, maximum and finiteness check; the
+                // tolerance test stays in fp32 (one mixed-precision subtraction per value)
+                uint32_t chk2 = 0u;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t w0[4] = {w[p][0].x, w[p][0].y, w[p][0].z, w[p][0].w};
+                    const uint32_t first = w0[q];
+                    const float x0a = half_of<DT>(first, 0), x0b = half_of<DT>(first, 1);
+                    const float thra = __fadd_rn(atol, __fmul_rn(rtol, fabsf(x0a)));
+                    const float thrb = __fadd_rn(atol, __fmul_rn(rtol, fabsf(x0b)));
+                    uint32_t lo2 = first, hi2 = first;
+                    chk2 = fma2_zero<DT>(first, chk2);
+#pragma unroll
+                    for (int c = 1; c < CH; ++c) {
+                        const uint32_t wc[4] = {w[p][c].x, w[p][c].y, w[p][c].z, w[p][c].w};
+                        const uint32_t x2 = wc[q];
+                        lo2 = min2<DT>(lo2, x2);
+                        hi2 = max2<DT>(hi2, x2);
+                        chk2 = fma2_zero<DT>(x2, chk2);
+                        far |= !(fabsf(sub_half_f32<DT>(x2, 0, x0a)) <= thra);
+                        far |= !(fabsf(sub_half_f32<DT>(x2, 1, x0b)) <= thrb);
+                    }
+                    const float da = __fsub_rn(half_of<DT>(hi2, 0), half_of<DT>(lo2, 0));
+                    const float db = __fsub_rn(half_of<DT>(hi2, 1), half_of<DT>(lo2, 1));
+                    if (da > best) { best = da; best_i = 2 * q; }
+                    if (db > best) { best = db; best_i = 2 * q + 1; }
+                }
+                chk = (chk2 & 0x7FFF7FFFu) ? 1.0f : 0.0f;
+            } else
 #pragma unroll
             for (int i = 0; i < VEC; ++i) {
                 const float x0 = elem_of<DT>(w[p][0], i);

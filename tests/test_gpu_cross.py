@@ -69,6 +69,31 @@ def test_cross_seed_matches_the_oracle(dtype, n, S):
         assert flags["nonfinite"] & rkv.CROSS_NONFINITE
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("S", [2, 4, 7, 11])
+def test_cross_seed_zeros_of_both_signs_and_subnormals(dtype, S):
+    """Outputs that differ across seeds only in the sign of a zero, and outputs of subnormal size:
+    the spread is a zero of the oracle's sign, the outputs are not identical but within tolerance;
+    minimum and maximum of 16-bit values are taken on pairs of values, which must not show."""
+    n = 4099
+    g = torch.Generator().manual_seed(5)
+    signs = [torch.where(torch.rand(n, generator=g) < 0.5, 0.0, -0.0) for _ in range(S)]
+    tiny = {"f32": 1e-41, "bf16": 1e-39, "f16": 3e-7}[dtype]
+    small = [(torch.randint(-3, 4, (n,), generator=g).double() * tiny).to(TD[dtype]) for _ in range(S)]
+    mixed = [torch.where(torch.rand(n, generator=g) < 0.3, sg.to(TD[dtype]), sm) for sg, sm in zip(signs, small)]
+    outs = [[t.to(TD[dtype]).contiguous() for t in signs], small, mixed]
+    stats, _ = rkv.cross_seed([[t.cuda() for t in row] for row in outs], 1e-5, 1e-5, 0.01)
+    got = rkv.cross_to_numpy(stats)
+    for k, row in enumerate(outs):
+        want = oracle.cross_seed([pop.bits_numpy(t) for t in row], 1e-5, 1e-5, 0.01)
+        assert int(got[k]["flags"]) == want["flags"], (k, dtype, S)
+        assert int(got[k]["n_nonfinite"]) == want["n_nonfinite"] == 0
+        assert int(got[k]["argmax_spread"]) == want["argmax_spread"], (k, dtype, S)
+        assert f32_bits(got[k]["max_spread"]) == f32_bits(want["max_spread"]), (k, dtype, S)
+    assert f32_bits(got[0]["max_spread"]) == 0 and int(got[0]["argmax_spread"]) == 0
+    assert int(got[0]["flags"]) & rkv.CROSS_WITHIN_TOL and not int(got[0]["flags"]) & rkv.CROSS_IDENTICAL
+
+
 def test_cross_seed_is_deterministic_and_validates():
     outs = [[t.cuda() for t in _candidate_outputs("honest", 123457, 5, "f32", seed=3)] for _ in range(3)]
     a, ws = rkv.cross_seed(outs, 1e-5, 1e-5)
