@@ -22,7 +22,10 @@ static int plan_one(uint64_t n, int cand_dtype, uint32_t* n_tiles, uint32_t* war
     const uint64_t tiles = (n + te - 1) / te;
     if (tiles > 0x3FFFFFFFull) return RKV_ERR_UNSUPPORTED;
     *n_tiles = (uint32_t)tiles;
-    *warm_tiles = tiles >= (uint64_t)kWarmMinTiles ? (uint32_t)kWarmTiles : (uint32_t)tiles;
+    // a shorter tensor warms up on the same share of its tiles, at least one
+    *warm_tiles = tiles >= (uint64_t)kWarmMinTiles
+                      ? (uint32_t)kWarmTiles
+                      : (uint32_t)((tiles * (uint64_t)kWarmTiles + (uint64_t)kWarmMinTiles - 1) / (uint64_t)kWarmMinTiles);
     return RKV_OK;
 }
 
@@ -144,12 +147,23 @@ int make_plan(const rkv_tensor_desc* tensors, int T, int K, int k_count, int num
     plan->n_cases = n_cases;
     plan->any_deferred = false;
     uint64_t rows = 0, sums = 0;
+    // A launch whose tiles all fit the first wave of blocks has nobody to warm up for: what a
+    // block publishes comes too late for the others, so every tile is a warm-up tile.
+    uint64_t launch_tiles = 0;
+    for (int t = 0; t < T; ++t) {
+        uint32_t nt = 0, wt = 0;
+        const int rc = plan_one(tensors[t].n, tensors[t].cand_dtype, &nt, &wt);
+        if (rc != RKV_OK) return rc;
+        launch_tiles += nt;
+    }
+    const bool one_wave = launch_tiles <= (uint64_t)grid;
     for (int t = 0; t < T; ++t) {
         const rkv_tensor_desc& s = tensors[t];
         DevTensor& d = plan->tensors[t];
         memset(&d, 0, sizeof d);
         const int rc = plan_one(s.n, s.cand_dtype, &d.n_tiles, &d.warm_tiles);
         if (rc != RKV_OK) return rc;
+        if (one_wave) d.warm_tiles = d.n_tiles;
         d.tail_tiles = tail_tiles_of(d.n_tiles, d.warm_tiles, grid);
         d.n = s.n;
         d.ref = s.ref_src == RKV_SRC_POINTER ? s.ref : nullptr;

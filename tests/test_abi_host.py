@@ -54,7 +54,7 @@ def test_stats_struct_is_88_bytes():
 
 
 @pytest.mark.parametrize("K", [1, 2, 8, 63, 64, 65, 128, 256, 1000])
-@pytest.mark.parametrize("n", [1, 127, 3584, 3585, 4096, 262144, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
+@pytest.mark.parametrize("n", [1, 127, 3584, 3585, 4096, 262144, 1200000, 4000000, 1 << 24, (1 << 25) + 3, (1 << 30) + 17])
 @pytest.mark.parametrize("dtype", [rkv.F32, rkv.BF16, rkv.F16])
 def test_item_plan_properties(n, K, dtype):
     sms = 148
@@ -67,10 +67,17 @@ def test_item_plan_properties(n, K, dtype):
     if warm < grid:
         # few tiles: the candidates are split so that every block gets an item, if K allows
         assert warm * parts_warm >= min(grid, warm * K)
+    if n_tiles <= grid:
+        assert warm == n_tiles           # everything fits the first wave of blocks: nobody to warm up for
+    else:
+        # 18 tiles of 2048 or more, the same share of fewer
+        assert warm == (18 if n_tiles >= 2048 else -(-n_tiles * 18 // 2048))
     if warm < n_tiles:
-        # a large tensor: a short warm-up group, then the fewest parts of at most 64
-        assert warm * tile >= 60000 and warm * 100 < n_tiles
-        assert parts_main == -(-K // 64)
+        # a short warm-up group, then the fewest parts of at most 64 (more while the tiles are fewer
+        # than the blocks)
+        assert warm * 100 < n_tiles + 100
+        main = n_tiles - warm - tail
+        assert parts_main == max(-(-K // 64), min(K, -(-grid // main) if main < grid else 1))
         # a long tensor ends with half a tile per block in parts a quarter that size
         if n_tiles - warm >= 4 * grid:
             assert tail == grid // 2 and parts_tail == min(K, 4 * parts_main)
