@@ -108,27 +108,35 @@ void plan_items(Plan* plan, int k_count) {
         const uint32_t p2 = (kc + kPartK - 1) / kPartK * tail_div;
         d.parts[2] = p2 > kc ? kc : p2;
     }
-    // Item numbering: group 0 of every tensor, then group 1 of every tensor, then group 2,
-    // the tensors one after the other inside a group.  (Dealing the items of an fp32 and of a
-    // 16-bit tensor out in turn, so that HBM-bound and issue-bound items share every SM, was
-    // measured 11 % slower than one tensor after the other.)
+    // Item numbering: group 0 of every tensor, then group 1 of every tensor, then group 2;
+    // inside a group the tensors of one storage type one after the other, then those of the
+    // next type.  The kernel has one instantiation of its item code per candidate storage type,
+    // and a block that changes type with every item runs out of its instruction cache: a sweep
+    // of alternating fp32 / bf16 / fp16 cases took twice the time of the same sweep in one
+    // type.  (Dealing the items of an fp32 and of a 16-bit tensor out in turn, so that
+    // HBM-bound and issue-bound items share every SM, was measured 11 % slower than one tensor
+    // after the other.)
     uint32_t n_seg = 0;
     uint64_t id = 0;
+    static const int32_t kTypeOrder[3] = {RKV_F32, RKV_BF16, RKV_F16};
     for (uint32_t g = 0; g < 3; ++g) {
-        for (int t = 0; t < plan->T; ++t) {
-            const DevTensor& d = plan->tensors[t];
-            const uint64_t cnt = (uint64_t)group_tiles(g, d.n_tiles, d.warm_tiles, d.tail_tiles) * d.parts[g];
-            if (!cnt) continue;
-            if ((size_t)n_seg + 1 >= plan->segment_capacity || id + cnt > 0x7FFFFFFFull) {
-                id = 0x100000000ull;          // cannot be numbered: the caller refuses the case
-                continue;
+        for (int ty = 0; ty < 3; ++ty) {
+            for (int t = 0; t < plan->T; ++t) {
+                const DevTensor& d = plan->tensors[t];
+                if (d.cand_dtype != kTypeOrder[ty]) continue;
+                const uint64_t cnt = (uint64_t)group_tiles(g, d.n_tiles, d.warm_tiles, d.tail_tiles) * d.parts[g];
+                if (!cnt) continue;
+                if ((size_t)n_seg + 1 >= plan->segment_capacity || id + cnt > 0x7FFFFFFFull) {
+                    id = 0x100000000ull;          // cannot be numbered: the caller refuses the case
+                    continue;
+                }
+                Segment& s = plan->segments[n_seg++];
+                s.first_id = (uint32_t)id;
+                s.first_local = 0;
+                s.tensor = (uint32_t)t;
+                s.group = g;
+                id += cnt;
             }
-            Segment& s = plan->segments[n_seg++];
-            s.first_id = (uint32_t)id;
-            s.first_local = 0;
-            s.tensor = (uint32_t)t;
-            s.group = g;
-            id += cnt;
         }
     }
     const bool too_many = id > 0x7FFFFFFFull;
