@@ -345,16 +345,18 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * elements per tile).  One work item is
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
- * part past them.  A large tensor has three groups of items: the first *warm_tiles
- * tiles, with the candidates cut into *parts_warm parts (many small ones, so that
- * every resident block -- 2 per SM -- starts with one of these items), are
- * verified first; the running maxima and loophole flags they publish let the
- * tiles after them, with *parts_main parts of at most 64 candidates, skip nearly
- * all rare-path work; the last *tail_tiles tiles, with *parts_tail parts of at most
- * 16 candidates, come last and even out the finishing times of the blocks.  A
- * smaller tensor has one group: *warm_tiles == *n_tiles, *parts_main == 0,
- * *tail_tiles == 0 and *parts_tail == 0.  Part p of P covers candidates
- * [p*K/P, (p+1)*K/P).
+ * part past them.  A tensor has up to three groups of items: the first *warm_tiles
+ * tiles (18 of 2048 tiles or more, the same share, at least one, of fewer), with the
+ * candidates cut into *parts_warm parts (many small ones, so that every resident
+ * block -- 2 per SM -- starts with one of these items), are verified first; the
+ * running maxima and loophole flags they publish let the tiles after them, with
+ * *parts_main parts of at most 64 candidates (more while these tiles are fewer than
+ * the blocks), skip nearly all rare-path work; the last *tail_tiles tiles of a long
+ * tensor, with *parts_tail parts of at most 16 candidates, come last and even out the
+ * finishing times of the blocks.  A tensor whose tiles all fit the first wave of
+ * blocks has one group: *warm_tiles == *n_tiles, *parts_main == 0, *tail_tiles == 0
+ * and *parts_tail == 0 (in a call of several tensors, the tiles of all of them
+ * count).  Part p of P covers candidates [p*K/P, (p+1)*K/P).
  *   cand_dtype  RKV_F32 | RKV_BF16 | RKV_F16 (storage type of the candidates)
  *   num_sms     SM count of the device
  * Errors: INVALID_ARG (n < 1, K < 1, num_sms < 1, bad dtype, null), UNSUPPORTED (n >= 2^40).
