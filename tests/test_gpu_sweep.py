@@ -127,3 +127,43 @@ def test_sweep_with_regenerated_references_and_a_large_case_among_small_ones():
             w = oracle.verify(pop.bits_numpy(ref), pop.bits_numpy(cands[k]), tol[0], tol[1], input=pop.bits_numpy(inp))
             assert_stats_equal(got[c * K + k], w, f"case {c} k={k}")
             assert int(case_pass[c, k]) == int(w["verdict"] == 0)
+
+
+def test_sweep_of_short_tensors_with_warm_up_and_split_main_groups():
+    """Three tensors of 30 to 151 tiles among forty of one tile: more tiles than the first wave of
+    blocks holds, so every tensor has a warm-up group of its own (one or two tiles), and fewer
+    main-group tiles than blocks, so the main group splits the candidates into parts.  Stored and
+    regenerated references, the three storage types, faults in every group; a copy of a regenerated
+    input goes through the copy check of a short tensor."""
+    K = 10
+    spec = [(3584 * 150 + 17, "f32", oracle.NORMAL, True), (7168 * 90 + 5, "bf16", oracle.STUDENT_T2, False),
+            (7168 * 29 + 7000, "f16", oracle.UNIFORM_PM1, False), (3584 * 40 + 1, "bf16", oracle.NORMAL_1E4, True)]
+    spec += [(1 + 97 * i, "f32" if i % 2 else "bf16", oracle.DISTS[i % 5], i % 4 == 0) for i in range(40)]
+    cases_gpu, cpu = [], []
+    for c, (n, cdt, dist, regenerated) in enumerate(spec):
+        rdt = "f32"
+        ref = oracle_gen_tensor(1300 + c, 0, dist, n, rdt)
+        inp = oracle_gen_tensor(1300 + c, 2, dist, n, "bf16" if cdt == "bf16" else "f32").to(TD[cdt])
+        cands = build_case_cpu(mixed_plan(K, n, seed=1300 + c, bf16=cdt != "f32"), ref, inp, cdt)
+        tol = (1e-5, 1e-5) if cdt == "f32" else (1e-2, 1.6e-2)
+        cpu.append((ref, inp, cands, tol))
+        if regenerated and cdt != "f16":
+            cases_gpu.append([rkv.TensorDesc(n=n, cands=[x.cuda() for x in cands], atol=tol[0], rtol=tol[1],
+                                             ref_gen=(1300 + c, 0, dist), input_gen=(1300 + c, 2, dist))])
+        else:
+            cases_gpu.append([rkv.TensorDesc(n=n, cands=[x.cuda() for x in cands], atol=tol[0], rtol=tol[1],
+                                             ref=ref.cuda(), input=inp.cuda())])
+    stats, case_pass, all_pass, ws = rkv.verify_sweep(cases_gpu, K)
+    assert rkv.device_status(ws) == rkv.OK
+    got = rkv.stats_to_numpy(stats)
+    seen_fail = 0
+    for c, (ref, inp, cands, tol) in enumerate(cpu):
+        for k in range(K):
+            w = oracle.verify(pop.bits_numpy(ref), pop.bits_numpy(cands[k]), tol[0], tol[1], input=pop.bits_numpy(inp))
+            assert_stats_equal(got[c * K + k], w, f"case {c} k={k}")
+            assert int(case_pass[c, k]) == int(w["verdict"] == 0)
+            seen_fail += int(w["verdict"] != 0)
+    assert seen_fail > 0
+    # the same launch twice: byte for byte
+    stats2, _, _, _ = rkv.verify_sweep(cases_gpu, K)
+    assert rkv.stats_to_numpy(stats2).tobytes() == got.tobytes()
