@@ -346,7 +346,7 @@ int rkv_verify_batch_static(const void *ref, const void *const *cands, int K, ui
  * one tile against a part of the K candidates: a thread block keeps the tile's
  * reference values in registers and streams that tile of each candidate of the
  * part past them.  A tensor has up to three groups of items: the first *warm_tiles
- * tiles (18 of 2048 tiles or more, the same share, at least one, of fewer), with the
+ * tiles (the square root of the tile count, rounded down, at most 18), with the
  * candidates cut into *parts_warm parts (many small ones, so that every resident
  * block -- 2 per SM -- starts with one of these items), are verified first; the
  * running maxima and loophole flags they publish let the tiles after them, with

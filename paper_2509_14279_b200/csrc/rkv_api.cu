@@ -14,18 +14,22 @@ namespace rkv {
 // planning
 // ----------------------------------------------------------------------------
 
-// How one tensor is cut: tiles of tile_elems(cand_dtype) elements; a large tensor's first
-// kWarmTiles tiles form the warm-up group (see DevTensor).
+// How one tensor is cut: tiles of tile_elems(cand_dtype) elements; its first tiles, up to
+// kWarmTiles of them, form the warm-up group (see DevTensor).
 static int plan_one(uint64_t n, int cand_dtype, uint32_t* n_tiles, uint32_t* warm_tiles) {
     if (n == 0 || n >= kMaxN) return RKV_ERR_INVALID_ARG;
     const uint64_t te = tile_elems(cand_dtype);
     const uint64_t tiles = (n + te - 1) / te;
     if (tiles > 0x3FFFFFFFull) return RKV_ERR_UNSUPPORTED;
     *n_tiles = (uint32_t)tiles;
-    // a shorter tensor warms up on the same share of its tiles, at least one
-    *warm_tiles = tiles >= (uint64_t)kWarmMinTiles
-                      ? (uint32_t)kWarmTiles
-                      : (uint32_t)((tiles * (uint64_t)kWarmTiles + (uint64_t)kWarmMinTiles - 1) / (uint64_t)kWarmMinTiles);
+    // The tiles that run at the same time as the first ones of the main group see what the
+    // warm-up tiles published and nothing else: with w warm-up tiles about 1 in w + 1 of them
+    // still has to locate a maximum, so w + c / (w + 1) tiles take the slow path, c the tiles
+    // running at once (the blocks of the grid, or all the tiles of a short tensor): least near
+    // w = sqrt(c).  kWarmTiles is that for two blocks on each of 148 SMs.
+    uint32_t w = 1;
+    while (w < (uint32_t)kWarmTiles && (uint64_t)(w + 1) * (w + 1) <= tiles) ++w;
+    *warm_tiles = w;
     return RKV_OK;
 }
 

@@ -27,8 +27,7 @@ __host__ __device__ constexpr uint32_t tile_elems(int cand_dtype) {
 }
 constexpr int kStages = 5;                           // ring depth (bulk copies in flight)
 constexpr int kPartK = 64;                           // candidates a block tracks at a time
-constexpr int kWarmTiles = 18;                       // leading tiles of a large tensor that are verified first
-constexpr int kWarmMinTiles = 2048;                  // ... of a tensor of at least this many tiles; a shorter one takes the same share, at least one tile
+constexpr int kWarmTiles = 18;                       // leading tiles of a tensor that are verified first: the square root of its tiles, at most this
 constexpr int kTailDiv = 4;                          // a tail item covers a quarter of a part's candidates ...
 constexpr int kTailDivGenerated = 2;                 // ... half, when every item regenerates its reference tile
 constexpr int kMaxTensors = 64;                      // rkv_verify_multi
@@ -73,8 +72,8 @@ static_assert(sizeof(CandState) == 64, "CandState layout");
 // the tiles after them with parts of up to kPartK candidates, group 2 its last
 // tail_tiles tiles with smaller parts.  Group 0 runs first: the maxima and loophole flags
 // it publishes let the rest skip almost all rare-path work.  Group 2 runs last: its
-// short items even out the finishing times of the blocks.  A shorter tensor warms up on the
-// same share of its tiles (at least one); in a launch whose tiles all fit the first wave of
+// short items even out the finishing times of the blocks.  A short tensor warms up on
+// the square root of its tiles; in a launch whose tiles all fit the first wave of
 // blocks every tile is in group 0.  Within a group, local item = part * tiles + tile.  The launch-wide item
 // numbering is given by the segment table (see Segment).
 struct DevTensor {

@@ -2,6 +2,7 @@
 symbol, validates arguments before touching CUDA, and plans slabs sensibly.
 No kernel is launched here."""
 import ctypes
+import math
 import os
 import re
 
@@ -70,12 +71,12 @@ def test_item_plan_properties(n, K, dtype):
     if n_tiles <= grid:
         assert warm == n_tiles           # everything fits the first wave of blocks: nobody to warm up for
     else:
-        # 18 tiles of 2048 or more, the same share of fewer
-        assert warm == (18 if n_tiles >= 2048 else -(-n_tiles * 18 // 2048))
+        # the square root of the tile count, at most 18
+        assert warm == min(18, math.isqrt(n_tiles))
     if warm < n_tiles:
         # a short warm-up group, then the fewest parts of at most 64 (more while the tiles are fewer
         # than the blocks)
-        assert warm * 100 < n_tiles + 100
+        assert warm * warm <= n_tiles
         main = n_tiles - warm - tail
         assert parts_main == max(-(-K // 64), min(K, -(-grid // main) if main < grid else 1))
         # a long tensor ends with half a tile per block in parts a quarter that size

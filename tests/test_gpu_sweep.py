@@ -131,7 +131,7 @@ def test_sweep_with_regenerated_references_and_a_large_case_among_small_ones():
 
 def test_sweep_of_short_tensors_with_warm_up_and_split_main_groups():
     """Three tensors of 30 to 151 tiles among forty of one tile: more tiles than the first wave of
-    blocks holds, so every tensor has a warm-up group of its own (one or two tiles), and fewer
+    blocks holds, so every tensor has a warm-up group of its own (the square root of its tiles), and fewer
     main-group tiles than blocks, so the main group splits the candidates into parts.  Stored and
     regenerated references, the three storage types, faults in every group; a copy of a regenerated
     input goes through the copy check of a short tensor."""
