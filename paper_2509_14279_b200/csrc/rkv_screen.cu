@@ -8,7 +8,8 @@
 //
 // Layout of the work: a thread takes 16-byte vectors (4 fp32 or 8 bf16 elements) at a
 // grid stride; for one vector position it visits the S outputs in turn, so the per-element
-// minimum and maximum across seeds never leave registers.  Sums are fp64, taken about a
+// minimum and maximum across seeds never leave registers (up to three fp32 outputs:
+// screen_few_kernel, which has the pieces of two positions in flight).  Sums are fp64, taken about a
 // pivot (the mean of the first finite values of the first output, computed identically by
 // every block) so that a large common offset costs the variance no digits.  Reductions are
 // deterministic: fixed shuffle trees, one partial per block, merged in block order;
@@ -138,18 +139,13 @@ __device__ __forceinline__ void screen_element(const ScreenArgs& A, Acc& a, doub
     }
 }
 
-// N outputs (s0 .. s0+N-1) at one vector position: their loads are issued together, then one
-// test tells whether all N * VEC values are finite (x * 0 is a zero for a finite x and NaN
-// otherwise) and the branch-free path can run.
+// The work of screen_chunk on N outputs whose pieces q[0 .. N-1] are already in registers.
 template <bool B16, int N>
-__device__ __forceinline__ void screen_chunk(const ScreenArgs& A, Acc& a, double pivot, int s0, uint64_t v,
-                                             uint32_t need, uint64_t r, uint64_t c0,
-                                             float (&lo)[B16 ? 8 : 4], float (&hi)[B16 ? 8 : 4],
-                                             bool (&ok)[B16 ? 8 : 4]) {
+__device__ __forceinline__ void screen_chunk_loaded(const ScreenArgs& A, Acc& a, double pivot, int s0,
+                                                    const uint4 (&q)[N], uint32_t need, uint64_t r, uint64_t c0,
+                                                    float (&lo)[B16 ? 8 : 4], float (&hi)[B16 ? 8 : 4],
+                                                    bool (&ok)[B16 ? 8 : 4]) {
     constexpr int VEC = B16 ? 8 : 4;
-    uint4 q[N];
-#pragma unroll
-    for (int u = 0; u < N; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[s0 + u]) + v);
     uint32_t b[N][VEC];
 #pragma unroll
     for (int u = 0; u < N; ++u) {
@@ -200,15 +196,26 @@ __device__ __forceinline__ void screen_chunk(const ScreenArgs& A, Acc& a, double
     }
 }
 
-template <bool B16>
-__global__ void __launch_bounds__(kScreenThreads, B16 ? kScreenBlocksPerSmB16 : kScreenBlocksPerSm)
-screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenPartial* __restrict__ partials) {
-    constexpr int VEC = B16 ? 8 : 4;
-    __shared__ double s_pivot;
-    __shared__ Acc s_acc[kScreenThreads / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // ---- pivot: mean of the finite values among the first elements of the first output ----
+// N outputs (s0 .. s0+N-1) at one vector position: their loads are issued together, then one
+// test tells whether all N * VEC values are finite (x * 0 is a zero for a finite x and NaN
+// otherwise) and the branch-free path can run.
+template <bool B16, int N>
+__device__ __forceinline__ void screen_chunk(const ScreenArgs& A, Acc& a, double pivot, int s0, uint64_t v,
+                                             uint32_t need, uint64_t r, uint64_t c0,
+                                             float (&lo)[B16 ? 8 : 4], float (&hi)[B16 ? 8 : 4],
+                                             bool (&ok)[B16 ? 8 : 4]) {
+    uint4 q[N];
+#pragma unroll
+    for (int u = 0; u < N; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[s0 + u]) + v);
+    screen_chunk_loaded<B16, N>(A, a, pivot, s0, q, need, r, c0, lo, hi, ok);
+}
+
+// The pivot: mean of the finite values among the first elements of the first output, computed
+// identically by every block (warp 0), handed to all threads through shared memory.
+template <bool B16>
+__device__ __forceinline__ double block_pivot(const ScreenArgs& A, double* s_pivot) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (warp == 0) {
         double ps = 0.0;
         uint32_t pc = 0;
@@ -226,14 +233,53 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
             ps += __shfl_xor_sync(kFull, ps, off);
             pc += __shfl_xor_sync(kFull, pc, off);
         }
-        if (lane == 0) s_pivot = pc ? ps / (double)pc : 0.0;
+        if (lane == 0) *s_pivot = pc ? ps / (double)pc : 0.0;
     }
     __syncthreads();
-    const double pivot = s_pivot;
+    return *s_pivot;
+}
 
-    Acc a;
+__device__ __forceinline__ void acc_clear(Acc& a) {
     a.sum = 0.0; a.sumsq = 0.0; a.n_fin = 0; a.n_nonfin = 0; a.arg = RKV_NO_INDEX;
     a.vmin = kInfF; a.vmax = -kInfF; a.spread = -1.0f; a.nonuniform = 0u;
+}
+
+// Block reduction (fixed shuffle tree, then the warps in order) and the block's partial.
+__device__ __forceinline__ void block_end(Acc a, uint32_t axes_wanted, double pivot, Acc* s_acc,
+                                          ScreenHeader* __restrict__ header, ScreenPartial* __restrict__ partials) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    a.nonuniform &= axes_wanted;
+    a.n_fin -= a.n_nonfin;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const Acc b = shfl_acc(a, off);
+        merge_acc(a, b);
+    }
+    if (lane == 0) s_acc[warp] = a;
+    __syncthreads();
+    if (tid == 0) {
+        Acc t = s_acc[0];
+        for (int w = 1; w < kScreenThreads / 32; ++w) merge_acc(t, s_acc[w]);
+        ScreenPartial p;
+        p.sum = t.sum; p.sumsq = t.sumsq; p.n_fin = t.n_fin; p.n_nonfin = t.n_nonfin; p.arg = t.arg;
+        p.vmin = t.vmin; p.vmax = t.vmax; p.spread = t.spread; p.nonuniform = t.nonuniform;
+        partials[blockIdx.x] = p;
+        if (blockIdx.x == 0) { header->pivot = pivot; header->grid = gridDim.x; }
+    }
+}
+
+template <bool B16>
+__global__ void __launch_bounds__(kScreenThreads, B16 ? kScreenBlocksPerSmB16 : kScreenBlocksPerSm)
+screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenPartial* __restrict__ partials) {
+    constexpr int VEC = B16 ? 8 : 4;
+    __shared__ double s_pivot;
+    __shared__ Acc s_acc[kScreenThreads / 32];
+    const int tid = threadIdx.x;
+
+    const double pivot = block_pivot<B16>(A, &s_pivot);
+
+    Acc a;
+    acc_clear(a);
 
     const bool vec_rows = (A.cols % VEC) == 0;       // every 16-byte vector lies inside one row
     const uint64_t nvec = A.n / VEC;
@@ -283,26 +329,73 @@ screen_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenParti
         for (uint64_t i = (uint64_t)blockIdx.x * kScreenThreads + tid; i < A.n; i += stride)
             screen_element<B16>(A, a, pivot, i, (axes_wanted & ~a.nonuniform) != 0u);
     }
-    a.nonuniform &= axes_wanted;
-    a.n_fin -= a.n_nonfin;
+    block_end(a, axes_wanted, pivot, s_acc, header, partials);
+}
 
-    // ---- block reduction: fixed shuffle tree, then the warps in order ----------------------
+// One vector position of fp32 outputs whose N = S pieces are already in registers: everything the
+// general kernel does for a position.
+template <int N>
+__device__ __forceinline__ void screen_position_loaded(const ScreenArgs& A, Acc& a, double pivot, uint64_t v,
+                                                       uint32_t axes_wanted, const uint4 (&q)[N]) {
+    constexpr int VEC = 4;
+    const uint64_t i0 = v * VEC;
+    a.n_fin += (unsigned long long)(VEC * N);
+    float lo[VEC], hi[VEC];
+    bool ok[VEC];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const Acc b = shfl_acc(a, off);
-        merge_acc(a, b);
+    for (int j = 0; j < VEC; ++j) { lo[j] = kInfF; hi[j] = -kInfF; ok[j] = true; }
+    const uint32_t need = axes_wanted & ~a.nonuniform;
+    uint64_t r = 0, c0 = 0;
+    if (need) { r = i0 / A.cols; c0 = i0 - r * A.cols; }
+    screen_chunk_loaded<false, N>(A, a, pivot, 0, q, need, r, c0, lo, hi, ok);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        a.vmin = fminf(a.vmin, lo[j]);
+        a.vmax = fmaxf(a.vmax, hi[j]);
     }
-    if (lane == 0) s_acc[warp] = a;
-    __syncthreads();
-    if (tid == 0) {
-        Acc t = s_acc[0];
-        for (int w = 1; w < kScreenThreads / 32; ++w) merge_acc(t, s_acc[w]);
-        ScreenPartial p;
-        p.sum = t.sum; p.sumsq = t.sumsq; p.n_fin = t.n_fin; p.n_nonfin = t.n_nonfin; p.arg = t.arg;
-        p.vmin = t.vmin; p.vmax = t.vmax; p.spread = t.spread; p.nonuniform = t.nonuniform;
-        partials[blockIdx.x] = p;
-        if (blockIdx.x == 0) { header->pivot = pivot; header->grid = gridDim.x; }
+    if (N >= 2) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            if (ok[j]) {
+                const float d = fabsf(__fsub_rn(hi[j], lo[j]));
+                if (d > a.spread) { a.spread = d; a.arg = i0 + j; }
+            }
+        }
     }
+}
+
+// N <= 3 fp32 outputs whose rows hold whole 16-byte vectors: the pieces of two positions (one grid
+// stride apart) are loaded before either is worked on, 2 * N loads per thread in flight instead of
+// N.  Same statistics as screen_kernel; a kernel of its own so that its registers do not weigh on
+// the general loop.
+template <int N>
+__global__ void __launch_bounds__(kScreenThreads, kScreenBlocksPerSm)
+screen_few_kernel(const ScreenArgs A, ScreenHeader* __restrict__ header, ScreenPartial* __restrict__ partials) {
+    constexpr int VEC = 4;
+    __shared__ double s_pivot;
+    __shared__ Acc s_acc[kScreenThreads / 32];
+    const int tid = threadIdx.x;
+    const double pivot = block_pivot<false>(A, &s_pivot);
+    Acc a;
+    acc_clear(a);
+    const uint64_t nvec = A.n / VEC;
+    const uint64_t stride = (uint64_t)gridDim.x * kScreenThreads;
+    const uint32_t axes_wanted = (A.rows >= 2 ? 1u : 0u) | (A.cols >= 2 ? 2u : 0u);
+    for (uint64_t v = (uint64_t)blockIdx.x * kScreenThreads + tid; v < nvec; v += 2 * stride) {
+        const uint64_t v2 = v + stride;
+        const bool two = v2 < nvec;
+        uint4 qa[N], qb[N];
+#pragma unroll
+        for (int u = 0; u < N; ++u) qa[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[u]) + v);
+        if (two) {
+#pragma unroll
+            for (int u = 0; u < N; ++u) qb[u] = __ldg(reinterpret_cast<const uint4*>(A.outs[u]) + v2);
+        }
+        screen_position_loaded<N>(A, a, pivot, v, axes_wanted, qa);
+        if (two) screen_position_loaded<N>(A, a, pivot, v2, axes_wanted, qb);
+    }
+    // (cols is a multiple of 4 here, so n is: no ragged end)
+    block_end(a, axes_wanted, pivot, s_acc, header, partials);
 }
 
 __global__ void __launch_bounds__(kScreenThreads)
@@ -407,7 +500,12 @@ int rkv_screen_outputs(const void* const* outs, int S, uint64_t rows, uint64_t c
     ScreenHeader* header = reinterpret_cast<ScreenHeader*>(workspace);
     ScreenPartial* partials = reinterpret_cast<ScreenPartial*>(header + 1);
     if (dtype == RKV_BF16) screen_kernel<true><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
-    else screen_kernel<false><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
+    else if (S <= 3 && (A.cols % 4) == 0) {
+        // (four outputs, eight loads in flight, spill at three blocks per SM and measure no faster)
+        if (S == 1) screen_few_kernel<1><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
+        else if (S == 2) screen_few_kernel<2><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
+        else screen_few_kernel<3><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
+    } else screen_kernel<false><<<grid, kScreenThreads, 0, stream>>>(A, header, partials);
     screen_finalize_kernel<<<1, kScreenThreads, 0, stream>>>(A, header, partials, grid, range_lim, std_lim,
                                                             spread_lim, stats_out);
     if (cudaGetLastError() != cudaSuccess) return RKV_ERR_CUDA;

@@ -125,6 +125,11 @@ def test_nonfinite_values():
     outs[2][64, :] = float("nan")
     got, want = check(outs, "nonfinite")
     assert int(got["n_nonfinite"]) == 3 + 384 and int(got["flags"]) & rkv.SCREEN_NONFINITE
+    # three and two outputs take the kernel that loads two positions at a time
+    got, _ = check(outs[:3], "nonfinite, three outputs")
+    assert int(got["n_nonfinite"]) == 2 + 384
+    got, _ = check(outs[1:3], "nonfinite, two outputs")
+    assert int(got["n_nonfinite"]) == 1 + 384
     allnan = [torch.full((8, 8), float("nan")) for _ in range(2)]
     got, _ = check(allnan, "all nan")
     assert int(got["argmax_seed_spread"]) == oracle.NO_INDEX and float(got["max_seed_spread"]) == -1.0
